@@ -1,0 +1,180 @@
+/*
+ * scap.h - C ABI of the SCAP sparse fully-connected library for NVIDIA B200 (sm_100a).
+ *
+ * SCAP (Statistical Calibrated Activation Pruning) sparsifies the INPUT activation of a
+ * fully-connected layer at decode time: the input is mode-centred (x' = x - m), every entry
+ * with |x'| < tau is dropped, and the matrix-vector product only fetches the weight rows of
+ * the surviving input channels; m W is folded into the bias offline so the layer's function is
+ * unchanged before pruning.
+ *
+ * Notation (paper's in brackets):  K input channels [IC], N output channels [OC], B batch rows.
+ *   x[B,K]      row-major activations, fp16 or bf16
+ *   W[K,N]      row-major weights, fp16 or bf16; row k holds every output of input channel k
+ *               [W in R^{IC x OC} of Eq. 1], so a kept channel is one contiguous row
+ *   m[K]        per-channel mode, fp32 (the paper's scalar eta is the constant vector)
+ *   tau[1]      pruning threshold, fp32, in DEVICE memory (no host round trip)
+ *   b_fused[N]  b + m W, fp32 (Eq. 6)
+ *   y[B,N]      fp32
+ *
+ * General rules for every entry point
+ *   - All data pointers are DEVICE pointers unless the parameter name ends in _host.
+ *   - The caller owns every buffer; the library allocates no device memory and keeps no state
+ *     between calls except the process-wide tuning set by scap_tune().
+ *   - Calls enqueue work on `stream` and return without synchronising; they perform no host
+ *     synchronisation, so they may be recorded into a CUDA graph.  Two calls that share a
+ *     workspace must be ordered on one stream.
+ *   - Data pointers must be 16-byte aligned and N (and F, D for the FFN calls) a multiple of 8,
+ *     else SCAP_ERR_ALIGN.  B outside 1..16, K < 1, K > 131072 or N < 1 give SCAP_ERR_SHAPE.  A
+ *     NULL required pointer gives SCAP_ERR_INVALID_ARG, a workspace smaller than the matching
+ *     *_workspace() query SCAP_ERR_WORKSPACE, an unknown dtype SCAP_ERR_DTYPE, a failed launch
+ *     SCAP_ERR_CUDA, a device that is not compute capability 10.x SCAP_ERR_UNSUPPORTED_ARCH.
+ *     Nothing throws, aborts, traps or prints.  On error nothing has been enqueued.
+ *   - Workspace contents are scratch: undefined on entry, undefined on exit.
+ */
+#ifndef SCAP_H_
+#define SCAP_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    SCAP_OK = 0,
+    SCAP_ERR_INVALID_ARG = 1,
+    SCAP_ERR_SHAPE = 2,
+    SCAP_ERR_DTYPE = 3,
+    SCAP_ERR_ALIGN = 4,
+    SCAP_ERR_WORKSPACE = 5,
+    SCAP_ERR_CUDA = 6,
+    SCAP_ERR_TIMEOUT = 7,
+    SCAP_ERR_UNSUPPORTED_ARCH = 8
+} scap_status;
+
+typedef enum { SCAP_F16 = 0, SCAP_BF16 = 1 } scap_dtype;
+
+/* A CUDA stream handle (cudaStream_t); NULL is the legacy default stream. */
+typedef struct CUstream_st *scap_stream_t;
+
+#define SCAP_MAX_BATCH 16
+#define SCAP_MAX_EXPERTS 32
+#define SCAP_MAX_TOP_K 4
+
+/* Static string naming a status code. */
+const char *scap_status_string(scap_status st);
+
+/* Library version, major * 1000 + minor. */
+int scap_version(void);
+
+/* Process-wide tuning knobs (plain ints, not thread-safe against concurrent calls):
+ *   "split_k"  force the split-K factor of the gather-GEMV (0 = automatic, at most 64)
+ *   "pdl"      1 = launch dependent kernels with programmatic dependent launch (default), 0 = off
+ * Unknown keys return SCAP_ERR_INVALID_ARG.  Tuning never changes what is computed; split_k
+ * changes the (fixed) summation order and therefore the last bits of y.  Query workspace sizes
+ * after tuning.                                                                               */
+scap_status scap_tune(const char *key, int value);
+
+/* ------------------------------------------------------------------------------------------
+ * Offline calibration (Section 3, "Mode-Centering Calibration"; Eq. 2 for tau)
+ *
+ * scap_calibrate reads calibration activations x_calib[T,K] (row-major, dtype dt) and writes
+ *   m_out[K]   per-channel mode: arg-max bin centre of an nbins-bin histogram over the channel's
+ *              [min, max] range (lowest bin wins ties; a constant channel returns that constant).
+ *              nbins = 0 disables centring and writes zeros.  1 <= nbins <= 2048 otherwise.
+ *   tau_out[1] the `sparsity` quantile (linear interpolation between order statistics) of the
+ *              importance |x - m| pooled over all T*K values; sparsity <= 0 gives tau = 0.
+ * Binary32 arithmetic with every operation rounded separately, so results are bit-reproducible.
+ * Inputs must be finite.  sparsity must lie in [0, 1); T*K < 2^31; T <= 65535.
+ * ------------------------------------------------------------------------------------------ */
+size_t scap_calibrate_workspace(int T, int K, int nbins);
+scap_status scap_calibrate(const void *x_calib, int T, int K, scap_dtype dt, double sparsity, int nbins,
+                           float *m_out, float *tau_out, void *ws, size_t ws_bytes, scap_stream_t stream);
+
+/* Eq. 5-6: b_fused[n] = b[n] + sum_k m[k] W[k,n].  b is in the weight dtype and may be NULL
+ * (zero bias).  Run once per layer after calibration.                                          */
+size_t scap_fold_bias_workspace(int K, int N);
+scap_status scap_fold_bias(const void *W, const float *m, const void *b, int K, int N, scap_dtype dt,
+                           float *b_fused, void *ws, size_t ws_bytes, scap_stream_t stream);
+
+/* ------------------------------------------------------------------------------------------
+ * Decode-time sparse FC (Eq. 2-3, Eq. 6; Alg. 3 "SCAP FC with Mode Centering")
+ *
+ *   d[b,k]   = float(x[b,k]) - m[k]            one binary32 subtraction (m == NULL: d = x)
+ *   keep     = |d| >= tau                      (a NaN is dropped)
+ *   y[b,n]   = b_fused[n] + sum_k keep[b,k] d[b,k] W[k,n]      fp32 accumulation, fixed order
+ * Only rows of W whose channel is kept by at least one batch row are read.  Pruning is per
+ * element, so row b of a batched call equals the batch-1 call on row b up to summation order.
+ * Optional outputs for inspection: idx_out[K] receives the ascending list of fetched channels
+ * (first *nnz_out entries valid), nnz_out[1] their number.  m, b_fused, idx_out, nnz_out may
+ * be NULL.  Results are bitwise reproducible for fixed shapes and tuning.
+ * ------------------------------------------------------------------------------------------ */
+size_t scap_fc_workspace(int B, int K, int N);
+scap_status scap_sparse_fc(const void *x, const void *W, const float *m, const float *tau, const float *b_fused,
+                           float *y, int B, int K, int N, scap_dtype dt, uint32_t *idx_out, int *nnz_out,
+                           void *ws, size_t ws_bytes, scap_stream_t stream);
+
+/* Eq. 1: y = x W + b over the same layout, no pruning; the library's own dense baseline.
+ * b is fp32 [N] or NULL.  Uses scap_fc_workspace(B, K, N).                                     */
+scap_status scap_dense_fc(const void *x, const void *W, const float *b, float *y, int B, int K, int N,
+                          scap_dtype dt, void *ws, size_t ws_bytes, scap_stream_t stream);
+
+/* scap_sparse_fc for a caller whose activations live in HOST memory: copies x_host[B,K]
+ * (dtype dt; pinned memory recommended) to the device, runs the sparse FC, and copies y back to
+ * y_host[B,N] (fp32), all enqueued on `stream`; y_host is valid once the stream has drained.
+ * W, m, tau, b_fused stay device-resident.  Needs scap_fc_host_workspace(B, K, N) bytes.        */
+size_t scap_fc_host_workspace(int B, int K, int N);
+scap_status scap_sparse_fc_host(const void *x_host, const void *W, const float *m, const float *tau,
+                                const float *b_fused, float *y_host, int B, int K, int N, scap_dtype dt,
+                                void *ws, size_t ws_bytes, scap_stream_t stream);
+
+/* ------------------------------------------------------------------------------------------
+ * SwiGLU FFN block (Alg. 2 "SCAP's SwiGLU")
+ *
+ *   [g | u] = sparse_fc(h; Wgu, m1, tau1, bgu_fused)     one mask shared by gate and up
+ *   z       = u * silu(g),  silu(g) = g / (1 + exp(-g))  kept in fp32
+ *   y       = sparse_fc(z; Wd, m2, tau2, bd_fused)
+ * h[B,D]; Wgu[D,2F] with gate in columns 0..F-1 and up in columns F..2F-1 of each row; Wd[F,D];
+ * bgu_fused[2F]; bd_fused[D]; y[B,D].  m1, m2 and the two fused biases may be NULL.  Optional
+ * outputs: z_out[B,F] (the fp32 z the second mask was taken on), idx1_out[D]/nnz1_out[1],
+ * idx2_out[F]/nnz2_out[1].  D and F must be multiples of 8.
+ * ------------------------------------------------------------------------------------------ */
+size_t scap_glu_workspace(int B, int D, int F);
+scap_status scap_glu_ffn(const void *h, const void *Wgu, const void *Wd, const float *m1, const float *tau1,
+                         const float *bgu_fused, const float *m2, const float *tau2, const float *bd_fused,
+                         float *y, int B, int D, int F, scap_dtype dt, float *z_out, uint32_t *idx1_out,
+                         int *nnz1_out, uint32_t *idx2_out, int *nnz2_out, void *ws, size_t ws_bytes,
+                         scap_stream_t stream);
+
+/* ------------------------------------------------------------------------------------------
+ * Mixture-of-experts FFN layer (the paper applies SCAP to Mixtral-8x7B, Table 4; it does not
+ * describe the router, so the convention is this library's): p = softmax(logits[b, 0..E-1]),
+ * the top_k largest are selected (ties to the lower index), their weights renormalised to sum
+ * to one, and y[b] = sum_j w[b,j] * glu_ffn_{e(b,j)}(h[b]), summed in selection order.  Each
+ * expert has its own calibration (m1, tau1, m2, tau2) and fused biases; the rows routed to one
+ * expert share that expert's union mask.
+ * experts_host: HOST array of E structs holding DEVICE pointers (read during the call only).
+ * logits[B,E] fp32.  Optional outputs expert_out[B,top_k] (int32), weight_out[B,top_k] (fp32).
+ * 1 <= E <= SCAP_MAX_EXPERTS, 1 <= top_k <= min(E, SCAP_MAX_TOP_K).
+ * ------------------------------------------------------------------------------------------ */
+typedef struct {
+    const void *Wgu;        /* [D,2F] */
+    const void *Wd;         /* [F,D]  */
+    const float *m1;        /* [D]  nullable */
+    const float *tau1;      /* [1]  */
+    const float *bgu_fused; /* [2F] nullable */
+    const float *m2;        /* [F]  nullable */
+    const float *tau2;      /* [1]  */
+    const float *bd_fused;  /* [D]  nullable */
+} scap_expert;
+
+size_t scap_moe_workspace(int B, int D, int F, int E, int top_k);
+scap_status scap_moe_ffn(const void *h, const float *logits, const scap_expert *experts_host, int E, int top_k,
+                         float *y, int B, int D, int F, scap_dtype dt, int *expert_out, float *weight_out,
+                         void *ws, size_t ws_bytes, scap_stream_t stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SCAP_H_ */

@@ -1,0 +1,100 @@
+// Shared device/host helpers of the SCAP sm_100a library (internal; the public ABI is scap.h).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "scap.h"
+
+namespace scap {
+
+constexpr int CH = 256;            // channels per compaction chunk (= threads of a compaction CTA)
+constexpr int TN = 256;            // output columns per gather-GEMV CTA: 32 lanes x 8 columns (16 B)
+constexpr int GEMV_THREADS = 256;  // 8 warps; the warps of a CTA take rows round-robin
+constexpr int GEMV_WARPS = GEMV_THREADS / 32;
+constexpr int LB = 256;            // kept rows staged in shared memory per fill
+constexpr int MAX_SPLIT = 64;      // upper bound on the split-K factor
+constexpr int MAX_CHUNKS_SMEM = 512;  // chunk-count prefix held in shared memory: K <= 512 * CH = 131072
+
+struct Tuning {
+    int split_k;  // 0 = automatic
+    int pdl;      // programmatic dependent launch between the kernels of one call
+};
+extern Tuning g_tune;
+
+// ---- status helpers -------------------------------------------------------------------------
+scap_status check_device();  // SCAP_OK on compute capability 10.x
+int sm_count();              // multiprocessors of the current device (148 when no device is present)
+
+inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+inline scap_status cuda_status(cudaError_t e) {
+    if (e == cudaSuccess) return SCAP_OK;
+    cudaGetLastError();
+    return SCAP_ERR_CUDA;
+}
+
+// ---- programmatic dependent launch ----------------------------------------------------------
+// wait: blocks until every kernel this grid depends on has finished and its writes are visible
+// (returns at once when the launch carried no programmatic dependency).
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+// launch_dependents: lets the next kernel in the stream begin its launch early; that kernel still
+// calls griddep_wait() before touching anything this grid produces.
+__device__ __forceinline__ void griddep_launch_dependents() {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, bool pdl,
+                          Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = pdl ? 1 : 0;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
+// ---- storage dtype widening -------------------------------------------------------------------
+// Two 16-bit values packed in one 32-bit word -> two floats (exact).
+template <bool BF16>
+__device__ __forceinline__ void widen2(uint32_t u, float &lo, float &hi) {
+    if constexpr (BF16) {
+        lo = __uint_as_float(u << 16);
+        hi = __uint_as_float(u & 0xffff0000u);
+    } else {
+        __half2 h = *reinterpret_cast<__half2 *>(&u);
+        float2 f = __half22float2(h);
+        lo = f.x;
+        hi = f.y;
+    }
+}
+
+__device__ __forceinline__ float widen1(const __nv_bfloat16 &v) { return __bfloat162float(v); }
+__device__ __forceinline__ float widen1(const __half &v) { return __half2float(v); }
+__device__ __forceinline__ float widen1(const float &v) { return v; }
+
+template <bool BF16>
+__device__ __forceinline__ float widen_at(const void *p, size_t i) {
+    if constexpr (BF16) return widen1(reinterpret_cast<const __nv_bfloat16 *>(p)[i]);
+    else return widen1(reinterpret_cast<const __half *>(p)[i]);
+}
+
+// 16-byte streaming load of weights: read-only path, no L1 allocation (each byte is used once).
+__device__ __forceinline__ uint4 ld_stream16(const void *p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
+}
+
+}  // namespace scap
