@@ -1,0 +1,85 @@
+"""scap_calibrate against the oracle: the mode vector and tau must match bit for bit (both sides follow the
+same binary32 recipe, and tau is an order statistic interpolated in binary64)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import scap_inputs as si
+from scap_testlib import dev, workspace
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def S():
+    import paper_2412_07174_b200 as scap
+    scap.lib()
+    return scap
+
+
+def run_calibrate(S, xbits, dt, s, nbins):
+    x = dev(xbits, dt)
+    T, K = x.shape
+    ws = workspace(S.scap_calibrate_workspace(T, K, nbins))
+    mg = workspace(K * 4)
+    tg = workspace(4)
+    m = mg.view(torch.float32, (K,))
+    tau = tg.view(torch.float32, (1,))
+    S.scap_calibrate(x, s, nbins, m, tau, ws.payload)
+    torch.cuda.synchronize()
+    assert ws.intact() and mg.intact() and tg.intact()
+    return m.cpu().numpy().copy(), np.float32(tau.item())
+
+
+@pytest.mark.parametrize("T,K,dt,nbins,s", [
+    (256, 1024, si.F16, 2048, 0.5),       # config 0's calibration set
+    (64, 40, si.BF16, 16, 0.3),           # one partial strip
+    (100, 264, si.BF16, 2048, 0.65),
+    (513, 72, si.F16, 7, 0.999),
+    (32, 8, si.BF16, 1, 0.01),
+    (300, 520, si.BF16, 333, 0.8),
+])
+def test_mode_and_tau_bit_exact(S, T, K, dt, nbins, s):
+    d = si.laplace_fc(0 if dt == si.F16 else 4, K, 8, dt, T, 1)
+    xf = si.to_f32(d["x_calib"], dt)
+    m_o, tau_o = oracle.calibrate(xf, s, nbins)
+    m_g, tau_g = run_calibrate(S, d["x_calib"], dt, s, nbins)
+    assert np.array_equal(m_g, m_o)
+    assert tau_g.view(np.uint32) == np.float32(tau_o).view(np.uint32)
+
+
+def test_no_centring_and_zero_sparsity(S):
+    d = si.laplace_fc(4, 128, 8, si.BF16, 200, 1)
+    xf = si.to_f32(d["x_calib"], si.BF16)
+    m_g, tau_g = run_calibrate(S, d["x_calib"], si.BF16, 0.7, 0)
+    assert not m_g.any() and tau_g == oracle.tau(xf, None, 0.7)
+    m_g, tau_g = run_calibrate(S, d["x_calib"], si.BF16, 0.0, 64)
+    assert np.array_equal(m_g, oracle.mode(xf, 64)) and tau_g == 0.0
+
+
+def test_constant_channels_and_heavy_ties(S):
+    # quantised data: many equal importances, constant channels, both order statistics in one bucket
+    T, K = 96, 48
+    rng = np.random.default_rng(11)
+    x = rng.integers(-3, 4, size=(T, K)).astype(np.float64) * 0.25
+    x[:, 5] = 1.5
+    x[:, 17] = 0.0
+    bits = si.to_bits(x, si.BF16)
+    xf = si.to_f32(bits, si.BF16)
+    for s in (0.1, 0.5, 0.9):
+        for nbins in (4, 2048):
+            m_o, tau_o = oracle.calibrate(xf, s, nbins)
+            m_g, tau_g = run_calibrate(S, bits, si.BF16, s, nbins)
+            assert np.array_equal(m_g, m_o) and tau_g == tau_o
+
+
+def test_config4_calibration_size(S):
+    # 2048 tokens x 14336 channels, 2048 bins: the calibration the sweep times
+    d = si.laplace_fc(4, 14336, 8, si.BF16, 2048, 1)
+    xf = si.to_f32(d["x_calib"], si.BF16)
+    m_o, tau_o = oracle.calibrate(xf, 0.6, 2048)
+    m_g, tau_g = run_calibrate(S, d["x_calib"], si.BF16, 0.6, 2048)
+    assert np.array_equal(m_g, m_o) and tau_g == tau_o
+    keep = oracle.mask(xf[:64], m_o, tau_o)[0]
+    assert abs((1 - keep.mean()) - 0.6) < 0.01

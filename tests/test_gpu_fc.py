@@ -1,0 +1,258 @@
+"""GPU parity of the sparse FC, the dense baseline and bias folding against the CPU oracle, through the
+C ABI.  Mask (kept-channel list) bit-exact; y within 2e-3 relative L2 per row of the oracle's binary64 y."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import scap_inputs as si
+from scap_testlib import REL_L2_TOL, dev, f32, oracle_fc, rel_l2_rows, workspace
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def S():
+    import paper_2412_07174_b200 as scap
+    scap.lib()
+    return scap
+
+
+def run_sparse(S, d, m, tau, bf, x_bits=None, want_idx=True):
+    dt = d["dt"]
+    x = dev(d["x"] if x_bits is None else x_bits, dt)
+    W = dev(d["W"], dt)
+    B, K = x.shape
+    N = W.shape[1]
+    ws = workspace(S.scap_fc_workspace(B, K, N))
+    yg = workspace(B * N * 4)
+    y = yg.view(torch.float32, (B, N))
+    idx = torch.full((K,), -1, dtype=torch.int32, device="cuda") if want_idx else None
+    nnz = torch.full((1,), -1, dtype=torch.int32, device="cuda") if want_idx else None
+    S.scap_sparse_fc(x, W, None if m is None else f32(m), f32([tau]), None if bf is None else f32(bf), y, ws.payload,
+                     idx_out=idx, nnz_out=nnz)
+    torch.cuda.synchronize()
+    assert ws.intact() and yg.intact()
+    if want_idx:
+        n = int(nnz.item())
+        return y.cpu().numpy().copy(), idx[:n].cpu().numpy().astype(np.uint32), n
+    return y.cpu().numpy().copy(), None, None
+
+
+def check_fc(S, d, m, tau, with_bias=True):
+    dt = d["dt"]
+    bf64 = oracle.fold_bias(d["W"], dt, m if m is not None else np.zeros(d["K"], np.float32), d.get("b")) if with_bias else None
+    bf32 = None if bf64 is None else bf64.astype(np.float32)
+    y64, keep, idx = oracle_fc(d, m, tau, bf64)
+    y, gidx, n = run_sparse(S, d, m, tau, bf32)
+    assert n == idx.size
+    assert np.array_equal(gidx, idx)
+    if np.linalg.norm(y64) > 0:
+        assert rel_l2_rows(y, y64) <= REL_L2_TOL
+    return y, y64, keep
+
+
+# ---------------------------------------------------------------- config 0 (fp16, 1024 x 1024, batch 1)
+
+def test_config0_single_fc_fp16(S):
+    d = si.config0()
+    xc = si.to_f32(d["x_calib"], d["dt"])
+    m, tau = oracle.calibrate(xc, 0.5, 2048)
+    y, y64, keep = check_fc(S, d, m, tau)
+    assert 0.3 < keep.mean() < 0.7
+
+
+# ---------------------------------------------------------------- shapes spanning tiles, ragged tails, batches
+
+@pytest.mark.parametrize("K,N,B,dt", [
+    (1000, 264, 1, si.BF16), (33, 8, 3, si.F16), (1, 16, 2, si.BF16), (777, 520, 5, si.BF16),
+    (2048, 1032, 16, si.F16), (300, 4096, 4, si.BF16), (5000, 256, 8, si.BF16), (256, 248, 2, si.F16),
+])
+def test_shapes_and_batches(S, K, N, B, dt):
+    d = si.laplace_fc(4, K, N, dt, 32, B)
+    m = d["m_true"]
+    tau = oracle.tau(si.to_f32(d["x_calib"], dt), m, 0.6)
+    check_fc(S, d, m, tau)
+    check_fc(S, d, None, tau, with_bias=False)
+
+
+@pytest.mark.parametrize("s", [0.0, 0.25, 0.5, 0.9, 0.99])
+def test_sparsity_levels(S, s):
+    d = si.laplace_fc(4, 1536, 776, si.BF16, 64, 2)
+    m = oracle.mode(si.to_f32(d["x_calib"], d["dt"]), 256)
+    tau = oracle.tau(si.to_f32(d["x_calib"], d["dt"]), m, s)
+    check_fc(S, d, m, tau)
+
+
+# ---------------------------------------------------------------- degenerate cases
+
+def test_tau_zero_is_dense_and_tau_inf_returns_bias(S):
+    d = si.laplace_fc(4, 640, 264, si.BF16, 8, 3)
+    dt = d["dt"]
+    bf = np.linspace(-1, 1, 264).astype(np.float32)
+    y, idx, n = run_sparse(S, d, None, 0.0, bf)
+    assert n == 640 and np.array_equal(idx, np.arange(640, dtype=np.uint32))
+    y64 = oracle.dense_fc(si.to_f32(d["x"], dt), d["W"], dt, bf)
+    assert rel_l2_rows(y, y64) <= REL_L2_TOL
+    y, idx, n = run_sparse(S, d, d["m_true"], np.inf, bf)
+    assert n == 0 and np.array_equal(y, np.tile(bf, (3, 1)))       # nnz = 0: y == b_fused exactly
+    y, idx, n = run_sparse(S, d, d["m_true"], np.inf, None)
+    assert n == 0 and not y.any()
+
+
+def test_ties_signed_zero_and_nan(S):
+    K, N = 40, 16
+    d = si.laplace_fc(4, K, N, si.BF16, 8, 2)
+    x = np.zeros((2, K))
+    x[0, 0], x[0, 1], x[0, 2], x[0, 3], x[0, 4] = 0.5, -0.5, 0.49, np.nan, -0.0
+    x[1, 5], x[1, 6] = 2.0, -0.25
+    xb = si.to_bits(x, si.BF16)
+    xb[0, 3] = 0x7FC0                                              # bf16 NaN
+    y64, keep, idx = oracle_fc(d, None, 0.5, None, x_bits=xb)
+    assert idx.tolist() == [0, 1, 5]                               # |x| == tau kept; NaN dropped
+    y, gidx, n = run_sparse(S, d, None, 0.5, None, x_bits=xb)
+    assert gidx.tolist() == [0, 1, 5] and np.isfinite(y).all()
+    assert rel_l2_rows(y, y64) <= REL_L2_TOL
+    # tau = 0 keeps +-0 too (all channels except the NaN)
+    y, gidx, n = run_sparse(S, d, None, 0.0, None, x_bits=xb)
+    assert n == K - 1 and 3 not in gidx.tolist()
+
+
+def test_mask_boundary_uses_one_binary32_subtraction(S):
+    # values straddling the threshold by one ulp after the subtraction
+    K, N = 512, 64
+    d = si.laplace_fc(4, K, N, si.F16, 8, 1)
+    m = d["m_true"]
+    xf = si.to_f32(d["x"], si.F16)
+    dd = np.abs((xf[0] - m).astype(np.float32))
+    for t in np.sort(dd)[[10, 100, 300]]:
+        for tau in (t, np.nextafter(t, np.float32(np.inf)), np.nextafter(t, np.float32(0))):
+            _, keep, idx = oracle_fc(d, m, tau, None)
+            _, gidx, n = run_sparse(S, d, m, float(tau), None)
+            assert np.array_equal(gidx, idx)
+
+
+# ---------------------------------------------------------------- properties
+
+def test_bitwise_determinism_and_row_independence(S):
+    d = si.laplace_fc(4, 2048, 1024, si.BF16, 16, 4)
+    m, tau = d["m_true"], 0.25
+    y1, i1, _ = run_sparse(S, d, m, tau, None)
+    y2, i2, _ = run_sparse(S, d, m, tau, None)
+    assert np.array_equal(y1, y2) and np.array_equal(i1, i2)
+    for b in range(4):
+        yb, _, _ = run_sparse(S, d, m, tau, None, x_bits=d["x"][b:b + 1])
+        y64 = oracle.sparse_fc(si.to_f32(d["x"][b:b + 1], d["dt"]), d["W"], d["dt"], m, tau, None)
+        assert rel_l2_rows(yb, y64) <= REL_L2_TOL
+        assert rel_l2_rows(y1[b:b + 1], y64) <= REL_L2_TOL
+
+
+@pytest.mark.parametrize("split", [1, 2, 7, 64])
+def test_any_split_k_gives_the_same_answer(S, split):
+    d = si.laplace_fc(4, 1500, 520, si.BF16, 16, 3)
+    try:
+        S.scap_tune("split_k", split)
+        check_fc(S, d, d["m_true"], 0.2)
+    finally:
+        S.scap_tune("split_k", 0)
+
+
+def test_pdl_off_gives_identical_bits(S):
+    d = si.laplace_fc(4, 1500, 520, si.BF16, 16, 2)
+    y1, _, _ = run_sparse(S, d, d["m_true"], 0.2, None)
+    try:
+        S.scap_tune("pdl", 0)
+        y2, _, _ = run_sparse(S, d, d["m_true"], 0.2, None)
+    finally:
+        S.scap_tune("pdl", 1)
+    assert np.array_equal(y1, y2)
+
+
+def test_back_to_back_calls_share_a_workspace(S):
+    # many calls in a row on one stream with different inputs: each must see only its own lists
+    d = si.laplace_fc(4, 1024, 512, si.BF16, 16, 8)
+    dt = d["dt"]
+    W = dev(d["W"], dt)
+    m = f32(d["m_true"])
+    tau = f32([0.3])
+    ws = workspace(S.scap_fc_workspace(1, 1024, 512))
+    xs = [dev(d["x"][b:b + 1], dt) for b in range(8)]
+    ys = [torch.empty((1, 512), dtype=torch.float32, device="cuda") for _ in range(8)]
+    for rep in range(3):
+        for b in range(8):
+            S.scap_sparse_fc(xs[b], W, m, tau, None, ys[b], ws.payload)
+    torch.cuda.synchronize()
+    assert ws.intact()
+    for b in range(8):
+        y64 = oracle.sparse_fc(si.to_f32(d["x"][b:b + 1], dt), d["W"], dt, d["m_true"], 0.3, None)
+        assert rel_l2_rows(ys[b].cpu().numpy(), y64) <= REL_L2_TOL
+
+
+def test_cuda_graph_replay_matches_eager(S):
+    d = si.laplace_fc(4, 1024, 512, si.BF16, 16, 2)
+    dt = d["dt"]
+    x, W, m, tau = dev(d["x"], dt), dev(d["W"], dt), f32(d["m_true"]), f32([0.3])
+    ws = workspace(S.scap_fc_workspace(2, 1024, 512))
+    y_e = torch.empty((2, 512), dtype=torch.float32, device="cuda")
+    y_g = torch.zeros((2, 512), dtype=torch.float32, device="cuda")
+    S.scap_sparse_fc(x, W, m, tau, None, y_e, ws.payload)
+    torch.cuda.synchronize()
+    st = torch.cuda.Stream()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(st):
+        with torch.cuda.graph(g, stream=st):
+            S.scap_sparse_fc(x, W, m, tau, None, y_g, ws.payload)
+            S.scap_sparse_fc(x, W, m, tau, None, y_g, ws.payload)
+    g.replay()
+    g.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(y_e, y_g)
+
+
+# ---------------------------------------------------------------- dense baseline, bias folding, host variant
+
+@pytest.mark.parametrize("K,N,B,dt", [(1000, 264, 1, si.BF16), (2048, 1032, 16, si.F16), (640, 4096, 3, si.BF16)])
+def test_dense_fc(S, K, N, B, dt):
+    d = si.laplace_fc(4, K, N, dt, 8, B)
+    x, W = dev(d["x"], dt), dev(d["W"], dt)
+    b = np.linspace(-2, 2, N).astype(np.float32)
+    ws = workspace(S.scap_fc_workspace(B, K, N))
+    yg = workspace(B * N * 4)
+    y = yg.view(torch.float32, (B, N))
+    S.scap_dense_fc(x, W, f32(b), y, ws.payload)
+    assert ws.intact() and yg.intact()
+    y64 = oracle.dense_fc(si.to_f32(d["x"], dt), d["W"], dt, b)
+    assert rel_l2_rows(y.cpu().numpy(), y64) <= REL_L2_TOL
+    S.scap_dense_fc(x, W, None, y, ws.payload)
+    torch.cuda.synchronize()
+    assert rel_l2_rows(y.cpu().numpy(), oracle.dense_fc(si.to_f32(d["x"], dt), d["W"], dt, None)) <= REL_L2_TOL
+
+
+@pytest.mark.parametrize("K,N,dt,bias", [(1024, 1024, si.F16, True), (1000, 264, si.BF16, False), (4096, 520, si.BF16, True)])
+def test_fold_bias(S, K, N, dt, bias):
+    d = si.laplace_fc(0, K, N, dt, 8, 1, with_bias=bias)
+    W = dev(d["W"], dt)
+    m = d["m_true"]
+    b = dev(d["b"], dt) if bias else None
+    ws = workspace(S.scap_fold_bias_workspace(K, N))
+    og = workspace(N * 4)
+    out = og.view(torch.float32, (N,))
+    S.scap_fold_bias(W, f32(m), b, out, ws.payload)
+    assert ws.intact() and og.intact()
+    want = oracle.fold_bias(d["W"], dt, m, d["b"])
+    got = out.cpu().numpy().astype(np.float64)
+    assert np.linalg.norm(got - want) / np.linalg.norm(want) <= 1e-6
+
+
+def test_host_buffer_variant_matches_device_variant(S):
+    d = si.laplace_fc(4, 1024, 520, si.BF16, 16, 4)
+    dt = d["dt"]
+    y_dev, _, _ = run_sparse(S, d, d["m_true"], 0.3, None, want_idx=False)
+    W, m, tau = dev(d["W"], dt), f32(d["m_true"]), f32([0.3])
+    xh = si.as_torch(d["x"], dt).pin_memory()
+    yh = torch.zeros((4, 520), dtype=torch.float32).pin_memory()
+    ws = workspace(S.scap_fc_host_workspace(4, 1024, 520))
+    S.scap_sparse_fc_host(xh, W, m, tau, None, yh, ws.payload)
+    torch.cuda.synchronize()
+    assert ws.intact()
+    assert np.array_equal(yh.numpy(), y_dev)
