@@ -107,7 +107,7 @@ def test_ties_signed_zero_and_nan(S):
     x[0, 0], x[0, 1], x[0, 2], x[0, 3], x[0, 4] = 0.5, -0.5, 0.49, np.nan, -0.0
     x[1, 5], x[1, 6] = 2.0, -0.25
     xb = si.to_bits(x, si.BF16)
-    xb[0, 3] = 0x7FC0                                              # bf16 NaN
+    xb[:, 3] = 0x7FC0                                              # bf16 NaN in both rows
     y64, keep, idx = oracle_fc(d, None, 0.5, None, x_bits=xb)
     assert idx.tolist() == [0, 1, 5]                               # |x| == tau kept; NaN dropped
     y, gidx, n = run_sparse(S, d, None, 0.5, None, x_bits=xb)
@@ -115,7 +115,7 @@ def test_ties_signed_zero_and_nan(S):
     assert rel_l2_rows(y, y64) <= REL_L2_TOL
     # tau = 0 keeps +-0 too (all channels except the NaN)
     y, gidx, n = run_sparse(S, d, None, 0.0, None, x_bits=xb)
-    assert n == K - 1 and 3 not in gidx.tolist()
+    assert n == K - 1 and 3 not in gidx.tolist() and np.isfinite(y).all()
 
 
 def test_mask_boundary_uses_one_binary32_subtraction(S):
