@@ -24,7 +24,7 @@
  *     synchronisation, so they may be recorded into a CUDA graph.  Two calls that share a
  *     workspace must be ordered on one stream.
  *   - Data pointers must be 16-byte aligned and N (and F, D for the FFN calls) a multiple of 8,
- *     else SCAP_ERR_ALIGN.  B outside 1..16, K < 1, K > 131072 or N < 1 give SCAP_ERR_SHAPE.  A
+ *     else SCAP_ERR_ALIGN.  B outside 1..16, K < 1, K > 1048576 or N < 1 give SCAP_ERR_SHAPE.  A
  *     NULL required pointer gives SCAP_ERR_INVALID_ARG, a workspace smaller than the matching
  *     *_workspace() query SCAP_ERR_WORKSPACE, an unknown dtype SCAP_ERR_DTYPE, a failed launch
  *     SCAP_ERR_CUDA, a device that is not compute capability 10.x SCAP_ERR_UNSUPPORTED_ARCH.
@@ -69,7 +69,7 @@ const char *scap_status_string(scap_status st);
 int scap_version(void);
 
 /* Process-wide tuning knobs (plain ints, not thread-safe against concurrent calls):
- *   "split_k"  force the split-K factor of the gather-GEMV (0 = automatic, at most 64)
+ *   "split_k"  cap the split-K factor (thread-block cluster size) of the FC kernel: 0 = automatic, else 1..8
  *   "pdl"      1 = launch dependent kernels with programmatic dependent launch (default), 0 = off
  * Unknown keys return SCAP_ERR_INVALID_ARG.  Tuning never changes what is computed; split_k
  * changes the (fixed) summation order and therefore the last bits of y.  Query workspace sizes

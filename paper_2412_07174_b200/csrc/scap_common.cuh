@@ -6,17 +6,13 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <type_traits>
+
 #include "scap.h"
 
 namespace scap {
 
-constexpr int CH = 256;            // channels per compaction chunk (= threads of a compaction CTA)
-constexpr int TN = 256;            // output columns per gather-GEMV CTA: 32 lanes x 8 columns (16 B)
-constexpr int GEMV_THREADS = 256;  // 8 warps; the warps of a CTA take rows round-robin
-constexpr int GEMV_WARPS = GEMV_THREADS / 32;
-constexpr int LB = 256;            // kept rows staged in shared memory per fill
-constexpr int MAX_SPLIT = 64;      // upper bound on the split-K factor
-constexpr int MAX_CHUNKS_SMEM = 512;  // chunk-count prefix held in shared memory: K <= 512 * CH = 131072
+constexpr int SCAP_MAX_K = 1 << 20;  // input channels per FC (keeps every index comfortably inside 32 bits)
 
 struct Tuning {
     int split_k;  // 0 = automatic

@@ -32,148 +32,143 @@ int sm_count() {
     if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
         n <= 0) {
         cudaGetLastError();
-        return 148;  // B200; used only so that workspace queries work on a machine without a GPU
+        return 148;  // B200; used only so that queries work on a machine without a GPU
     }
     cached = n;
     return n;
 }
 
-// Split-K factor: fill every SM with four resident CTAs in a single wave, but keep at least 32 rows
-// per slice at full density.
-int choose_split(int K, int tiles_total) {
-    if (g_tune.split_k > 0) return g_tune.split_k < MAX_SPLIT ? g_tune.split_k : MAX_SPLIT;
-    const int target = sm_count() * 4;
-    int S = (target + tiles_total / 2) / tiles_total;
-    const int by_rows = (K + 31) / 32;
-    if (S > by_rows) S = by_rows;
-    if (S > MAX_SPLIT) S = MAX_SPLIT;
-    if (S < 1) S = 1;
+// Largest power of two <= 8 that keeps the whole grid co-resident (about two CTAs per SM) and leaves
+// every slice at least 64 input channels.
+int choose_split(int K, int tiles, int groups) {
+    int S = MAX_CLUSTER;
+    if (g_tune.split_k > 0) {
+        while (S > g_tune.split_k) S >>= 1;
+        return S;
+    }
+    const int budget = 2 * sm_count();
+    while (S > 1 && ((long long)tiles * groups * S > budget || K / S < 64)) S >>= 1;
     return S;
 }
 
-FcLayout fc_layout(int B, int K, int N, int halves, size_t base) {
-    FcLayout L;
-    const int Nh = N / halves;
-    L.nchunks = (K + CH - 1) / CH;
-    L.Kpad = L.nchunks * CH;
-    L.tiles = halves * ((Nh + TN - 1) / TN);
-    L.S = choose_split(K, L.tiles);
-    size_t off = align_up(base, 256);
-    L.counts = off;
-    off = align_up(off + sizeof(int) * L.nchunks, 256);
-    L.tickets = off;
-    off = align_up(off + sizeof(int) * L.tiles, 256);
-    L.idx_local = off;
-    off = align_up(off + sizeof(uint32_t) * L.Kpad, 256);
-    L.xs_local = off;
-    off = align_up(off + sizeof(float) * (size_t)B * L.Kpad, 256);
-    L.partials = off;
-    off = align_up(off + sizeof(float) * (size_t)L.S * B * N, 256);
-    L.total = off;
-    return L;
-}
-
-void bind_layout(GemvArgs &a, const FcLayout &L, unsigned char *ws) {
-    a.S = L.S;
-    a.counts = reinterpret_cast<const int *>(ws + L.counts);
-    a.idx_local = reinterpret_cast<const uint32_t *>(ws + L.idx_local);
-    a.xs_local = reinterpret_cast<const float *>(ws + L.xs_local);
-    a.Kpad = L.Kpad;
-    a.nchunks = L.nchunks;
-    a.partials = reinterpret_cast<float *>(ws + L.partials);
-    a.tickets = reinterpret_cast<int *>(ws + L.tickets);
-}
-
-template <typename XT>
-cudaError_t launch_compact(const XT *x, const float *m, const float *tau, int B, int K, const FcLayout &L, unsigned char *ws,
-                           int ntickets, cudaStream_t st) {
-    return launch(compact_kernel<XT>, dim3(L.nchunks), dim3(CH), 0, st, g_tune.pdl != 0, x, m, tau, B, K,
-                  reinterpret_cast<int *>(ws + L.counts), reinterpret_cast<uint32_t *>(ws + L.idx_local),
-                  reinterpret_cast<float *>(ws + L.xs_local), L.Kpad, reinterpret_cast<int *>(ws + L.tickets), ntickets);
-}
-template cudaError_t launch_compact<__half>(const __half *, const float *, const float *, int, int, const FcLayout &,
-                                            unsigned char *, int, cudaStream_t);
-template cudaError_t launch_compact<__nv_bfloat16>(const __nv_bfloat16 *, const float *, const float *, int, int,
-                                                   const FcLayout &, unsigned char *, int, cudaStream_t);
-
 template <bool BF16, int BT, int MODE, typename XT, int EPI>
-static cudaError_t launch_gemv_t(const GemvArgs &a, cudaStream_t st) {
-    const int tiles = a.halves * ((a.Nh + TN - 1) / TN);
-    return launch(gemv_kernel<BF16, BT, MODE, XT, EPI>, dim3(tiles, a.S), dim3(GEMV_THREADS), 0, st, g_tune.pdl != 0, a);
+static cudaError_t launch_fc_t(const FcArgs &a, cudaStream_t st) {
+    static bool attr_done = false;
+    auto kern = fc_kernel<BF16, BT, MODE, XT, EPI>;
+    if (!attr_done) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, fc_smem_bytes(BT));
+        if (e != cudaSuccess) return e;
+        attr_done = true;
+    }
+    return launch_cluster(kern, dim3(fc_tiles(a.Nh, EPI), a.S), dim3(fc_threads(BT)), fc_smem_bytes(BT), a.S, st,
+                          g_tune.pdl != 0, a);
 }
 
 template <bool BF16, int MODE, typename XT, int EPI>
-static cudaError_t launch_gemv_bt(const GemvArgs &a, cudaStream_t st) {
+static cudaError_t launch_fc_bt(const FcArgs &a, cudaStream_t st) {
     switch (batch_tile(a.B)) {
-        case 1: return launch_gemv_t<BF16, 1, MODE, XT, EPI>(a, st);
-        case 2: return launch_gemv_t<BF16, 2, MODE, XT, EPI>(a, st);
-        case 4: return launch_gemv_t<BF16, 4, MODE, XT, EPI>(a, st);
-        case 8: return launch_gemv_t<BF16, 8, MODE, XT, EPI>(a, st);
-        default: return launch_gemv_t<BF16, 16, MODE, XT, EPI>(a, st);
+        case 1: return launch_fc_t<BF16, 1, MODE, XT, EPI>(a, st);
+        case 2: return launch_fc_t<BF16, 2, MODE, XT, EPI>(a, st);
+        case 4: return launch_fc_t<BF16, 4, MODE, XT, EPI>(a, st);
+        case 8: return launch_fc_t<BF16, 8, MODE, XT, EPI>(a, st);
+        default: return launch_fc_t<BF16, 16, MODE, XT, EPI>(a, st);
     }
 }
 
-cudaError_t launch_gemv(bool bf16, int mode, int xkind, int epi, const GemvArgs &a, cudaStream_t st) {
-    if (mode == MODE_GATHER) {
-        if (epi == EPI_GLU)
-            return bf16 ? launch_gemv_bt<true, MODE_GATHER, float, EPI_GLU>(a, st)
-                        : launch_gemv_bt<false, MODE_GATHER, float, EPI_GLU>(a, st);
-        return bf16 ? launch_gemv_bt<true, MODE_GATHER, float, EPI_BIAS>(a, st)
-                    : launch_gemv_bt<false, MODE_GATHER, float, EPI_BIAS>(a, st);
+template <bool BF16>
+static cudaError_t launch_fc_w(int mode, int xkind, int epi, const FcArgs &a, cudaStream_t st) {
+    using ST = typename std::conditional<BF16, __nv_bfloat16, __half>::type;
+    if (mode == MODE_DENSE) {
+        if (xkind == 2) return launch_fc_t<BF16, 1, MODE_DENSE, float, EPI_BIAS>(a, st);  // bias folding: x = m, batch 1
+        return launch_fc_bt<BF16, MODE_DENSE, ST, EPI_BIAS>(a, st);
     }
-    if (xkind == 2)  // fp32 activation (the mode vector when folding the bias): batch 1 only
-        return bf16 ? launch_gemv_t<true, 1, MODE_DENSE, float, EPI_BIAS>(a, st)
-                    : launch_gemv_t<false, 1, MODE_DENSE, float, EPI_BIAS>(a, st);
-    return bf16 ? launch_gemv_bt<true, MODE_DENSE, __nv_bfloat16, EPI_BIAS>(a, st)
-                : launch_gemv_bt<false, MODE_DENSE, __half, EPI_BIAS>(a, st);
+    if (epi == EPI_GLU) return launch_fc_bt<BF16, MODE_GATHER, ST, EPI_GLU>(a, st);
+    if (xkind == 2) return launch_fc_bt<BF16, MODE_GATHER, float, EPI_BIAS>(a, st);  // down projection reading fp32 z
+    return launch_fc_bt<BF16, MODE_GATHER, ST, EPI_BIAS>(a, st);
+}
+
+cudaError_t launch_fc(bool bf16, int mode, int xkind, int epi, const FcArgs &a, cudaStream_t st) {
+    return bf16 ? launch_fc_w<true>(mode, xkind, epi, a, st) : launch_fc_w<false>(mode, xkind, epi, a, st);
+}
+
+// One CTA of 1024 threads: popcount prefix over the mask words, then every word's thread writes its set bits.
+__global__ void __launch_bounds__(1024) expand_bits_kernel(const uint32_t *__restrict__ bits, int K,
+                                                          uint32_t *__restrict__ idx_out, int *__restrict__ nnz_out) {
+    __shared__ int s_warp[32];
+    __shared__ int s_carry;
+    griddep_wait();
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int nwords = (K + 31) >> 5;
+    if (tid == 0) s_carry = 0;
+    __syncthreads();
+    for (int w0 = 0; w0 < nwords; w0 += 1024) {
+        const int w = w0 + tid;
+        const uint32_t word = w < nwords ? bits[w] : 0u;
+        const int c = __popc(word);
+        int v = c;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int t = __shfl_up_sync(0xffffffffu, v, o);
+            if (lane >= o) v += t;
+        }
+        if (lane == 31) s_warp[warp] = v;
+        __syncthreads();
+        int base = s_carry;
+        for (int q = 0; q < warp; ++q) base += s_warp[q];
+        int pos = base + v - c;
+        if (idx_out) {
+            uint32_t rem = word;
+            while (rem) {
+                const int bit = __ffs(rem) - 1;
+                rem &= rem - 1;
+                idx_out[pos++] = (uint32_t)(w * 32 + bit);
+            }
+        }
+        __syncthreads();
+        if (tid == 1023) s_carry = base + v;
+        __syncthreads();
+    }
+    if (tid == 0 && nnz_out) *nnz_out = s_carry;
+}
+
+cudaError_t launch_expand_bits(const uint32_t *bits, int K, uint32_t *idx_out, int *nnz_out, cudaStream_t st) {
+    return launch(expand_bits_kernel, dim3(1), dim3(1024), 0, st, false, bits, K, idx_out, nnz_out);
 }
 
 static scap_status validate_fc(const void *x, const void *W, const float *y, int B, int K, int N, int dt) {
     if (!x || !W || !y) return SCAP_ERR_INVALID_ARG;
     if (dt != SCAP_F16 && dt != SCAP_BF16) return SCAP_ERR_DTYPE;
-    if (B < 1 || B > SCAP_MAX_BATCH || K < 1 || N < 1 || K > MAX_CHUNKS_SMEM * CH) return SCAP_ERR_SHAPE;
+    if (B < 1 || B > SCAP_MAX_BATCH || K < 1 || N < 1 || K > SCAP_MAX_K) return SCAP_ERR_SHAPE;
     if (N % 8 != 0 || !aligned16(x) || !aligned16(W) || !aligned16(y)) return SCAP_ERR_ALIGN;
     return SCAP_OK;
 }
 
+static size_t bits_bytes(int K) { return align_up(sizeof(uint32_t) * ((K + 31) / 32), 256); }
+
 static scap_status sparse_fc_impl(const void *x, const void *W, const float *m, const float *tau, const float *b_fused,
                                   float *y, int B, int K, int N, scap_dtype dt, uint32_t *idx_out, int *nnz_out,
                                   unsigned char *ws, cudaStream_t st) {
-    const FcLayout L = fc_layout(B, K, N, 1, 0);
-    cudaError_t e = dt == SCAP_BF16
-                        ? launch_compact(reinterpret_cast<const __nv_bfloat16 *>(x), m, tau, B, K, L, ws, L.tiles, st)
-                        : launch_compact(reinterpret_cast<const __half *>(x), m, tau, B, K, L, ws, L.tiles, st);
-    if (e != cudaSuccess) return cuda_status(e);
-    GemvArgs a;
+    FcArgs a;
     memset(&a, 0, sizeof(a));
-    a.W = W; a.K = K; a.ldw = N; a.halves = 1; a.Nh = N; a.B = B;
-    bind_layout(a, L, ws);
-    a.bias = b_fused; a.y = y; a.idx_out = idx_out; a.nnz_out = nnz_out;
-    return cuda_status(launch_gemv(dt == SCAP_BF16, MODE_GATHER, 0, EPI_BIAS, a, st));
-}
-
-// The tickets of a dense call are cleared by a one-CTA kernel (the sparse path clears them in its compaction).
-__global__ void clear_tickets_kernel(int *tickets, int n) {
-    griddep_wait();
-    griddep_launch_dependents();
-    for (int i = threadIdx.x; i < n; i += blockDim.x) tickets[i] = 0;
+    a.W = W; a.K = K; a.ldw = N; a.Nh = N; a.B = B;
+    a.S = choose_split(K, fc_tiles(N, EPI_BIAS), 1);
+    a.x = x; a.x_ld = K; a.m = m; a.tau = tau; a.bias = b_fused; a.y = y; a.y_ld = N;
+    const bool inspect = idx_out || nnz_out;
+    if (inspect) a.bits = reinterpret_cast<uint32_t *>(ws);
+    cudaError_t e = launch_fc(dt == SCAP_BF16, MODE_GATHER, dt == SCAP_BF16 ? 1 : 0, EPI_BIAS, a, st);
+    if (e != cudaSuccess) return cuda_status(e);
+    if (inspect) e = launch_expand_bits(a.bits, K, idx_out, nnz_out, st);
+    return cuda_status(e);
 }
 
 static scap_status dense_impl(const void *x, int xkind, const void *W, const float *b, const void *b16, float *y, int B,
-                              int K, int N, scap_dtype dt, unsigned char *ws, cudaStream_t st) {
-    const FcLayout L = fc_layout(B, K, N, 1, 0);
-    if (L.S > 1) {
-        cudaError_t e = launch(clear_tickets_kernel, dim3(1), dim3(256), 0, st, g_tune.pdl != 0,
-                               reinterpret_cast<int *>(ws + L.tickets), L.tiles);
-        if (e != cudaSuccess) return cuda_status(e);
-    }
-    GemvArgs a;
+                              int K, int N, scap_dtype dt, cudaStream_t st) {
+    FcArgs a;
     memset(&a, 0, sizeof(a));
-    a.W = W; a.K = K; a.ldw = N; a.halves = 1; a.Nh = N; a.B = B;
-    bind_layout(a, L, ws);
-    a.x = x;
-    a.bias = b; a.bias16 = b16; a.y = y;
-    return cuda_status(launch_gemv(dt == SCAP_BF16, MODE_DENSE, xkind, EPI_BIAS, a, st));
+    a.W = W; a.K = K; a.ldw = N; a.Nh = N; a.B = B;
+    a.S = choose_split(K, fc_tiles(N, EPI_BIAS), 1);
+    a.x = x; a.x_ld = K; a.bias = b; a.bias16 = b16; a.y = y; a.y_ld = N;
+    return cuda_status(launch_fc(dt == SCAP_BF16, MODE_DENSE, xkind, EPI_BIAS, a, st));
 }
 
 }  // namespace scap
@@ -197,12 +192,12 @@ const char *scap_status_string(scap_status st) {
     return "SCAP_ERR_UNKNOWN";
 }
 
-int scap_version(void) { return 1000; }
+int scap_version(void) { return 1001; }
 
 scap_status scap_tune(const char *key, int value) {
     if (!key) return SCAP_ERR_INVALID_ARG;
     if (!strcmp(key, "split_k")) {
-        if (value < 0 || value > MAX_SPLIT) return SCAP_ERR_INVALID_ARG;
+        if (value < 0 || value > MAX_CLUSTER) return SCAP_ERR_INVALID_ARG;
         g_tune.split_k = value;
         return SCAP_OK;
     }
@@ -214,8 +209,8 @@ scap_status scap_tune(const char *key, int value) {
 }
 
 size_t scap_fc_workspace(int B, int K, int N) {
-    if (B < 1 || B > SCAP_MAX_BATCH || K < 1 || N < 1 || K > MAX_CHUNKS_SMEM * CH) return 0;
-    return fc_layout(B, K, N, 1, 0).total;
+    if (B < 1 || B > SCAP_MAX_BATCH || K < 1 || N < 1 || K > SCAP_MAX_K) return 0;
+    return bits_bytes(K);
 }
 
 scap_status scap_sparse_fc(const void *x, const void *W, const float *m, const float *tau, const float *b_fused, float *y,
@@ -239,8 +234,7 @@ scap_status scap_dense_fc(const void *x, const void *W, const float *b, float *y
     if (!aligned16(ws) || (b && !aligned16(b))) return SCAP_ERR_ALIGN;
     if (ws_bytes < scap_fc_workspace(B, K, N)) return SCAP_ERR_WORKSPACE;
     if ((st = check_device()) != SCAP_OK) return st;
-    return dense_impl(x, dt == SCAP_BF16 ? 1 : 0, W, b, nullptr, y, B, K, N, dt, static_cast<unsigned char *>(ws),
-                      reinterpret_cast<cudaStream_t>(stream));
+    return dense_impl(x, dt == SCAP_BF16 ? 1 : 0, W, b, nullptr, y, B, K, N, dt, reinterpret_cast<cudaStream_t>(stream));
 }
 
 size_t scap_fold_bias_workspace(int K, int N) { return scap_fc_workspace(1, K, N); }
@@ -253,8 +247,7 @@ scap_status scap_fold_bias(const void *W, const float *m, const void *b, int K, 
     if (!aligned16(ws) || (b && !aligned16(b))) return SCAP_ERR_ALIGN;
     if (ws_bytes < scap_fold_bias_workspace(K, N)) return SCAP_ERR_WORKSPACE;
     if ((st = check_device()) != SCAP_OK) return st;
-    return dense_impl(m, 2, W, nullptr, b, b_fused, 1, K, N, dt, static_cast<unsigned char *>(ws),
-                      reinterpret_cast<cudaStream_t>(stream));
+    return dense_impl(m, 2, W, nullptr, b, b_fused, 1, K, N, dt, reinterpret_cast<cudaStream_t>(stream));
 }
 
 size_t scap_fc_host_workspace(int B, int K, int N) {
@@ -268,7 +261,7 @@ scap_status scap_sparse_fc_host(const void *x_host, const void *W, const float *
                                 scap_stream_t stream) {
     if (!x_host || !y_host || !W || !tau || !ws) return SCAP_ERR_INVALID_ARG;
     if (dt != SCAP_F16 && dt != SCAP_BF16) return SCAP_ERR_DTYPE;
-    if (B < 1 || B > SCAP_MAX_BATCH || K < 1 || N < 1 || K > MAX_CHUNKS_SMEM * CH) return SCAP_ERR_SHAPE;
+    if (B < 1 || B > SCAP_MAX_BATCH || K < 1 || N < 1 || K > SCAP_MAX_K) return SCAP_ERR_SHAPE;
     if (N % 8 != 0 || !aligned16(W) || !aligned16(ws) || (m && !aligned16(m)) || (b_fused && !aligned16(b_fused)))
         return SCAP_ERR_ALIGN;
     if (ws_bytes < scap_fc_host_workspace(B, K, N)) return SCAP_ERR_WORKSPACE;

@@ -1,48 +1,22 @@
-// SwiGLU FFN block (Alg. 2): compaction of h -> gather-GEMV over the packed gate|up weight whose
-// second pass also forms z = up * silu(gate) and compacts it -> gather-GEMV over the down weight.
+// SwiGLU FFN block (Alg. 2): one fused FC kernel over the packed gate|up weight whose cluster
+// reduction also forms z = up * silu(gate), then one fused FC kernel over the down weight that
+// thresholds z itself.  z (fp32, B x F) is the only intermediate and stays L2-resident.
 #include <string.h>
 
 #include "scap_fc.cuh"
 
 namespace scap {
 
-// One CTA: prefix over the chunk counts, then every chunk's local list is copied to its global offset.
-__global__ void expand_idx_kernel(const int *__restrict__ counts, const uint32_t *__restrict__ idx_local, int nchunks,
-                                  uint32_t *__restrict__ idx_out, int *__restrict__ nnz_out) {
-    __shared__ int s_prefix[MAX_CHUNKS_SMEM + 1];
-    griddep_wait();
-    if (threadIdx.x == 0) {
-        int acc = 0;
-        for (int c = 0; c < nchunks; ++c) {
-            s_prefix[c] = acc;
-            acc += counts[c];
-        }
-        s_prefix[nchunks] = acc;
-        if (nnz_out) *nnz_out = acc;
-    }
-    __syncthreads();
-    if (!idx_out) return;
-    for (int c = 0; c < nchunks; ++c) {
-        const int n = s_prefix[c + 1] - s_prefix[c];
-        for (int j = threadIdx.x; j < n; j += blockDim.x) idx_out[s_prefix[c] + j] = idx_local[(size_t)c * CH + j];
-    }
-}
-
-cudaError_t launch_expand_idx(const int *counts, const uint32_t *idx_local, int nchunks, uint32_t *idx_out, int *nnz_out,
-                              cudaStream_t st) {
-    return launch(expand_idx_kernel, dim3(1), dim3(256), 0, st, false, counts, idx_local, nchunks, idx_out, nnz_out);
-}
-
 struct GluLayout {
-    FcLayout s1, s2;  // stage 1: K = D, N = 2F (two halves); stage 2: K = F, N = D
-    size_t total;
+    size_t bits1, z, bits2, total;
 };
 
 static GluLayout glu_layout(int B, int D, int F) {
     GluLayout G;
-    G.s1 = fc_layout(B, D, 2 * F, 2, 0);
-    G.s2 = fc_layout(B, F, D, 1, G.s1.total);
-    G.total = G.s2.total;
+    G.bits1 = 0;
+    G.z = align_up(sizeof(uint32_t) * ((D + 31) / 32), 256);
+    G.bits2 = G.z + align_up(sizeof(float) * (size_t)B * F, 256);
+    G.total = G.bits2 + align_up(sizeof(uint32_t) * ((F + 31) / 32), 256);
     return G;
 }
 
@@ -53,7 +27,7 @@ using namespace scap;
 extern "C" {
 
 size_t scap_glu_workspace(int B, int D, int F) {
-    if (B < 1 || B > SCAP_MAX_BATCH || D < 1 || F < 1 || D > MAX_CHUNKS_SMEM * CH || F > MAX_CHUNKS_SMEM * CH) return 0;
+    if (B < 1 || B > SCAP_MAX_BATCH || D < 1 || F < 1 || D > SCAP_MAX_K || F > SCAP_MAX_K) return 0;
     return glu_layout(B, D, F).total;
 }
 
@@ -63,8 +37,7 @@ scap_status scap_glu_ffn(const void *h, const void *Wgu, const void *Wd, const f
                          int *nnz2_out, void *ws, size_t ws_bytes, scap_stream_t stream) {
     if (!h || !Wgu || !Wd || !tau1 || !tau2 || !y || !ws) return SCAP_ERR_INVALID_ARG;
     if (dt != SCAP_F16 && dt != SCAP_BF16) return SCAP_ERR_DTYPE;
-    if (B < 1 || B > SCAP_MAX_BATCH || D < 1 || F < 1 || D > MAX_CHUNKS_SMEM * CH || F > MAX_CHUNKS_SMEM * CH)
-        return SCAP_ERR_SHAPE;
+    if (B < 1 || B > SCAP_MAX_BATCH || D < 1 || F < 1 || D > SCAP_MAX_K || F > SCAP_MAX_K) return SCAP_ERR_SHAPE;
     if (D % 8 != 0 || F % 8 != 0 || !aligned16(h) || !aligned16(Wgu) || !aligned16(Wd) || !aligned16(y) || !aligned16(ws) ||
         (m1 && !aligned16(m1)) || (m2 && !aligned16(m2)) || (bgu_fused && !aligned16(bgu_fused)) ||
         (bd_fused && !aligned16(bd_fused)) || (z_out && !aligned16(z_out)))
@@ -77,43 +50,36 @@ scap_status scap_glu_ffn(const void *h, const void *Wgu, const void *Wd, const f
     unsigned char *w = static_cast<unsigned char *>(ws);
     const GluLayout G = glu_layout(B, D, F);
     const bool bf16 = dt == SCAP_BF16;
+    float *z = reinterpret_cast<float *>(w + G.z);
 
-    // stage 1: centre + threshold h; the tickets cleared are the per-pair tickets (tiles / 2)
-    cudaError_t e = bf16 ? launch_compact(reinterpret_cast<const __nv_bfloat16 *>(h), m1, tau1, B, D, G.s1, w, G.s1.tiles, st)
-                         : launch_compact(reinterpret_cast<const __half *>(h), m1, tau1, B, D, G.s1, w, G.s1.tiles, st);
-    if (e != cudaSuccess) return cuda_status(e);
-
-    GemvArgs a;
+    FcArgs a;
     memset(&a, 0, sizeof(a));
-    a.W = Wgu; a.K = D; a.ldw = 2 * F; a.halves = 2; a.Nh = F; a.B = B;
-    bind_layout(a, G.s1, w);
-    a.bias = bgu_fused;
-    a.m2 = m2; a.tau2 = tau2; a.z_out = z_out;
-    a.counts2 = reinterpret_cast<int *>(w + G.s2.counts);
-    a.idx_local2 = reinterpret_cast<uint32_t *>(w + G.s2.idx_local);
-    a.xs_local2 = reinterpret_cast<float *>(w + G.s2.xs_local);
-    a.Kpad2 = G.s2.Kpad;
-    a.tickets_next = reinterpret_cast<int *>(w + G.s2.tickets);
-    a.ntickets_next = G.s2.tiles;
-    e = launch_gemv(bf16, MODE_GATHER, 0, EPI_GLU, a, st);
+    a.W = Wgu; a.K = D; a.ldw = 2 * F; a.Nh = F; a.B = B;
+    a.S = choose_split(D, fc_tiles(F, EPI_GLU), 1);
+    a.x = h; a.x_ld = D; a.m = m1; a.tau = tau1; a.bias = bgu_fused;
+    a.y = z; a.y_ld = F; a.z_copy = z_out;
+    if (idx1_out || nnz1_out) a.bits = reinterpret_cast<uint32_t *>(w + G.bits1);
+    cudaError_t e = launch_fc(bf16, MODE_GATHER, bf16 ? 1 : 0, EPI_GLU, a, st);
     if (e != cudaSuccess) return cuda_status(e);
 
-    GemvArgs d;
+    FcArgs d;
     memset(&d, 0, sizeof(d));
-    d.W = Wd; d.K = F; d.ldw = D; d.halves = 1; d.Nh = D; d.B = B;
-    bind_layout(d, G.s2, w);
-    d.bias = bd_fused; d.y = y; d.idx_out = idx2_out; d.nnz_out = nnz2_out;
-    e = launch_gemv(bf16, MODE_GATHER, 0, EPI_BIAS, d, st);
+    d.W = Wd; d.K = F; d.ldw = D; d.Nh = D; d.B = B;
+    d.S = choose_split(F, fc_tiles(D, EPI_BIAS), 1);
+    d.x = z; d.x_ld = F; d.m = m2; d.tau = tau2; d.bias = bd_fused; d.y = y; d.y_ld = D;
+    if (idx2_out || nnz2_out) d.bits = reinterpret_cast<uint32_t *>(w + G.bits2);
+    e = launch_fc(bf16, MODE_GATHER, 2, EPI_BIAS, d, st);
     if (e != cudaSuccess) return cuda_status(e);
 
-    if (idx1_out || nnz1_out) {
-        // inspection only: expand the stage-1 chunk-local lists into the global ascending list
-        e = launch_expand_idx(reinterpret_cast<const int *>(w + G.s1.counts), reinterpret_cast<const uint32_t *>(w + G.s1.idx_local),
-                              G.s1.nchunks, idx1_out, nnz1_out, st);
+    if (a.bits) {
+        e = launch_expand_bits(a.bits, D, idx1_out, nnz1_out, st);
+        if (e != cudaSuccess) return cuda_status(e);
+    }
+    if (d.bits) {
+        e = launch_expand_bits(d.bits, F, idx2_out, nnz2_out, st);
         if (e != cudaSuccess) return cuda_status(e);
     }
     return SCAP_OK;
 }
 
 }  // extern "C"
-

@@ -40,7 +40,7 @@ def test_status_strings_and_version(L):
 
 def test_workspace_queries_without_a_device(L):
     assert L.scap_fc_workspace(1, 11008, 4096) > 0
-    assert L.scap_fc_workspace(16, 14336, 4096) > L.scap_fc_workspace(1, 14336, 4096)
+    assert L.scap_glu_workspace(16, 4096, 14336) > L.scap_glu_workspace(1, 4096, 14336)
     assert L.scap_fc_workspace(17, 64, 64) == 0 and L.scap_fc_workspace(1, 0, 64) == 0
     assert L.scap_glu_workspace(8, 4096, 11008) > 0
     assert L.scap_moe_workspace(4, 4096, 14336, 8, 2) > 0
@@ -62,7 +62,7 @@ def test_argument_validation_returns_codes(L):
     assert call(N=60) == 4 and call(W=P + 2) == 4  # SCAP_ERR_ALIGN
     assert call(wsb=ws - 1) == 5                  # SCAP_ERR_WORKSPACE
     assert L.scap_tune(b"no_such_key", 1) == 1
-    assert L.scap_tune(b"split_k", 1000) == 1
+    assert L.scap_tune(b"split_k", 9) == 1
     assert L.scap_tune(b"split_k", 0) == 0
     assert L.scap_calibrate(P, 16, 12, 1, 0.5, 16, P, P, P, 1 << 20, None) == 4   # K not a multiple of 8
     assert L.scap_calibrate(P, 16, 16, 1, 1.5, 16, P, P, P, 1 << 20, None) == 1   # sparsity outside [0, 1)

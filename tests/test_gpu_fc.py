@@ -147,7 +147,7 @@ def test_bitwise_determinism_and_row_independence(S):
         assert rel_l2_rows(y1[b:b + 1], y64) <= REL_L2_TOL
 
 
-@pytest.mark.parametrize("split", [1, 2, 7, 64])
+@pytest.mark.parametrize("split", [1, 2, 3, 8])
 def test_any_split_k_gives_the_same_answer(S, split):
     d = si.laplace_fc(4, 1500, 520, si.BF16, 16, 3)
     try:
