@@ -60,7 +60,7 @@ static cudaError_t launch_fc_t(const FcArgs &a, cudaStream_t st) {
         if (e != cudaSuccess) return e;
         attr_done = true;
     }
-    return launch_cluster(kern, dim3(fc_tiles(a.Nh, EPI), a.S), dim3(fc_threads(BT)), fc_smem_bytes(BT), a.S, st,
+    return launch_cluster(kern, dim3(fc_tiles(a.Nh, EPI), a.S), dim3(FC_THREADS), fc_smem_bytes(BT), a.S, st,
                           g_tune.pdl != 0, a);
 }
 

@@ -1,11 +1,11 @@
 // The fused decode-time sparse FC kernel (Eq. 2-3, Eq. 6, Alg. 3).
 //
 // One kernel does centre + threshold + compaction + gather-GEMV + reduction:
-//   grid  = (column tiles, S)   block = 512 threads (256 when 16 batch rows are tiled)
+//   grid  = (column tiles, S)   block = 256 threads
 //   the S CTAs of a column tile form one thread-block cluster; CTA s owns the 32-channel chunks
 //   c = s, s+S, s+2S, ... of the input, thresholds them itself (ballot + popcount, order kept),
 //   streams the surviving weight rows of its tile with 16-byte loads kept U deep per thread, and
-//   the cluster sums its S partial tiles through distributed shared memory in rank order.
+//   the cluster exchanges its S partial tiles through distributed shared memory and adds them in rank order.
 // No global scratch, no atomics, no second kernel; the summation order is fixed, so results are
 // bitwise reproducible.  Internal header shared by the FC, SwiGLU and MoE entry points.
 #pragma once
@@ -24,18 +24,21 @@ enum { EPI_BIAS = 0, EPI_GLU = 1 };
 constexpr int TN = 256;         // columns per CTA: 32 lanes x 8 columns (one 16-byte load per lane and row)
 constexpr int MAX_CLUSTER = 8;  // portable cluster size: upper bound of the split-K factor S
 
-__host__ __device__ constexpr int fc_threads(int BT) { return BT <= 8 ? 512 : 256; }
-__host__ __device__ constexpr int fc_min_blocks(int BT) { return BT <= 2 ? 2 : 1; }
-__host__ __device__ constexpr int fc_cap(int BT) { return BT <= 2 ? 4096 : BT <= 4 ? 2048 : 1024; }  // channels staged per fill
-__host__ __device__ constexpr int fc_rb(int BT) { return BT < 4 ? BT : 4; }                          // batch rows per cross-warp round
-__host__ __device__ constexpr int fc_unroll(int BT) { return BT <= 2 ? 8 : 4; }                      // row loads in flight per thread
+constexpr int FC_THREADS = 256;  // 8 warps; two CTAs fit on an SM, so every cluster of the grid is resident at once
+constexpr int FC_WARPS = FC_THREADS / 32;
+__host__ __device__ constexpr int fc_min_blocks(int BT) { return BT <= 8 ? 2 : 1; }
+// chunks (of 32 channels) each warp thresholds per fill; their centred values stay in registers
+__host__ __device__ constexpr int fc_pu(int BT) { return BT <= 2 ? 8 : BT <= 4 ? 4 : BT <= 8 ? 2 : 1; }
+__host__ __device__ constexpr int fc_cap(int BT) { return FC_WARPS * fc_pu(BT) * 32; }  // channels staged per fill
+__host__ __device__ constexpr int fc_rb(int BT) { return BT < 4 ? BT : 4; }              // batch rows per cross-warp round
+__host__ __device__ constexpr int fc_unroll(int BT) { return BT <= 1 ? 16 : BT <= 4 ? 8 : 4; }  // row loads in flight per thread
 
 __host__ __device__ constexpr int fc_main_bytes(int BT) {
     const int stage = fc_cap(BT) * 4 * (1 + BT);
-    const int red = (fc_threads(BT) / 32) * fc_rb(BT) * TN * 4;
+    const int red = FC_WARPS * fc_rb(BT) * TN * 4;
     return stage > red ? stage : red;
 }
-__host__ __device__ constexpr int fc_smem_bytes(int BT) {  // main | partial tile | chunk masks | chunk offsets
+__host__ __device__ constexpr int fc_smem_bytes(int BT) {  // main | gathered partials | chunk masks | chunk offsets
     return fc_main_bytes(BT) + BT * TN * 4 + (fc_cap(BT) / 32) * 4 + (fc_cap(BT) / 32 + 1) * 4 + 16;
 }
 
@@ -57,26 +60,6 @@ struct FcArgs {
     float *z_copy;        // EPI_GLU: optional second copy of z, [B, F] dense rows
     uint32_t *bits;       // optional [ceil(K/32)]: union keep mask, one word per 32-channel chunk
 };
-
-// Centre + threshold of one channel for every batch row (Alg. 3): one binary32 subtraction, one compare.
-template <typename XT>
-__device__ __forceinline__ uint32_t centre_threshold(const FcArgs &a, float tau, int k, float (&d)[SCAP_MAX_BATCH]) {
-    uint32_t keepmask = 0;
-    const float mk = a.m ? __ldg(a.m + k) : 0.0f;
-    const XT *x = reinterpret_cast<const XT *>(a.x);
-#pragma unroll
-    for (int b = 0; b < SCAP_MAX_BATCH; ++b) {
-        d[b] = 0.0f;
-        if (b < a.B) {
-            const int row = a.in_rows ? a.in_rows[b] : b;
-            const float xv = widen1(x[(size_t)row * a.x_ld + k]);
-            const float dv = a.m ? __fsub_rn(xv, mk) : xv;
-            d[b] = dv;
-            if (fabsf(dv) >= tau) keepmask |= 1u << b;
-        }
-    }
-    return keepmask;
-}
 
 template <bool BF16, int BT, int CAP>
 __device__ __forceinline__ void fma_row(float (&acc)[BT][8], const uint4 &v, const float *__restrict__ s_xs, int i) {
@@ -103,18 +86,19 @@ __device__ __forceinline__ float load_bias(const FcArgs &a, int n) {
 // Body for column tile `tile` and cluster rank `s`; every thread of every CTA of the cluster calls it.
 template <bool BF16, int BT, int MODE, typename XT, int EPI>
 __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const int s) {
-    constexpr int NT = fc_threads(BT), NW = NT / 32, CAP = fc_cap(BT), RB = fc_rb(BT), U = fc_unroll(BT);
+    constexpr int NT = FC_THREADS, NW = FC_WARPS, PU = fc_pu(BT), CAP = fc_cap(BT), RB = fc_rb(BT), U = fc_unroll(BT);
     constexpr int CAPC = CAP / 32;  // chunks per fill
     extern __shared__ __align__(16) unsigned char smem[];
     uint32_t *s_k = reinterpret_cast<uint32_t *>(smem);
     float *s_xs = reinterpret_cast<float *>(smem) + CAP;
     float *s_red = reinterpret_cast<float *>(smem);
-    float *s_part = reinterpret_cast<float *>(smem + fc_main_bytes(BT));
-    uint32_t *s_bits = reinterpret_cast<uint32_t *>(s_part + BT * TN);
+    float *s_gather = reinterpret_cast<float *>(smem + fc_main_bytes(BT));  // [S][BT][columns owned by this rank]
+    uint32_t *s_bits = reinterpret_cast<uint32_t *>(s_gather + BT * TN);
     int *s_off = reinterpret_cast<int *>(s_bits + CAPC);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int B = a.B, S = a.S, K = a.K;
+    const XT *xg = reinterpret_cast<const XT *>(a.x);
 
     // this lane's 8 columns
     int col;
@@ -130,6 +114,25 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
     const unsigned char *Wb = reinterpret_cast<const unsigned char *>(a.W) + (size_t)col * 2;
     const size_t row_bytes = (size_t)a.ldw * 2;
 
+    // Columns this rank finishes after the cluster exchange, and their bias, fetched now so that the
+    // load is off the critical path.  EPI_BIAS: `per` columns; EPI_GLU: `per` gate/up pairs.
+    const int per = (EPI == EPI_GLU ? TN / 2 : TN) / S;
+    float bias0[2] = {0.0f, 0.0f}, bias1[2] = {0.0f, 0.0f};
+#pragma unroll
+    for (int it = 0; it < 2; ++it) {
+        const int i = tid + it * NT;
+        if (i < per * B) {
+            const int cl = i % per;
+            if constexpr (EPI == EPI_GLU) {
+                const int f = tile * (TN / 2) + s * per + cl;
+                if (f < a.Nh && a.bias) { bias0[it] = __ldg(a.bias + f); bias1[it] = __ldg(a.bias + a.Nh + f); }
+            } else {
+                const int n = tile * TN + s * per + cl;
+                if (n < a.Nh) bias0[it] = load_bias<BF16>(a, n);
+            }
+        }
+    }
+
     float acc[BT][8];
 #pragma unroll
     for (int b = 0; b < BT; ++b)
@@ -143,94 +146,117 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
 
     for (int j0 = 0; j0 < my_chunks; j0 += CAPC) {
         const int nj = min(CAPC, my_chunks - j0);
-        int cnt;
-        if constexpr (MODE == MODE_GATHER) {
-            // ---- A: keep mask of each chunk (one ballot word), recorded for the prefix sum
-            for (int j = warp; j < nj; j += NW) {
-                const int c = s + S * (j0 + j), k = c * 32 + lane;
-                float d[SCAP_MAX_BATCH];
-                const uint32_t km = k < K ? centre_threshold<XT>(a, tau, k, d) : 0u;
-                const unsigned bal = __ballot_sync(0xffffffffu, km != 0);
-                if (lane == 0) {
-                    s_bits[j] = bal;
-                    if (a.bits && tile == 0) a.bits[c] = bal;
-                }
-            }
-            __syncthreads();
-            // ---- exclusive prefix of the chunk counts (warp 0)
-            if (warp == 0) {
-                int carry = 0;
-                for (int c0 = 0; c0 < nj; c0 += 32) {
-                    const int v0 = (c0 + lane < nj) ? __popc(s_bits[c0 + lane]) : 0;
-                    int v = v0;
+        // ---- A: every warp loads PU chunks at once (all loads issued before any use), centres and thresholds them
+        // (Alg. 3: one binary32 subtraction, one compare per element) and keeps the values in registers.
+        float xv[PU][BT], mk[PU];
 #pragma unroll
-                    for (int o = 1; o < 32; o <<= 1) {
-                        const int t = __shfl_up_sync(0xffffffffu, v, o);
-                        if (lane >= o) v += t;
-                    }
-                    if (c0 + lane < nj) s_off[c0 + lane] = carry + v - v0;
-                    carry += __shfl_sync(0xffffffffu, v, 31);
-                }
-                if (lane == 0) s_off[nj] = carry;
-            }
-            __syncthreads();
-            cnt = s_off[nj];
-            // ---- B: write the kept channels and their pruned values, ascending
-            for (int j = warp; j < nj; j += NW) {
-                const unsigned bal = s_bits[j];
-                if (bal == 0) continue;
-                const int c = s + S * (j0 + j), k = c * 32 + lane;
-                float d[SCAP_MAX_BATCH];
-                const uint32_t km = k < K ? centre_threshold<XT>(a, tau, k, d) : 0u;
-                if (km) {
-                    const int pos = s_off[j] + __popc(bal & ((1u << lane) - 1u));
-                    s_k[pos] = (uint32_t)k;
+        for (int p = 0; p < PU; ++p) {
+            const int j = warp * PU + p;
+            const int k = (s + S * (j0 + j)) * 32 + lane;
+            const bool ok = j < nj && k < K;
+            mk[p] = (ok && a.m) ? __ldg(a.m + k) : 0.0f;
 #pragma unroll
-                    for (int b = 0; b < BT; ++b) s_xs[b * CAP + pos] = ((km >> b) & 1u) ? d[b] : 0.0f;
-                }
+            for (int b = 0; b < BT; ++b) {
+                xv[p][b] = 0.0f;
+                if (ok && b < B) xv[p][b] = widen1(xg[(size_t)(a.in_rows ? a.in_rows[b] : b) * a.x_ld + k]);
             }
-        } else {
-            // dense: every channel of the slice, no compare
-            const XT *x = reinterpret_cast<const XT *>(a.x);
-            for (int j = warp; j < nj; j += NW) {
-                const int c = s + S * (j0 + j), k = c * 32 + lane;
-                const int pos = j * 32 + lane;
-                s_k[pos] = (uint32_t)min(k, K - 1);
+        }
+        uint32_t km[PU];
+        unsigned bal[PU];
 #pragma unroll
-                for (int b = 0; b < BT; ++b) {
-                    float v = 0.0f;
-                    if (b < B && k < K) v = widen1(x[(size_t)(a.in_rows ? a.in_rows[b] : b) * a.x_ld + k]);
-                    s_xs[b * CAP + pos] = v;
+        for (int p = 0; p < PU; ++p) {
+            const int j = warp * PU + p;
+            const int c = s + S * (j0 + j), k = c * 32 + lane;
+            const bool ok = j < nj && k < K;
+            km[p] = 0;
+#pragma unroll
+            for (int b = 0; b < BT; ++b) {
+                if constexpr (MODE == MODE_GATHER) {
+                    const float dv = a.m ? __fsub_rn(xv[p][b], mk[p]) : xv[p][b];
+                    xv[p][b] = dv;
+                    if (ok && b < B && fabsf(dv) >= tau) km[p] |= 1u << b;
+                } else {
+                    if (ok) km[p] = 1u;  // dense: every channel, no compare
                 }
             }
-            // only the globally last chunk can be partial, and it is the last one of its slice
-            cnt = nj * 32 - ((s + S * (j0 + nj - 1) == nchunks - 1) ? nchunks * 32 - K : 0);
+            bal[p] = __ballot_sync(0xffffffffu, km[p] != 0);
+            if (lane == 0 && j < nj) {
+                s_bits[j] = bal[p];
+                if (MODE == MODE_GATHER && a.bits && tile == 0) a.bits[c] = bal[p];
+            }
+        }
+        __syncthreads();
+        // ---- exclusive prefix of the chunk counts (warp 0)
+        if (warp == 0) {
+            int carry = 0;
+#pragma unroll
+            for (int c0 = 0; c0 < CAPC; c0 += 32) {
+                const int v0 = (c0 + lane < nj) ? __popc(s_bits[c0 + lane]) : 0;
+                int v = v0;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const int t = __shfl_up_sync(0xffffffffu, v, o);
+                    if (lane >= o) v += t;
+                }
+                if (c0 + lane < nj) s_off[c0 + lane] = carry + v - v0;
+                carry += __shfl_sync(0xffffffffu, v, 31);
+            }
+            if (lane == 0) s_off[nj] = carry;
+        }
+        __syncthreads();
+        const int cnt = s_off[nj];
+        // ---- B: kept channels and their pruned values, in ascending channel order
+#pragma unroll
+        for (int p = 0; p < PU; ++p) {
+            const int j = warp * PU + p;
+            if (km[p]) {
+                const int pos = s_off[j] + __popc(bal[p] & ((1u << lane) - 1u));
+                s_k[pos] = (uint32_t)((s + S * (j0 + j)) * 32 + lane);
+#pragma unroll
+                for (int b = 0; b < BT; ++b)
+                    s_xs[b * CAP + pos] = (MODE == MODE_DENSE || ((km[p] >> b) & 1u)) ? xv[p][b] : 0.0f;
+            }
         }
         __syncthreads();
 
-        // ---- stream the kept rows: warp w takes rows w, w+NW, ...; U loads stay in flight per thread
+        // ---- stream the kept rows: warp w takes rows w, w+NW, ...  Two register groups of G loads alternate
+        // (one is consumed while the other is in flight).
         if (col_ok) {
+            constexpr int G = U / 2;
             const int nrows = cnt > warp ? (cnt - warp + NW - 1) / NW : 0;
-            uint4 buf[U];
+            uint4 ga[G], gb[G];
 #pragma unroll
-            for (int u = 0; u < U; ++u)
-                if (u < nrows) buf[u] = ld_stream16(Wb + (size_t)s_k[warp + NW * u] * row_bytes);
-            for (int t0 = 0; t0 < nrows; t0 += U) {
+            for (int u = 0; u < G; ++u)
+                if (u < nrows) ga[u] = ld_stream16(Wb + (size_t)s_k[warp + NW * u] * row_bytes);
 #pragma unroll
-                for (int u = 0; u < U; ++u) {
-                    const int t = t0 + u;
-                    if (t < nrows) {
-                        const uint4 v = buf[u];
-                        if (t + U < nrows) buf[u] = ld_stream16(Wb + (size_t)s_k[warp + NW * (t + U)] * row_bytes);
-                        fma_row<BF16, BT, CAP>(acc, v, s_xs, warp + NW * t);
-                    }
-                }
+            for (int u = 0; u < G; ++u)
+                if (G + u < nrows) gb[u] = ld_stream16(Wb + (size_t)s_k[warp + NW * (G + u)] * row_bytes);
+            for (int t0 = 0; t0 < nrows; t0 += 2 * G) {
+#pragma unroll
+                for (int u = 0; u < G; ++u)
+                    if (t0 + u < nrows) fma_row<BF16, BT, CAP>(acc, ga[u], s_xs, warp + NW * (t0 + u));
+#pragma unroll
+                for (int u = 0; u < G; ++u)
+                    if (t0 + 2 * G + u < nrows) ga[u] = ld_stream16(Wb + (size_t)s_k[warp + NW * (t0 + 2 * G + u)] * row_bytes);
+#pragma unroll
+                for (int u = 0; u < G; ++u)
+                    if (t0 + G + u < nrows) fma_row<BF16, BT, CAP>(acc, gb[u], s_xs, warp + NW * (t0 + G + u));
+#pragma unroll
+                for (int u = 0; u < G; ++u)
+                    if (t0 + 3 * G + u < nrows) gb[u] = ld_stream16(Wb + (size_t)s_k[warp + NW * (t0 + 3 * G + u)] * row_bytes);
             }
         }
         __syncthreads();
     }
 
-    // ---- cross-warp reduction in warp order -> this CTA's partial tile s_part[b][c]
+    // ---- cross-warp reduction in warp order; each finished element of this CTA's partial tile is pushed into
+    // the shared memory of the cluster rank that owns its column (slot = this rank), so one cluster barrier later
+    // every rank holds all S partials of its columns and adds them in rank order.
+    cg::cluster_group cluster = cg::this_cluster();
+    float *owner[MAX_CLUSTER];
+#pragma unroll
+    for (int q = 0; q < MAX_CLUSTER; ++q) owner[q] = (S > 1 && q < S) ? cluster.map_shared_rank(s_gather, q) : s_gather;
+    constexpr int HALF = TN / 2;
 #pragma unroll
     for (int b0 = 0; b0 < BT; b0 += RB) {
 #pragma unroll
@@ -241,66 +267,64 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
         }
         __syncthreads();
         for (int i = tid; i < RB * TN; i += NT) {
-            const int rb = i / TN, c = i - rb * TN;
+            const int rb = i / TN, c = i - rb * TN, b = b0 + rb;
             float v = 0.0f;
 #pragma unroll
             for (int w = 0; w < NW; ++w) v += s_red[(w * RB + rb) * TN + c];
-            s_part[(b0 + rb) * TN + c] = v;
+            if (b < B) {
+                int r, slot;
+                if constexpr (EPI == EPI_GLU) {  // owner by pair index j = c mod 128; gate and up of a pair sit side by side
+                    const int j = c & (HALF - 1), hf = c / HALF;
+                    r = j / per;
+                    slot = ((s * BT + b) * 2 + hf) * per + (j - r * per);
+                } else {
+                    r = c / per;
+                    slot = (s * BT + b) * per + (c - r * per);
+                }
+#pragma unroll
+                for (int q = 0; q < MAX_CLUSTER; ++q)
+                    if (q == r) owner[q][slot] = v;
+            }
         }
         __syncthreads();
     }
+    if (S > 1) cluster.sync();  // all pushes have landed; nothing remote is touched after this point
+    else __syncthreads();
 
-    // ---- cluster reduction through distributed shared memory, partials added in rank order
-    cg::cluster_group cluster = cg::this_cluster();
-    const float *peer[MAX_CLUSTER];
-    if (S > 1) {
-        cluster.sync();
-#pragma unroll
-        for (int q = 0; q < MAX_CLUSTER; ++q) peer[q] = cluster.map_shared_rank(s_part, q < S ? q : 0);
-    } else {
-        peer[0] = s_part;
-    }
-    if constexpr (EPI == EPI_BIAS) {
-        const int per = TN / S;  // columns finished by this rank
-        for (int i = tid; i < per * B; i += NT) {
-            const int b = i / per, c = s * per + (i - b * per);
-            const int n = tile * TN + c;
+    for (int it = 0; tid + it * NT < per * B; ++it) {
+        const int i = tid + it * NT;
+        const int b = i / per, cl = i - b * per;
+        const int row = a.out_rows ? a.out_rows[b] : b;
+        if constexpr (EPI == EPI_BIAS) {
+            const int n = tile * TN + s * per + cl;
             if (n < a.Nh) {
-                float v = load_bias<BF16>(a, n);
+                float v = it == 0 ? bias0[0] : it == 1 ? bias0[1] : load_bias<BF16>(a, n);
 #pragma unroll
                 for (int q = 0; q < MAX_CLUSTER; ++q)
-                    if (q < S) v += peer[q][b * TN + c];
-                const int row = a.out_rows ? a.out_rows[b] : b;
+                    if (q < S) v += s_gather[(q * BT + b) * per + cl];
                 a.y[(size_t)row * a.y_ld + n] = v;
             }
-        }
-    } else {
-        const int per = (TN / 2) / S;  // gate/up pairs finished by this rank
-        const int F = a.Nh;
-        for (int i = tid; i < per * B; i += NT) {
-            const int b = i / per, j = s * per + (i - b * per);
-            const int f = tile * (TN / 2) + j;
+        } else {
+            const int F = a.Nh, f = tile * HALF + s * per + cl;
             if (f < F) {
-                float g = a.bias ? __ldg(a.bias + f) : 0.0f;
-                float u = a.bias ? __ldg(a.bias + F + f) : 0.0f;
+                float g = it == 0 ? bias0[0] : it == 1 ? bias0[1] : (a.bias ? __ldg(a.bias + f) : 0.0f);
+                float u = it == 0 ? bias1[0] : it == 1 ? bias1[1] : (a.bias ? __ldg(a.bias + F + f) : 0.0f);
 #pragma unroll
                 for (int q = 0; q < MAX_CLUSTER; ++q)
                     if (q < S) {
-                        g += peer[q][b * TN + j];
-                        u += peer[q][b * TN + TN / 2 + j];
+                        g += s_gather[((q * BT + b) * 2 + 0) * per + cl];
+                        u += s_gather[((q * BT + b) * 2 + 1) * per + cl];
                     }
                 const float z = u * (g / (1.0f + expf(-g)));  // up * silu(gate)
-                const int row = a.out_rows ? a.out_rows[b] : b;
                 a.y[(size_t)row * a.y_ld + f] = z;
                 if (a.z_copy) a.z_copy[(size_t)b * F + f] = z;
             }
         }
     }
-    if (S > 1) cluster.sync();  // peers may still be reading this CTA's partial tile
 }
 
 template <bool BF16, int BT, int MODE, typename XT, int EPI>
-__global__ void __launch_bounds__(fc_threads(BT), fc_min_blocks(BT)) fc_kernel(const FcArgs a) {
+__global__ void __launch_bounds__(FC_THREADS, fc_min_blocks(BT)) fc_kernel(const FcArgs a) {
     griddep_wait();               // inputs produced by the previous kernel in the stream are complete
     griddep_launch_dependents();  // the next kernel may begin launching; it waits for this grid's completion itself
     fc_body<BF16, BT, MODE, XT, EPI>(a, blockIdx.x, blockIdx.y);

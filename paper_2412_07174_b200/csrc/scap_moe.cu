@@ -77,7 +77,7 @@ __global__ void __launch_bounds__(64) moe_route_kernel(const float *__restrict__
 // grid (tiles, S, E).  STAGE 1: packed gate|up FC of the rows routed to expert blockIdx.z, writing that
 // expert's z; STAGE 2: down FC reading z and writing each row to its (row, selection position) slot.
 template <bool BF16, int BT, int STAGE>
-__global__ void __launch_bounds__(fc_threads(BT), fc_min_blocks(BT)) moe_fc_kernel(const MoeArgs a) {
+__global__ void __launch_bounds__(FC_THREADS, fc_min_blocks(BT)) moe_fc_kernel(const MoeArgs a) {
     using ST = typename std::conditional<BF16, __nv_bfloat16, __half>::type;
     griddep_wait();
     griddep_launch_dependents();
@@ -137,7 +137,7 @@ static cudaError_t launch_moe_fc_t(const MoeArgs &a, int tiles, int S, cudaStrea
         if (e != cudaSuccess) return e;
         attr_done = true;
     }
-    return launch_cluster(kern, dim3(tiles, S, a.E), dim3(fc_threads(BT)), fc_smem_bytes(BT), S, st, g_tune.pdl != 0, a);
+    return launch_cluster(kern, dim3(tiles, S, a.E), dim3(FC_THREADS), fc_smem_bytes(BT), S, st, g_tune.pdl != 0, a);
 }
 
 template <bool BF16, int STAGE>
