@@ -93,4 +93,22 @@ __device__ __forceinline__ uint4 ld_stream16(const void *p) {
     return v;
 }
 
+// Ordered read-only loads: being volatile asm, they are issued where they are written (the compiler neither
+// sinks them towards their first use nor reorders them), which is what keeps a batch of them in flight together.
+__device__ __forceinline__ float ld_nc(const float *p) {
+    float v;
+    asm volatile("ld.global.nc.f32 %0, [%1];" : "=f"(v) : "l"(p));
+    return v;
+}
+__device__ __forceinline__ __nv_bfloat16 ld_nc(const __nv_bfloat16 *p) {
+    unsigned short v;
+    asm volatile("ld.global.nc.u16 %0, [%1];" : "=h"(v) : "l"(p));
+    return __ushort_as_bfloat16(v);
+}
+__device__ __forceinline__ __half ld_nc(const __half *p) {
+    unsigned short v;
+    asm volatile("ld.global.nc.u16 %0, [%1];" : "=h"(v) : "l"(p));
+    return __ushort_as_half(v);
+}
+
 }  // namespace scap

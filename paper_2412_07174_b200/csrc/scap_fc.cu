@@ -162,12 +162,13 @@ static scap_status sparse_fc_impl(const void *x, const void *W, const float *m, 
 }
 
 static scap_status dense_impl(const void *x, int xkind, const void *W, const float *b, const void *b16, float *y, int B,
-                              int K, int N, scap_dtype dt, cudaStream_t st) {
+                              int K, int N, scap_dtype dt, cudaStream_t st, bool writes_parameters) {
     FcArgs a;
     memset(&a, 0, sizeof(a));
     a.W = W; a.K = K; a.ldw = N; a.Nh = N; a.B = B;
     a.S = choose_split(K, fc_tiles(N, EPI_BIAS), 1);
     a.x = x; a.x_ld = K; a.bias = b; a.bias16 = b16; a.y = y; a.y_ld = N;
+    a.hold_dependents = writes_parameters ? 1 : 0;
     return cuda_status(launch_fc(dt == SCAP_BF16, MODE_DENSE, xkind, EPI_BIAS, a, st));
 }
 
@@ -234,7 +235,7 @@ scap_status scap_dense_fc(const void *x, const void *W, const float *b, float *y
     if (!aligned16(ws) || (b && !aligned16(b))) return SCAP_ERR_ALIGN;
     if (ws_bytes < scap_fc_workspace(B, K, N)) return SCAP_ERR_WORKSPACE;
     if ((st = check_device()) != SCAP_OK) return st;
-    return dense_impl(x, dt == SCAP_BF16 ? 1 : 0, W, b, nullptr, y, B, K, N, dt, reinterpret_cast<cudaStream_t>(stream));
+    return dense_impl(x, dt == SCAP_BF16 ? 1 : 0, W, b, nullptr, y, B, K, N, dt, reinterpret_cast<cudaStream_t>(stream), false);
 }
 
 size_t scap_fold_bias_workspace(int K, int N) { return scap_fc_workspace(1, K, N); }
@@ -247,7 +248,7 @@ scap_status scap_fold_bias(const void *W, const float *m, const void *b, int K, 
     if (!aligned16(ws) || (b && !aligned16(b))) return SCAP_ERR_ALIGN;
     if (ws_bytes < scap_fold_bias_workspace(K, N)) return SCAP_ERR_WORKSPACE;
     if ((st = check_device()) != SCAP_OK) return st;
-    return dense_impl(m, 2, W, nullptr, b, b_fused, 1, K, N, dt, reinterpret_cast<cudaStream_t>(stream));
+    return dense_impl(m, 2, W, nullptr, b, b_fused, 1, K, N, dt, reinterpret_cast<cudaStream_t>(stream), true);
 }
 
 size_t scap_fc_host_workspace(int B, int K, int N) {

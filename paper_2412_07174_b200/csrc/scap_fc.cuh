@@ -38,8 +38,8 @@ __host__ __device__ constexpr int fc_main_bytes(int BT) {
     const int red = FC_WARPS * fc_rb(BT) * TN * 4;
     return stage > red ? stage : red;
 }
-__host__ __device__ constexpr int fc_smem_bytes(int BT) {  // main | gathered partials | chunk masks | chunk offsets
-    return fc_main_bytes(BT) + BT * TN * 4 + (fc_cap(BT) / 32) * 4 + (fc_cap(BT) / 32 + 1) * 4 + 16;
+__host__ __device__ constexpr int fc_smem_bytes(int BT) {  // main | gathered partials | chunk masks
+    return fc_main_bytes(BT) + BT * TN * 4 + (fc_cap(BT) / 32) * 4 + 16;
 }
 
 struct FcArgs {
@@ -59,6 +59,7 @@ struct FcArgs {
     const int *out_rows;  // batch row b writes row out_rows[b] of y (NULL: row b)
     float *z_copy;        // EPI_GLU: optional second copy of z, [B, F] dense rows
     uint32_t *bits;       // optional [ceil(K/32)]: union keep mask, one word per 32-channel chunk
+    int hold_dependents;  // 1: do not let the next kernel start before this grid completes (it writes parameters)
 };
 
 template <bool BF16, int BT, int CAP>
@@ -84,8 +85,11 @@ __device__ __forceinline__ float load_bias(const FcArgs &a, int n) {
 }
 
 // Body for column tile `tile` and cluster rank `s`; every thread of every CTA of the cluster calls it.
+// With wait_inside the body itself waits for the previous kernel in the stream, and does so as late as it can:
+// W, m, tau and the biases are layer parameters, not outputs of the previous kernel, so they are read first and
+// only the activation x is read after the wait.
 template <bool BF16, int BT, int MODE, typename XT, int EPI>
-__device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const int s) {
+__device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const int s, const bool wait_inside) {
     constexpr int NT = FC_THREADS, NW = FC_WARPS, PU = fc_pu(BT), CAP = fc_cap(BT), RB = fc_rb(BT), U = fc_unroll(BT);
     constexpr int CAPC = CAP / 32;  // chunks per fill
     extern __shared__ __align__(16) unsigned char smem[];
@@ -94,7 +98,6 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
     float *s_red = reinterpret_cast<float *>(smem);
     float *s_gather = reinterpret_cast<float *>(smem + fc_main_bytes(BT));  // [S][BT][columns owned by this rank]
     uint32_t *s_bits = reinterpret_cast<uint32_t *>(s_gather + BT * TN);
-    int *s_off = reinterpret_cast<int *>(s_bits + CAPC);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int B = a.B, S = a.S, K = a.K;
@@ -142,25 +145,45 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
     const int nchunks = (K + 31) >> 5;
     const int my_chunks = nchunks > s ? (nchunks - s + S - 1) / S : 0;  // chunks s, s+S, ...
     float tau = 0.0f;
-    if constexpr (MODE == MODE_GATHER) tau = __ldg(a.tau);
+    if constexpr (MODE == MODE_GATHER) tau = ld_nc(a.tau);
 
+    if (wait_inside && my_chunks == 0) {
+        griddep_wait();
+        griddep_launch_dependents();
+    }
     for (int j0 = 0; j0 < my_chunks; j0 += CAPC) {
         const int nj = min(CAPC, my_chunks - j0);
         // ---- A: every warp loads PU chunks at once (all loads issued before any use), centres and thresholds them
         // (Alg. 3: one binary32 subtraction, one compare per element) and keeps the values in registers.
+        // Loads use clamped (always valid) addresses and no data-dependent branch, and nothing consumes
+        // them inside this loop, so the PU * (BT + 1) loads of a lane are all in flight together.
+        XT xraw[PU][BT];
         float xv[PU][BT], mk[PU];
 #pragma unroll
         for (int p = 0; p < PU; ++p) {
             const int j = warp * PU + p;
             const int k = (s + S * (j0 + j)) * 32 + lane;
-            const bool ok = j < nj && k < K;
-            mk[p] = (ok && a.m) ? __ldg(a.m + k) : 0.0f;
+            mk[p] = a.m ? ld_nc(a.m + ((j < nj && k < K) ? k : 0)) : 0.0f;
+        }
+        if (wait_inside && j0 == 0) {
+            griddep_wait();               // x (produced by the previous kernel in the stream) is complete
+            griddep_launch_dependents();  // the next kernel may begin launching; it waits for this grid itself
+        }
+#pragma unroll
+        for (int p = 0; p < PU; ++p) {
+            const int j = warp * PU + p;
+            const int k = (s + S * (j0 + j)) * 32 + lane;
+            const int kk = (j < nj && k < K) ? k : 0;
 #pragma unroll
             for (int b = 0; b < BT; ++b) {
-                xv[p][b] = 0.0f;
-                if (ok && b < B) xv[p][b] = widen1(xg[(size_t)(a.in_rows ? a.in_rows[b] : b) * a.x_ld + k]);
+                const int bb = b < B ? b : 0;
+                xraw[p][b] = ld_nc(xg + (size_t)(a.in_rows ? a.in_rows[bb] : bb) * a.x_ld + kk);
             }
         }
+#pragma unroll
+        for (int p = 0; p < PU; ++p)
+#pragma unroll
+            for (int b = 0; b < BT; ++b) xv[p][b] = widen1(xraw[p][b]);
         uint32_t km[PU];
         unsigned bal[PU];
 #pragma unroll
@@ -186,8 +209,9 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
             }
         }
         __syncthreads();
-        // ---- exclusive prefix of the chunk counts (warp 0)
-        if (warp == 0) {
+        // ---- exclusive prefix of the chunk counts: every warp scans all CAPC counts itself (no second barrier)
+        int my_off[PU], cnt;
+        {
             int carry = 0;
 #pragma unroll
             for (int c0 = 0; c0 < CAPC; c0 += 32) {
@@ -198,19 +222,23 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
                     const int t = __shfl_up_sync(0xffffffffu, v, o);
                     if (lane >= o) v += t;
                 }
-                if (c0 + lane < nj) s_off[c0 + lane] = carry + v - v0;
+                const int excl = carry + v - v0;
+#pragma unroll
+                for (int p = 0; p < PU; ++p) {  // chunk warp*PU+p lives in lane (warp*PU+p) % 32 of block (warp*PU+p) / 32
+                    const int j = warp * PU + p;
+                    const int t = __shfl_sync(0xffffffffu, excl, j & 31);
+                    if ((j >> 5) == (c0 >> 5)) my_off[p] = t;
+                }
                 carry += __shfl_sync(0xffffffffu, v, 31);
             }
-            if (lane == 0) s_off[nj] = carry;
+            cnt = carry;
         }
-        __syncthreads();
-        const int cnt = s_off[nj];
         // ---- B: kept channels and their pruned values, in ascending channel order
 #pragma unroll
         for (int p = 0; p < PU; ++p) {
-            const int j = warp * PU + p;
             if (km[p]) {
-                const int pos = s_off[j] + __popc(bal[p] & ((1u << lane) - 1u));
+                const int j = warp * PU + p;
+                const int pos = my_off[p] + __popc(bal[p] & ((1u << lane) - 1u));
                 s_k[pos] = (uint32_t)((s + S * (j0 + j)) * 32 + lane);
 #pragma unroll
                 for (int b = 0; b < BT; ++b)
@@ -325,9 +353,12 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
 
 template <bool BF16, int BT, int MODE, typename XT, int EPI>
 __global__ void __launch_bounds__(FC_THREADS, fc_min_blocks(BT)) fc_kernel(const FcArgs a) {
-    griddep_wait();               // inputs produced by the previous kernel in the stream are complete
-    griddep_launch_dependents();  // the next kernel may begin launching; it waits for this grid's completion itself
-    fc_body<BF16, BT, MODE, XT, EPI>(a, blockIdx.x, blockIdx.y);
+    if (a.hold_dependents) {  // parameter-producing call: ordinary stream order on both sides
+        griddep_wait();
+        fc_body<BF16, BT, MODE, XT, EPI>(a, blockIdx.x, blockIdx.y, false);
+    } else {
+        fc_body<BF16, BT, MODE, XT, EPI>(a, blockIdx.x, blockIdx.y, true);
+    }
 }
 
 // ---- host-side plumbing shared by the entry points ------------------------------------------------
