@@ -38,30 +38,44 @@ int sm_count() {
     return n;
 }
 
-// Largest power of two <= 8 that keeps the whole grid co-resident (about two CTAs per SM) and leaves
-// every slice at least 64 input channels.
-int choose_split(int K, int tiles, int groups) {
-    int S = MAX_CLUSTER;
-    if (g_tune.split_k > 0) {
-        while (S > g_tune.split_k) S >>= 1;
-        return S;
-    }
+// Two CTAs fit on an SM, so up to 2 * SMs CTAs are resident at once.  Among tile widths {256, 128} and cluster
+// sizes {8, 4, 2, 1} pick the pair with the most CTAs within that budget (ties: wider tile, then larger
+// cluster), keeping at least 64 input channels per slice.
+void choose_config(int K, int Nh, int epi, int groups, int *tn_out, int *S_out) {
     const int budget = 2 * sm_count();
-    while (S > 1 && ((long long)tiles * groups * S > budget || K / S < 64)) S >>= 1;
-    return S;
+    int best_tn = 256, best_S = 1;
+    long long best = -1;
+    for (int tn = 256; tn >= 128; tn >>= 1) {
+        const int tiles = fc_tiles(Nh, epi, tn);
+        for (int S = MAX_CLUSTER; S >= 1; S >>= 1) {
+            if (g_tune.split_k > 0 && S > g_tune.split_k) continue;
+            if (S > 1 && K / S < 64) continue;
+            const long long ctas = (long long)tiles * groups * S;
+            if (ctas > budget && !(S == 1 && tn == 256)) continue;
+            const long long score = ctas > budget ? 0 : ctas;
+            if (score > best) { best = score; best_tn = tn; best_S = S; }
+        }
+    }
+    *tn_out = best_tn;
+    *S_out = best_S;
 }
 
-template <bool BF16, int BT, int MODE, typename XT, int EPI>
-static cudaError_t launch_fc_t(const FcArgs &a, cudaStream_t st) {
+template <bool BF16, int BT, int MODE, typename XT, int EPI, int TNT>
+static cudaError_t launch_fc_tn(const FcArgs &a, cudaStream_t st) {
     static bool attr_done = false;
-    auto kern = fc_kernel<BF16, BT, MODE, XT, EPI>;
+    auto kern = fc_kernel<BF16, BT, MODE, XT, EPI, TNT>;
     if (!attr_done) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, fc_smem_bytes(BT));
         if (e != cudaSuccess) return e;
         attr_done = true;
     }
-    return launch_cluster(kern, dim3(fc_tiles(a.Nh, EPI), a.S), dim3(FC_THREADS), fc_smem_bytes(BT), a.S, st,
+    return launch_cluster(kern, dim3(fc_tiles(a.Nh, EPI, TNT), a.S), dim3(FC_THREADS), fc_smem_bytes(BT), a.S, st,
                           g_tune.pdl != 0, a);
+}
+
+template <bool BF16, int BT, int MODE, typename XT, int EPI>
+static cudaError_t launch_fc_t(const FcArgs &a, cudaStream_t st) {
+    return a.tn == 128 ? launch_fc_tn<BF16, BT, MODE, XT, EPI, 128>(a, st) : launch_fc_tn<BF16, BT, MODE, XT, EPI, 256>(a, st);
 }
 
 template <bool BF16, int MODE, typename XT, int EPI>
@@ -151,7 +165,7 @@ static scap_status sparse_fc_impl(const void *x, const void *W, const float *m, 
     FcArgs a;
     memset(&a, 0, sizeof(a));
     a.W = W; a.K = K; a.ldw = N; a.Nh = N; a.B = B;
-    a.S = choose_split(K, fc_tiles(N, EPI_BIAS), 1);
+    choose_config(K, N, EPI_BIAS, 1, &a.tn, &a.S);
     a.x = x; a.x_ld = K; a.m = m; a.tau = tau; a.bias = b_fused; a.y = y; a.y_ld = N;
     const bool inspect = idx_out || nnz_out;
     if (inspect) a.bits = reinterpret_cast<uint32_t *>(ws);
@@ -166,7 +180,7 @@ static scap_status dense_impl(const void *x, int xkind, const void *W, const flo
     FcArgs a;
     memset(&a, 0, sizeof(a));
     a.W = W; a.K = K; a.ldw = N; a.Nh = N; a.B = B;
-    a.S = choose_split(K, fc_tiles(N, EPI_BIAS), 1);
+    choose_config(K, N, EPI_BIAS, 1, &a.tn, &a.S);
     a.x = x; a.x_ld = K; a.bias = b; a.bias16 = b16; a.y = y; a.y_ld = N;
     a.hold_dependents = writes_parameters ? 1 : 0;
     return cuda_status(launch_fc(dt == SCAP_BF16, MODE_DENSE, xkind, EPI_BIAS, a, st));

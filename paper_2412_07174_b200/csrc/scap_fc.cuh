@@ -21,7 +21,7 @@ namespace cg = cooperative_groups;
 enum { MODE_GATHER = 0, MODE_DENSE = 1 };
 enum { EPI_BIAS = 0, EPI_GLU = 1 };
 
-constexpr int TN = 256;         // columns per CTA: 32 lanes x 8 columns (one 16-byte load per lane and row)
+constexpr int TN = 256;         // widest column tile per CTA (each thread owns 8 columns = one 16-byte load per row)
 constexpr int MAX_CLUSTER = 8;  // portable cluster size: upper bound of the split-K factor S
 
 constexpr int FC_THREADS = 256;  // 8 warps; two CTAs fit on an SM, so every cluster of the grid is resident at once
@@ -47,6 +47,7 @@ struct FcArgs {
     int K, ldw;           // ldw: columns of a weight row (N, or 2F for the packed gate|up weight)
     int Nh;               // EPI_BIAS: N.  EPI_GLU: F (gate columns 0..F-1, up columns F..2F-1)
     int B, S;             // batch rows; split-K factor = cluster size (1, 2, 4 or 8)
+    int tn;               // columns per CTA: 256 or 128
     const void *x;        // activations [rows, x_ld] of type XT
     int x_ld;
     const int *in_rows;   // batch row b reads row in_rows[b] of x (NULL: row b)
@@ -85,13 +86,17 @@ __device__ __forceinline__ float load_bias(const FcArgs &a, int n) {
 }
 
 // Body for column tile `tile` and cluster rank `s`; every thread of every CTA of the cluster calls it.
+// TNT = columns per CTA (256 or 128): a row segment is TNT/8 lanes wide, so a warp streams 1 or 2 rows per load.
 // With wait_inside the body itself waits for the previous kernel in the stream, and does so as late as it can:
 // W, m, tau and the biases are layer parameters, not outputs of the previous kernel, so they are read first and
 // only the activation x is read after the wait.
-template <bool BF16, int BT, int MODE, typename XT, int EPI>
+template <bool BF16, int BT, int MODE, typename XT, int EPI, int TNT>
 __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const int s, const bool wait_inside) {
-    constexpr int NT = FC_THREADS, NW = FC_WARPS, PU = fc_pu(BT), CAP = fc_cap(BT), RB = fc_rb(BT), U = fc_unroll(BT);
-    constexpr int CAPC = CAP / 32;  // chunks per fill
+    constexpr int NT = FC_THREADS, PU = fc_pu(BT), CAP = fc_cap(BT), RB = fc_rb(BT), U = fc_unroll(BT);
+    constexpr int CAPC = CAP / 32;    // chunks per fill
+    constexpr int LPR = TNT / 8;      // lanes per row segment
+    constexpr int NR = NT / LPR;      // row groups per CTA: group g streams rows g, g+NR, ...
+    constexpr int HALF = TNT / 2;
     extern __shared__ __align__(16) unsigned char smem[];
     uint32_t *s_k = reinterpret_cast<uint32_t *>(smem);
     float *s_xs = reinterpret_cast<float *>(smem) + CAP;
@@ -100,18 +105,19 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
     uint32_t *s_bits = reinterpret_cast<uint32_t *>(s_gather + BT * TN);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int rg = tid / LPR, cl = tid % LPR;  // row group and column lane of this thread
     const int B = a.B, S = a.S, K = a.K;
     const XT *xg = reinterpret_cast<const XT *>(a.x);
 
-    // this lane's 8 columns
+    // this thread's 8 columns
     int col;
     bool col_ok;
-    if constexpr (EPI == EPI_GLU) {  // lanes 0..15: gate columns of 128 f's; lanes 16..31: the matching up columns
-        const int f = tile * (TN / 2) + (lane & 15) * 8;
+    if constexpr (EPI == EPI_GLU) {  // first half of the column lanes: gate columns; second half: the matching up columns
+        const int f = tile * HALF + (cl % (LPR / 2)) * 8;
         col_ok = f < a.Nh;
-        col = (lane >> 4) * a.Nh + f;
+        col = (cl / (LPR / 2)) * a.Nh + f;
     } else {
-        col = tile * TN + lane * 8;
+        col = tile * TNT + cl * 8;
         col_ok = col < a.Nh;
     }
     const unsigned char *Wb = reinterpret_cast<const unsigned char *>(a.W) + (size_t)col * 2;
@@ -119,18 +125,18 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
 
     // Columns this rank finishes after the cluster exchange, and their bias, fetched now so that the
     // load is off the critical path.  EPI_BIAS: `per` columns; EPI_GLU: `per` gate/up pairs.
-    const int per = (EPI == EPI_GLU ? TN / 2 : TN) / S;
+    const int per = (EPI == EPI_GLU ? HALF : TNT) / S;
     float bias0[2] = {0.0f, 0.0f}, bias1[2] = {0.0f, 0.0f};
 #pragma unroll
     for (int it = 0; it < 2; ++it) {
         const int i = tid + it * NT;
         if (i < per * B) {
-            const int cl = i % per;
+            const int c = i % per;
             if constexpr (EPI == EPI_GLU) {
-                const int f = tile * (TN / 2) + s * per + cl;
+                const int f = tile * HALF + s * per + c;
                 if (f < a.Nh && a.bias) { bias0[it] = __ldg(a.bias + f); bias1[it] = __ldg(a.bias + a.Nh + f); }
             } else {
-                const int n = tile * TN + s * per + cl;
+                const int n = tile * TNT + s * per + c;
                 if (n < a.Nh) bias0[it] = load_bias<BF16>(a, n);
             }
         }
@@ -153,10 +159,10 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
     }
     for (int j0 = 0; j0 < my_chunks; j0 += CAPC) {
         const int nj = min(CAPC, my_chunks - j0);
-        // ---- A: every warp loads PU chunks at once (all loads issued before any use), centres and thresholds them
-        // (Alg. 3: one binary32 subtraction, one compare per element) and keeps the values in registers.
-        // Loads use clamped (always valid) addresses and no data-dependent branch, and nothing consumes
-        // them inside this loop, so the PU * (BT + 1) loads of a lane are all in flight together.
+        // ---- A: every warp loads PU chunks at once, centres and thresholds them (Alg. 3: one binary32
+        // subtraction, one compare per element) and keeps the values in registers.  Loads use clamped (always
+        // valid) addresses and no data-dependent branch, and nothing consumes them inside the load loops, so the
+        // PU * (BT + 1) loads of a lane are all in flight together.
         XT xraw[PU][BT];
         float xv[PU][BT], mk[PU];
 #pragma unroll
@@ -184,54 +190,57 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
         for (int p = 0; p < PU; ++p)
 #pragma unroll
             for (int b = 0; b < BT; ++b) xv[p][b] = widen1(xraw[p][b]);
+        // Branch-free so that the PU independent chains interleave: keep masks, then one ballot word per chunk.
         uint32_t km[PU];
         unsigned bal[PU];
 #pragma unroll
         for (int p = 0; p < PU; ++p) {
             const int j = warp * PU + p;
-            const int c = s + S * (j0 + j), k = c * 32 + lane;
+            const int k = (s + S * (j0 + j)) * 32 + lane;
             const bool ok = j < nj && k < K;
-            km[p] = 0;
+            uint32_t m_ = 0;
 #pragma unroll
             for (int b = 0; b < BT; ++b) {
                 if constexpr (MODE == MODE_GATHER) {
                     const float dv = a.m ? __fsub_rn(xv[p][b], mk[p]) : xv[p][b];
                     xv[p][b] = dv;
-                    if (ok && b < B && fabsf(dv) >= tau) km[p] |= 1u << b;
+                    m_ |= (ok && b < B && fabsf(dv) >= tau) ? (1u << b) : 0u;
                 } else {
-                    if (ok) km[p] = 1u;  // dense: every channel, no compare
+                    m_ = ok ? 1u : 0u;  // dense: every channel, no compare
                 }
             }
-            bal[p] = __ballot_sync(0xffffffffu, km[p] != 0);
-            if (lane == 0 && j < nj) {
-                s_bits[j] = bal[p];
-                if (MODE == MODE_GATHER && a.bits && tile == 0) a.bits[c] = bal[p];
+            km[p] = m_;
+            bal[p] = __ballot_sync(0xffffffffu, m_ != 0);
+        }
+        {   // lane p publishes the word of chunk warp*PU + p
+            unsigned mine = 0;
+#pragma unroll
+            for (int p = 0; p < PU; ++p) mine = lane == p ? bal[p] : mine;
+            const int j = warp * PU + lane;
+            if (lane < PU && j < nj) {
+                s_bits[j] = mine;
+                if (MODE == MODE_GATHER && a.bits && tile == 0) a.bits[s + S * (j0 + j)] = mine;
             }
         }
         __syncthreads();
-        // ---- exclusive prefix of the chunk counts: every warp scans all CAPC counts itself (no second barrier)
-        int my_off[PU], cnt;
+        // ---- position of each chunk in the kept list: every warp sums the counts of the chunks before its own
+        // with warp-wide integer reductions (no second barrier, no serial scan)
+        int my_off[PU], cnt = 0;
         {
-            int carry = 0;
+            int c_lo[(CAPC + 31) / 32];
 #pragma unroll
-            for (int c0 = 0; c0 < CAPC; c0 += 32) {
-                const int v0 = (c0 + lane < nj) ? __popc(s_bits[c0 + lane]) : 0;
-                int v = v0;
-#pragma unroll
-                for (int o = 1; o < 32; o <<= 1) {
-                    const int t = __shfl_up_sync(0xffffffffu, v, o);
-                    if (lane >= o) v += t;
-                }
-                const int excl = carry + v - v0;
-#pragma unroll
-                for (int p = 0; p < PU; ++p) {  // chunk warp*PU+p lives in lane (warp*PU+p) % 32 of block (warp*PU+p) / 32
-                    const int j = warp * PU + p;
-                    const int t = __shfl_sync(0xffffffffu, excl, j & 31);
-                    if ((j >> 5) == (c0 >> 5)) my_off[p] = t;
-                }
-                carry += __shfl_sync(0xffffffffu, v, 31);
+            for (int q = 0; q < (CAPC + 31) / 32; ++q) {
+                c_lo[q] = (q * 32 + lane < nj) ? __popc(s_bits[q * 32 + lane]) : 0;
+                cnt += __reduce_add_sync(0xffffffffu, c_lo[q]);
             }
-            cnt = carry;
+#pragma unroll
+            for (int p = 0; p < PU; ++p) {
+                const int j = warp * PU + p;
+                int o = 0;
+#pragma unroll
+                for (int q = 0; q < (CAPC + 31) / 32; ++q) o += __reduce_add_sync(0xffffffffu, (q * 32 + lane < j) ? c_lo[q] : 0);
+                my_off[p] = o;
+            }
         }
         // ---- B: kept channels and their pruned values, in ascending channel order
 #pragma unroll
@@ -247,62 +256,61 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
         }
         __syncthreads();
 
-        // ---- stream the kept rows: warp w takes rows w, w+NW, ...  Two register groups of G loads alternate
+        // ---- stream the kept rows: row group g takes rows g, g+NR, ...  Two register groups of G loads alternate
         // (one is consumed while the other is in flight).
         if (col_ok) {
             constexpr int G = U / 2;
-            const int nrows = cnt > warp ? (cnt - warp + NW - 1) / NW : 0;
+            const int nrows = cnt > rg ? (cnt - rg + NR - 1) / NR : 0;
             uint4 ga[G], gb[G];
 #pragma unroll
             for (int u = 0; u < G; ++u)
-                if (u < nrows) ga[u] = ld_stream16(Wb + (size_t)s_k[warp + NW * u] * row_bytes);
+                if (u < nrows) ga[u] = ld_stream16(Wb + (size_t)s_k[rg + NR * u] * row_bytes);
 #pragma unroll
             for (int u = 0; u < G; ++u)
-                if (G + u < nrows) gb[u] = ld_stream16(Wb + (size_t)s_k[warp + NW * (G + u)] * row_bytes);
+                if (G + u < nrows) gb[u] = ld_stream16(Wb + (size_t)s_k[rg + NR * (G + u)] * row_bytes);
             for (int t0 = 0; t0 < nrows; t0 += 2 * G) {
 #pragma unroll
                 for (int u = 0; u < G; ++u)
-                    if (t0 + u < nrows) fma_row<BF16, BT, CAP>(acc, ga[u], s_xs, warp + NW * (t0 + u));
+                    if (t0 + u < nrows) fma_row<BF16, BT, CAP>(acc, ga[u], s_xs, rg + NR * (t0 + u));
 #pragma unroll
                 for (int u = 0; u < G; ++u)
-                    if (t0 + 2 * G + u < nrows) ga[u] = ld_stream16(Wb + (size_t)s_k[warp + NW * (t0 + 2 * G + u)] * row_bytes);
+                    if (t0 + 2 * G + u < nrows) ga[u] = ld_stream16(Wb + (size_t)s_k[rg + NR * (t0 + 2 * G + u)] * row_bytes);
 #pragma unroll
                 for (int u = 0; u < G; ++u)
-                    if (t0 + G + u < nrows) fma_row<BF16, BT, CAP>(acc, gb[u], s_xs, warp + NW * (t0 + G + u));
+                    if (t0 + G + u < nrows) fma_row<BF16, BT, CAP>(acc, gb[u], s_xs, rg + NR * (t0 + G + u));
 #pragma unroll
                 for (int u = 0; u < G; ++u)
-                    if (t0 + 3 * G + u < nrows) gb[u] = ld_stream16(Wb + (size_t)s_k[warp + NW * (t0 + 3 * G + u)] * row_bytes);
+                    if (t0 + 3 * G + u < nrows) gb[u] = ld_stream16(Wb + (size_t)s_k[rg + NR * (t0 + 3 * G + u)] * row_bytes);
             }
         }
         __syncthreads();
     }
 
-    // ---- cross-warp reduction in warp order; each finished element of this CTA's partial tile is pushed into
-    // the shared memory of the cluster rank that owns its column (slot = this rank), so one cluster barrier later
-    // every rank holds all S partials of its columns and adds them in rank order.
+    // ---- reduction over the row groups in group order; each finished element of this CTA's partial tile is
+    // pushed into the shared memory of the cluster rank that owns its column (slot = this rank), so one cluster
+    // barrier later every rank holds all S partials of its columns and adds them in rank order.
     cg::cluster_group cluster = cg::this_cluster();
     float *owner[MAX_CLUSTER];
 #pragma unroll
     for (int q = 0; q < MAX_CLUSTER; ++q) owner[q] = (S > 1 && q < S) ? cluster.map_shared_rank(s_gather, q) : s_gather;
-    constexpr int HALF = TN / 2;
 #pragma unroll
     for (int b0 = 0; b0 < BT; b0 += RB) {
 #pragma unroll
         for (int rb = 0; rb < RB; ++rb) {
-            float4 *dst = reinterpret_cast<float4 *>(s_red + ((warp * RB + rb) * TN + lane * 8));
+            float4 *dst = reinterpret_cast<float4 *>(s_red + ((rg * RB + rb) * TNT + cl * 8));
             dst[0] = make_float4(acc[b0 + rb][0], acc[b0 + rb][1], acc[b0 + rb][2], acc[b0 + rb][3]);
             dst[1] = make_float4(acc[b0 + rb][4], acc[b0 + rb][5], acc[b0 + rb][6], acc[b0 + rb][7]);
         }
         __syncthreads();
-        for (int i = tid; i < RB * TN; i += NT) {
-            const int rb = i / TN, c = i - rb * TN, b = b0 + rb;
+        for (int i = tid; i < RB * TNT; i += NT) {
+            const int rb = i / TNT, c = i - rb * TNT, b = b0 + rb;
             float v = 0.0f;
 #pragma unroll
-            for (int w = 0; w < NW; ++w) v += s_red[(w * RB + rb) * TN + c];
+            for (int g = 0; g < NR; ++g) v += s_red[(g * RB + rb) * TNT + c];
             if (b < B) {
                 int r, slot;
-                if constexpr (EPI == EPI_GLU) {  // owner by pair index j = c mod 128; gate and up of a pair sit side by side
-                    const int j = c & (HALF - 1), hf = c / HALF;
+                if constexpr (EPI == EPI_GLU) {  // owner by pair index j = c mod HALF; gate and up of a pair sit side by side
+                    const int j = c % HALF, hf = c / HALF;
                     r = j / per;
                     slot = ((s * BT + b) * 2 + hf) * per + (j - r * per);
                 } else {
@@ -321,27 +329,27 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
 
     for (int it = 0; tid + it * NT < per * B; ++it) {
         const int i = tid + it * NT;
-        const int b = i / per, cl = i - b * per;
+        const int b = i / per, c = i - b * per;
         const int row = a.out_rows ? a.out_rows[b] : b;
         if constexpr (EPI == EPI_BIAS) {
-            const int n = tile * TN + s * per + cl;
+            const int n = tile * TNT + s * per + c;
             if (n < a.Nh) {
                 float v = it == 0 ? bias0[0] : it == 1 ? bias0[1] : load_bias<BF16>(a, n);
 #pragma unroll
                 for (int q = 0; q < MAX_CLUSTER; ++q)
-                    if (q < S) v += s_gather[(q * BT + b) * per + cl];
+                    if (q < S) v += s_gather[(q * BT + b) * per + c];
                 a.y[(size_t)row * a.y_ld + n] = v;
             }
         } else {
-            const int F = a.Nh, f = tile * HALF + s * per + cl;
+            const int F = a.Nh, f = tile * HALF + s * per + c;
             if (f < F) {
                 float g = it == 0 ? bias0[0] : it == 1 ? bias0[1] : (a.bias ? __ldg(a.bias + f) : 0.0f);
                 float u = it == 0 ? bias1[0] : it == 1 ? bias1[1] : (a.bias ? __ldg(a.bias + F + f) : 0.0f);
 #pragma unroll
                 for (int q = 0; q < MAX_CLUSTER; ++q)
                     if (q < S) {
-                        g += s_gather[((q * BT + b) * 2 + 0) * per + cl];
-                        u += s_gather[((q * BT + b) * 2 + 1) * per + cl];
+                        g += s_gather[((q * BT + b) * 2 + 0) * per + c];
+                        u += s_gather[((q * BT + b) * 2 + 1) * per + c];
                     }
                 const float z = u * (g / (1.0f + expf(-g)));  // up * silu(gate)
                 a.y[(size_t)row * a.y_ld + f] = z;
@@ -351,23 +359,24 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
     }
 }
 
-template <bool BF16, int BT, int MODE, typename XT, int EPI>
+template <bool BF16, int BT, int MODE, typename XT, int EPI, int TNT>
 __global__ void __launch_bounds__(FC_THREADS, fc_min_blocks(BT)) fc_kernel(const FcArgs a) {
     if (a.hold_dependents) {  // parameter-producing call: ordinary stream order on both sides
         griddep_wait();
-        fc_body<BF16, BT, MODE, XT, EPI>(a, blockIdx.x, blockIdx.y, false);
+        fc_body<BF16, BT, MODE, XT, EPI, TNT>(a, blockIdx.x, blockIdx.y, false);
     } else {
-        fc_body<BF16, BT, MODE, XT, EPI>(a, blockIdx.x, blockIdx.y, true);
+        fc_body<BF16, BT, MODE, XT, EPI, TNT>(a, blockIdx.x, blockIdx.y, true);
     }
 }
 
 // ---- host-side plumbing shared by the entry points ------------------------------------------------
 
 inline int batch_tile(int B) { return B <= 1 ? 1 : B <= 2 ? 2 : B <= 4 ? 4 : B <= 8 ? 8 : 16; }
-inline int fc_tiles(int Nh, int epi) { return epi == EPI_GLU ? (Nh + TN / 2 - 1) / (TN / 2) : (Nh + TN - 1) / TN; }
+inline int fc_tiles(int Nh, int epi, int tn) { return epi == EPI_GLU ? (Nh + tn / 2 - 1) / (tn / 2) : (Nh + tn - 1) / tn; }
 
-// Split-K factor (cluster size) for `tiles` column tiles per group and `groups` concurrently active groups.
-int choose_split(int K, int tiles, int groups);
+// Tile width (256 or 128 columns) and split-K factor (cluster size) for an FC with Nh columns per half and
+// `groups` concurrently active groups (experts): the pair with the most CTAs that are still all co-resident.
+void choose_config(int K, int Nh, int epi, int groups, int *tn, int *S);
 
 // Launch with cluster dimension (1, S, 1) and, if enabled, programmatic dependent launch.
 template <typename... KArgs, typename... Args>

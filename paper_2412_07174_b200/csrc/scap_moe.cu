@@ -16,7 +16,7 @@ struct Route {  // device-resident routing table
 
 struct MoeArgs {
     scap_expert ex[SCAP_MAX_EXPERTS];
-    int E, top_k, B, D, F, S1, S2;
+    int E, top_k, B, D, F, S1, S2, tn1, tn2;
     const void *h;
     const float *logits;
     unsigned char *groups;  // per-expert scratch: z[B, F]
@@ -76,7 +76,7 @@ __global__ void __launch_bounds__(64) moe_route_kernel(const float *__restrict__
 
 // grid (tiles, S, E).  STAGE 1: packed gate|up FC of the rows routed to expert blockIdx.z, writing that
 // expert's z; STAGE 2: down FC reading z and writing each row to its (row, selection position) slot.
-template <bool BF16, int BT, int STAGE>
+template <bool BF16, int BT, int STAGE, int TNT>
 __global__ void __launch_bounds__(FC_THREADS, fc_min_blocks(BT)) moe_fc_kernel(const MoeArgs a) {
     using ST = typename std::conditional<BF16, __nv_bfloat16, __half>::type;
     griddep_wait();
@@ -92,13 +92,13 @@ __global__ void __launch_bounds__(FC_THREADS, fc_min_blocks(BT)) moe_fc_kernel(c
         g.x = a.h; g.x_ld = a.D; g.in_rows = a.route->rows[e];
         g.m = a.ex[e].m1; g.tau = a.ex[e].tau1; g.bias = a.ex[e].bgu_fused;
         g.y = z; g.y_ld = a.F;
-        fc_body<BF16, BT, MODE_GATHER, ST, EPI_GLU>(g, blockIdx.x, blockIdx.y, false);
+        fc_body<BF16, BT, MODE_GATHER, ST, EPI_GLU, TNT>(g, blockIdx.x, blockIdx.y, false);
     } else {
         g.W = a.ex[e].Wd; g.K = a.F; g.ldw = a.D; g.Nh = a.D; g.S = a.S2;
         g.x = z; g.x_ld = a.F;
         g.m = a.ex[e].m2; g.tau = a.ex[e].tau2; g.bias = a.ex[e].bd_fused;
         g.y = a.yslot; g.y_ld = a.D; g.out_rows = a.route->slots[e];
-        fc_body<BF16, BT, MODE_GATHER, float, EPI_BIAS>(g, blockIdx.x, blockIdx.y, false);
+        fc_body<BF16, BT, MODE_GATHER, float, EPI_BIAS, TNT>(g, blockIdx.x, blockIdx.y, false);
     }
 }
 
@@ -128,16 +128,22 @@ static MoeLayout moe_layout(int B, int D, int F, int E, int top_k) {
     return M;
 }
 
-template <bool BF16, int BT, int STAGE>
-static cudaError_t launch_moe_fc_t(const MoeArgs &a, int tiles, int S, cudaStream_t st) {
+template <bool BF16, int BT, int STAGE, int TNT>
+static cudaError_t launch_moe_fc_tn(const MoeArgs &a, int tiles, int S, cudaStream_t st) {
     static bool attr_done = false;
-    auto kern = moe_fc_kernel<BF16, BT, STAGE>;
+    auto kern = moe_fc_kernel<BF16, BT, STAGE, TNT>;
     if (!attr_done) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, fc_smem_bytes(BT));
         if (e != cudaSuccess) return e;
         attr_done = true;
     }
     return launch_cluster(kern, dim3(tiles, S, a.E), dim3(FC_THREADS), fc_smem_bytes(BT), S, st, g_tune.pdl != 0, a);
+}
+
+template <bool BF16, int BT, int STAGE>
+static cudaError_t launch_moe_fc_t(const MoeArgs &a, int tiles, int S, cudaStream_t st) {
+    const int tn = STAGE == 1 ? a.tn1 : a.tn2;
+    return tn == 128 ? launch_moe_fc_tn<BF16, BT, STAGE, 128>(a, tiles, S, st) : launch_moe_fc_tn<BF16, BT, STAGE, 256>(a, tiles, S, st);
 }
 
 template <bool BF16, int STAGE>
@@ -198,9 +204,9 @@ scap_status scap_moe_ffn(const void *h, const float *logits, const scap_expert *
     a.yslot = reinterpret_cast<float *>(w + M.yslot);
     a.y = y; a.expert_out = expert_out; a.weight_out = weight_out;
     const int active = B * top_k < E ? B * top_k : E;  // experts that can have rows at once
-    const int tiles1 = fc_tiles(F, EPI_GLU), tiles2 = fc_tiles(D, EPI_BIAS);
-    a.S1 = choose_split(D, tiles1, active);
-    a.S2 = choose_split(F, tiles2, active);
+    choose_config(D, F, EPI_GLU, active, &a.tn1, &a.S1);
+    choose_config(F, D, EPI_BIAS, active, &a.tn2, &a.S2);
+    const int tiles1 = fc_tiles(F, EPI_GLU, a.tn1), tiles2 = fc_tiles(D, EPI_BIAS, a.tn2);
     const bool bf16 = dt == SCAP_BF16, pdl = g_tune.pdl != 0;
 
     cudaError_t e = launch(moe_route_kernel, dim3(1), dim3(64), 0, st, pdl, logits, B, E, top_k, a.route, expert_out, weight_out);
