@@ -5,8 +5,9 @@
 
 Workload (N = 1): the Llama-2-7B-shaped FFN down projection, bf16, batch 1 - W[K=11008, N=4096] ~ N(0, 0.02^2),
 inputs silu(g)*u with g, u ~ N(0,1), mode and tau calibrated on 1024 tokens at sparsity targets 50 / 65 / 80 %.
-One step = one sparse FC call (compaction + gather-GEMV) per sparsity target on each of R device copies of W,
-R chosen so that the copies total at least four times the L2 size: no call finds its weight rows in L2.
+One step = one sparse FC call (one fused kernel: threshold + compaction + gather-GEMV + reduction) per sparsity target on
+each of R device copies of W, R chosen so that even the sparsest call pattern touches at least four times the L2 size
+per cycle: no call finds its weight rows in L2.
 The metric is effective HBM GB/s on the bytes a call must touch (kept rows + activations + mode + bias + output),
 summed over the step; the JSON line also carries us/call per sparsity, the library's own dense GEMV on the same
 rotation, the speedup over it, the roofline fraction against the measured copy bandwidth, an end-to-end number
@@ -200,8 +201,10 @@ def main():
     # ------------------------------------------------------------------ inputs (seeded, synthetic)
     d = si.config1(B=N_INPUTS)
     dt = si.BF16
+    # Cold-HBM rule: every call of a replay must miss L2, also at the highest sparsity, where a call touches only
+    # (1 - s) of its weight copy.  So the copies are sized on the smallest touched footprint: R * (1 - s_max) * |W| >= 4 * L2.
     l2 = torch.cuda.get_device_properties(local_rank).L2_cache_size
-    R = max(2, -(-4 * l2 // (K * N * 2)))
+    R = max(2, int(np.ceil(4 * l2 / ((1.0 - max(SPARSITIES)) * K * N * 2))))
     W0 = si.as_torch(d["W"], dt).cuda()
     Ws = [W0] + [W0.clone() for _ in range(R - 1)]
     xs = si.as_torch(d["x"], dt).cuda()
@@ -286,7 +289,7 @@ def main():
 
     g_step, step_bytes = capture(lambda: sparse_calls(SPARSITIES, [0]))
     calls_per_step = len(SPARSITIES) * R
-    launches_per_step = 2 * calls_per_step
+    launches_per_step = calls_per_step  # one fused kernel per call
 
     # ------------------------------------------------------------------ timed region: K steps, device time, max over ranks
     with torch.cuda.stream(stream):
@@ -370,7 +373,7 @@ def main():
         "config": {
             "workload": "llama2_7b_down_proj_bf16_b1 (K=11008,N=4096), sparsity targets 50/65/80%",
             "weights": "bf16", "accumulate": "f32", "batch": 1, "calls_per_step": calls_per_step,
-            "l2_policy": "inputs larger than L2: %d weight copies (%.0f MB) rotated, %d input vectors" % (R, R * K * N * 2 / 1e6, N_INPUTS),
+            "l2_policy": "inputs larger than L2: %d weight copies (%.0f MB) rotated so that even the sparsest call pattern touches >= 4x L2 per cycle, %d input vectors" % (R, R * K * N * 2 / 1e6, N_INPUTS),
             "launch": "CUDA graph replay of one step", "parallelism": "replicas only" if world > 1 else "single GPU",
         },
         "us_per_call": {("%d%%" % round(100 * s)): round(detail[s]["us_per_call"], 3) for s in SPARSITIES},
@@ -381,7 +384,7 @@ def main():
         "calibrate_ms": {("%d%%" % round(100 * s)): round(cal_ms[s], 3) for s in SPARSITIES},
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "traffic": None, "peak_kind": peak_kind, "frac_of_nominal_8000": achieved / 8000.0,
-                     "kernel": "gemv_kernel (gather-GEMV); time per call includes the compaction kernel"},
+                     "kernel": "fc_kernel (fused threshold + compaction + gather-GEMV + cluster reduction), one launch per call"},
         "e2e": {"value": e2e_value, "unit": "GB/s", "h2d_bytes_per_step": calls_per_step * K * 2,
                 "d2h_bytes_per_step": calls_per_step * N * 4, "steps": e2e_steps},
         "gpu_launches": launches_per_step * args.steps,
@@ -392,7 +395,7 @@ def main():
         cores = os.cpu_count() or 1
         cal_o = {s: (cal[s][0].cpu().numpy(), float(cal[s][1].item()), cal[s][2].cpu().numpy()) for s in SPARSITIES}
         tot_t, tot_b, n = 0.0, 0, 0
-        while tot_t < 10.0 and n < 200:
+        while tot_t < 10.0 and n < 2000:
             t, b = oracle_step(d, cal_o, d["x"][3 * (n % 20):], cores)
             tot_t += t
             tot_b += b
