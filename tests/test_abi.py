@@ -57,7 +57,7 @@ def test_argument_validation_returns_codes(L):
     assert call(x=None) == 1                      # SCAP_ERR_INVALID_ARG
     assert call(tau=None) == 1
     assert call(B=0) == 2 and call(B=17) == 2     # SCAP_ERR_SHAPE
-    assert call(K=0) == 2 and call(K=131073) == 2
+    assert call(K=0) == 2 and call(K=(1 << 20) + 1) == 2
     assert call(dt=7) == 3                        # SCAP_ERR_DTYPE
     assert call(N=60) == 4 and call(W=P + 2) == 4  # SCAP_ERR_ALIGN
     assert call(wsb=ws - 1) == 5                  # SCAP_ERR_WORKSPACE
