@@ -153,6 +153,30 @@ scap_status scap_glu_ffn(const void *h, const void *Wgu, const void *Wd, const f
                          int *nnz1_out, uint32_t *idx2_out, int *nnz2_out, void *ws, size_t ws_bytes,
                          scap_stream_t stream);
 
+/* scap_glu_ffn without a workspace argument (the paper has no counterpart; this is a deployment aid).
+ *
+ * Some callers must not allocate device memory on the decode path: a serving process that handed all
+ * free HBM to its KV-cache pool at start-up, a plug-in that runs inside a host framework's memory
+ * budget, or code on a latency-critical path where cudaMalloc's implicit device synchronisation is not
+ * acceptable.  For them the scratch of the SwiGLU block (the fp32 intermediate z[B,F] plus a few mask
+ * words) lives in a fixed array inside the library image instead of a caller workspace.  The call
+ * performs no cudaMalloc / cudaFree and uses no allocating library routine.
+ *
+ *   - Capacity: scap_glu_static_capacity() bytes (2 MiB), held by every GPU that loads the library
+ *     until the process exits.  A shape needing more (scap_glu_workspace(B, D, F) > capacity, i.e.
+ *     roughly B * F > 520000) is rejected with SCAP_ERR_WORKSPACE and nothing is enqueued.
+ *   - The first call on each device looks up the array's device address (cudaGetSymbolAddress) and
+ *     caches it; make that first call outside any stream capture.
+ *   - All calls on a device share the one array.  It keeps whatever the last call left there; nothing
+ *     needs clearing because each call writes every word before reading it.  Two calls that overlap
+ *     on the GPU (different streams, or graphs replayed concurrently) race on it: keep them on one
+ *     stream or order them with events.
+ *   - Arguments, results and error codes are otherwise those of scap_glu_ffn (no idx/nnz outputs).   */
+size_t scap_glu_static_capacity(void);
+scap_status scap_glu_ffn_static(const void *h, const void *Wgu, const void *Wd, const float *m1, const float *tau1,
+                                const float *bgu_fused, const float *m2, const float *tau2, const float *bd_fused,
+                                float *y, int B, int D, int F, scap_dtype dt, float *z_out, scap_stream_t stream);
+
 /* ------------------------------------------------------------------------------------------
  * Mixture-of-experts FFN layer (the paper applies SCAP to Mixtral-8x7B, Table 4; it does not
  * describe the router, so the convention is this library's): p = softmax(logits[b, 0..E-1]),

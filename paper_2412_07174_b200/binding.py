@@ -10,8 +10,8 @@ __all__ = [
     "SCAP_F16", "SCAP_BF16", "ScapError", "lib", "lib_path", "status_string", "scap_version", "scap_tune",
     "scap_calibrate_workspace", "scap_calibrate", "scap_fold_bias_workspace", "scap_fold_bias",
     "scap_fc_workspace", "scap_sparse_fc", "scap_dense_fc", "scap_fc_host_workspace", "scap_sparse_fc_host",
-    "scap_glu_workspace", "scap_glu_ffn", "scap_moe_workspace", "scap_moe_ffn", "ScapExpert", "dtype_of",
-    "EXPORTS",
+    "scap_glu_workspace", "scap_glu_ffn", "scap_glu_static_capacity", "scap_glu_ffn_static", "scap_moe_workspace",
+    "scap_moe_ffn", "ScapExpert", "dtype_of", "EXPORTS",
 ]
 
 SCAP_F16, SCAP_BF16 = 0, 1
@@ -22,7 +22,7 @@ EXPORTS = [
     "scap_status_string", "scap_version", "scap_tune", "scap_calibrate_workspace", "scap_calibrate",
     "scap_fold_bias_workspace", "scap_fold_bias", "scap_fc_workspace", "scap_sparse_fc", "scap_dense_fc",
     "scap_fc_host_workspace", "scap_sparse_fc_host", "scap_glu_workspace", "scap_glu_ffn",
-    "scap_moe_workspace", "scap_moe_ffn",
+    "scap_glu_static_capacity", "scap_glu_ffn_static", "scap_moe_workspace", "scap_moe_ffn",
 ]
 
 
@@ -82,6 +82,10 @@ def lib():
     L.scap_glu_workspace.restype = sz
     L.scap_glu_ffn.argtypes = [vp] * 10 + [i, i, i, i] + [vp] * 5 + [vp, sz, vp]
     L.scap_glu_ffn.restype = i
+    L.scap_glu_static_capacity.argtypes = []
+    L.scap_glu_static_capacity.restype = sz
+    L.scap_glu_ffn_static.argtypes = [vp] * 10 + [i, i, i, i] + [vp, vp]
+    L.scap_glu_ffn_static.restype = i
     L.scap_moe_workspace.argtypes = [i, i, i, i, i]
     L.scap_moe_workspace.restype = sz
     L.scap_moe_ffn.argtypes = [vp, vp, C.POINTER(ScapExpert), i, i, vp, i, i, i, i, vp, vp, vp, sz, vp]
@@ -203,6 +207,19 @@ def scap_glu_ffn(h, Wgu, Wd, m1, tau1, bgu_fused, m2, tau2, bd_fused, y, ws, z_o
     _check(lib().scap_glu_ffn(_ptr(h), _ptr(Wgu), _ptr(Wd), _ptr(m1), _ptr(tau1), _ptr(bgu_fused), _ptr(m2), _ptr(tau2),
                               _ptr(bd_fused), _ptr(y), B, D, F, dtype_of(Wgu), _ptr(z_out), _ptr(idx1_out), _ptr(nnz1_out),
                               _ptr(idx2_out), _ptr(nnz2_out), p, n, _stream(stream)), "scap_glu_ffn")
+
+
+def scap_glu_static_capacity() -> int:
+    return lib().scap_glu_static_capacity()
+
+
+def scap_glu_ffn_static(h, Wgu, Wd, m1, tau1, bgu_fused, m2, tau2, bd_fused, y, z_out=None, stream=None) -> None:
+    """scap_glu_ffn for callers that may not allocate: the scratch is a fixed array inside the library (see scap.h)."""
+    B, D = h.shape
+    F = Wd.shape[0]
+    _check(lib().scap_glu_ffn_static(_ptr(h), _ptr(Wgu), _ptr(Wd), _ptr(m1), _ptr(tau1), _ptr(bgu_fused), _ptr(m2),
+                                     _ptr(tau2), _ptr(bd_fused), _ptr(y), B, D, F, dtype_of(Wgu), _ptr(z_out),
+                                     _stream(stream)), "scap_glu_ffn_static")
 
 
 def scap_moe_workspace(B: int, D: int, F: int, E: int, top_k: int) -> int:

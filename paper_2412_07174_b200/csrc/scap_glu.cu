@@ -83,3 +83,62 @@ scap_status scap_glu_ffn(const void *h, const void *Wgu, const void *Wd, const f
 }
 
 }  // extern "C"
+
+// ------------------------------------------------------------------------------------------------
+// SwiGLU block for callers that cannot allocate device memory.
+//
+// The intermediate z and the mask words of scap_glu_ffn normally live in a caller-provided workspace.
+// Here they live in the file-scope array below, which is part of the library image: every GPU that
+// loads the library holds these 2 MiB until the process exits.  The array's name is only a host-side
+// handle; kernels need its device address, which is looked up once per device with
+// cudaGetSymbolAddress (with that device current) and cached.
+// ------------------------------------------------------------------------------------------------
+namespace scap {
+
+constexpr size_t GLU_STATIC_BYTES = (size_t)2 << 20;
+static __device__ __align__(256) unsigned char g_glu_static_scratch[GLU_STATIC_BYTES];
+
+static scap_status glu_static_address(unsigned char **out) {
+    static unsigned char *cached[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) {
+        cudaGetLastError();
+        return SCAP_ERR_CUDA;
+    }
+    if (dev >= 0 && dev < 64 && cached[dev]) {
+        *out = cached[dev];
+        return SCAP_OK;
+    }
+    void *p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_glu_static_scratch) != cudaSuccess || p == nullptr) {
+        cudaGetLastError();
+        return SCAP_ERR_CUDA;
+    }
+    if (dev >= 0 && dev < 64) cached[dev] = static_cast<unsigned char *>(p);
+    *out = static_cast<unsigned char *>(p);
+    return SCAP_OK;
+}
+
+}  // namespace scap
+
+extern "C" {
+
+size_t scap_glu_static_capacity(void) { return GLU_STATIC_BYTES; }
+
+scap_status scap_glu_ffn_static(const void *h, const void *Wgu, const void *Wd, const float *m1, const float *tau1,
+                                const float *bgu_fused, const float *m2, const float *tau2, const float *bd_fused, float *y,
+                                int B, int D, int F, scap_dtype dt, float *z_out, scap_stream_t stream) {
+    const size_t need = scap_glu_workspace(B, D, F);
+    if (need == 0) return SCAP_ERR_SHAPE;
+    if (need > GLU_STATIC_BYTES) return SCAP_ERR_WORKSPACE;  // B * F too large for the built-in scratch
+    scap_status st = check_device();
+    if (st != SCAP_OK) return st;
+    unsigned char *scratch = nullptr;
+    if ((st = glu_static_address(&scratch)) != SCAP_OK) return st;
+    // Every scratch word that is read is written earlier in the same call (z by the gate|up kernel before the
+    // down kernel reads it), so nothing has to be cleared even though the array keeps the previous call's data.
+    return scap_glu_ffn(h, Wgu, Wd, m1, tau1, bgu_fused, m2, tau2, bd_fused, y, B, D, F, dt, z_out, nullptr, nullptr, nullptr,
+                        nullptr, scratch, GLU_STATIC_BYTES, stream);
+}
+
+}  // extern "C"
