@@ -171,6 +171,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--detail", action="store_true", help="also print a per-sparsity table to stderr")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--copies", type=int, default=0,
+                    help="number of weight copies to rotate (default: enough for the cold-HBM rule); a small value keeps "
+                         "device memory low for a profiler capture and is recorded in config.l2_policy")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -205,6 +208,8 @@ def main():
     # (1 - s) of its weight copy.  So the copies are sized on the smallest touched footprint: R * (1 - s_max) * |W| >= 4 * L2.
     l2 = torch.cuda.get_device_properties(local_rank).L2_cache_size
     R = max(2, int(np.ceil(4 * l2 / ((1.0 - max(SPARSITIES)) * K * N * 2))))
+    if args.copies > 0:
+        R = args.copies
     W0 = si.as_torch(d["W"], dt).cuda()
     Ws = [W0] + [W0.clone() for _ in range(R - 1)]
     xs = si.as_torch(d["x"], dt).cuda()
