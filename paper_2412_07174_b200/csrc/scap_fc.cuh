@@ -167,7 +167,7 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
         float xv[PU][BT], mk[PU];
 #pragma unroll
         for (int p = 0; p < PU; ++p) {
-            const int j = warp * PU + p;
+            const int j = p * FC_WARPS + warp;
             const int k = (s + S * (j0 + j)) * 32 + lane;
             mk[p] = a.m ? ld_nc(a.m + ((j < nj && k < K) ? k : 0)) : 0.0f;
         }
@@ -177,7 +177,7 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
         }
 #pragma unroll
         for (int p = 0; p < PU; ++p) {
-            const int j = warp * PU + p;
+            const int j = p * FC_WARPS + warp;
             const int k = (s + S * (j0 + j)) * 32 + lane;
             const int kk = (j < nj && k < K) ? k : 0;
 #pragma unroll
@@ -195,7 +195,7 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
         unsigned bal[PU];
 #pragma unroll
         for (int p = 0; p < PU; ++p) {
-            const int j = warp * PU + p;
+            const int j = p * FC_WARPS + warp;
             const int k = (s + S * (j0 + j)) * 32 + lane;
             const bool ok = j < nj && k < K;
             uint32_t m_ = 0;
@@ -212,11 +212,12 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
             km[p] = m_;
             bal[p] = __ballot_sync(0xffffffffu, m_ != 0);
         }
-        {   // lane p publishes the word of chunk warp*PU + p
+        {   // lane p publishes the word of this warp's p-th chunk (chunk index p * FC_WARPS + warp: the chunks of
+            // a fill are dealt round-robin to the warps so that every warp has about the same number)
             unsigned mine = 0;
 #pragma unroll
             for (int p = 0; p < PU; ++p) mine = lane == p ? bal[p] : mine;
-            const int j = warp * PU + lane;
+            const int j = lane * FC_WARPS + warp;
             if (lane < PU && j < nj) {
                 s_bits[j] = mine;
                 if (MODE == MODE_GATHER && a.bits && tile == 0) a.bits[s + S * (j0 + j)] = mine;
@@ -235,7 +236,7 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
             }
 #pragma unroll
             for (int p = 0; p < PU; ++p) {
-                const int j = warp * PU + p;
+                const int j = p * FC_WARPS + warp;
                 int o = 0;
 #pragma unroll
                 for (int q = 0; q < (CAPC + 31) / 32; ++q) o += __reduce_add_sync(0xffffffffu, (q * 32 + lane < j) ? c_lo[q] : 0);
@@ -246,7 +247,7 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
 #pragma unroll
         for (int p = 0; p < PU; ++p) {
             if (km[p]) {
-                const int j = warp * PU + p;
+                const int j = p * FC_WARPS + warp;
                 const int pos = my_off[p] + __popc(bal[p] & ((1u << lane) - 1u));
                 s_k[pos] = (uint32_t)((s + S * (j0 + j)) * 32 + lane);
 #pragma unroll
