@@ -163,6 +163,209 @@ def run_reference(args, rank):
     print(json.dumps(line), flush=True)
 
 
+# ---------------------------------------------------------------------------------------------------------
+# --suite: the other workload descriptions (SwiGLU block, MoE layer, sparsity/batch sweep, calibration).
+# Same timing protocol as the headline line (CUDA-graph replay, device events, cold-HBM rotation); results go
+# to stdout as one JSON object per line and are not part of the one-line contract of the default run.
+# ---------------------------------------------------------------------------------------------------------
+
+def _time_graph(torch, stream, fn, reps=30, warm=5):
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(stream):
+        fn()
+        stream.synchronize()
+        with torch.cuda.graph(g, stream=stream):
+            fn()
+        for _ in range(warm):
+            g.replay()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        stream.synchronize()
+        e0.record(stream)
+        for _ in range(reps):
+            g.replay()
+        e1.record(stream)
+        stream.synchronize()
+    return e0.elapsed_time(e1) / reps * 1e3  # us per replay
+
+
+def suite_sweep(torch, scap, peak, shapes, sparsities, batches, out):
+    """Config 4: sparse FC over sparsity x batch x shape, bf16, Laplace-around-mode inputs, vs the dense GEMV."""
+    stream = torch.cuda.Stream()
+    l2 = torch.cuda.get_device_properties(0).L2_cache_size
+    for (Kk, Nn) in shapes:
+        d = si.config4_fc(Kk, Nn, 16 * 8, T_calib=2048)
+        W0 = si.as_torch(d["W"], si.BF16).cuda()
+        xc = si.as_torch(d["x_calib"], si.BF16).cuda()
+        xs = si.as_torch(d["x"], si.BF16).cuda()          # 128 rows = 8 batches of 16
+        Rmax = int(np.ceil(4 * l2 / (0.1 * Kk * Nn * 2)))
+        Ws = [W0] + [W0.clone() for _ in range(Rmax - 1)]
+        cws = torch.empty(scap.scap_calibrate_workspace(2048, Kk, NBINS), dtype=torch.uint8, device="cuda")
+        m = torch.empty(Kk, dtype=torch.float32, device="cuda")
+        bf = torch.empty(Nn, dtype=torch.float32, device="cuda")
+        nnz = torch.zeros(1, dtype=torch.int32, device="cuda")
+        for B in batches:
+            ws = torch.empty(scap.scap_fc_workspace(B, Kk, Nn), dtype=torch.uint8, device="cuda")
+            y = torch.empty((B, Nn), dtype=torch.float32, device="cuda")
+            xb = [xs[i * 16:i * 16 + B] for i in range(8)]
+            Rd = max(2, int(np.ceil(4 * l2 / (Kk * Nn * 2))))
+            t_dense = _time_graph(torch, stream, lambda: [scap.scap_dense_fc(xb[r % 8], Ws[r], None, y, ws) for r in range(Rd)]) / Rd
+            dense_b = Kk * Nn * 2 + B * Kk * 2 + 4 * Nn + 4 * B * Nn
+            for s in sparsities:
+                tau = torch.empty(1, dtype=torch.float32, device="cuda")
+                scap.scap_calibrate(xc, s, NBINS, m, tau, cws)
+                scap.scap_fold_bias(W0, m, None, bf, ws)
+                kept = []
+                for i in range(8):
+                    scap.scap_sparse_fc(xb[i], W0, m, tau, bf, y, ws, nnz_out=nnz)
+                    kept.append(int(nnz.item()))
+                rho = float(np.mean(kept)) / Kk
+                R = max(2, min(Rmax, int(np.ceil(4 * l2 / (max(rho, 0.1) * Kk * Nn * 2)))))
+                t = _time_graph(torch, stream, lambda: [scap.scap_sparse_fc(xb[r % 8], Ws[r], m, tau, bf, y, ws) for r in range(R)]) / R
+                nb = float(np.mean(kept)) * Nn * 2 + B * Kk * 2 + 4 * Kk + 4 + 4 * Nn + 4 * B * Nn
+                rec = {"suite": "sweep", "K": Kk, "N": Nn, "B": B, "sparsity_target": s, "union_kept_fraction": round(rho, 4),
+                       "us_per_call": round(t, 3), "gbs": round(nb / t / 1e3, 1), "frac_of_measured_peak": round(nb / t / 1e3 / peak, 3),
+                       "dense_us": round(t_dense, 3), "dense_gbs": round(dense_b / t_dense / 1e3, 1), "speedup_vs_dense": round(t_dense / t, 3),
+                       "weight_copies": R}
+                out(rec)
+        del Ws
+        torch.cuda.empty_cache()
+
+
+def suite_calibrate(torch, scap, out):
+    """Config 4's timed calibration: 2048 tokens x 14336 channels, 2048 bins, plus the tau quantile."""
+    T, Kk = 2048, 14336
+    d = si.laplace_fc(4, Kk, 8, si.BF16, T, 1, with_bias=False)
+    xc = si.as_torch(d["x_calib"], si.BF16).cuda()
+    cws = torch.empty(scap.scap_calibrate_workspace(T, Kk, NBINS), dtype=torch.uint8, device="cuda")
+    m = torch.empty(Kk, dtype=torch.float32, device="cuda")
+    tau = torch.empty(1, dtype=torch.float32, device="cuda")
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
+    times = []
+    for _ in range(8):
+        flush.fill_(1)  # L2 flush: the calibration tensor (58.7 MB) would otherwise be L2-resident from the last run
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        scap.scap_calibrate(xc, 0.6, NBINS, m, tau, cws)
+        e1.record()
+        torch.cuda.synchronize()
+        times.append(e0.elapsed_time(e1) * 1e3)
+    t = float(np.median(times[2:]))
+    out({"suite": "calibrate", "T": T, "K": Kk, "nbins": NBINS, "sparsity": 0.6, "us": round(t, 1),
+         "compulsory_bytes": T * Kk * 2, "gbs_on_compulsory_bytes": round(T * Kk * 2 / t / 1e3, 1), "passes_over_input": 5,
+         "l2": "flushed before each run"})
+
+
+def suite_glu(torch, scap, peak, out):
+    """Config 2: full Llama-2-7B-shaped SwiGLU block, batch 1 / 4 / 8, 40 % / 70 % targets."""
+    D, F = 4096, 11008
+    g = si.config2(B=64)
+    dt = si.BF16
+    stream = torch.cuda.Stream()
+    l2 = torch.cuda.get_device_properties(0).L2_cache_size
+    Wgu0, Wd0 = si.as_torch(g["Wgu"], dt).cuda(), si.as_torch(g["Wd"], dt).cuda()
+    hc, hs = si.as_torch(g["h_calib"], dt).cuda(), si.as_torch(g["h"], dt).cuda()
+    ws = torch.empty(max(scap.scap_glu_workspace(16, D, F), scap.scap_calibrate_workspace(1024, F, NBINS)), dtype=torch.uint8, device="cuda")
+    m1 = torch.empty(D, dtype=torch.float32, device="cuda")
+    tau1 = torch.empty(1, dtype=torch.float32, device="cuda")
+    m2 = torch.empty(F, dtype=torch.float32, device="cuda")
+    tau2 = torch.zeros(1, dtype=torch.float32, device="cuda")
+    b1 = torch.empty(2 * F, dtype=torch.float32, device="cuda")
+    b2 = torch.empty(D, dtype=torch.float32, device="cuda")
+    scap.scap_calibrate(hc, 0.4, NBINS, m1, tau1, ws)
+    scap.scap_fold_bias(Wgu0, m1, None, b1, ws)
+    # stage-2 calibration set: z of the calibration tokens from the product path (16 rows per call), rounded to bf16
+    zc = torch.empty((1024, F), dtype=torch.float32, device="cuda")
+    ytmp = torch.empty((16, D), dtype=torch.float32, device="cuda")
+    for i in range(0, 1024, 16):
+        scap.scap_glu_ffn(hc[i:i + 16], Wgu0, Wd0, m1, tau1, b1, None, tau2, None, ytmp, ws, z_out=zc[i:i + 16])
+    scap.scap_calibrate(zc.to(torch.bfloat16), 0.7, NBINS, m2, tau2, ws)
+    scap.scap_fold_bias(Wd0, m2, None, b2, ws)
+    R = max(2, int(np.ceil(4 * l2 / (0.6 * D * 2 * F * 2 + 0.3 * F * D * 2))))
+    Wgus = [Wgu0] + [Wgu0.clone() for _ in range(R - 1)]
+    Wds = [Wd0] + [Wd0.clone() for _ in range(R - 1)]
+    n1 = torch.zeros(1, dtype=torch.int32, device="cuda")
+    n2 = torch.zeros(1, dtype=torch.int32, device="cuda")
+    for B in (1, 4, 8):
+        y = torch.empty((B, D), dtype=torch.float32, device="cuda")
+        hb = [hs[i * 8:i * 8 + B] for i in range(8)]
+        k1, k2 = [], []
+        for i in range(8):
+            scap.scap_glu_ffn(hb[i], Wgu0, Wd0, m1, tau1, b1, m2, tau2, b2, y, ws, nnz1_out=n1, nnz2_out=n2)
+            k1.append(int(n1.item()))
+            k2.append(int(n2.item()))
+        t = _time_graph(torch, stream, lambda: [scap.scap_glu_ffn(hb[r % 8], Wgus[r], Wds[r], m1, tau1, b1, m2, tau2, b2, y, ws) for r in range(R)]) / R
+        nb = np.mean(k1) * 2 * F * 2 + np.mean(k2) * D * 2 + B * D * 2 + 4 * D + 4 * 2 * F + 4 * F + 4 * D + 4 * B * D + 8
+        dense_b = D * 2 * F * 2 + F * D * 2
+        out({"suite": "glu", "D": D, "F": F, "B": B, "targets": [0.4, 0.7], "kept_fraction_stage1": round(float(np.mean(k1)) / D, 4),
+             "kept_fraction_stage2": round(float(np.mean(k2)) / F, 4), "us_per_call": round(t, 2), "gbs": round(nb / t / 1e3, 1),
+             "frac_of_measured_peak": round(nb / t / 1e3 / peak, 3), "dense_weight_bytes": dense_b,
+             "ffn_sparsity_paper_accounting": round(1 - (2 * np.mean(k1) / D + np.mean(k2) / F) / 3, 4), "weight_copies": R, "kernels_per_call": 2})
+
+
+def suite_moe(torch, scap, peak, out):
+    """Config 3: Mixtral-8x7B-shaped MoE layer, 8 experts, top-2, batch 1..4, 40 % / 60 % targets."""
+    D, F, E = 4096, 14336, 8
+    dt = si.BF16
+    stream = torch.cuda.Stream()
+    mo = si.moe_layer(3, D, F, E, dt, 2048, 64)
+    ws = torch.empty(max(scap.scap_moe_workspace(4, D, F, E, 2), scap.scap_glu_workspace(16, D, F),
+                         scap.scap_calibrate_workspace(2048, F, NBINS)), dtype=torch.uint8, device="cuda")
+    experts = []
+    ytmp = torch.empty((16, D), dtype=torch.float32, device="cuda")
+    for p in mo["experts"]:
+        Wgu, Wd = si.as_torch(p["Wgu"], dt).cuda(), si.as_torch(p["Wd"], dt).cuda()
+        hc = si.as_torch(p["h_calib"], dt).cuda()
+        t = dict(Wgu=Wgu, Wd=Wd, m1=torch.empty(D, dtype=torch.float32, device="cuda"), tau1=torch.empty(1, dtype=torch.float32, device="cuda"),
+                 bgu_fused=torch.empty(2 * F, dtype=torch.float32, device="cuda"), m2=torch.empty(F, dtype=torch.float32, device="cuda"),
+                 tau2=torch.zeros(1, dtype=torch.float32, device="cuda"), bd_fused=torch.empty(D, dtype=torch.float32, device="cuda"))
+        scap.scap_calibrate(hc, 0.4, NBINS, t["m1"], t["tau1"], ws)
+        scap.scap_fold_bias(Wgu, t["m1"], None, t["bgu_fused"], ws)
+        zc = torch.empty((512, F), dtype=torch.float32, device="cuda")
+        for i in range(0, 512, 16):
+            scap.scap_glu_ffn(hc[i:i + 16], Wgu, Wd, t["m1"], t["tau1"], t["bgu_fused"], None, t["tau2"], None, ytmp, ws, z_out=zc[i:i + 16])
+        scap.scap_calibrate(zc.to(torch.bfloat16), 0.6, NBINS, t["m2"], t["tau2"], ws)
+        scap.scap_fold_bias(Wd, t["m2"], None, t["bd_fused"], ws)
+        experts.append(t)
+    hs = si.as_torch(mo["h"], dt).cuda()
+    logits = torch.from_numpy(mo["logits"]).cuda()
+    for B in (1, 2, 4):
+        y = torch.empty((B, D), dtype=torch.float32, device="cuda")
+        hb = [hs[i * 4:i * 4 + B] for i in range(16)]
+        lb = [logits[i * 4:i * 4 + B].contiguous() for i in range(16)]
+        t = _time_graph(torch, stream, lambda: [scap.scap_moe_ffn(hb[r], lb[r], experts, 2, y, ws) for r in range(16)]) / 16
+        sel = [len(set(torch.topk(lb[r], 2, dim=1).indices.flatten().tolist())) for r in range(16)]
+        out({"suite": "moe", "D": D, "F": F, "E": E, "top_k": 2, "B": B, "targets": [0.4, 0.6], "us_per_call": round(t, 2),
+             "distinct_experts_per_call": round(float(np.mean(sel)), 2), "dense_bytes_per_expert": D * 2 * F * 2 + F * D * 2,
+             "gbs_vs_dense_expert_bytes": round(float(np.mean(sel)) * (D * 2 * F * 2 + F * D * 2) / t / 1e3, 1), "kernels_per_call": 4})
+
+
+def run_suite(args):
+    import torch
+    import paper_2412_07174_b200 as scap
+    scap.lib()
+    torch.cuda.set_device(0)
+    peak, _ = measured_peaks()
+
+    def out(rec):
+        print(json.dumps(rec), flush=True)
+
+    which = args.suite
+    if which in ("calibrate", "all"):
+        suite_calibrate(torch, scap, out)
+    if which in ("glu", "all"):
+        suite_glu(torch, scap, peak, out)
+    if which in ("sweep", "all", "sweep-small"):
+        shapes = [(4096, 4096), (4096, 11008), (11008, 4096), (14336, 4096)]
+        if which == "sweep-small":
+            suite_sweep(torch, scap, peak, [(11008, 4096)], (0.0, 0.5, 0.8), (1, 4, 8, 16), out)
+        else:
+            suite_sweep(torch, scap, peak, shapes, (0.0, 0.25, 0.5, 0.6, 0.7, 0.8, 0.9), (1, 2, 4, 8, 16), out)
+    if which in ("moe", "all"):
+        suite_moe(torch, scap, peak, out)
+
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -171,6 +374,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--detail", action="store_true", help="also print a per-sparsity table to stderr")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--suite", default="", choices=["", "calibrate", "glu", "moe", "sweep", "sweep-small", "all"],
+                    help="run the other workload descriptions instead of the headline line (one JSON object per line)")
     ap.add_argument("--copies", type=int, default=0,
                     help="number of weight copies to rotate (default: enough for the cold-HBM rule); a small value keeps "
                          "device memory low for a profiler capture and is recorded in config.l2_policy")
@@ -183,6 +388,10 @@ def main():
 
     if args.impl == "reference":
         run_reference(args, rank)
+        return
+    if args.suite:
+        if rank == 0:
+            run_suite(args)
         return
 
     import torch
