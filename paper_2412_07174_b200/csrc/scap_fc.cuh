@@ -85,6 +85,96 @@ __device__ __forceinline__ float load_bias(const FcArgs &a, int n) {
     return bv;
 }
 
+// One round of the reduction over NRED row groups (in group order) for RBX batch rows starting at b0: thread i
+// sums column c of row rb from s_red[g][rb][c] and pushes the result into the shared memory of the cluster rank
+// that owns the column (slot = this rank s).  EPI_GLU: owner by pair index j = c mod HALF; the gate and up
+// values of a pair sit side by side in the owner's slot.
+template <int BT, int EPI, int TNT, int NRED, int RBX>
+__device__ __forceinline__ void reduce_push_round(const float *__restrict__ s_red, int b0, int B, int s, int per,
+                                                  float *const (&owner)[MAX_CLUSTER]) {
+    constexpr int HALF = TNT / 2;
+    for (int i = threadIdx.x; i < RBX * TNT; i += FC_THREADS) {
+        const int rb = i / TNT, c = i - rb * TNT, b = b0 + rb;
+        float v = 0.0f;
+#pragma unroll
+        for (int g = 0; g < NRED; ++g) v += s_red[(g * RBX + rb) * TNT + c];
+        if (b < B) {
+            int r, slot;
+            if constexpr (EPI == EPI_GLU) {
+                const int j = c % HALF, hf = c / HALF;
+                r = j / per;
+                slot = ((s * BT + b) * 2 + hf) * per + (j - r * per);
+            } else {
+                r = c / per;
+                slot = (s * BT + b) * per + (c - r * per);
+            }
+#pragma unroll
+            for (int q = 0; q < MAX_CLUSTER; ++q)
+                if (q == r) owner[q][slot] = v;
+        }
+    }
+}
+
+// After the cluster barrier: every rank adds the S partials of its columns in rank order, adds the bias (or forms
+// z = up * silu(gate)) and writes the result.
+template <bool BF16, int BT, int EPI, int TNT>
+__device__ __forceinline__ void finish_columns(const FcArgs &a, int tile, int s, int per, const float *__restrict__ s_gather,
+                                               const float (&bias0)[2], const float (&bias1)[2]) {
+    constexpr int HALF = TNT / 2;
+    const int B = a.B, S = a.S, tid = threadIdx.x;
+    for (int it = 0; tid + it * FC_THREADS < per * B; ++it) {
+        const int i = tid + it * FC_THREADS;
+        const int b = i / per, c = i - b * per;
+        const int row = a.out_rows ? a.out_rows[b] : b;
+        if constexpr (EPI == EPI_BIAS) {
+            const int n = tile * TNT + s * per + c;
+            if (n < a.Nh) {
+                float v = it == 0 ? bias0[0] : it == 1 ? bias0[1] : load_bias<BF16>(a, n);
+#pragma unroll
+                for (int q = 0; q < MAX_CLUSTER; ++q)
+                    if (q < S) v += s_gather[(q * BT + b) * per + c];
+                a.y[(size_t)row * a.y_ld + n] = v;
+            }
+        } else {
+            const int F = a.Nh, f = tile * HALF + s * per + c;
+            if (f < F) {
+                float g = it == 0 ? bias0[0] : it == 1 ? bias0[1] : (a.bias ? __ldg(a.bias + f) : 0.0f);
+                float u = it == 0 ? bias1[0] : it == 1 ? bias1[1] : (a.bias ? __ldg(a.bias + F + f) : 0.0f);
+#pragma unroll
+                for (int q = 0; q < MAX_CLUSTER; ++q)
+                    if (q < S) {
+                        g += s_gather[((q * BT + b) * 2 + 0) * per + c];
+                        u += s_gather[((q * BT + b) * 2 + 1) * per + c];
+                    }
+                const float z = u * (g / (1.0f + expf(-g)));  // up * silu(gate)
+                a.y[(size_t)row * a.y_ld + f] = z;
+                if (a.z_copy) a.z_copy[(size_t)b * F + f] = z;
+            }
+        }
+    }
+}
+
+// Bias of the columns this rank finishes, fetched at kernel start so that the load is off the critical path.
+template <bool BF16, int EPI, int TNT>
+__device__ __forceinline__ void prefetch_bias(const FcArgs &a, int tile, int s, int per, float (&bias0)[2], float (&bias1)[2]) {
+    constexpr int HALF = TNT / 2;
+#pragma unroll
+    for (int it = 0; it < 2; ++it) {
+        bias0[it] = bias1[it] = 0.0f;
+        const int i = threadIdx.x + it * FC_THREADS;
+        if (i < per * a.B) {
+            const int c = i % per;
+            if constexpr (EPI == EPI_GLU) {
+                const int f = tile * HALF + s * per + c;
+                if (f < a.Nh && a.bias) { bias0[it] = __ldg(a.bias + f); bias1[it] = __ldg(a.bias + a.Nh + f); }
+            } else {
+                const int n = tile * TNT + s * per + c;
+                if (n < a.Nh) bias0[it] = load_bias<BF16>(a, n);
+            }
+        }
+    }
+}
+
 // Body for column tile `tile` and cluster rank `s`; every thread of every CTA of the cluster calls it.
 // TNT = columns per CTA (256 or 128): a row segment is TNT/8 lanes wide, so a warp streams 1 or 2 rows per load.
 // With wait_inside the body itself waits for the previous kernel in the stream, and does so as late as it can:
@@ -123,24 +213,10 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
     const unsigned char *Wb = reinterpret_cast<const unsigned char *>(a.W) + (size_t)col * 2;
     const size_t row_bytes = (size_t)a.ldw * 2;
 
-    // Columns this rank finishes after the cluster exchange, and their bias, fetched now so that the
-    // load is off the critical path.  EPI_BIAS: `per` columns; EPI_GLU: `per` gate/up pairs.
+    // columns (EPI_GLU: gate/up pairs) this rank finishes after the cluster exchange
     const int per = (EPI == EPI_GLU ? HALF : TNT) / S;
-    float bias0[2] = {0.0f, 0.0f}, bias1[2] = {0.0f, 0.0f};
-#pragma unroll
-    for (int it = 0; it < 2; ++it) {
-        const int i = tid + it * NT;
-        if (i < per * B) {
-            const int c = i % per;
-            if constexpr (EPI == EPI_GLU) {
-                const int f = tile * HALF + s * per + c;
-                if (f < a.Nh && a.bias) { bias0[it] = __ldg(a.bias + f); bias1[it] = __ldg(a.bias + a.Nh + f); }
-            } else {
-                const int n = tile * TNT + s * per + c;
-                if (n < a.Nh) bias0[it] = load_bias<BF16>(a, n);
-            }
-        }
-    }
+    float bias0[2], bias1[2];
+    prefetch_bias<BF16, EPI, TNT>(a, tile, s, per, bias0, bias1);
 
     float acc[BT][8];
 #pragma unroll
@@ -303,61 +379,13 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
             dst[1] = make_float4(acc[b0 + rb][4], acc[b0 + rb][5], acc[b0 + rb][6], acc[b0 + rb][7]);
         }
         __syncthreads();
-        for (int i = tid; i < RB * TNT; i += NT) {
-            const int rb = i / TNT, c = i - rb * TNT, b = b0 + rb;
-            float v = 0.0f;
-#pragma unroll
-            for (int g = 0; g < NR; ++g) v += s_red[(g * RB + rb) * TNT + c];
-            if (b < B) {
-                int r, slot;
-                if constexpr (EPI == EPI_GLU) {  // owner by pair index j = c mod HALF; gate and up of a pair sit side by side
-                    const int j = c % HALF, hf = c / HALF;
-                    r = j / per;
-                    slot = ((s * BT + b) * 2 + hf) * per + (j - r * per);
-                } else {
-                    r = c / per;
-                    slot = (s * BT + b) * per + (c - r * per);
-                }
-#pragma unroll
-                for (int q = 0; q < MAX_CLUSTER; ++q)
-                    if (q == r) owner[q][slot] = v;
-            }
-        }
+        reduce_push_round<BT, EPI, TNT, NR, RB>(s_red, b0, B, s, per, owner);
         __syncthreads();
     }
     if (S > 1) cluster.sync();  // all pushes have landed; nothing remote is touched after this point
     else __syncthreads();
 
-    for (int it = 0; tid + it * NT < per * B; ++it) {
-        const int i = tid + it * NT;
-        const int b = i / per, c = i - b * per;
-        const int row = a.out_rows ? a.out_rows[b] : b;
-        if constexpr (EPI == EPI_BIAS) {
-            const int n = tile * TNT + s * per + c;
-            if (n < a.Nh) {
-                float v = it == 0 ? bias0[0] : it == 1 ? bias0[1] : load_bias<BF16>(a, n);
-#pragma unroll
-                for (int q = 0; q < MAX_CLUSTER; ++q)
-                    if (q < S) v += s_gather[(q * BT + b) * per + c];
-                a.y[(size_t)row * a.y_ld + n] = v;
-            }
-        } else {
-            const int F = a.Nh, f = tile * HALF + s * per + c;
-            if (f < F) {
-                float g = it == 0 ? bias0[0] : it == 1 ? bias0[1] : (a.bias ? __ldg(a.bias + f) : 0.0f);
-                float u = it == 0 ? bias1[0] : it == 1 ? bias1[1] : (a.bias ? __ldg(a.bias + F + f) : 0.0f);
-#pragma unroll
-                for (int q = 0; q < MAX_CLUSTER; ++q)
-                    if (q < S) {
-                        g += s_gather[((q * BT + b) * 2 + 0) * per + c];
-                        u += s_gather[((q * BT + b) * 2 + 1) * per + c];
-                    }
-                const float z = u * (g / (1.0f + expf(-g)));  // up * silu(gate)
-                a.y[(size_t)row * a.y_ld + f] = z;
-                if (a.z_copy) a.z_copy[(size_t)b * F + f] = z;
-            }
-        }
-    }
+    finish_columns<BF16, BT, EPI, TNT>(a, tile, s, per, s_gather, bias0, bias1);
 }
 
 template <bool BF16, int BT, int MODE, typename XT, int EPI, int TNT>
