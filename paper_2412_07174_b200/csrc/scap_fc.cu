@@ -65,11 +65,11 @@ static cudaError_t launch_fc_tn(const FcArgs &a, cudaStream_t st) {
     static bool attr_done = false;
     auto kern = fc_kernel<BF16, BT, MODE, XT, EPI, TNT>;
     if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, fc_smem_bytes(BT));
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, fc_smem_for(BT));
         if (e != cudaSuccess) return e;
         attr_done = true;
     }
-    return launch_cluster(kern, dim3(fc_tiles(a.Nh, EPI, TNT), a.S), dim3(FC_THREADS), fc_smem_bytes(BT), a.S, st,
+    return launch_cluster(kern, dim3(fc_tiles(a.Nh, EPI, TNT), a.S), dim3(FC_THREADS), fc_smem_for(BT), a.S, st,
                           g_tune.pdl != 0, a);
 }
 
@@ -83,8 +83,6 @@ static cudaError_t launch_fc_bt(const FcArgs &a, cudaStream_t st) {
     switch (batch_tile(a.B)) {
         case 1: return launch_fc_t<BF16, 1, MODE, XT, EPI>(a, st);
         case 2: return launch_fc_t<BF16, 2, MODE, XT, EPI>(a, st);
-        case 4: return launch_fc_t<BF16, 4, MODE, XT, EPI>(a, st);
-        case 8: return launch_fc_t<BF16, 8, MODE, XT, EPI>(a, st);
         default: return launch_fc_t<BF16, 16, MODE, XT, EPI>(a, st);
     }
 }

@@ -26,7 +26,7 @@ constexpr int MAX_CLUSTER = 8;  // portable cluster size: upper bound of the spl
 
 constexpr int FC_THREADS = 256;  // 8 warps; two CTAs fit on an SM, so every cluster of the grid is resident at once
 constexpr int FC_WARPS = FC_THREADS / 32;
-__host__ __device__ constexpr int fc_min_blocks(int BT) { return BT <= 8 ? 2 : 1; }
+__host__ __device__ constexpr int fc_min_blocks(int BT) { return 2; }
 // chunks (of 32 channels) each warp thresholds per fill; their centred values stay in registers
 __host__ __device__ constexpr int fc_pu(int BT) { return BT <= 2 ? 8 : BT <= 4 ? 4 : BT <= 8 ? 2 : 1; }
 __host__ __device__ constexpr int fc_cap(int BT) { return FC_WARPS * fc_pu(BT) * 32; }  // channels staged per fill
@@ -388,9 +388,268 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
     finish_columns<BF16, BT, EPI, TNT>(a, tile, s, per, s_gather, bias0, bias1);
 }
 
+// ------------------------------------------------------------------------------------------------
+// Batch 3..16: the same kernel with the multiply-accumulate on the tensor cores.
+//
+// At more than two batch rows the fp32 FMA path issues 8 * B instructions per 16-byte weight load and the
+// SM's issue rate, not HBM, becomes the limit.  Here a warp owns a 64-column chunk of the tile and streams
+// blocks of 8 kept rows: lane (g, t) = (lane / 4, lane % 4) loads rows t and t + 4 of the block at columns
+// 8g .. 8g+7 of the chunk, which after widening to fp32 bit patterns is exactly the B fragment (k8 x n8, tf32)
+// of eight mma.m16n8k8 instructions - MMA number i takes column i of every lane's eight, i.e. the column set
+// {8g' + i}.  The A fragment (16 batch rows x 8 kept channels) comes from the staged activations, rounded to
+// tf32 (10 mantissa bits: relative error 2^-11 per term, about 3e-4 on y).  Weights are exact in tf32 (bf16 and
+// fp16 have at most 10 mantissa bits).  Accumulation is fp32 in the MMA.
+// ------------------------------------------------------------------------------------------------
+constexpr int MMA_BT = 16;
+constexpr int MMA_PU = 3;                          // chunks per warp per fill
+constexpr int MMA_CAP = FC_WARPS * MMA_PU * 32;    // 768 channels staged per fill
+constexpr int MMA_XLD = MMA_CAP + 4;               // row pitch of the staged activations: conflict-free fragment reads
+__host__ __device__ constexpr int mma_main_bytes() {
+    const int stage = MMA_CAP * 4 + MMA_BT * MMA_XLD * 4;
+    const int red = FC_WARPS * 64 * MMA_BT * 4;  // (8 / NCW) row groups x 16 rows x (64 NCW) columns
+    return stage > red ? stage : red;
+}
+__host__ __device__ constexpr int mma_smem_bytes() { return mma_main_bytes() + MMA_BT * TN * 4 + (MMA_CAP / 32) * 4 + 16; }
+__host__ __device__ constexpr int fc_smem_for(int BT) { return BT == MMA_BT ? mma_smem_bytes() : fc_smem_bytes(BT); }
+
+__device__ __forceinline__ uint32_t to_tf32(float v) {
+    uint32_t r;
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(v));
+    return r;
+}
+__device__ __forceinline__ void mma_tf32(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+template <bool BF16>
+__device__ __forceinline__ void widen8_bits(const uint4 &v, uint32_t (&w)[8]) {
+    float f[8];
+    widen2<BF16>(v.x, f[0], f[1]);
+    widen2<BF16>(v.y, f[2], f[3]);
+    widen2<BF16>(v.z, f[4], f[5]);
+    widen2<BF16>(v.w, f[6], f[7]);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) w[j] = __float_as_uint(f[j]);
+}
+
+template <bool BF16, int MODE, typename XT, int EPI, int TNT>
+__device__ __forceinline__ void fc_body_mma(const FcArgs &a, const int tile, const int s, const bool wait_inside) {
+    constexpr int BT = MMA_BT, PU = MMA_PU, CAP = MMA_CAP, XLD = MMA_XLD, CAPC = CAP / 32;
+    constexpr int NCW = TNT / 64;          // warps across the columns of the tile
+    constexpr int NRW = FC_WARPS / NCW;    // warps across row blocks: warp row rw streams blocks rw, rw+NRW, ...
+    constexpr int HALF = TNT / 2;
+    constexpr int UB = 4;                  // row blocks in flight per warp (2 loads per lane each), in two groups
+    extern __shared__ __align__(16) unsigned char smem[];
+    uint32_t *s_k = reinterpret_cast<uint32_t *>(smem);
+    float *s_xs = reinterpret_cast<float *>(smem) + CAP;   // [16][XLD]
+    float *s_red = reinterpret_cast<float *>(smem);        // [NRW][16][TNT]
+    float *s_gather = reinterpret_cast<float *>(smem + mma_main_bytes());
+    uint32_t *s_bits = reinterpret_cast<uint32_t *>(s_gather + BT * TN);
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int g = lane >> 2, t = lane & 3, cw = warp % NCW, rw = warp / NCW;
+    const int B = a.B, S = a.S, K = a.K;
+    const XT *xg = reinterpret_cast<const XT *>(a.x);
+
+    // this lane's 8 columns inside its warp's 64-column chunk
+    int col;
+    bool col_ok;
+    if constexpr (EPI == EPI_GLU) {  // first half of the chunks: gate columns; second half: the matching up columns
+        const int f = tile * HALF + (cw % (NCW / 2)) * 64 + g * 8;
+        col_ok = f < a.Nh;
+        col = (cw / (NCW / 2)) * a.Nh + f;
+    } else {
+        col = tile * TNT + cw * 64 + g * 8;
+        col_ok = col < a.Nh;
+    }
+    const unsigned char *Wb = reinterpret_cast<const unsigned char *>(a.W) + (size_t)col * 2;
+    const size_t row_bytes = (size_t)a.ldw * 2;
+
+    const int per = (EPI == EPI_GLU ? HALF : TNT) / S;
+    float bias0[2], bias1[2];
+    prefetch_bias<BF16, EPI, TNT>(a, tile, s, per, bias0, bias1);
+
+    float acc[8][4];
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = 0.0f;
+
+    const int nchunks = (K + 31) >> 5;
+    const int my_chunks = nchunks > s ? (nchunks - s + S - 1) / S : 0;
+    float tau = 0.0f;
+    if constexpr (MODE == MODE_GATHER) tau = ld_nc(a.tau);
+    int rows_of[BT];  // source row of x for every batch row (clamped for the unused ones)
+#pragma unroll
+    for (int b = 0; b < BT; ++b) rows_of[b] = a.in_rows ? a.in_rows[b < B ? b : 0] : (b < B ? b : 0);
+
+    if (wait_inside && my_chunks == 0) {
+        griddep_wait();
+        griddep_launch_dependents();
+    }
+    for (int j0 = 0; j0 < my_chunks; j0 += CAPC) {
+        const int nj = min(CAPC, my_chunks - j0);
+        // ---- A: keep masks.  Each warp takes PU chunks; all 16 * PU activation loads of a lane are in flight
+        // together; the values are not kept (they are re-read from L1 in pass B) to stay within the registers.
+        float mk[PU];
+#pragma unroll
+        for (int p = 0; p < PU; ++p) {
+            const int j = p * FC_WARPS + warp;
+            const int k = (s + S * (j0 + j)) * 32 + lane;
+            mk[p] = a.m ? ld_nc(a.m + ((j < nj && k < K) ? k : 0)) : 0.0f;
+        }
+        if (wait_inside && j0 == 0) {
+            griddep_wait();
+            griddep_launch_dependents();
+        }
+        uint32_t km[PU];
+        unsigned bal[PU];
+        {
+            XT xraw[PU][BT];
+#pragma unroll
+            for (int p = 0; p < PU; ++p) {
+                const int j = p * FC_WARPS + warp;
+                const int k = (s + S * (j0 + j)) * 32 + lane;
+                const int kk = (j < nj && k < K) ? k : 0;
+#pragma unroll
+                for (int b = 0; b < BT; ++b) xraw[p][b] = ld_nc(xg + (size_t)rows_of[b] * a.x_ld + kk);
+            }
+#pragma unroll
+            for (int p = 0; p < PU; ++p) {
+                const int j = p * FC_WARPS + warp;
+                const int k = (s + S * (j0 + j)) * 32 + lane;
+                const bool ok = j < nj && k < K;
+                uint32_t m_ = 0;
+                if constexpr (MODE == MODE_GATHER) {
+#pragma unroll
+                    for (int b = 0; b < BT; ++b) {
+                        const float xv = widen1(xraw[p][b]);
+                        const float dv = a.m ? __fsub_rn(xv, mk[p]) : xv;
+                        m_ |= (ok && b < B && fabsf(dv) >= tau) ? (1u << b) : 0u;
+                    }
+                } else {
+                    m_ = ok ? 1u : 0u;
+                }
+                km[p] = m_;
+                bal[p] = __ballot_sync(0xffffffffu, m_ != 0);
+            }
+        }
+        {
+            unsigned mine = 0;
+#pragma unroll
+            for (int p = 0; p < PU; ++p) mine = lane == p ? bal[p] : mine;
+            const int j = lane * FC_WARPS + warp;
+            if (lane < PU && j < nj) {
+                s_bits[j] = mine;
+                if (MODE == MODE_GATHER && a.bits && tile == 0) a.bits[s + S * (j0 + j)] = mine;
+            }
+        }
+        __syncthreads();
+        int my_off[PU], cnt;
+        {
+            const int c_lo = (lane < nj) ? __popc(s_bits[lane]) : 0;  // CAPC = 24 <= 32
+            cnt = __reduce_add_sync(0xffffffffu, c_lo);
+#pragma unroll
+            for (int p = 0; p < PU; ++p) my_off[p] = __reduce_add_sync(0xffffffffu, (lane < p * FC_WARPS + warp) ? c_lo : 0);
+        }
+        // ---- B: kept channels and their pruned values (activations re-read; same arithmetic as in pass A)
+#pragma unroll
+        for (int p = 0; p < PU; ++p) {
+            const int j = p * FC_WARPS + warp;
+            const int k = (s + S * (j0 + j)) * 32 + lane;
+            const int kk = (j < nj && k < K) ? k : 0;
+            const int pos = my_off[p] + __popc(bal[p] & ((1u << lane) - 1u));
+            if (km[p]) s_k[pos] = (uint32_t)k;
+#pragma unroll
+            for (int b0 = 0; b0 < BT; b0 += 8) {
+                XT xr[8];
+#pragma unroll
+                for (int b = 0; b < 8; ++b) xr[b] = ld_nc(xg + (size_t)rows_of[b0 + b] * a.x_ld + kk);
+#pragma unroll
+                for (int b = 0; b < 8; ++b) {
+                    const float xv = widen1(xr[b]);
+                    const float dv = (MODE == MODE_GATHER && a.m) ? __fsub_rn(xv, mk[p]) : xv;
+                    const bool kept = MODE == MODE_DENSE ? (b0 + b < B) : (((km[p] >> (b0 + b)) & 1u) != 0);
+                    if (km[p]) s_xs[(b0 + b) * XLD + pos] = kept ? dv : 0.0f;
+                }
+            }
+        }
+        __syncthreads();
+
+        // ---- stream blocks of 8 kept rows; two groups of UB/2 blocks alternate (one consumed, one in flight)
+        {
+            constexpr int G = UB / 2;
+            const int nblk = (cnt + 7) >> 3;
+            const int nq = nblk > rw ? (nblk - rw + NRW - 1) / NRW : 0;  // blocks rw, rw+NRW, ...
+            uint4 ga[G][2], gb[G][2];
+            auto load_block = [&](uint4(&dst)[2], int q) {
+                const int i0 = 8 * (rw + NRW * q) + t, i1 = i0 + 4;
+                dst[0] = make_uint4(0, 0, 0, 0);
+                dst[1] = make_uint4(0, 0, 0, 0);
+                if (q < nq && col_ok) {
+                    if (i0 < cnt) dst[0] = ld_stream16(Wb + (size_t)s_k[i0] * row_bytes);
+                    if (i1 < cnt) dst[1] = ld_stream16(Wb + (size_t)s_k[i1] * row_bytes);
+                }
+            };
+            auto use_block = [&](const uint4(&src)[2], int q) {
+                if (q >= nq) return;  // warp-uniform
+                const int i0 = 8 * (rw + NRW * q) + t, i1 = i0 + 4;
+                uint32_t af[4];
+                af[0] = to_tf32(i0 < cnt ? s_xs[g * XLD + i0] : 0.0f);
+                af[1] = to_tf32(i0 < cnt ? s_xs[(g + 8) * XLD + i0] : 0.0f);
+                af[2] = to_tf32(i1 < cnt ? s_xs[g * XLD + i1] : 0.0f);
+                af[3] = to_tf32(i1 < cnt ? s_xs[(g + 8) * XLD + i1] : 0.0f);
+                uint32_t w0[8], w1[8];
+                widen8_bits<BF16>(src[0], w0);
+                widen8_bits<BF16>(src[1], w1);
+#pragma unroll
+                for (int i = 0; i < 8; ++i) mma_tf32(acc[i], af, w0[i], w1[i]);
+            };
+#pragma unroll
+            for (int u = 0; u < G; ++u) load_block(ga[u], u);
+#pragma unroll
+            for (int u = 0; u < G; ++u) load_block(gb[u], G + u);
+            for (int q0 = 0; q0 < nq; q0 += 2 * G) {
+#pragma unroll
+                for (int u = 0; u < G; ++u) use_block(ga[u], q0 + u);
+#pragma unroll
+                for (int u = 0; u < G; ++u) load_block(ga[u], q0 + 2 * G + u);
+#pragma unroll
+                for (int u = 0; u < G; ++u) use_block(gb[u], q0 + G + u);
+#pragma unroll
+                for (int u = 0; u < G; ++u) load_block(gb[u], q0 + 3 * G + u);
+            }
+        }
+        __syncthreads();
+    }
+
+    // ---- accumulator fragments -> s_red[rw][b][column]; MMA i holds columns {8 g' + i} of the chunk, and in its
+    // D fragment this lane has batch rows g and g + 8 at fragment columns 2t and 2t + 1 (g' = 2t, 2t + 1).
+    cg::cluster_group cluster = cg::this_cluster();
+    float *owner[MAX_CLUSTER];
+#pragma unroll
+    for (int q = 0; q < MAX_CLUSTER; ++q) owner[q] = (S > 1 && q < S) ? cluster.map_shared_rank(s_gather, q) : s_gather;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const int c0 = cw * 64 + 8 * (2 * t) + i, c1 = c0 + 8;
+        s_red[(rw * BT + g) * TNT + c0] = acc[i][0];
+        s_red[(rw * BT + g) * TNT + c1] = acc[i][1];
+        s_red[(rw * BT + g + 8) * TNT + c0] = acc[i][2];
+        s_red[(rw * BT + g + 8) * TNT + c1] = acc[i][3];
+    }
+    __syncthreads();
+    reduce_push_round<BT, EPI, TNT, NRW, BT>(s_red, 0, B, s, per, owner);
+    if (S > 1) cluster.sync();
+    else __syncthreads();
+    finish_columns<BF16, BT, EPI, TNT>(a, tile, s, per, s_gather, bias0, bias1);
+}
+
 template <bool BF16, int BT, int MODE, typename XT, int EPI, int TNT>
 __global__ void __launch_bounds__(FC_THREADS, fc_min_blocks(BT)) fc_kernel(const FcArgs a) {
-    if (a.hold_dependents) {  // parameter-producing call: ordinary stream order on both sides
+    if constexpr (BT == MMA_BT) {
+        fc_body_mma<BF16, MODE, XT, EPI, TNT>(a, blockIdx.x, blockIdx.y, true);
+    } else if (a.hold_dependents) {  // parameter-producing call: ordinary stream order on both sides
         griddep_wait();
         fc_body<BF16, BT, MODE, XT, EPI, TNT>(a, blockIdx.x, blockIdx.y, false);
     } else {
@@ -400,7 +659,7 @@ __global__ void __launch_bounds__(FC_THREADS, fc_min_blocks(BT)) fc_kernel(const
 
 // ---- host-side plumbing shared by the entry points ------------------------------------------------
 
-inline int batch_tile(int B) { return B <= 1 ? 1 : B <= 2 ? 2 : B <= 4 ? 4 : B <= 8 ? 8 : 16; }
+inline int batch_tile(int B) { return B <= 1 ? 1 : B <= 2 ? 2 : 16; }  // 3..16 rows: tensor-core variant
 inline int fc_tiles(int Nh, int epi, int tn) { return epi == EPI_GLU ? (Nh + tn / 2 - 1) / (tn / 2) : (Nh + tn - 1) / tn; }
 
 // Tile width (256 or 128 columns) and split-K factor (cluster size) for an FC with Nh columns per half and
