@@ -111,4 +111,23 @@ __device__ __forceinline__ __half ld_nc(const __half *p) {
     return __ushort_as_half(v);
 }
 
+// Activation loads.  With programmatic dependent launch a kernel is resident on an SM while its predecessor is
+// still writing the activations, and the non-coherent path may serve a line that an earlier kernel left in that
+// SM's L1; activations are therefore read through L2 (.cg), in issue order like ld_nc.
+__device__ __forceinline__ float ld_act(const float *p) {
+    float v;
+    asm volatile("ld.global.cg.f32 %0, [%1];" : "=f"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ __nv_bfloat16 ld_act(const __nv_bfloat16 *p) {
+    unsigned short v;
+    asm volatile("ld.global.cg.u16 %0, [%1];" : "=h"(v) : "l"(p) : "memory");
+    return __ushort_as_bfloat16(v);
+}
+__device__ __forceinline__ __half ld_act(const __half *p) {
+    unsigned short v;
+    asm volatile("ld.global.cg.u16 %0, [%1];" : "=h"(v) : "l"(p) : "memory");
+    return __ushort_as_half(v);
+}
+
 }  // namespace scap

@@ -115,7 +115,7 @@ __global__ void __launch_bounds__(1024) expand_bits_kernel(const uint32_t *__res
     __syncthreads();
     for (int w0 = 0; w0 < nwords; w0 += 1024) {
         const int w = w0 + tid;
-        const uint32_t word = w < nwords ? bits[w] : 0u;
+        const uint32_t word = w < nwords ? __ldcg(bits + w) : 0u;
         const int c = __popc(word);
         int v = c;
 #pragma unroll

@@ -125,7 +125,7 @@ __device__ __forceinline__ void finish_columns(const FcArgs &a, int tile, int s,
     for (int it = 0; tid + it * FC_THREADS < per * B; ++it) {
         const int i = tid + it * FC_THREADS;
         const int b = i / per, c = i - b * per;
-        const int row = a.out_rows ? a.out_rows[b] : b;
+        const int row = a.out_rows ? __ldcg(a.out_rows + b) : b;
         if constexpr (EPI == EPI_BIAS) {
             const int n = tile * TNT + s * per + c;
             if (n < a.Nh) {
@@ -259,7 +259,7 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
 #pragma unroll
             for (int b = 0; b < BT; ++b) {
                 const int bb = b < B ? b : 0;
-                xraw[p][b] = ld_nc(xg + (size_t)(a.in_rows ? a.in_rows[bb] : bb) * a.x_ld + kk);
+                xraw[p][b] = ld_act(xg + (size_t)(a.in_rows ? __ldcg(a.in_rows + bb) : bb) * a.x_ld + kk);
             }
         }
 #pragma unroll
@@ -396,9 +396,9 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
 // blocks of 8 kept rows: lane (g, t) = (lane / 4, lane % 4) loads rows t and t + 4 of the block at columns
 // 8g .. 8g+7 of the chunk, which after widening to fp32 bit patterns is exactly the B fragment (k8 x n8, tf32)
 // of eight mma.m16n8k8 instructions - MMA number i takes column i of every lane's eight, i.e. the column set
-// {8g' + i}.  The A fragment (16 batch rows x 8 kept channels) comes from the staged activations, rounded to
-// tf32 (10 mantissa bits: relative error 2^-11 per term, about 3e-4 on y).  Weights are exact in tf32 (bf16 and
-// fp16 have at most 10 mantissa bits).  Accumulation is fp32 in the MMA.
+// {8g' + i}.  The A fragment (16 batch rows x 8 kept channels) comes from the staged activations, split into
+// hi + lo tf32 parts (two MMAs per tile) so that no precision is lost against the fp32 FMA path.  Weights are
+// exact in tf32 (bf16 and fp16 have at most 10 mantissa bits).  Accumulation is fp32 in the MMA.
 // ------------------------------------------------------------------------------------------------
 constexpr int MMA_BT = 16;
 constexpr int MMA_PU = 3;                          // chunks per warp per fill
@@ -482,7 +482,7 @@ __device__ __forceinline__ void fc_body_mma(const FcArgs &a, const int tile, con
     if constexpr (MODE == MODE_GATHER) tau = ld_nc(a.tau);
     int rows_of[BT];  // source row of x for every batch row (clamped for the unused ones)
 #pragma unroll
-    for (int b = 0; b < BT; ++b) rows_of[b] = a.in_rows ? a.in_rows[b < B ? b : 0] : (b < B ? b : 0);
+    for (int b = 0; b < BT; ++b) rows_of[b] = a.in_rows ? __ldcg(a.in_rows + (b < B ? b : 0)) : (b < B ? b : 0);
 
     if (wait_inside && my_chunks == 0) {
         griddep_wait();
@@ -513,7 +513,7 @@ __device__ __forceinline__ void fc_body_mma(const FcArgs &a, const int tile, con
                 const int k = (s + S * (j0 + j)) * 32 + lane;
                 const int kk = (j < nj && k < K) ? k : 0;
 #pragma unroll
-                for (int b = 0; b < BT; ++b) xraw[p][b] = ld_nc(xg + (size_t)rows_of[b] * a.x_ld + kk);
+                for (int b = 0; b < BT; ++b) xraw[p][b] = ld_act(xg + (size_t)rows_of[b] * a.x_ld + kk);
             }
 #pragma unroll
             for (int p = 0; p < PU; ++p) {
@@ -565,7 +565,7 @@ __device__ __forceinline__ void fc_body_mma(const FcArgs &a, const int tile, con
             for (int b0 = 0; b0 < BT; b0 += 8) {
                 XT xr[8];
 #pragma unroll
-                for (int b = 0; b < 8; ++b) xr[b] = ld_nc(xg + (size_t)rows_of[b0 + b] * a.x_ld + kk);
+                for (int b = 0; b < 8; ++b) xr[b] = ld_act(xg + (size_t)rows_of[b0 + b] * a.x_ld + kk);
 #pragma unroll
                 for (int b = 0; b < 8; ++b) {
                     const float xv = widen1(xr[b]);
@@ -575,6 +575,14 @@ __device__ __forceinline__ void fc_body_mma(const FcArgs &a, const int tile, con
                 }
             }
         }
+        // The last block of 8 is completed with copies of the last kept row and zero activations, so that the
+        // streaming loop needs no per-row predicate (a padded row adds exactly 0 for finite weights).
+        __syncthreads();
+        if (tid < 8 && cnt > 0 && cnt + tid < ((cnt + 7) & ~7)) {
+            s_k[cnt + tid] = s_k[cnt - 1];
+#pragma unroll
+            for (int b = 0; b < BT; ++b) s_xs[b * XLD + cnt + tid] = 0.0f;
+        }
         __syncthreads();
 
         // ---- stream blocks of 8 kept rows; two groups of UB/2 blocks alternate (one consumed, one in flight)
@@ -583,28 +591,38 @@ __device__ __forceinline__ void fc_body_mma(const FcArgs &a, const int tile, con
             const int nblk = (cnt + 7) >> 3;
             const int nq = nblk > rw ? (nblk - rw + NRW - 1) / NRW : 0;  // blocks rw, rw+NRW, ...
             uint4 ga[G][2], gb[G][2];
+#pragma unroll
+            for (int u = 0; u < G; ++u) ga[u][0] = ga[u][1] = gb[u][0] = gb[u][1] = make_uint4(0, 0, 0, 0);
             auto load_block = [&](uint4(&dst)[2], int q) {
-                const int i0 = 8 * (rw + NRW * q) + t, i1 = i0 + 4;
-                dst[0] = make_uint4(0, 0, 0, 0);
-                dst[1] = make_uint4(0, 0, 0, 0);
-                if (q < nq && col_ok) {
-                    if (i0 < cnt) dst[0] = ld_stream16(Wb + (size_t)s_k[i0] * row_bytes);
-                    if (i1 < cnt) dst[1] = ld_stream16(Wb + (size_t)s_k[i1] * row_bytes);
+                if (q < nq) {  // warp-uniform; lanes outside the matrix keep their zeros
+                    const int i0 = 8 * (rw + NRW * q) + t;
+                    if (col_ok) {
+                        dst[0] = ld_stream16(Wb + (size_t)s_k[i0] * row_bytes);
+                        dst[1] = ld_stream16(Wb + (size_t)s_k[i0 + 4] * row_bytes);
+                    }
                 }
             };
             auto use_block = [&](const uint4(&src)[2], int q) {
                 if (q >= nq) return;  // warp-uniform
-                const int i0 = 8 * (rw + NRW * q) + t, i1 = i0 + 4;
-                uint32_t af[4];
-                af[0] = to_tf32(i0 < cnt ? s_xs[g * XLD + i0] : 0.0f);
-                af[1] = to_tf32(i0 < cnt ? s_xs[(g + 8) * XLD + i0] : 0.0f);
-                af[2] = to_tf32(i1 < cnt ? s_xs[g * XLD + i1] : 0.0f);
-                af[3] = to_tf32(i1 < cnt ? s_xs[(g + 8) * XLD + i1] : 0.0f);
+                const int i0 = 8 * (rw + NRW * q) + t;
+                // activation = hi + lo with both parts in tf32: the pair carries 21 mantissa bits, so the product
+                // is as accurate as the fp32 FMA path (the weights are exact in tf32)
+                const float xf[4] = {s_xs[g * XLD + i0], s_xs[(g + 8) * XLD + i0], s_xs[g * XLD + i0 + 4],
+                                     s_xs[(g + 8) * XLD + i0 + 4]};
+                uint32_t af[4], al[4];
+#pragma unroll
+                for (int r = 0; r < 4; ++r) {
+                    af[r] = to_tf32(xf[r]);
+                    al[r] = to_tf32(xf[r] - __uint_as_float(af[r]));
+                }
                 uint32_t w0[8], w1[8];
                 widen8_bits<BF16>(src[0], w0);
                 widen8_bits<BF16>(src[1], w1);
 #pragma unroll
-                for (int i = 0; i < 8; ++i) mma_tf32(acc[i], af, w0[i], w1[i]);
+                for (int i = 0; i < 8; ++i) {
+                    mma_tf32(acc[i], al, w0[i], w1[i]);
+                    mma_tf32(acc[i], af, w0[i], w1[i]);
+                }
             };
 #pragma unroll
             for (int u = 0; u < G; ++u) load_block(ga[u], u);

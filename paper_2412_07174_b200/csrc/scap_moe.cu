@@ -82,7 +82,7 @@ __global__ void __launch_bounds__(FC_THREADS, fc_min_blocks(BT)) moe_fc_kernel(c
     griddep_wait();
     griddep_launch_dependents();
     const int e = blockIdx.z;
-    const int nb = a.route->nb[e];
+    const int nb = __ldcg(&a.route->nb[e]);  // through L2: written by the routing kernel just before
     if (nb == 0) return;  // the whole cluster belongs to this expert, so every CTA of it leaves together
     float *z = reinterpret_cast<float *>(a.groups + (size_t)e * a.group_bytes);
     FcArgs g = {};
@@ -112,7 +112,7 @@ __global__ void __launch_bounds__(256) moe_combine_kernel(const Route *__restric
     const int n = blockIdx.x * blockDim.x + threadIdx.x, b = blockIdx.y;
     if (n >= D) return;
     float acc = 0.0f;
-    for (int j = 0; j < top_k; ++j) acc = fmaf(r->w[b][j], yslot[(size_t)(b * top_k + j) * D + n], acc);
+    for (int j = 0; j < top_k; ++j) acc = fmaf(__ldcg(&r->w[b][j]), __ldcg(yslot + (size_t)(b * top_k + j) * D + n), acc);
     y[(size_t)b * D + n] = acc;
 }
 
