@@ -393,57 +393,73 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
 //
 // At more than two batch rows the fp32 FMA path issues 8 * B instructions per 16-byte weight load and the
 // SM's issue rate, not HBM, becomes the limit.  Here a warp owns a 64-column chunk of the tile and streams
-// blocks of 8 kept rows: lane (g, t) = (lane / 4, lane % 4) loads rows t and t + 4 of the block at columns
-// 8g .. 8g+7 of the chunk, which after widening to fp32 bit patterns is exactly the B fragment (k8 x n8, tf32)
-// of eight mma.m16n8k8 instructions - MMA number i takes column i of every lane's eight, i.e. the column set
-// {8g' + i}.  The A fragment (16 batch rows x 8 kept channels) comes from the staged activations, split into
-// hi + lo tf32 parts (two MMAs per tile) so that no precision is lost against the fp32 FMA path.  Weights are
-// exact in tf32 (bf16 and fp16 have at most 10 mantissa bits).  Accumulation is fp32 in the MMA.
+// blocks of 16 kept rows through mma.m16n8k16 (bf16 or fp16 operands, fp32 accumulation):
+//   - lane (g, t) = (lane / 4, lane % 4) loads rows 2t, 2t+1, 2t+8, 2t+9 of the block at columns 8g .. 8g+7 of
+//     the chunk; a byte permute pairs the two rows of each column, which is exactly the B fragment (k16 x n8)
+//     of eight MMAs - MMA number i takes column i of every lane's eight, i.e. the column set {8g' + i};
+//   - the A fragment (16 batch rows x 16 kept channels) comes from the staged activations.  They are fp32 values
+//     (x - m), so each is split into NSPLIT parts of the weight dtype (bf16: hi + mid + lo = 24 mantissa bits,
+//     fp16: hi + lo = 22 bits) and the tile is multiplied once per part: nothing is lost against the fp32 path.
+//     (fp16 parts overflow for |x - m| > 65504.)
 // ------------------------------------------------------------------------------------------------
 constexpr int MMA_BT = 16;
 constexpr int MMA_PU = 3;                          // chunks per warp per fill
 constexpr int MMA_CAP = FC_WARPS * MMA_PU * 32;    // 768 channels staged per fill
-constexpr int MMA_XLD = MMA_CAP + 4;               // row pitch of the staged activations: conflict-free fragment reads
+constexpr int MMA_XLD2 = MMA_CAP / 2 + 4;          // 32-bit words per batch row of one staged part (conflict-free reads)
+__host__ __device__ constexpr int mma_nsplit(bool bf16) { return bf16 ? 3 : 2; }
 __host__ __device__ constexpr int mma_main_bytes() {
-    const int stage = MMA_CAP * 4 + MMA_BT * MMA_XLD * 4;
+    const int stage = MMA_CAP * 4 + 3 * MMA_BT * MMA_XLD2 * 4;
     const int red = FC_WARPS * 64 * MMA_BT * 4;  // (8 / NCW) row groups x 16 rows x (64 NCW) columns
     return stage > red ? stage : red;
 }
 __host__ __device__ constexpr int mma_smem_bytes() { return mma_main_bytes() + MMA_BT * TN * 4 + (MMA_CAP / 32) * 4 + 16; }
 __host__ __device__ constexpr int fc_smem_for(int BT) { return BT == MMA_BT ? mma_smem_bytes() : fc_smem_bytes(BT); }
 
-__device__ __forceinline__ uint32_t to_tf32(float v) {
-    uint32_t r;
-    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(v));
-    return r;
-}
-__device__ __forceinline__ void mma_tf32(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-    asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
 template <bool BF16>
-__device__ __forceinline__ void widen8_bits(const uint4 &v, uint32_t (&w)[8]) {
-    float f[8];
-    widen2<BF16>(v.x, f[0], f[1]);
-    widen2<BF16>(v.y, f[2], f[3]);
-    widen2<BF16>(v.z, f[4], f[5]);
-    widen2<BF16>(v.w, f[6], f[7]);
-#pragma unroll
-    for (int j = 0; j < 8; ++j) w[j] = __float_as_uint(f[j]);
+__device__ __forceinline__ void mma_k16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    if constexpr (BF16)
+        asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                     : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                     : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+    else
+        asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                     : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                     : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+// Splits v into NSPLIT values of the weight dtype whose sum is v to 2^-22 or better; part[0] is the leading one.
+template <bool BF16>
+__device__ __forceinline__ void split_parts(float v, unsigned short (&part)[3]) {
+    if constexpr (BF16) {
+        const __nv_bfloat16 h = __float2bfloat16_rn(v);
+        const float r1 = v - __bfloat162float(h);
+        const __nv_bfloat16 m = __float2bfloat16_rn(r1);
+        const __nv_bfloat16 l = __float2bfloat16_rn(r1 - __bfloat162float(m));
+        part[0] = __bfloat16_as_ushort(h);
+        part[1] = __bfloat16_as_ushort(m);
+        part[2] = __bfloat16_as_ushort(l);
+    } else {
+        const __half h = __float2half_rn(v);
+        const __half l = __float2half_rn(v - __half2float(h));
+        part[0] = __half_as_ushort(h);
+        part[1] = __half_as_ushort(l);
+        part[2] = 0;
+    }
 }
 
 template <bool BF16, int MODE, typename XT, int EPI, int TNT>
 __device__ __forceinline__ void fc_body_mma(const FcArgs &a, const int tile, const int s, const bool wait_inside) {
-    constexpr int BT = MMA_BT, PU = MMA_PU, CAP = MMA_CAP, XLD = MMA_XLD, CAPC = CAP / 32;
+    constexpr int BT = MMA_BT, PU = MMA_PU, CAP = MMA_CAP, XLD2 = MMA_XLD2, CAPC = CAP / 32;
+    constexpr int NSPLIT = mma_nsplit(BF16);
     constexpr int NCW = TNT / 64;          // warps across the columns of the tile
     constexpr int NRW = FC_WARPS / NCW;    // warps across row blocks: warp row rw streams blocks rw, rw+NRW, ...
     constexpr int HALF = TNT / 2;
-    constexpr int UB = 4;                  // row blocks in flight per warp (2 loads per lane each), in two groups
+    constexpr int G = 1;                   // row blocks per register group (two groups alternate); 4 loads per lane each
     extern __shared__ __align__(16) unsigned char smem[];
     uint32_t *s_k = reinterpret_cast<uint32_t *>(smem);
-    float *s_xs = reinterpret_cast<float *>(smem) + CAP;   // [16][XLD]
-    float *s_red = reinterpret_cast<float *>(smem);        // [NRW][16][TNT]
+    uint32_t *s_xp = reinterpret_cast<uint32_t *>(smem) + CAP;                 // [NSPLIT][16][XLD2] packed pairs
+    unsigned short *s_xh = reinterpret_cast<unsigned short *>(s_xp);           // same, addressed per element
+    float *s_red = reinterpret_cast<float *>(smem);                            // [NRW][16][TNT]
     float *s_gather = reinterpret_cast<float *>(smem + mma_main_bytes());
     uint32_t *s_bits = reinterpret_cast<uint32_t *>(s_gather + BT * TN);
 
@@ -480,28 +496,25 @@ __device__ __forceinline__ void fc_body_mma(const FcArgs &a, const int tile, con
     const int my_chunks = nchunks > s ? (nchunks - s + S - 1) / S : 0;
     float tau = 0.0f;
     if constexpr (MODE == MODE_GATHER) tau = ld_nc(a.tau);
+
+    if (wait_inside) {  // the row map and the activations are outputs of the previous kernel
+        griddep_wait();
+        griddep_launch_dependents();
+    }
     int rows_of[BT];  // source row of x for every batch row (clamped for the unused ones)
 #pragma unroll
     for (int b = 0; b < BT; ++b) rows_of[b] = a.in_rows ? __ldcg(a.in_rows + (b < B ? b : 0)) : (b < B ? b : 0);
 
-    if (wait_inside && my_chunks == 0) {
-        griddep_wait();
-        griddep_launch_dependents();
-    }
     for (int j0 = 0; j0 < my_chunks; j0 += CAPC) {
         const int nj = min(CAPC, my_chunks - j0);
         // ---- A: keep masks.  Each warp takes PU chunks; all 16 * PU activation loads of a lane are in flight
-        // together; the values are not kept (they are re-read from L1 in pass B) to stay within the registers.
+        // together; the values are not kept (they are re-read in pass B) to stay within the registers.
         float mk[PU];
 #pragma unroll
         for (int p = 0; p < PU; ++p) {
             const int j = p * FC_WARPS + warp;
             const int k = (s + S * (j0 + j)) * 32 + lane;
             mk[p] = a.m ? ld_nc(a.m + ((j < nj && k < K) ? k : 0)) : 0.0f;
-        }
-        if (wait_inside && j0 == 0) {
-            griddep_wait();
-            griddep_launch_dependents();
         }
         uint32_t km[PU];
         unsigned bal[PU];
@@ -553,7 +566,7 @@ __device__ __forceinline__ void fc_body_mma(const FcArgs &a, const int tile, con
 #pragma unroll
             for (int p = 0; p < PU; ++p) my_off[p] = __reduce_add_sync(0xffffffffu, (lane < p * FC_WARPS + warp) ? c_lo : 0);
         }
-        // ---- B: kept channels and their pruned values (activations re-read; same arithmetic as in pass A)
+        // ---- B: kept channels and the parts of their pruned values (activations re-read; same arithmetic as in A)
 #pragma unroll
         for (int p = 0; p < PU; ++p) {
             const int j = p * FC_WARPS + warp;
@@ -571,57 +584,67 @@ __device__ __forceinline__ void fc_body_mma(const FcArgs &a, const int tile, con
                     const float xv = widen1(xr[b]);
                     const float dv = (MODE == MODE_GATHER && a.m) ? __fsub_rn(xv, mk[p]) : xv;
                     const bool kept = MODE == MODE_DENSE ? (b0 + b < B) : (((km[p] >> (b0 + b)) & 1u) != 0);
-                    if (km[p]) s_xs[(b0 + b) * XLD + pos] = kept ? dv : 0.0f;
+                    unsigned short part[3];
+                    split_parts<BF16>(kept ? dv : 0.0f, part);
+                    if (km[p]) {
+#pragma unroll
+                        for (int q = 0; q < NSPLIT; ++q) s_xh[((q * BT + b0 + b) * XLD2) * 2 + pos] = part[q];
+                    }
                 }
             }
         }
-        // The last block of 8 is completed with copies of the last kept row and zero activations, so that the
-        // streaming loop needs no per-row predicate (a padded row adds exactly 0 for finite weights).
         __syncthreads();
-        if (tid < 8 && cnt > 0 && cnt + tid < ((cnt + 7) & ~7)) {
+        // The last block of 16 is completed with copies of the last kept row and zero activations, so that the
+        // streaming loop needs no per-row predicate (a padded row adds exactly 0 for finite weights).
+        const int cnt_pad = (cnt + 15) & ~15;
+        if (tid < 16 && cnt > 0 && cnt + tid < cnt_pad) {
             s_k[cnt + tid] = s_k[cnt - 1];
 #pragma unroll
-            for (int b = 0; b < BT; ++b) s_xs[b * XLD + cnt + tid] = 0.0f;
+            for (int q = 0; q < NSPLIT; ++q)
+#pragma unroll
+                for (int b = 0; b < BT; ++b) s_xh[((q * BT + b) * XLD2) * 2 + cnt + tid] = 0;
         }
         __syncthreads();
 
-        // ---- stream blocks of 8 kept rows; two groups of UB/2 blocks alternate (one consumed, one in flight)
+        // ---- stream blocks of 16 kept rows; two register groups of G blocks alternate (one consumed, one in flight)
         {
-            constexpr int G = UB / 2;
-            const int nblk = (cnt + 7) >> 3;
+            const int nblk = cnt_pad >> 4;
             const int nq = nblk > rw ? (nblk - rw + NRW - 1) / NRW : 0;  // blocks rw, rw+NRW, ...
-            uint4 ga[G][2], gb[G][2];
+            uint4 ga[G][4], gb[G][4];
 #pragma unroll
-            for (int u = 0; u < G; ++u) ga[u][0] = ga[u][1] = gb[u][0] = gb[u][1] = make_uint4(0, 0, 0, 0);
-            auto load_block = [&](uint4(&dst)[2], int q) {
-                if (q < nq) {  // warp-uniform; lanes outside the matrix keep their zeros
-                    const int i0 = 8 * (rw + NRW * q) + t;
-                    if (col_ok) {
-                        dst[0] = ld_stream16(Wb + (size_t)s_k[i0] * row_bytes);
-                        dst[1] = ld_stream16(Wb + (size_t)s_k[i0 + 4] * row_bytes);
-                    }
+            for (int u = 0; u < G; ++u)
+#pragma unroll
+                for (int r = 0; r < 4; ++r) ga[u][r] = gb[u][r] = make_uint4(0, 0, 0, 0);
+            auto load_block = [&](uint4(&dst)[4], int q) {
+                if (q < nq && col_ok) {  // q < nq is warp-uniform; lanes outside the matrix keep their zeros
+                    const int i0 = 16 * (rw + NRW * q) + 2 * t;
+                    dst[0] = ld_stream16(Wb + (size_t)s_k[i0] * row_bytes);
+                    dst[1] = ld_stream16(Wb + (size_t)s_k[i0 + 1] * row_bytes);
+                    dst[2] = ld_stream16(Wb + (size_t)s_k[i0 + 8] * row_bytes);
+                    dst[3] = ld_stream16(Wb + (size_t)s_k[i0 + 9] * row_bytes);
                 }
             };
-            auto use_block = [&](const uint4(&src)[2], int q) {
+            auto use_block = [&](const uint4(&src)[4], int q) {
                 if (q >= nq) return;  // warp-uniform
-                const int i0 = 8 * (rw + NRW * q) + t;
-                // activation = hi + lo with both parts in tf32: the pair carries 21 mantissa bits, so the product
-                // is as accurate as the fp32 FMA path (the weights are exact in tf32)
-                const float xf[4] = {s_xs[g * XLD + i0], s_xs[(g + 8) * XLD + i0], s_xs[g * XLD + i0 + 4],
-                                     s_xs[(g + 8) * XLD + i0 + 4]};
-                uint32_t af[4], al[4];
+                // B fragments: pair rows (2t, 2t+1) and (2t+8, 2t+9) column by column
+                uint32_t b0[8], b1[8];
+                const uint32_t r0[4] = {src[0].x, src[0].y, src[0].z, src[0].w}, r1[4] = {src[1].x, src[1].y, src[1].z, src[1].w};
+                const uint32_t r2[4] = {src[2].x, src[2].y, src[2].z, src[2].w}, r3[4] = {src[3].x, src[3].y, src[3].z, src[3].w};
 #pragma unroll
-                for (int r = 0; r < 4; ++r) {
-                    af[r] = to_tf32(xf[r]);
-                    al[r] = to_tf32(xf[r] - __uint_as_float(af[r]));
+                for (int i = 0; i < 4; ++i) {
+                    b0[2 * i] = __byte_perm(r0[i], r1[i], 0x5410);
+                    b0[2 * i + 1] = __byte_perm(r0[i], r1[i], 0x7632);
+                    b1[2 * i] = __byte_perm(r2[i], r3[i], 0x5410);
+                    b1[2 * i + 1] = __byte_perm(r2[i], r3[i], 0x7632);
                 }
-                uint32_t w0[8], w1[8];
-                widen8_bits<BF16>(src[0], w0);
-                widen8_bits<BF16>(src[1], w1);
+                const int w0 = 8 * (rw + NRW * q) + t;  // pair index of kept rows (2t, 2t+1) of this block
 #pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    mma_tf32(acc[i], al, w0[i], w1[i]);
-                    mma_tf32(acc[i], af, w0[i], w1[i]);
+                for (int qs = NSPLIT - 1; qs >= 0; --qs) {  // smallest part first
+                    const uint32_t *pl = s_xp + qs * BT * XLD2;
+                    const uint32_t af[4] = {pl[g * XLD2 + w0], pl[(g + 8) * XLD2 + w0], pl[g * XLD2 + w0 + 4],
+                                            pl[(g + 8) * XLD2 + w0 + 4]};
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) mma_k16<BF16>(acc[i], af, b0[i], b1[i]);
                 }
             };
 #pragma unroll
