@@ -83,6 +83,7 @@ static cudaError_t launch_fc_bt(const FcArgs &a, cudaStream_t st) {
     switch (batch_tile(a.B)) {
         case 1: return launch_fc_t<BF16, 1, MODE, XT, EPI>(a, st);
         case 2: return launch_fc_t<BF16, 2, MODE, XT, EPI>(a, st);
+        case 8: return launch_fc_t<BF16, 8, MODE, XT, EPI>(a, st);
         default: return launch_fc_t<BF16, 16, MODE, XT, EPI>(a, st);
     }
 }

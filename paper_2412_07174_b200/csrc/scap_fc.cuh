@@ -402,18 +402,22 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
 //     fp16: hi + lo = 22 bits) and the tile is multiplied once per part: nothing is lost against the fp32 path.
 //     (fp16 parts overflow for |x - m| > 65504.)
 // ------------------------------------------------------------------------------------------------
-constexpr int MMA_BT = 16;
-constexpr int MMA_PU = 3;                          // chunks per warp per fill
-constexpr int MMA_CAP = FC_WARPS * MMA_PU * 32;    // 768 channels staged per fill
-constexpr int MMA_XLD2 = MMA_CAP / 2 + 4;          // 32-bit words per batch row of one staged part (conflict-free reads)
+// Two instantiations: ROWS = 8 (batch 3..8; the upper half of the 16-row tile is fed zeros and twice as many
+// channels fit per fill) and ROWS = 16 (batch 9..16).  The template parameter BT of the kernels carries ROWS.
+__host__ __device__ constexpr bool is_mma(int BT) { return BT == 8 || BT == 16; }
+__host__ __device__ constexpr int mma_pu(int ROWS) { return ROWS == 8 ? 6 : 3; }              // chunks per warp per fill
+__host__ __device__ constexpr int mma_cap(int ROWS) { return FC_WARPS * mma_pu(ROWS) * 32; }  // 1536 / 768 channels per fill
+__host__ __device__ constexpr int mma_xld2(int ROWS) { return mma_cap(ROWS) / 2 + 4; }  // words per batch row of one staged part
 __host__ __device__ constexpr int mma_nsplit(bool bf16) { return bf16 ? 3 : 2; }
-__host__ __device__ constexpr int mma_main_bytes() {
-    const int stage = MMA_CAP * 4 + 3 * MMA_BT * MMA_XLD2 * 4;
-    const int red = FC_WARPS * 64 * MMA_BT * 4;  // (8 / NCW) row groups x 16 rows x (64 NCW) columns
+__host__ __device__ constexpr int mma_main_bytes(int ROWS) {
+    const int stage = mma_cap(ROWS) * 4 + 3 * ROWS * mma_xld2(ROWS) * 4;
+    const int red = FC_WARPS * 64 * ROWS * 4;  // (8 / NCW) row groups x ROWS x (64 NCW) columns
     return stage > red ? stage : red;
 }
-__host__ __device__ constexpr int mma_smem_bytes() { return mma_main_bytes() + MMA_BT * TN * 4 + (MMA_CAP / 32) * 4 + 16; }
-__host__ __device__ constexpr int fc_smem_for(int BT) { return BT == MMA_BT ? mma_smem_bytes() : fc_smem_bytes(BT); }
+__host__ __device__ constexpr int mma_smem_bytes(int ROWS) {
+    return mma_main_bytes(ROWS) + ROWS * TN * 4 + (mma_cap(ROWS) / 32) * 4 + 16;
+}
+__host__ __device__ constexpr int fc_smem_for(int BT) { return is_mma(BT) ? mma_smem_bytes(BT) : fc_smem_bytes(BT); }
 
 template <bool BF16>
 __device__ __forceinline__ void mma_k16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
@@ -447,9 +451,9 @@ __device__ __forceinline__ void split_parts(float v, unsigned short (&part)[3]) 
     }
 }
 
-template <bool BF16, int MODE, typename XT, int EPI, int TNT>
+template <bool BF16, int ROWS, int MODE, typename XT, int EPI, int TNT>
 __device__ __forceinline__ void fc_body_mma(const FcArgs &a, const int tile, const int s, const bool wait_inside) {
-    constexpr int BT = MMA_BT, PU = MMA_PU, CAP = MMA_CAP, XLD2 = MMA_XLD2, CAPC = CAP / 32;
+    constexpr int BT = ROWS, PU = mma_pu(ROWS), CAP = mma_cap(ROWS), XLD2 = mma_xld2(ROWS), CAPC = CAP / 32;
     constexpr int NSPLIT = mma_nsplit(BF16);
     constexpr int NCW = TNT / 64;          // warps across the columns of the tile
     constexpr int NRW = FC_WARPS / NCW;    // warps across row blocks: warp row rw streams blocks rw, rw+NRW, ...
@@ -460,7 +464,7 @@ __device__ __forceinline__ void fc_body_mma(const FcArgs &a, const int tile, con
     uint32_t *s_xp = reinterpret_cast<uint32_t *>(smem) + CAP;                 // [NSPLIT][16][XLD2] packed pairs
     unsigned short *s_xh = reinterpret_cast<unsigned short *>(s_xp);           // same, addressed per element
     float *s_red = reinterpret_cast<float *>(smem);                            // [NRW][16][TNT]
-    float *s_gather = reinterpret_cast<float *>(smem + mma_main_bytes());
+    float *s_gather = reinterpret_cast<float *>(smem + mma_main_bytes(ROWS));
     uint32_t *s_bits = reinterpret_cast<uint32_t *>(s_gather + BT * TN);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -505,6 +509,8 @@ __device__ __forceinline__ void fc_body_mma(const FcArgs &a, const int tile, con
 #pragma unroll
     for (int b = 0; b < BT; ++b) rows_of[b] = a.in_rows ? __ldcg(a.in_rows + (b < B ? b : 0)) : (b < B ? b : 0);
 
+    const int Bp = (B + 3) & ~3;  // batch rows staged (groups of 4); fragment rows beyond them are fed zeros
+
     for (int j0 = 0; j0 < my_chunks; j0 += CAPC) {
         const int nj = min(CAPC, my_chunks - j0);
         // ---- A: keep masks.  Each warp takes PU chunks; all 16 * PU activation loads of a lane are in flight
@@ -518,15 +524,18 @@ __device__ __forceinline__ void fc_body_mma(const FcArgs &a, const int tile, con
         }
         uint32_t km[PU];
         unsigned bal[PU];
+        XT xraw[PU][BT];  // stays in registers until pass B
         {
-            XT xraw[PU][BT];
 #pragma unroll
             for (int p = 0; p < PU; ++p) {
                 const int j = p * FC_WARPS + warp;
                 const int k = (s + S * (j0 + j)) * 32 + lane;
                 const int kk = (j < nj && k < K) ? k : 0;
 #pragma unroll
-                for (int b = 0; b < BT; ++b) xraw[p][b] = ld_act(xg + (size_t)rows_of[b] * a.x_ld + kk);
+                for (int b = 0; b < BT; ++b) {
+                    xraw[p][b] = XT();
+                    if ((b & ~3) < B) xraw[p][b] = ld_act(xg + (size_t)rows_of[b] * a.x_ld + kk);  // groups of 4 rows in use
+                }
             }
 #pragma unroll
             for (int p = 0; p < PU; ++p) {
@@ -561,34 +570,40 @@ __device__ __forceinline__ void fc_body_mma(const FcArgs &a, const int tile, con
         __syncthreads();
         int my_off[PU], cnt;
         {
-            const int c_lo = (lane < nj) ? __popc(s_bits[lane]) : 0;  // CAPC = 24 <= 32
-            cnt = __reduce_add_sync(0xffffffffu, c_lo);
+            int c_lo[(CAPC + 31) / 32];
+            cnt = 0;
 #pragma unroll
-            for (int p = 0; p < PU; ++p) my_off[p] = __reduce_add_sync(0xffffffffu, (lane < p * FC_WARPS + warp) ? c_lo : 0);
+            for (int q = 0; q < (CAPC + 31) / 32; ++q) {
+                c_lo[q] = (q * 32 + lane < nj) ? __popc(s_bits[q * 32 + lane]) : 0;
+                cnt += __reduce_add_sync(0xffffffffu, c_lo[q]);
+            }
+#pragma unroll
+            for (int p = 0; p < PU; ++p) {
+                int o = 0;
+#pragma unroll
+                for (int q = 0; q < (CAPC + 31) / 32; ++q)
+                    o += __reduce_add_sync(0xffffffffu, (q * 32 + lane < p * FC_WARPS + warp) ? c_lo[q] : 0);
+                my_off[p] = o;
+            }
         }
-        // ---- B: kept channels and the parts of their pruned values (activations re-read; same arithmetic as in A)
+        // ---- B: kept channels and the parts of their pruned values (same arithmetic as in A, from the same registers)
 #pragma unroll
         for (int p = 0; p < PU; ++p) {
             const int j = p * FC_WARPS + warp;
             const int k = (s + S * (j0 + j)) * 32 + lane;
-            const int kk = (j < nj && k < K) ? k : 0;
             const int pos = my_off[p] + __popc(bal[p] & ((1u << lane) - 1u));
-            if (km[p]) s_k[pos] = (uint32_t)k;
+            if (km[p]) {
+                s_k[pos] = (uint32_t)k;
 #pragma unroll
-            for (int b0 = 0; b0 < BT; b0 += 8) {
-                XT xr[8];
+                for (int b = 0; b < BT; ++b) {
+                    if (b < Bp) {  // rows beyond Bp are never read
+                        const float xv = widen1(xraw[p][b]);
+                        const float dv = (MODE == MODE_GATHER && a.m) ? __fsub_rn(xv, mk[p]) : xv;
+                        const bool kept = MODE == MODE_DENSE ? (b < B) : (((km[p] >> b) & 1u) != 0);
+                        unsigned short part[3];
+                        split_parts<BF16>(kept ? dv : 0.0f, part);
 #pragma unroll
-                for (int b = 0; b < 8; ++b) xr[b] = ld_act(xg + (size_t)rows_of[b0 + b] * a.x_ld + kk);
-#pragma unroll
-                for (int b = 0; b < 8; ++b) {
-                    const float xv = widen1(xr[b]);
-                    const float dv = (MODE == MODE_GATHER && a.m) ? __fsub_rn(xv, mk[p]) : xv;
-                    const bool kept = MODE == MODE_DENSE ? (b0 + b < B) : (((km[p] >> (b0 + b)) & 1u) != 0);
-                    unsigned short part[3];
-                    split_parts<BF16>(kept ? dv : 0.0f, part);
-                    if (km[p]) {
-#pragma unroll
-                        for (int q = 0; q < NSPLIT; ++q) s_xh[((q * BT + b0 + b) * XLD2) * 2 + pos] = part[q];
+                        for (int q = 0; q < NSPLIT; ++q) s_xh[((q * BT + b) * XLD2) * 2 + pos] = part[q];
                     }
                 }
             }
@@ -602,7 +617,8 @@ __device__ __forceinline__ void fc_body_mma(const FcArgs &a, const int tile, con
 #pragma unroll
             for (int q = 0; q < NSPLIT; ++q)
 #pragma unroll
-                for (int b = 0; b < BT; ++b) s_xh[((q * BT + b) * XLD2) * 2 + cnt + tid] = 0;
+                for (int b = 0; b < BT; ++b)
+                    if (b < Bp) s_xh[((q * BT + b) * XLD2) * 2 + cnt + tid] = 0;
         }
         __syncthreads();
 
@@ -641,8 +657,15 @@ __device__ __forceinline__ void fc_body_mma(const FcArgs &a, const int tile, con
 #pragma unroll
                 for (int qs = NSPLIT - 1; qs >= 0; --qs) {  // smallest part first
                     const uint32_t *pl = s_xp + qs * BT * XLD2;
-                    const uint32_t af[4] = {pl[g * XLD2 + w0], pl[(g + 8) * XLD2 + w0], pl[g * XLD2 + w0 + 4],
-                                            pl[(g + 8) * XLD2 + w0 + 4]};
+                    uint32_t af[4] = {0u, 0u, 0u, 0u};
+                    if (g < Bp) {
+                        af[0] = pl[g * XLD2 + w0];
+                        af[2] = pl[g * XLD2 + w0 + 4];
+                    }
+                    if (ROWS == 16 && g + 8 < Bp) {
+                        af[1] = pl[(g + 8) * XLD2 + w0];
+                        af[3] = pl[(g + 8) * XLD2 + w0 + 4];
+                    }
 #pragma unroll
                     for (int i = 0; i < 8; ++i) mma_k16<BF16>(acc[i], af, b0[i], b1[i]);
                 }
@@ -667,29 +690,79 @@ __device__ __forceinline__ void fc_body_mma(const FcArgs &a, const int tile, con
 
     // ---- accumulator fragments -> s_red[rw][b][column]; MMA i holds columns {8 g' + i} of the chunk, and in its
     // D fragment this lane has batch rows g and g + 8 at fragment columns 2t and 2t + 1 (g' = 2t, 2t + 1).
-    cg::cluster_group cluster = cg::this_cluster();
-    float *owner[MAX_CLUSTER];
-#pragma unroll
-    for (int q = 0; q < MAX_CLUSTER; ++q) owner[q] = (S > 1 && q < S) ? cluster.map_shared_rank(s_gather, q) : s_gather;
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
         const int c0 = cw * 64 + 8 * (2 * t) + i, c1 = c0 + 8;
         s_red[(rw * BT + g) * TNT + c0] = acc[i][0];
         s_red[(rw * BT + g) * TNT + c1] = acc[i][1];
-        s_red[(rw * BT + g + 8) * TNT + c0] = acc[i][2];
-        s_red[(rw * BT + g + 8) * TNT + c1] = acc[i][3];
+        if constexpr (ROWS == 16) {
+            s_red[(rw * BT + g + 8) * TNT + c0] = acc[i][2];
+            s_red[(rw * BT + g + 8) * TNT + c1] = acc[i][3];
+        }
     }
     __syncthreads();
-    reduce_push_round<BT, EPI, TNT, NRW, BT>(s_red, 0, B, s, per, owner);
+    // this CTA's partial tile, row groups added in order; s_gather is used as [b][column] here
+    for (int i = tid; i < BT * TNT; i += FC_THREADS) {
+        float v = 0.0f;
+#pragma unroll
+        for (int q = 0; q < NRW; ++q) v += s_red[q * BT * TNT + i];
+        s_gather[i] = v;
+    }
+    // ---- cluster exchange, pull form: with up to 16 batch rows a rank owns per * B results, each the sum of S
+    // partials; it reads them from its peers' shared memory (S independent loads in flight per result) in rank
+    // order.  The second barrier keeps every partial tile alive until all peers have read it.
+    cg::cluster_group cluster = cg::this_cluster();
     if (S > 1) cluster.sync();
     else __syncthreads();
-    finish_columns<BF16, BT, EPI, TNT>(a, tile, s, per, s_gather, bias0, bias1);
+    const float *peer[MAX_CLUSTER];
+#pragma unroll
+    for (int q = 0; q < MAX_CLUSTER; ++q) peer[q] = (S > 1 && q < S) ? cluster.map_shared_rank(s_gather, q) : s_gather;
+    for (int it = 0; tid + it * FC_THREADS < per * B; ++it) {
+        const int i = tid + it * FC_THREADS;
+        const int b = i / per, c = i - b * per;
+        const int row = a.out_rows ? __ldcg(a.out_rows + b) : b;
+        if constexpr (EPI == EPI_BIAS) {
+            const int n = tile * TNT + s * per + c;
+            if (n < a.Nh) {
+                float part[MAX_CLUSTER];
+#pragma unroll
+                for (int q = 0; q < MAX_CLUSTER; ++q) part[q] = q < S ? peer[q][b * TNT + s * per + c] : 0.0f;
+                float v = it == 0 ? bias0[0] : it == 1 ? bias0[1] : load_bias<BF16>(a, n);
+#pragma unroll
+                for (int q = 0; q < MAX_CLUSTER; ++q)
+                    if (q < S) v += part[q];
+                a.y[(size_t)row * a.y_ld + n] = v;
+            }
+        } else {
+            const int F = a.Nh, f = tile * HALF + s * per + c;
+            if (f < F) {
+                float pg[MAX_CLUSTER], pu[MAX_CLUSTER];
+#pragma unroll
+                for (int q = 0; q < MAX_CLUSTER; ++q) {
+                    pg[q] = q < S ? peer[q][b * TNT + s * per + c] : 0.0f;
+                    pu[q] = q < S ? peer[q][b * TNT + HALF + s * per + c] : 0.0f;
+                }
+                float gt = it == 0 ? bias0[0] : it == 1 ? bias0[1] : (a.bias ? __ldg(a.bias + f) : 0.0f);
+                float up = it == 0 ? bias1[0] : it == 1 ? bias1[1] : (a.bias ? __ldg(a.bias + F + f) : 0.0f);
+#pragma unroll
+                for (int q = 0; q < MAX_CLUSTER; ++q)
+                    if (q < S) {
+                        gt += pg[q];
+                        up += pu[q];
+                    }
+                const float z = up * (gt / (1.0f + expf(-gt)));  // up * silu(gate)
+                a.y[(size_t)row * a.y_ld + f] = z;
+                if (a.z_copy) a.z_copy[(size_t)b * F + f] = z;
+            }
+        }
+    }
+    if (S > 1) cluster.sync();
 }
 
 template <bool BF16, int BT, int MODE, typename XT, int EPI, int TNT>
 __global__ void __launch_bounds__(FC_THREADS, fc_min_blocks(BT)) fc_kernel(const FcArgs a) {
-    if constexpr (BT == MMA_BT) {
-        fc_body_mma<BF16, MODE, XT, EPI, TNT>(a, blockIdx.x, blockIdx.y, true);
+    if constexpr (is_mma(BT)) {
+        fc_body_mma<BF16, BT, MODE, XT, EPI, TNT>(a, blockIdx.x, blockIdx.y, true);
     } else if (a.hold_dependents) {  // parameter-producing call: ordinary stream order on both sides
         griddep_wait();
         fc_body<BF16, BT, MODE, XT, EPI, TNT>(a, blockIdx.x, blockIdx.y, false);
@@ -700,7 +773,7 @@ __global__ void __launch_bounds__(FC_THREADS, fc_min_blocks(BT)) fc_kernel(const
 
 // ---- host-side plumbing shared by the entry points ------------------------------------------------
 
-inline int batch_tile(int B) { return B <= 1 ? 1 : B <= 2 ? 2 : 16; }  // 3..16 rows: tensor-core variant
+inline int batch_tile(int B) { return B <= 1 ? 1 : B <= 2 ? 2 : B <= 8 ? 8 : 16; }  // 3..16 rows: tensor-core variants
 inline int fc_tiles(int Nh, int epi, int tn) { return epi == EPI_GLU ? (Nh + tn / 2 - 1) / (tn / 2) : (Nh + tn - 1) / tn; }
 
 // Tile width (256 or 128 columns) and split-K factor (cluster size) for an FC with Nh columns per half and
