@@ -92,15 +92,24 @@ __global__ void __launch_bounds__(FC_THREADS, fc_min_blocks(BT)) moe_fc_kernel(c
         g.x = a.h; g.x_ld = a.D; g.in_rows = a.route->rows[e];
         g.m = a.ex[e].m1; g.tau = a.ex[e].tau1; g.bias = a.ex[e].bgu_fused;
         g.y = z; g.y_ld = a.F;
-        if constexpr (is_mma(BT)) fc_body_mma<BF16, BT, MODE_GATHER, ST, EPI_GLU, TNT>(g, blockIdx.x, blockIdx.y, false);
-        else fc_body<BF16, BT, MODE_GATHER, ST, EPI_GLU, TNT>(g, blockIdx.x, blockIdx.y, false);
+        // an expert that got one or two rows of a larger batch takes the FMA body (cluster-uniform choice)
+        if constexpr (is_mma(BT)) {
+            if (nb <= 2) fc_body<BF16, 2, MODE_GATHER, ST, EPI_GLU, TNT>(g, blockIdx.x, blockIdx.y, false);
+            else fc_body_mma<BF16, BT, MODE_GATHER, ST, EPI_GLU, TNT>(g, blockIdx.x, blockIdx.y, false);
+        } else {
+            fc_body<BF16, BT, MODE_GATHER, ST, EPI_GLU, TNT>(g, blockIdx.x, blockIdx.y, false);
+        }
     } else {
         g.W = a.ex[e].Wd; g.K = a.F; g.ldw = a.D; g.Nh = a.D; g.S = a.S2;
         g.x = z; g.x_ld = a.F;
         g.m = a.ex[e].m2; g.tau = a.ex[e].tau2; g.bias = a.ex[e].bd_fused;
         g.y = a.yslot; g.y_ld = a.D; g.out_rows = a.route->slots[e];
-        if constexpr (is_mma(BT)) fc_body_mma<BF16, BT, MODE_GATHER, float, EPI_BIAS, TNT>(g, blockIdx.x, blockIdx.y, false);
-        else fc_body<BF16, BT, MODE_GATHER, float, EPI_BIAS, TNT>(g, blockIdx.x, blockIdx.y, false);
+        if constexpr (is_mma(BT)) {
+            if (nb <= 2) fc_body<BF16, 2, MODE_GATHER, float, EPI_BIAS, TNT>(g, blockIdx.x, blockIdx.y, false);
+            else fc_body_mma<BF16, BT, MODE_GATHER, float, EPI_BIAS, TNT>(g, blockIdx.x, blockIdx.y, false);
+        } else {
+            fc_body<BF16, BT, MODE_GATHER, float, EPI_BIAS, TNT>(g, blockIdx.x, blockIdx.y, false);
+        }
     }
 }
 
