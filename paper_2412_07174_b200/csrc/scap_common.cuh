@@ -129,5 +129,31 @@ __device__ __forceinline__ __half ld_act(const __half *p) {
     asm volatile("ld.global.cg.u16 %0, [%1];" : "=h"(v) : "l"(p) : "memory");
     return __ushort_as_half(v);
 }
+// Predicated forms: the load is issued only where `on` holds and the result is 0 elsewhere.  No branch, so a batch
+// of them still goes out together; and - unlike clamping the address of an unused slot to element 0 - the unused
+// slots of all CTAs do not converge on one L2 sector (which serialises them there).
+__device__ __forceinline__ float ld_nc_if(const float *p, bool on) {
+    float v;
+    asm volatile("{ .reg .pred q; setp.ne.u32 q, %2, 0; mov.f32 %0, 0f00000000; @q ld.global.nc.f32 %0, [%1]; }"
+                 : "=f"(v) : "l"(p), "r"((unsigned)on));
+    return v;
+}
+__device__ __forceinline__ float ld_act_if(const float *p, bool on) {
+    float v;
+    asm volatile("{ .reg .pred q; setp.ne.u32 q, %2, 0; mov.f32 %0, 0f00000000; @q ld.global.cg.f32 %0, [%1]; }"
+                 : "=f"(v) : "l"(p), "r"((unsigned)on) : "memory");
+    return v;
+}
+__device__ __forceinline__ unsigned short ld_act_if_u16(const void *p, bool on) {
+    unsigned short v;
+    asm volatile("{ .reg .pred q; setp.ne.u32 q, %2, 0; mov.u16 %0, 0; @q ld.global.cg.u16 %0, [%1]; }"
+                 : "=h"(v) : "l"(p), "r"((unsigned)on) : "memory");
+    return v;
+}
+__device__ __forceinline__ __nv_bfloat16 ld_act_if(const __nv_bfloat16 *p, bool on) { return __ushort_as_bfloat16(ld_act_if_u16(p, on)); }
+__device__ __forceinline__ __half ld_act_if(const __half *p, bool on) { return __ushort_as_half(ld_act_if_u16(p, on)); }
+
+// Hint: bring the line that holds *p into L2 (no register result, no ordering effect).
+__device__ __forceinline__ void prefetch_l2(const void *p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
 
 }  // namespace scap

@@ -39,15 +39,15 @@ int sm_count() {
 }
 
 // Two CTAs fit on an SM, so up to 2 * SMs CTAs are resident at once.  Among tile widths {256, 128} and cluster
-// sizes {8, 4, 2, 1} pick the pair with the most CTAs within that budget (ties: wider tile, then larger
-// cluster), keeping at least 64 input channels per slice.
+// sizes 8 .. 1 pick the pair with the most CTAs within that budget (ties: narrower tile - the smaller cluster
+// exchanges less - then larger cluster), keeping at least 64 input channels per slice.
 void choose_config(int K, int Nh, int epi, int groups, int *tn_out, int *S_out) {
     const int budget = 2 * sm_count();
     int best_tn = 256, best_S = 1;
     long long best = -1;
-    for (int tn = 256; tn >= 128; tn >>= 1) {
+    for (int tn = 128; tn <= 256; tn <<= 1) {
         const int tiles = fc_tiles(Nh, epi, tn);
-        for (int S = MAX_CLUSTER; S >= 1; S >>= 1) {
+        for (int S = MAX_CLUSTER; S >= 1; --S) {
             if (g_tune.split_k > 0 && S > g_tune.split_k) continue;
             if (S > 1 && K / S < 64) continue;
             const long long ctas = (long long)tiles * groups * S;

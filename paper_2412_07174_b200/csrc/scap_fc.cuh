@@ -38,15 +38,18 @@ __host__ __device__ constexpr int fc_main_bytes(int BT) {
     const int red = FC_WARPS * fc_rb(BT) * TN * 4;
     return stage > red ? stage : red;
 }
-__host__ __device__ constexpr int fc_smem_bytes(int BT) {  // main | gathered partials | chunk masks
-    return fc_main_bytes(BT) + BT * TN * 4 + (fc_cap(BT) / 32) * 4 + 16;
+// Row pitch of the gathered-partials region: a rank finishes ceil(columns / S) columns, so with a cluster size
+// that does not divide the tile the S slices together are up to 2 * (S - 1) entries longer than the tile.
+constexpr int GATHER_LD = TN + 16;
+__host__ __device__ constexpr int fc_smem_bytes(int BT) {  // main | gathered partials | chunk masks | row map
+    return fc_main_bytes(BT) + BT * GATHER_LD * 4 + (fc_cap(BT) / 32) * 4 + 16 * 4 + 16;
 }
 
 struct FcArgs {
     const void *W;        // [K, ldw] storage dtype, row k = all outputs of input channel k
     int K, ldw;           // ldw: columns of a weight row (N, or 2F for the packed gate|up weight)
     int Nh;               // EPI_BIAS: N.  EPI_GLU: F (gate columns 0..F-1, up columns F..2F-1)
-    int B, S;             // batch rows; split-K factor = cluster size (1, 2, 4 or 8)
+    int B, S;             // batch rows; split-K factor = cluster size (1 .. 8)
     int tn;               // columns per CTA: 256 or 128
     const void *x;        // activations [rows, x_ld] of type XT
     int x_ld;
@@ -128,7 +131,7 @@ __device__ __forceinline__ void finish_columns(const FcArgs &a, int tile, int s,
         const int row = a.out_rows ? __ldcg(a.out_rows + b) : b;
         if constexpr (EPI == EPI_BIAS) {
             const int n = tile * TNT + s * per + c;
-            if (n < a.Nh) {
+            if (s * per + c < TNT && n < a.Nh) {
                 float v = it == 0 ? bias0[0] : it == 1 ? bias0[1] : load_bias<BF16>(a, n);
 #pragma unroll
                 for (int q = 0; q < MAX_CLUSTER; ++q)
@@ -137,7 +140,7 @@ __device__ __forceinline__ void finish_columns(const FcArgs &a, int tile, int s,
             }
         } else {
             const int F = a.Nh, f = tile * HALF + s * per + c;
-            if (f < F) {
+            if (s * per + c < HALF && f < F) {
                 float g = it == 0 ? bias0[0] : it == 1 ? bias0[1] : (a.bias ? __ldg(a.bias + f) : 0.0f);
                 float u = it == 0 ? bias1[0] : it == 1 ? bias1[1] : (a.bias ? __ldg(a.bias + F + f) : 0.0f);
 #pragma unroll
@@ -166,10 +169,10 @@ __device__ __forceinline__ void prefetch_bias(const FcArgs &a, int tile, int s, 
             const int c = i % per;
             if constexpr (EPI == EPI_GLU) {
                 const int f = tile * HALF + s * per + c;
-                if (f < a.Nh && a.bias) { bias0[it] = __ldg(a.bias + f); bias1[it] = __ldg(a.bias + a.Nh + f); }
+                if (s * per + c < HALF && f < a.Nh && a.bias) { bias0[it] = __ldg(a.bias + f); bias1[it] = __ldg(a.bias + a.Nh + f); }
             } else {
                 const int n = tile * TNT + s * per + c;
-                if (n < a.Nh) bias0[it] = load_bias<BF16>(a, n);
+                if (s * per + c < TNT && n < a.Nh) bias0[it] = load_bias<BF16>(a, n);
             }
         }
     }
@@ -192,7 +195,8 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
     float *s_xs = reinterpret_cast<float *>(smem) + CAP;
     float *s_red = reinterpret_cast<float *>(smem);
     float *s_gather = reinterpret_cast<float *>(smem + fc_main_bytes(BT));  // [S][BT][columns owned by this rank]
-    uint32_t *s_bits = reinterpret_cast<uint32_t *>(s_gather + BT * TN);
+    uint32_t *s_bits = reinterpret_cast<uint32_t *>(s_gather + BT * GATHER_LD);
+    int *s_rows = reinterpret_cast<int *>(s_bits + CAPC);  // source row of x per batch row (when a row map is given)
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int rg = tid / LPR, cl = tid % LPR;  // row group and column lane of this thread
@@ -214,7 +218,7 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
     const size_t row_bytes = (size_t)a.ldw * 2;
 
     // columns (EPI_GLU: gate/up pairs) this rank finishes after the cluster exchange
-    const int per = (EPI == EPI_GLU ? HALF : TNT) / S;
+    const int per = ((EPI == EPI_GLU ? HALF : TNT) + S - 1) / S;  // the last rank may own fewer
     float bias0[2], bias1[2];
     prefetch_bias<BF16, EPI, TNT>(a, tile, s, per, bias0, bias1);
 
@@ -229,25 +233,41 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
     float tau = 0.0f;
     if constexpr (MODE == MODE_GATHER) tau = ld_nc(a.tau);
 
-    if (wait_inside && my_chunks == 0) {
+    if (wait_inside && (my_chunks == 0 || a.in_rows)) {
         griddep_wait();
         griddep_launch_dependents();
+    }
+    if (a.in_rows) {  // one L2 read per CTA and row (the map is an output of the previous kernel), then broadcast
+        if (tid < BT) s_rows[tid] = __ldcg(a.in_rows + (tid < B ? tid : 0));
+        __syncthreads();
     }
     for (int j0 = 0; j0 < my_chunks; j0 += CAPC) {
         const int nj = min(CAPC, my_chunks - j0);
         // ---- A: every warp loads PU chunks at once, centres and thresholds them (Alg. 3: one binary32
-        // subtraction, one compare per element) and keeps the values in registers.  Loads use clamped (always
-        // valid) addresses and no data-dependent branch, and nothing consumes them inside the load loops, so the
-        // PU * (BT + 1) loads of a lane are all in flight together.
+        // subtraction, one compare per element) and keeps the values in registers.  Loads of unused slots are
+        // predicated off (no branch) and nothing consumes a value inside the load loops, so the PU * (BT + 1)
+        // loads of a lane are all in flight together.
         XT xraw[PU][BT];
         float xv[PU][BT], mk[PU];
 #pragma unroll
         for (int p = 0; p < PU; ++p) {
             const int j = p * FC_WARPS + warp;
             const int k = (s + S * (j0 + j)) * 32 + lane;
-            mk[p] = a.m ? ld_nc(a.m + ((j < nj && k < K) ? k : 0)) : 0.0f;
+            mk[p] = a.m ? ld_nc_if(a.m + k, j < nj && k < K) : 0.0f;
         }
-        if (wait_inside && j0 == 0) {
+        if (wait_inside && j0 == 0 && !a.in_rows) {
+            // Pull this CTA's slice of x towards L2 while the previous kernel drains.  L2 is the coherence point,
+            // so a line the previous kernel still writes stays correct; the values are only read after the wait.
+#pragma unroll
+            for (int p = 0; p < PU; ++p) {
+                const int j = p * FC_WARPS + warp;
+                const int k = (s + S * j) * 32 + lane;
+                if (j < nj && k < K) {
+#pragma unroll
+                    for (int b = 0; b < BT; ++b)
+                        if (b < B) prefetch_l2(xg + (size_t)b * a.x_ld + k);
+                }
+            }
             griddep_wait();               // x (produced by the previous kernel in the stream) is complete
             griddep_launch_dependents();  // the next kernel may begin launching; it waits for this grid itself
         }
@@ -255,11 +275,11 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
         for (int p = 0; p < PU; ++p) {
             const int j = p * FC_WARPS + warp;
             const int k = (s + S * (j0 + j)) * 32 + lane;
-            const int kk = (j < nj && k < K) ? k : 0;
+            const bool ok = j < nj && k < K;
 #pragma unroll
             for (int b = 0; b < BT; ++b) {
                 const int bb = b < B ? b : 0;
-                xraw[p][b] = ld_act(xg + (size_t)(a.in_rows ? __ldcg(a.in_rows + bb) : bb) * a.x_ld + kk);
+                xraw[p][b] = ld_act_if(xg + (size_t)(a.in_rows ? s_rows[bb] : bb) * a.x_ld + k, ok && b < B);
             }
         }
 #pragma unroll
@@ -415,7 +435,7 @@ __host__ __device__ constexpr int mma_main_bytes(int ROWS) {
     return stage > red ? stage : red;
 }
 __host__ __device__ constexpr int mma_smem_bytes(int ROWS) {
-    return mma_main_bytes(ROWS) + ROWS * TN * 4 + (mma_cap(ROWS) / 32) * 4 + 16;
+    return mma_main_bytes(ROWS) + ROWS * GATHER_LD * 4 + (mma_cap(ROWS) / 32) * 4 + 16 * 4 + 16;
 }
 __host__ __device__ constexpr int fc_smem_for(int BT) { return is_mma(BT) ? mma_smem_bytes(BT) : fc_smem_bytes(BT); }
 
@@ -465,7 +485,8 @@ __device__ __forceinline__ void fc_body_mma(const FcArgs &a, const int tile, con
     unsigned short *s_xh = reinterpret_cast<unsigned short *>(s_xp);           // same, addressed per element
     float *s_red = reinterpret_cast<float *>(smem);                            // [NRW][16][TNT]
     float *s_gather = reinterpret_cast<float *>(smem + mma_main_bytes(ROWS));
-    uint32_t *s_bits = reinterpret_cast<uint32_t *>(s_gather + BT * TN);
+    uint32_t *s_bits = reinterpret_cast<uint32_t *>(s_gather + BT * GATHER_LD);
+    int *s_rows = reinterpret_cast<int *>(s_bits + CAPC);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int g = lane >> 2, t = lane & 3, cw = warp % NCW, rw = warp / NCW;
@@ -486,7 +507,7 @@ __device__ __forceinline__ void fc_body_mma(const FcArgs &a, const int tile, con
     const unsigned char *Wb = reinterpret_cast<const unsigned char *>(a.W) + (size_t)col * 2;
     const size_t row_bytes = (size_t)a.ldw * 2;
 
-    const int per = (EPI == EPI_GLU ? HALF : TNT) / S;
+    const int per = ((EPI == EPI_GLU ? HALF : TNT) + S - 1) / S;  // the last rank may own fewer
     float bias0[2], bias1[2];
     prefetch_bias<BF16, EPI, TNT>(a, tile, s, per, bias0, bias1);
 
@@ -505,9 +526,13 @@ __device__ __forceinline__ void fc_body_mma(const FcArgs &a, const int tile, con
         griddep_wait();
         griddep_launch_dependents();
     }
+    if (a.in_rows) {  // one L2 read per CTA and row, then broadcast
+        if (tid < BT) s_rows[tid] = __ldcg(a.in_rows + (tid < B ? tid : 0));
+        __syncthreads();
+    }
     int rows_of[BT];  // source row of x for every batch row (clamped for the unused ones)
 #pragma unroll
-    for (int b = 0; b < BT; ++b) rows_of[b] = a.in_rows ? __ldcg(a.in_rows + (b < B ? b : 0)) : (b < B ? b : 0);
+    for (int b = 0; b < BT; ++b) rows_of[b] = a.in_rows ? s_rows[b] : (b < B ? b : 0);
 
     const int Bp = (B + 3) & ~3;  // batch rows staged (groups of 4); fragment rows beyond them are fed zeros
 
@@ -520,7 +545,7 @@ __device__ __forceinline__ void fc_body_mma(const FcArgs &a, const int tile, con
         for (int p = 0; p < PU; ++p) {
             const int j = p * FC_WARPS + warp;
             const int k = (s + S * (j0 + j)) * 32 + lane;
-            mk[p] = a.m ? ld_nc(a.m + ((j < nj && k < K) ? k : 0)) : 0.0f;
+            mk[p] = a.m ? ld_nc_if(a.m + k, j < nj && k < K) : 0.0f;
         }
         uint32_t km[PU];
         unsigned bal[PU];
@@ -530,12 +555,9 @@ __device__ __forceinline__ void fc_body_mma(const FcArgs &a, const int tile, con
             for (int p = 0; p < PU; ++p) {
                 const int j = p * FC_WARPS + warp;
                 const int k = (s + S * (j0 + j)) * 32 + lane;
-                const int kk = (j < nj && k < K) ? k : 0;
+                const bool ok = j < nj && k < K;
 #pragma unroll
-                for (int b = 0; b < BT; ++b) {
-                    xraw[p][b] = XT();
-                    if ((b & ~3) < B) xraw[p][b] = ld_act(xg + (size_t)rows_of[b] * a.x_ld + kk);  // groups of 4 rows in use
-                }
+                for (int b = 0; b < BT; ++b) xraw[p][b] = ld_act_if(xg + (size_t)rows_of[b] * a.x_ld + k, ok && b < B);
             }
 #pragma unroll
             for (int p = 0; p < PU; ++p) {
@@ -723,7 +745,7 @@ __device__ __forceinline__ void fc_body_mma(const FcArgs &a, const int tile, con
         const int row = a.out_rows ? __ldcg(a.out_rows + b) : b;
         if constexpr (EPI == EPI_BIAS) {
             const int n = tile * TNT + s * per + c;
-            if (n < a.Nh) {
+            if (s * per + c < TNT && n < a.Nh) {
                 float part[MAX_CLUSTER];
 #pragma unroll
                 for (int q = 0; q < MAX_CLUSTER; ++q) part[q] = q < S ? peer[q][b * TNT + s * per + c] : 0.0f;
@@ -735,7 +757,7 @@ __device__ __forceinline__ void fc_body_mma(const FcArgs &a, const int tile, con
             }
         } else {
             const int F = a.Nh, f = tile * HALF + s * per + c;
-            if (f < F) {
+            if (s * per + c < HALF && f < F) {
                 float pg[MAX_CLUSTER], pu[MAX_CLUSTER];
 #pragma unroll
                 for (int q = 0; q < MAX_CLUSTER; ++q) {

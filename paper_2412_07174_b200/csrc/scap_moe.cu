@@ -82,7 +82,10 @@ __global__ void __launch_bounds__(FC_THREADS, fc_min_blocks(BT)) moe_fc_kernel(c
     griddep_wait();
     griddep_launch_dependents();
     const int e = blockIdx.z;
-    const int nb = __ldcg(&a.route->nb[e]);  // through L2: written by the routing kernel just before
+    __shared__ int s_nb;  // one L2 read per CTA (written by the routing kernel just before), then broadcast
+    if (threadIdx.x == 0) s_nb = __ldcg(&a.route->nb[e]);
+    __syncthreads();
+    const int nb = s_nb;
     if (nb == 0) return;  // the whole cluster belongs to this expert, so every CTA of it leaves together
     float *z = reinterpret_cast<float *>(a.groups + (size_t)e * a.group_bytes);
     FcArgs g = {};

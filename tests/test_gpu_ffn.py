@@ -86,6 +86,18 @@ def test_glu_small_shapes(S, D, F, B):
     assert kept2 < 0.9
 
 
+@pytest.mark.parametrize("split", [3, 5, 6, 7])
+@pytest.mark.parametrize("B", [1, 5])
+def test_glu_cluster_sizes_that_do_not_divide_the_tile(S, split, B):
+    g = si.glu_block(2, 520, 1000, si.BF16, 64, B)
+    c = calibrate_glu(g, 0.4, 0.7)
+    try:
+        S.scap_tune("split_k", split)
+        check_glu(S, g, c)
+    finally:
+        S.scap_tune("split_k", 0)
+
+
 def test_glu_fp16_and_no_centring(S):
     g = si.glu_block(2, 256, 520, si.F16, 64, 2)
     c = calibrate_glu(g, 0.3, 0.6, centre2=False)
