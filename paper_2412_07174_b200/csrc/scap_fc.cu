@@ -38,11 +38,42 @@ int sm_count() {
     return n;
 }
 
-// Two CTAs fit on an SM, so up to 2 * SMs CTAs are resident at once.  Among tile widths {256, 128} and cluster
-// sizes 8 .. 1 pick the pair with the most CTAs within that budget (ties: narrower tile - the smaller cluster
-// exchanges less - then larger cluster), keeping at least 64 input channels per slice.
-void choose_config(int K, int Nh, int epi, int groups, int *tn_out, int *S_out) {
-    const int budget = 2 * sm_count();
+// CTAs of clusters of size S that can be resident at once, as the runtime reports it for this device (a cluster
+// needs S SMs of one GPC with a free CTA slot, so the figure depends on how the device's SMs are grouped and is a
+// little below 2 * SMs for S > 1).  Queried once per size for the batch-1 kernel, which has the launch shape of
+// all variants (256 threads, two CTAs per SM); 2 * SMs where the query is not possible.
+static int resident_ctas(int S) {
+    static int cached[MAX_CLUSTER + 1];
+    if (cached[S]) return cached[S];
+    int n = 2 * sm_count();
+    if (S > 1) {
+        auto kern = fc_kernel<true, 1, MODE_GATHER, __nv_bfloat16, EPI_BIAS, 128>;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(1, S);
+        cfg.blockDim = dim3(FC_THREADS);
+        cfg.dynamicSmemBytes = fc_smem_for(1);
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 1;
+        attr[0].val.clusterDim.y = S;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        int clusters = 0;
+        if (cudaOccupancyMaxActiveClusters(&clusters, kern, &cfg) == cudaSuccess && clusters > 0) n = clusters * S;
+        else cudaGetLastError();
+    }
+    cached[S] = n;
+    return n;
+}
+
+// Two CTAs fit on an SM, so up to 2 * SMs CTAs are resident at once (fewer in clusters, see above).  Among tile widths {128, 256} and cluster
+// sizes 8 .. 1 pick the pair with the most CTAs within that budget, keeping at least 64 input channels per slice.
+// Ties: fewer fills of the kept-channel stage per CTA (B decides the stage capacity), then the narrower tile (its
+// smaller cluster exchanges less), then the larger cluster.
+void choose_config(int K, int Nh, int epi, int groups, int B, int *tn_out, int *S_out) {
+    const int bt = batch_tile(B), cap = is_mma(bt) ? mma_cap(bt) : fc_cap(bt);
+    const int nchunks = (K + 31) / 32;
     int best_tn = 256, best_S = 1;
     long long best = -1;
     for (int tn = 128; tn <= 256; tn <<= 1) {
@@ -51,8 +82,10 @@ void choose_config(int K, int Nh, int epi, int groups, int *tn_out, int *S_out) 
             if (g_tune.split_k > 0 && S > g_tune.split_k) continue;
             if (S > 1 && K / S < 64) continue;
             const long long ctas = (long long)tiles * groups * S;
+            const int budget = resident_ctas(S);
             if (ctas > budget && !(S == 1 && tn == 256)) continue;
-            const long long score = ctas > budget ? 0 : ctas;
+            const int fills = ((nchunks + S - 1) / S * 32 + cap - 1) / cap;
+            const long long score = ctas > budget ? 0 : ctas * 64 + (63 - (fills < 63 ? fills : 63));
             if (score > best) { best = score; best_tn = tn; best_S = S; }
         }
     }
@@ -164,7 +197,7 @@ static scap_status sparse_fc_impl(const void *x, const void *W, const float *m, 
     FcArgs a;
     memset(&a, 0, sizeof(a));
     a.W = W; a.K = K; a.ldw = N; a.Nh = N; a.B = B;
-    choose_config(K, N, EPI_BIAS, 1, &a.tn, &a.S);
+    choose_config(K, N, EPI_BIAS, 1, B, &a.tn, &a.S);
     a.x = x; a.x_ld = K; a.m = m; a.tau = tau; a.bias = b_fused; a.y = y; a.y_ld = N;
     const bool inspect = idx_out || nnz_out;
     if (inspect) a.bits = reinterpret_cast<uint32_t *>(ws);
@@ -179,7 +212,7 @@ static scap_status dense_impl(const void *x, int xkind, const void *W, const flo
     FcArgs a;
     memset(&a, 0, sizeof(a));
     a.W = W; a.K = K; a.ldw = N; a.Nh = N; a.B = B;
-    choose_config(K, N, EPI_BIAS, 1, &a.tn, &a.S);
+    choose_config(K, N, EPI_BIAS, 1, B, &a.tn, &a.S);
     a.x = x; a.x_ld = K; a.bias = b; a.bias16 = b16; a.y = y; a.y_ld = N;
     a.hold_dependents = writes_parameters ? 1 : 0;
     return cuda_status(launch_fc(dt == SCAP_BF16, MODE_DENSE, xkind, EPI_BIAS, a, st));

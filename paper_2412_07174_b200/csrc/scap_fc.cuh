@@ -42,7 +42,7 @@ __host__ __device__ constexpr int fc_main_bytes(int BT) {
 // that does not divide the tile the S slices together are up to 2 * (S - 1) entries longer than the tile.
 constexpr int GATHER_LD = TN + 16;
 __host__ __device__ constexpr int fc_smem_bytes(int BT) {  // main | gathered partials | chunk masks | row map
-    return fc_main_bytes(BT) + BT * GATHER_LD * 4 + (fc_cap(BT) / 32) * 4 + 16 * 4 + 16;
+    return fc_main_bytes(BT) + BT * GATHER_LD * 4 + (fc_cap(BT) / 32) * 4 + 16 * 4 + FC_WARPS * 4 + 16;
 }
 
 struct FcArgs {
@@ -197,6 +197,7 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
     float *s_gather = reinterpret_cast<float *>(smem + fc_main_bytes(BT));  // [S][BT][columns owned by this rank]
     uint32_t *s_bits = reinterpret_cast<uint32_t *>(s_gather + BT * GATHER_LD);
     int *s_rows = reinterpret_cast<int *>(s_bits + CAPC);  // source row of x per batch row (when a row map is given)
+    int *s_wcnt = s_rows + 16;                             // kept channels per warp, this fill
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int rg = tid / LPR, cl = tid % LPR;  // row group and column lane of this thread
@@ -251,7 +252,7 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
         float xv[PU][BT], mk[PU];
 #pragma unroll
         for (int p = 0; p < PU; ++p) {
-            const int j = p * FC_WARPS + warp;
+            const int j = warp * PU + p;
             const int k = (s + S * (j0 + j)) * 32 + lane;
             mk[p] = a.m ? ld_nc_if(a.m + k, j < nj && k < K) : 0.0f;
         }
@@ -260,7 +261,7 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
             // so a line the previous kernel still writes stays correct; the values are only read after the wait.
 #pragma unroll
             for (int p = 0; p < PU; ++p) {
-                const int j = p * FC_WARPS + warp;
+                const int j = warp * PU + p;
                 const int k = (s + S * j) * 32 + lane;
                 if (j < nj && k < K) {
 #pragma unroll
@@ -273,7 +274,7 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
         }
 #pragma unroll
         for (int p = 0; p < PU; ++p) {
-            const int j = p * FC_WARPS + warp;
+            const int j = warp * PU + p;
             const int k = (s + S * (j0 + j)) * 32 + lane;
             const bool ok = j < nj && k < K;
 #pragma unroll
@@ -291,7 +292,7 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
         unsigned bal[PU];
 #pragma unroll
         for (int p = 0; p < PU; ++p) {
-            const int j = p * FC_WARPS + warp;
+            const int j = warp * PU + p;
             const int k = (s + S * (j0 + j)) * 32 + lane;
             const bool ok = j < nj && k < K;
             uint32_t m_ = 0;
@@ -308,43 +309,36 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
             km[p] = m_;
             bal[p] = __ballot_sync(0xffffffffu, m_ != 0);
         }
-        {   // lane p publishes the word of this warp's p-th chunk (chunk index p * FC_WARPS + warp: the chunks of
-            // a fill are dealt round-robin to the warps so that every warp has about the same number)
+        // ---- position of each chunk in the kept list.  A warp owns PU consecutive chunks, so the positions inside
+        // the warp's stretch follow from its own ballot words; only the eight per-warp totals cross warps.
+        int my_off[PU], wtotal = 0;
+#pragma unroll
+        for (int p = 0; p < PU; ++p) {
+            my_off[p] = wtotal;
+            wtotal += __popc(bal[p]);
+        }
+        if (lane == 0) s_wcnt[warp] = wtotal;
+        if (MODE == MODE_GATHER && a.bits && tile == 0) {  // lane p publishes the mask word of the warp's p-th chunk
             unsigned mine = 0;
 #pragma unroll
             for (int p = 0; p < PU; ++p) mine = lane == p ? bal[p] : mine;
-            const int j = lane * FC_WARPS + warp;
-            if (lane < PU && j < nj) {
-                s_bits[j] = mine;
-                if (MODE == MODE_GATHER && a.bits && tile == 0) a.bits[s + S * (j0 + j)] = mine;
-            }
+            const int j = warp * PU + lane;
+            if (lane < PU && j < nj) a.bits[s + S * (j0 + j)] = mine;
         }
         __syncthreads();
-        // ---- position of each chunk in the kept list: every warp sums the counts of the chunks before its own
-        // with warp-wide integer reductions (no second barrier, no serial scan)
-        int my_off[PU], cnt = 0;
-        {
-            int c_lo[(CAPC + 31) / 32];
+        int cnt = 0, wbase = 0;
 #pragma unroll
-            for (int q = 0; q < (CAPC + 31) / 32; ++q) {
-                c_lo[q] = (q * 32 + lane < nj) ? __popc(s_bits[q * 32 + lane]) : 0;
-                cnt += __reduce_add_sync(0xffffffffu, c_lo[q]);
-            }
-#pragma unroll
-            for (int p = 0; p < PU; ++p) {
-                const int j = p * FC_WARPS + warp;
-                int o = 0;
-#pragma unroll
-                for (int q = 0; q < (CAPC + 31) / 32; ++q) o += __reduce_add_sync(0xffffffffu, (q * 32 + lane < j) ? c_lo[q] : 0);
-                my_off[p] = o;
-            }
+        for (int w = 0; w < FC_WARPS; ++w) {
+            const int c = s_wcnt[w];
+            cnt += c;
+            wbase += w < warp ? c : 0;
         }
         // ---- B: kept channels and their pruned values, in ascending channel order
 #pragma unroll
         for (int p = 0; p < PU; ++p) {
             if (km[p]) {
-                const int j = p * FC_WARPS + warp;
-                const int pos = my_off[p] + __popc(bal[p] & ((1u << lane) - 1u));
+                const int j = warp * PU + p;
+                const int pos = wbase + my_off[p] + __popc(bal[p] & ((1u << lane) - 1u));
                 s_k[pos] = (uint32_t)((s + S * (j0 + j)) * 32 + lane);
 #pragma unroll
                 for (int b = 0; b < BT; ++b)
@@ -800,7 +794,7 @@ inline int fc_tiles(int Nh, int epi, int tn) { return epi == EPI_GLU ? (Nh + tn 
 
 // Tile width (256 or 128 columns) and split-K factor (cluster size) for an FC with Nh columns per half and
 // `groups` concurrently active groups (experts): the pair with the most CTAs that are still all co-resident.
-void choose_config(int K, int Nh, int epi, int groups, int *tn, int *S);
+void choose_config(int K, int Nh, int epi, int groups, int B, int *tn, int *S);
 
 // Launch with cluster dimension (1, S, 1) and, if enabled, programmatic dependent launch.
 template <typename... KArgs, typename... Args>

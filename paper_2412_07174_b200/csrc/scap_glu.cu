@@ -55,7 +55,7 @@ scap_status scap_glu_ffn(const void *h, const void *Wgu, const void *Wd, const f
     FcArgs a;
     memset(&a, 0, sizeof(a));
     a.W = Wgu; a.K = D; a.ldw = 2 * F; a.Nh = F; a.B = B;
-    choose_config(D, F, EPI_GLU, 1, &a.tn, &a.S);
+    choose_config(D, F, EPI_GLU, 1, B, &a.tn, &a.S);
     a.x = h; a.x_ld = D; a.m = m1; a.tau = tau1; a.bias = bgu_fused;
     a.y = z; a.y_ld = F; a.z_copy = z_out;
     if (idx1_out || nnz1_out) a.bits = reinterpret_cast<uint32_t *>(w + G.bits1);
@@ -65,7 +65,7 @@ scap_status scap_glu_ffn(const void *h, const void *Wgu, const void *Wd, const f
     FcArgs d;
     memset(&d, 0, sizeof(d));
     d.W = Wd; d.K = F; d.ldw = D; d.Nh = D; d.B = B;
-    choose_config(F, D, EPI_BIAS, 1, &d.tn, &d.S);
+    choose_config(F, D, EPI_BIAS, 1, B, &d.tn, &d.S);
     d.x = z; d.x_ld = F; d.m = m2; d.tau = tau2; d.bias = bd_fused; d.y = y; d.y_ld = D;
     if (idx2_out || nnz2_out) d.bits = reinterpret_cast<uint32_t *>(w + G.bits2);
     e = launch_fc(bf16, MODE_GATHER, 2, EPI_BIAS, d, st);

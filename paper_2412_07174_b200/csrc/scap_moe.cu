@@ -217,8 +217,8 @@ scap_status scap_moe_ffn(const void *h, const float *logits, const scap_expert *
     a.yslot = reinterpret_cast<float *>(w + M.yslot);
     a.y = y; a.expert_out = expert_out; a.weight_out = weight_out;
     const int active = B * top_k < E ? B * top_k : E;  // experts that can have rows at once
-    choose_config(D, F, EPI_GLU, active, &a.tn1, &a.S1);
-    choose_config(F, D, EPI_BIAS, active, &a.tn2, &a.S2);
+    choose_config(D, F, EPI_GLU, active, B, &a.tn1, &a.S1);
+    choose_config(F, D, EPI_BIAS, active, B, &a.tn2, &a.S2);
     const int tiles1 = fc_tiles(F, EPI_GLU, a.tn1), tiles2 = fc_tiles(D, EPI_BIAS, a.tn2);
     const bool bf16 = dt == SCAP_BF16, pdl = g_tune.pdl != 0;
 
