@@ -115,6 +115,10 @@ scap_status scap_fold_bias(const void *W, const float *m, const void *b, int K, 
  * Optional outputs for inspection: idx_out[K] receives the ascending list of fetched channels
  * (first *nnz_out entries valid), nnz_out[1] their number.  m, b_fused, idx_out, nnz_out may
  * be NULL.  Results are bitwise reproducible for fixed shapes and tuning.
+ * Arithmetic: batch 1-2 multiply-accumulates in fp32 FMAs.  Batch 3-16 runs on the tensor cores
+ * with d split exactly into parts of the weight dtype (bf16: three parts, fp16: two) and fp32
+ * accumulation, so the result carries the same information as the FMA path; with fp16 weights
+ * the parts overflow for |d| > 65504 (such an activation yields inf/NaN in its row only).
  * ------------------------------------------------------------------------------------------ */
 size_t scap_fc_workspace(int B, int K, int N);
 scap_status scap_sparse_fc(const void *x, const void *W, const float *m, const float *tau, const float *b_fused,
