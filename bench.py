@@ -366,6 +366,12 @@ def run_suite(args):
 
 
 
+# dram__bytes_read.sum + dram__bytes_write.sum of one fc_kernel launch from the ncu capture summarised under
+# profiles/ (None whenever the kernel has changed since that capture).
+NCU_TRAFFIC_BYTES = 31949568
+NCU_TRAFFIC_NOTE = "ncu capture of one launch at the 65% target (algorithmic bytes of that launch: 31.8 MB)"
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -597,7 +603,7 @@ def main():
         "speedup_vs_dense": {("%d%%" % round(100 * s)): round(dense_us / detail[s]["us_per_call"], 3) for s in SPARSITIES},
         "calibrate_ms": {("%d%%" % round(100 * s)): round(cal_ms[s], 3) for s in SPARSITIES},
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "traffic": None, "peak_kind": peak_kind, "frac_of_nominal_8000": achieved / 8000.0,
+                     "traffic": NCU_TRAFFIC_BYTES, "traffic_note": NCU_TRAFFIC_NOTE, "peak_kind": peak_kind, "frac_of_nominal_8000": achieved / 8000.0,
                      "kernel": "fc_kernel (fused threshold + compaction + gather-GEMV + cluster reduction), one launch per call"},
         "e2e": {"value": e2e_value, "unit": "GB/s", "h2d_bytes_per_step": calls_per_step * K * 2,
                 "d2h_bytes_per_step": calls_per_step * N * 4, "steps": e2e_steps},
