@@ -77,10 +77,18 @@ int scap_version(void);
 /* Process-wide tuning knobs (plain ints, not thread-safe against concurrent calls):
  *   "split_k"  cap the split-K factor (thread-block cluster size) of the FC kernel: 0 = automatic, else 1..8
  *   "pdl"      1 = launch dependent kernels with programmatic dependent launch (default), 0 = off
+ *   "tcgen05"  1 = batch 3..16 calls of the FC and SwiGLU entry points run the TMA-gather + tcgen05
+ *              kernel, 0 = the mma.sync variants
  * Unknown keys return SCAP_ERR_INVALID_ARG.  Tuning never changes what is computed; split_k
  * changes the (fixed) summation order and therefore the last bits of y.  Query workspace sizes
  * after tuning.                                                                               */
 scap_status scap_tune(const char *key, int value);
+
+/* The tcgen05 kernel bounds every wait on a shared-memory barrier; a wait that runs out (which a
+ * correct run never does) makes the CTA stop issuing work, so y is then incomplete.  This call
+ * synchronises the device, returns SCAP_ERR_TIMEOUT if that happened since the last call (and
+ * clears the record), SCAP_OK otherwise.  Not for use during stream capture.                   */
+scap_status scap_device_status(void);
 
 /* ------------------------------------------------------------------------------------------
  * Offline calibration (Section 3, "Mode-Centering Calibration"; Eq. 2 for tau)

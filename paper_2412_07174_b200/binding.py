@@ -7,7 +7,7 @@ import os
 import torch
 
 __all__ = [
-    "SCAP_F16", "SCAP_BF16", "ScapError", "lib", "lib_path", "status_string", "scap_version", "scap_tune",
+    "SCAP_F16", "SCAP_BF16", "ScapError", "lib", "lib_path", "status_string", "scap_version", "scap_tune", "scap_device_status",
     "scap_calibrate_workspace", "scap_calibrate", "scap_fold_bias_workspace", "scap_fold_bias",
     "scap_fc_workspace", "scap_sparse_fc", "scap_dense_fc", "scap_fc_host_workspace", "scap_sparse_fc_host",
     "scap_glu_workspace", "scap_glu_ffn", "scap_glu_static_capacity", "scap_glu_ffn_static", "scap_moe_workspace",
@@ -19,7 +19,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 
 # every symbol include/scap.h declares
 EXPORTS = [
-    "scap_status_string", "scap_version", "scap_tune", "scap_calibrate_workspace", "scap_calibrate",
+    "scap_status_string", "scap_version", "scap_tune", "scap_device_status", "scap_calibrate_workspace", "scap_calibrate",
     "scap_fold_bias_workspace", "scap_fold_bias", "scap_fc_workspace", "scap_sparse_fc", "scap_dense_fc",
     "scap_fc_host_workspace", "scap_sparse_fc_host", "scap_glu_workspace", "scap_glu_ffn",
     "scap_glu_static_capacity", "scap_glu_ffn_static", "scap_moe_workspace", "scap_moe_ffn",
@@ -60,6 +60,8 @@ def lib():
     L.scap_version.restype = i
     L.scap_tune.argtypes = [C.c_char_p, i]
     L.scap_tune.restype = i
+    L.scap_device_status.argtypes = []
+    L.scap_device_status.restype = i
     L.scap_calibrate_workspace.argtypes = [i, i, i]
     L.scap_calibrate_workspace.restype = sz
     L.scap_calibrate.argtypes = [vp, i, i, i, d, i, vp, vp, vp, sz, vp]
@@ -109,6 +111,11 @@ def _check(code: int, where: str) -> None:
 
 def scap_tune(key: str, value: int) -> None:
     _check(lib().scap_tune(key.encode(), int(value)), "scap_tune")
+
+
+def scap_device_status() -> None:
+    """Synchronises the device; raises ScapError(SCAP_ERR_TIMEOUT) if a bounded wait of the tcgen05 kernel ran out."""
+    _check(lib().scap_device_status(), "scap_device_status")
 
 
 def _ptr(t):

@@ -17,6 +17,7 @@ constexpr int SCAP_MAX_K = 1 << 20;  // input channels per FC (keeps every index
 struct Tuning {
     int split_k;  // 0 = automatic
     int pdl;      // programmatic dependent launch between the kernels of one call
+    int tc;       // batch 3..16 on the tcgen05 kernel (0: the mma.sync variants)
 };
 extern Tuning g_tune;
 

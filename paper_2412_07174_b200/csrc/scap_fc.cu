@@ -6,7 +6,7 @@
 
 namespace scap {
 
-Tuning g_tune = {0, 1};
+Tuning g_tune = {0, 1, 0};
 
 scap_status check_device() {
     static int cached[64];  // 0 unknown, 1 ok, 2 unsupported
@@ -134,6 +134,12 @@ static cudaError_t launch_fc_w(int mode, int xkind, int epi, const FcArgs &a, cu
 }
 
 cudaError_t launch_fc(bool bf16, int mode, int xkind, int epi, const FcArgs &a, cudaStream_t st) {
+    if (tc_applicable(a, xkind)) {
+        FcArgs t = a;
+        t.tn = 256;
+        t.S = tc_choose_split(a.K, a.Nh, epi, a.B, bf16);
+        return launch_fc_tc(bf16, mode, xkind, epi, t, st);
+    }
     return bf16 ? launch_fc_w<true>(mode, xkind, epi, a, st) : launch_fc_w<false>(mode, xkind, epi, a, st);
 }
 
@@ -239,7 +245,13 @@ const char *scap_status_string(scap_status st) {
     return "SCAP_ERR_UNKNOWN";
 }
 
-int scap_version(void) { return 1001; }
+int scap_version(void) { return 1002; }
+
+scap_status scap_device_status(void) {
+    const int v = tc_take_status();
+    if (v < 0) return SCAP_ERR_CUDA;
+    return v == 0 ? SCAP_OK : SCAP_ERR_TIMEOUT;
+}
 
 scap_status scap_tune(const char *key, int value) {
     if (!key) return SCAP_ERR_INVALID_ARG;
@@ -250,6 +262,10 @@ scap_status scap_tune(const char *key, int value) {
     }
     if (!strcmp(key, "pdl")) {
         g_tune.pdl = value != 0;
+        return SCAP_OK;
+    }
+    if (!strcmp(key, "tcgen05")) {
+        g_tune.tc = value != 0;
         return SCAP_OK;
     }
     return SCAP_ERR_INVALID_ARG;

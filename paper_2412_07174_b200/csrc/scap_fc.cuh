@@ -796,6 +796,13 @@ inline int fc_tiles(int Nh, int epi, int tn) { return epi == EPI_GLU ? (Nh + tn 
 // `groups` concurrently active groups (experts): the pair with the most CTAs that are still all co-resident.
 void choose_config(int K, int Nh, int epi, int groups, int B, int *tn, int *S);
 
+// tcgen05 kernel for batch 3..16 (scap_fc_tc.cu): whether it can take this call, its split-K factor, its launch,
+// and the status word of its bounded waits (0 = none ran out; reading synchronises the device and clears it).
+bool tc_applicable(const FcArgs &a, int xkind);
+int tc_choose_split(int K, int Nh, int epi, int B, bool bf16);
+cudaError_t launch_fc_tc(bool bf16, int mode, int xkind, int epi, const FcArgs &a, cudaStream_t st);
+int tc_take_status();
+
 // Launch with cluster dimension (1, S, 1) and, if enabled, programmatic dependent launch.
 template <typename... KArgs, typename... Args>
 inline cudaError_t launch_cluster(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, int cluster_y,

@@ -1,0 +1,554 @@
+// Batch 3..16 on the 5th-generation tensor cores: the sparse FC of Eq. 2-3 / Eq. 6 / Alg. 3 as
+//   TMA row gather (cp.async.bulk.tensor tile::gather4)  ->  shared-memory ring  ->  tcgen05.mma  ->  TMEM.
+//
+// Same decomposition as the FMA kernel (grid = column tiles x S, the S CTAs of a tile form a cluster and split the
+// input channels by interleaved 32-channel chunks, cluster exchange of the partial tiles at the end), but one CTA
+// per SM with a deep ring:
+//   prologue   all 8 warps: d = x - m, |d| >= tau, union over the batch, ballot compaction (ascending kept list),
+//              and the pruned values split exactly into parts of the weight dtype (bf16: hi+mid+lo, fp16: hi+lo)
+//              written as the A operand: row (part * Bp + b), K-major core matrices of 8 rows x 16 bytes;
+//   warp 0     producer: per block of 16 kept rows, 16 gather4 copies (4 rows x 64 columns each, 128-byte swizzle)
+//              fill one 8 KB stage laid out as the MN-major B operand (N = 256 columns of W);
+//   warp 1     one lane issues tcgen05.mma M=128 N=256 K=16 per block (all parts of all batch rows at once, rows
+//              beyond parts * Bp read whatever follows in shared memory and produce accumulator rows nobody reads)
+//              and commits to the stage's "empty" barrier; the accumulator (128 lanes x 256 fp32 columns) stays in
+//              TMEM across blocks and fills;
+//   epilogue   warps 0-1 read the accumulator rows, the parts are added smallest first, and the cluster exchange
+//              and bias / SwiGLU epilogue are those of the other variants.
+// Every wait on an mbarrier is bounded; a wait that runs out sets a device status word, the CTA stops issuing work,
+// still passes every cluster barrier and frees its TMEM.
+#include <cuda.h>
+#include <string.h>
+
+#include "scap_fc.cuh"
+
+namespace scap {
+
+constexpr int TC_TN = 256;                          // columns per CTA
+constexpr int TC_STAGE = 16 * TC_TN * 2;            // bytes of one block of 16 kept rows
+constexpr int TC_NST = 16;                          // ring stages (128 KB in flight per SM)
+constexpr int TC_CAP = 1408;                        // most kept channels per fill (44 chunks)
+constexpr int TC_PLANE = TC_CAP * 48 + 2048;        // A-operand bytes: 48 per channel (3 parts x 8 rows x 2) + read slack
+constexpr int TC_PU = 6;                            // chunks per warp per fill, at most
+constexpr int TC_PART_LD = 257;                     // row pitch of the accumulator copy (conflict-free)
+constexpr uint32_t TC_SPIN = 1u << 20;              // polls before a wait gives up (tens of milliseconds)
+
+// shared-memory map (offsets from a 1024-byte aligned base)
+constexpr int TC_OFF_RING = 0;
+constexpr int TC_OFF_PLANE = TC_OFF_RING + TC_NST * TC_STAGE;
+constexpr int TC_OFF_K = TC_OFF_PLANE + TC_PLANE;
+constexpr int TC_OFF_GATHER = TC_OFF_K + TC_CAP * 4;
+constexpr int TC_OFF_MISC = TC_OFF_GATHER + 16 * GATHER_LD * 4;
+constexpr int TC_SMEM = TC_OFF_MISC + 1024 + 1024;  // misc block + alignment slack
+static_assert(48 * TC_PART_LD * 4 <= TC_NST * TC_STAGE, "accumulator copy must fit in the ring");
+static_assert(TC_SMEM <= 232448, "exceeds the shared memory of an SM");
+
+__device__ int g_tc_status;  // 0, or the code of the first bounded wait that ran out
+
+struct TcMisc {
+    unsigned long long full[TC_NST];
+    unsigned long long empty[TC_NST];
+    unsigned long long fill_done;
+    uint32_t tmem_base;
+    int abort;
+    int wcnt[FC_WARPS];
+    int rows[16];
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(unsigned long long *bar, int count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(unsigned long long *bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_test(unsigned long long *bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{ .reg .pred p; mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+                 : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait: false (and the status word set) when the phase did not complete within TC_SPIN polls.
+__device__ __forceinline__ bool mbar_wait(unsigned long long *bar, uint32_t parity, int code, volatile int *abort_flag) {
+    for (uint32_t i = 0; i < TC_SPIN; ++i) {
+        if (mbar_test(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (i > 64) __nanosleep(32);
+    }
+    atomicCAS(&g_tc_status, 0, code);
+    *abort_flag = 1;
+    return false;
+}
+
+__device__ __forceinline__ void tma_gather4(const CUtensorMap *tmap, unsigned long long *bar, void *dst, int x, int y0, int y1,
+                                            int y2, int y3) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile::gather4.mbarrier::complete_tx::bytes"
+        " [%0], [%1, {%3, %4, %5, %6, %7}], [%2];" ::"r"(smem_u32(dst)),
+        "l"(reinterpret_cast<uint64_t>(tmap)), "r"(smem_u32(bar)), "r"(x), "r"(y0), "r"(y1), "r"(y2), "r"(y3)
+        : "memory");
+}
+
+__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}\n" ::"r"(d_tmem),
+        "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(0u)
+        : "memory");
+}
+__device__ __forceinline__ void tc_commit(unsigned long long *bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// Shared-memory matrix descriptor (start address, leading / stride byte offsets in 16-byte units, version 1, swizzle).
+__device__ __forceinline__ uint64_t tc_desc(uint32_t addr, uint32_t lbo, uint32_t sbo, uint32_t layout) {
+    return (uint64_t)((addr >> 4) & 0x3fffu) | ((uint64_t)((lbo >> 4) & 0x3fffu) << 16) |
+           ((uint64_t)((sbo >> 4) & 0x3fffu) << 32) | (1ull << 46) | ((uint64_t)layout << 61);
+}
+
+template <bool BF16, int MODE, typename XT, int EPI>
+__global__ void __launch_bounds__(FC_THREADS, 1) fc_tc_kernel(const FcArgs a, const __grid_constant__ CUtensorMap tmap) {
+    constexpr int TNT = TC_TN, HALF = TNT / 2, NSPLIT = mma_nsplit(BF16);
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    unsigned char *s_ring = smem + TC_OFF_RING;
+    unsigned char *s_plane = smem + TC_OFF_PLANE;
+    uint32_t *s_k = reinterpret_cast<uint32_t *>(smem + TC_OFF_K);
+    float *s_gather = reinterpret_cast<float *>(smem + TC_OFF_GATHER);  // this CTA's partial tile [b][TNT]
+    TcMisc *misc = reinterpret_cast<TcMisc *>(smem + TC_OFF_MISC);
+    float *s_part = reinterpret_cast<float *>(s_ring);                   // accumulator rows, after the stream
+    volatile int *abort_flag = &misc->abort;
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int tile = blockIdx.x, s = blockIdx.y;
+    const int B = a.B, S = a.S, K = a.K;
+    const int Bp = B <= 8 ? 8 : 16;            // batch rows per part in the A operand
+    const int G = NSPLIT * Bp / 8;             // 8-row groups of the A operand in use
+    const uint32_t LBO = G * 128, BLK = 2 * LBO;  // bytes: between the two K halves of a block, and per block
+    const int cap_chunks = min(TC_CAP / 32, (TC_CAP * 48) / (NSPLIT * Bp * 2) / 32);
+    const XT *xg = reinterpret_cast<const XT *>(a.x);
+
+    if (tid == 0) {
+        for (int i = 0; i < TC_NST; ++i) {
+            mbar_init(&misc->full[i], 1);
+            mbar_init(&misc->empty[i], 1);
+        }
+        mbar_init(&misc->fill_done, 1);
+        misc->abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0) {  // the accumulator: 256 TMEM columns, allocated by warp 0 and freed by it at the end
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&misc->tmem_base)), "r"(256)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+
+    const int per = ((EPI == EPI_GLU ? HALF : TNT) + S - 1) / S;
+    float bias0[2], bias1[2];
+    prefetch_bias<BF16, EPI, TNT>(a, tile, s, per, bias0, bias1);
+
+    const int nchunks = (K + 31) >> 5;
+    const int my_chunks = nchunks > s ? (nchunks - s + S - 1) / S : 0;
+    float tau = 0.0f;
+    if constexpr (MODE == MODE_GATHER) tau = ld_nc(a.tau);
+
+    griddep_wait();  // the row map and the activations are outputs of the previous kernel
+    griddep_launch_dependents();
+    if (a.in_rows && tid < 16) misc->rows[tid] = __ldcg(a.in_rows + (tid < B ? tid : 0));
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = misc->tmem_base;
+
+    uint32_t blocks_done = 0;  // blocks streamed so far by this CTA (ring position), the same in every thread
+    int fills_done = 0;
+    const uint32_t idesc = (1u << 4) | ((BF16 ? 1u : 0u) << 7) | ((BF16 ? 1u : 0u) << 10) | (0u << 15) | (1u << 16) |
+                           ((uint32_t)(TNT >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+
+    for (int j0 = 0; j0 < my_chunks; j0 += cap_chunks) {
+        const int nj = min(cap_chunks, my_chunks - j0);
+        const int pu = (nj + FC_WARPS - 1) / FC_WARPS;  // consecutive chunks per warp
+        // ---- keep masks: all activation loads of a lane in flight together, values kept in registers
+        float mk[TC_PU];
+        XT xraw[TC_PU][16];
+        uint32_t km[TC_PU];
+        unsigned bal[TC_PU];
+#pragma unroll
+        for (int p = 0; p < TC_PU; ++p) {
+            const int j = warp * pu + p;
+            const int k = (s + S * (j0 + j)) * 32 + lane;
+            mk[p] = a.m ? ld_nc_if(a.m + k, p < pu && j < nj && k < K) : 0.0f;
+        }
+#pragma unroll
+        for (int p = 0; p < TC_PU; ++p) {
+            const int j = warp * pu + p;
+            const int k = (s + S * (j0 + j)) * 32 + lane;
+            const bool ok = p < pu && j < nj && k < K;
+#pragma unroll
+            for (int b = 0; b < 16; ++b) {
+                const int row = a.in_rows ? misc->rows[b] : b;
+                xraw[p][b] = ld_act_if(xg + (size_t)row * a.x_ld + k, ok && b < B);
+            }
+        }
+        int my_off[TC_PU], wtotal = 0;
+#pragma unroll
+        for (int p = 0; p < TC_PU; ++p) {
+            const int j = warp * pu + p;
+            const int k = (s + S * (j0 + j)) * 32 + lane;
+            const bool ok = p < pu && j < nj && k < K;
+            uint32_t m_ = 0;
+            if constexpr (MODE == MODE_GATHER) {
+#pragma unroll
+                for (int b = 0; b < 16; ++b) {
+                    const float xv = widen1(xraw[p][b]);
+                    const float dv = a.m ? __fsub_rn(xv, mk[p]) : xv;
+                    m_ |= (ok && b < B && fabsf(dv) >= tau) ? (1u << b) : 0u;
+                }
+            } else {
+                m_ = ok ? 1u : 0u;
+            }
+            km[p] = m_;
+            bal[p] = __ballot_sync(0xffffffffu, m_ != 0);
+            my_off[p] = wtotal;
+            wtotal += __popc(bal[p]);
+        }
+        if (lane == 0) misc->wcnt[warp] = wtotal;
+        if (MODE == MODE_GATHER && a.bits && tile == 0) {
+            unsigned mine = 0;
+#pragma unroll
+            for (int p = 0; p < TC_PU; ++p) mine = lane == p ? bal[p] : mine;
+            const int j = warp * pu + lane;
+            if (lane < pu && j < nj) a.bits[s + S * (j0 + j)] = mine;
+        }
+        __syncthreads();
+        int cnt = 0, wbase = 0;
+#pragma unroll
+        for (int w = 0; w < FC_WARPS; ++w) {
+            const int c = misc->wcnt[w];
+            cnt += c;
+            wbase += w < warp ? c : 0;
+        }
+        // ---- kept list and A operand.  Element (row r = part * Bp + b, kept position pos): block pos / 16,
+        // K half (pos / 8) & 1, 8-row group r / 8, then 16 bytes per row of the group, 2 bytes per position.
+#pragma unroll
+        for (int p = 0; p < TC_PU; ++p) {
+            if (km[p]) {
+                const int j = warp * pu + p;
+                const int k = (s + S * (j0 + j)) * 32 + lane;
+                const int pos = wbase + my_off[p] + __popc(bal[p] & ((1u << lane) - 1u));
+                s_k[pos] = (uint32_t)k;
+                unsigned char *blk = s_plane + (size_t)(pos >> 4) * BLK + ((pos >> 3) & 1) * LBO + (pos & 7) * 2;
+#pragma unroll
+                for (int b = 0; b < 16; ++b) {
+                    if (b < Bp) {
+                        const float xv = widen1(xraw[p][b]);
+                        const float dv = (MODE == MODE_GATHER && a.m) ? __fsub_rn(xv, mk[p]) : xv;
+                        const bool kept = MODE == MODE_DENSE ? (b < B) : (((km[p] >> b) & 1u) != 0);
+                        unsigned short part[3];
+                        split_parts<BF16>(kept ? dv : 0.0f, part);
+#pragma unroll
+                        for (int q = 0; q < NSPLIT; ++q) {
+                            const int r = q * Bp + b;
+                            *reinterpret_cast<unsigned short *>(blk + (r >> 3) * 128 + (r & 7) * 16) = part[q];
+                        }
+                    }
+                }
+            }
+        }
+        __syncthreads();
+        // The last block is completed with copies of the last kept row and zero activations (a padded row adds
+        // exactly 0 for finite weights).
+        const int cnt_pad = (cnt + 15) & ~15;
+        if (tid < 16 && cnt > 0 && cnt + tid < cnt_pad) {
+            const int pos = cnt + tid;
+            s_k[pos] = s_k[cnt - 1];
+            unsigned char *blk = s_plane + (size_t)(pos >> 4) * BLK + ((pos >> 3) & 1) * LBO + (pos & 7) * 2;
+            for (int r = 0; r < NSPLIT * Bp; ++r) *reinterpret_cast<unsigned short *>(blk + (r >> 3) * 128 + (r & 7) * 16) = 0;
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes -> visible to the tensor core
+        __syncthreads();
+
+        const uint32_t nblk = (uint32_t)cnt_pad >> 4;
+        if (warp == 0) {
+            // ---- producer: block q goes to ring stage (blocks_done + q) % TC_NST
+            for (uint32_t q = 0; q < nblk; ++q) {
+                const uint32_t it = blocks_done + q, st = it % TC_NST, n = it / TC_NST;
+                bool ok = true;
+                if (lane == 0) {
+                    ok = mbar_wait(&misc->empty[st], (n & 1u) ^ 1u, 1, abort_flag);
+                    if (ok) mbar_expect_tx(&misc->full[st], TC_STAGE);
+                }
+                ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+                if (!ok) break;
+                if (lane < 16) {  // lane = (column quarter, row quad): 4 rows x 64 columns = 512 bytes each
+                    const int nh = lane >> 2, rq = lane & 3;
+                    int xc;
+                    if constexpr (EPI == EPI_GLU) xc = (nh >> 1) * a.Nh + tile * HALF + (nh & 1) * 64;
+                    else xc = tile * TNT + nh * 64;
+                    const uint32_t *rows = s_k + q * 16 + rq * 4;
+                    unsigned char *dst = s_ring + st * TC_STAGE + (rq >> 1) * 4096 + nh * 1024 + (rq & 1) * 512;
+                    tma_gather4(&tmap, &misc->full[st], dst, xc, (int)rows[0], (int)rows[1], (int)rows[2], (int)rows[3]);
+                }
+                __syncwarp();
+            }
+        } else if (warp == 1) {
+            // ---- MMA issuer
+            for (uint32_t q = 0; q < nblk; ++q) {
+                const uint32_t it = blocks_done + q, st = it % TC_NST, n = it / TC_NST;
+                bool ok = true;
+                if (lane == 0) {
+                    ok = mbar_wait(&misc->full[st], n & 1u, 2, abort_flag);
+                    if (ok) {
+                        tc_fence_after();
+                        const uint64_t da = tc_desc(smem_u32(s_plane) + q * BLK, LBO, 128, 0);
+                        const uint64_t db = tc_desc(smem_u32(s_ring) + st * TC_STAGE, 1024, 4096, 2);
+                        tc_mma(tmem, da, db, idesc, it > 0 ? 1u : 0u);
+                        tc_commit(&misc->empty[st]);  // arrives once the MMA has read the stage
+                    }
+                }
+                ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+                if (!ok) break;
+            }
+            if (nblk > 0 && lane == 0 && !*abort_flag) tc_commit(&misc->fill_done);
+            __syncwarp();
+        }
+        // ---- the A operand and the kept list are reused by the next fill: wait until this fill's MMAs are done
+        if (nblk > 0) {
+            mbar_wait(&misc->fill_done, (uint32_t)fills_done & 1u, 3, abort_flag);
+            ++fills_done;
+        }
+        blocks_done += nblk;
+        tc_fence_before();
+        __syncthreads();
+        tc_fence_after();
+        if (*abort_flag) break;
+    }
+
+    // ---- accumulator rows -> shared memory (the ring is idle now), parts added smallest first
+    const bool have_acc = blocks_done > 0 && !*abort_flag;
+    const int acc_rows = NSPLIT * Bp;
+    if (have_acc && warp * 32 < acc_rows && warp < 2) {
+#pragma unroll 1
+        for (int c0 = 0; c0 < TNT; c0 += 32) {
+            uint32_t v[32];
+            asm volatile(
+                "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+                "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+                : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+                  "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
+                  "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
+                  "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+                : "r"(tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0));
+            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+            const int r = warp * 32 + lane;
+            if (r < acc_rows) {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) s_part[r * TC_PART_LD + c0 + j] = __uint_as_float(v[j]);
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(256) : "memory");
+    for (int i = tid; i < 16 * TNT; i += FC_THREADS) {
+        const int b = i / TNT, c = i - b * TNT;
+        float v = 0.0f;
+        if (have_acc && b < Bp) {
+#pragma unroll
+            for (int q = NSPLIT - 1; q >= 0; --q) v += s_part[(q * Bp + b) * TC_PART_LD + c];
+        }
+        s_gather[i] = v;
+    }
+
+    // ---- cluster exchange, pull form, and the bias / SwiGLU epilogue
+    cg::cluster_group cluster = cg::this_cluster();
+    if (S > 1) cluster.sync();
+    else __syncthreads();
+    const float *peer[MAX_CLUSTER];
+#pragma unroll
+    for (int q = 0; q < MAX_CLUSTER; ++q) peer[q] = (S > 1 && q < S) ? cluster.map_shared_rank(s_gather, q) : s_gather;
+    for (int it = 0; tid + it * FC_THREADS < per * B; ++it) {
+        const int i = tid + it * FC_THREADS;
+        const int b = i / per, c = i - b * per;
+        const int row = a.out_rows ? __ldcg(a.out_rows + b) : b;
+        if constexpr (EPI == EPI_BIAS) {
+            const int n = tile * TNT + s * per + c;
+            if (s * per + c < TNT && n < a.Nh) {
+                float v = it == 0 ? bias0[0] : it == 1 ? bias0[1] : load_bias<BF16>(a, n);
+#pragma unroll
+                for (int q = 0; q < MAX_CLUSTER; ++q)
+                    if (q < S) v += peer[q][b * TNT + s * per + c];
+                a.y[(size_t)row * a.y_ld + n] = v;
+            }
+        } else {
+            const int F = a.Nh, f = tile * HALF + s * per + c;
+            if (s * per + c < HALF && f < F) {
+                float gt = it == 0 ? bias0[0] : it == 1 ? bias0[1] : (a.bias ? __ldg(a.bias + f) : 0.0f);
+                float up = it == 0 ? bias1[0] : it == 1 ? bias1[1] : (a.bias ? __ldg(a.bias + F + f) : 0.0f);
+#pragma unroll
+                for (int q = 0; q < MAX_CLUSTER; ++q)
+                    if (q < S) {
+                        gt += peer[q][b * TNT + s * per + c];
+                        up += peer[q][b * TNT + HALF + s * per + c];
+                    }
+                const float z = up * (gt / (1.0f + expf(-gt)));  // up * silu(gate)
+                a.y[(size_t)row * a.y_ld + f] = z;
+                if (a.z_copy) a.z_copy[(size_t)b * F + f] = z;
+            }
+        }
+    }
+    if (S > 1) cluster.sync();
+}
+
+// ---- host side ------------------------------------------------------------------------------------------------
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
+                                  const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult qr;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qr) == cudaSuccess &&
+            qr == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+        else
+            cudaGetLastError();
+    }
+    return fn;
+}
+
+// Tensor map of W[K, ldw] for row gathers: box = 64 columns x 1 row, 128-byte swizzle, zero fill outside.
+static bool make_map(const void *W, int K, int ldw, bool bf16, CUtensorMap *out) {
+    struct Key { const void *W; int K, ldw, bf16; };
+    struct Slot { Key k; CUtensorMap m; bool used; };
+    static Slot cache[64];
+    static int next = 0;
+    for (int i = 0; i < 64; ++i)
+        if (cache[i].used && cache[i].k.W == W && cache[i].k.K == K && cache[i].k.ldw == ldw && cache[i].k.bf16 == (int)bf16) {
+            *out = cache[i].m;
+            return true;
+        }
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)ldw, (cuuint64_t)K};
+    const cuuint64_t strides[1] = {(cuuint64_t)ldw * 2};
+    const cuuint32_t box[2] = {64, 1};
+    const cuuint32_t estr[2] = {1, 1};
+    CUtensorMap m;
+    if (fn(&m, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void *>(W), dims, strides, box,
+           estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return false;
+    Slot &sl = cache[next];
+    next = (next + 1) % 64;
+    sl.k = Key{W, K, ldw, (int)bf16};
+    sl.m = m;
+    sl.used = true;
+    *out = m;
+    return true;
+}
+
+template <bool BF16, int MODE, typename XT, int EPI>
+static cudaError_t launch_tc_t(const FcArgs &a, const CUtensorMap &map, cudaStream_t st) {
+    static bool attr_done = false;
+    auto kern = fc_tc_kernel<BF16, MODE, XT, EPI>;
+    if (!attr_done) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM);
+        if (e != cudaSuccess) return e;
+        attr_done = true;
+    }
+    return launch_cluster(kern, dim3(fc_tiles(a.Nh, EPI, TC_TN), a.S), dim3(FC_THREADS), TC_SMEM, a.S, st, g_tune.pdl != 0, a, map);
+}
+
+template <bool BF16, int MODE, typename XT>
+static cudaError_t launch_tc_e(int epi, const FcArgs &a, const CUtensorMap &map, cudaStream_t st) {
+    return epi == EPI_GLU ? launch_tc_t<BF16, MODE, XT, EPI_GLU>(a, map, st) : launch_tc_t<BF16, MODE, XT, EPI_BIAS>(a, map, st);
+}
+
+template <bool BF16>
+static cudaError_t launch_tc_w(int mode, int xkind, int epi, const FcArgs &a, const CUtensorMap &map, cudaStream_t st) {
+    using ST = typename std::conditional<BF16, __nv_bfloat16, __half>::type;
+    if (mode == MODE_DENSE)
+        return xkind == 2 ? launch_tc_e<BF16, MODE_DENSE, float>(epi, a, map, st) : launch_tc_e<BF16, MODE_DENSE, ST>(epi, a, map, st);
+    return xkind == 2 ? launch_tc_e<BF16, MODE_GATHER, float>(epi, a, map, st) : launch_tc_e<BF16, MODE_GATHER, ST>(epi, a, map, st);
+}
+
+// CTAs of clusters of size S resident at once with one CTA per SM.
+static int tc_resident(int S) {
+    static int cached[MAX_CLUSTER + 1];
+    if (cached[S]) return cached[S];
+    int n = sm_count();
+    if (S > 1) {
+        auto kern = fc_tc_kernel<true, MODE_GATHER, __nv_bfloat16, EPI_BIAS>;
+        cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM);
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(1, S);
+        cfg.blockDim = dim3(FC_THREADS);
+        cfg.dynamicSmemBytes = TC_SMEM;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 1;
+        attr[0].val.clusterDim.y = S;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        int clusters = 0;
+        if (cudaOccupancyMaxActiveClusters(&clusters, kern, &cfg) == cudaSuccess && clusters > 0) n = clusters * S;
+        else { cudaGetLastError(); n = (sm_count() / S - 2) * S; }
+    }
+    cached[S] = n;
+    return n;
+}
+
+bool tc_applicable(const FcArgs &a, int xkind) {
+    (void)xkind;
+    return g_tune.tc != 0 && a.B >= 3 && a.B <= 16 && a.ldw % 8 == 0 && aligned16(a.W) && !a.hold_dependents && encode_fn() != nullptr;
+}
+
+// Split-K factor for the tensor-core kernel (tile width is fixed at 256): most CTAs that are all resident with
+// one CTA per SM; ties: fewer fills, then the smaller cluster.
+int tc_choose_split(int K, int Nh, int epi, int B, bool bf16) {
+    const int tiles = fc_tiles(Nh, epi, TC_TN);
+    const int nchunks = (K + 31) / 32;
+    const int bp = B <= 8 ? 8 : 16, nsplit = bf16 ? 3 : 2;
+    int cap_chunks = (TC_CAP * 48) / (nsplit * bp * 2) / 32;
+    if (cap_chunks > TC_CAP / 32) cap_chunks = TC_CAP / 32;
+    int best_S = 1;
+    long long best = -1;
+    for (int S = 1; S <= MAX_CLUSTER; ++S) {
+        if (g_tune.split_k > 0 && S > g_tune.split_k) continue;
+        if (S > 1 && K / S < 64) continue;
+        const long long ctas = (long long)tiles * S;
+        if (S > 1 && ctas > tc_resident(S)) continue;
+        const int fills = ((nchunks + S - 1) / S + cap_chunks - 1) / cap_chunks;
+        const long long score = (ctas > sm_count() ? 0 : ctas * 64) + (63 - (fills < 63 ? fills : 63));
+        if (score > best) { best = score; best_S = S; }
+    }
+    return best_S;
+}
+
+cudaError_t launch_fc_tc(bool bf16, int mode, int xkind, int epi, const FcArgs &a, cudaStream_t st) {
+    CUtensorMap map;
+    if (!make_map(a.W, a.K, a.ldw, bf16, &map)) return cudaErrorNotSupported;
+    return bf16 ? launch_tc_w<true>(mode, xkind, epi, a, map, st) : launch_tc_w<false>(mode, xkind, epi, a, map, st);
+}
+
+// Reads and clears the status word of the bounded waits (synchronises the device).
+int tc_take_status() {
+    int v = 0, zero = 0;
+    if (cudaDeviceSynchronize() != cudaSuccess) { cudaGetLastError(); return -1; }
+    if (cudaMemcpyFromSymbol(&v, g_tc_status, sizeof(int)) != cudaSuccess) { cudaGetLastError(); return -1; }
+    if (v) cudaMemcpyToSymbol(g_tc_status, &zero, sizeof(int));
+    return v;
+}
+
+}  // namespace scap
