@@ -1,5 +1,5 @@
 // Batch 3..16 on the 5th-generation tensor cores: the sparse FC of Eq. 2-3 / Eq. 6 / Alg. 3 as
-//   TMA row gather (cp.async.bulk.tensor tile::gather4)  ->  shared-memory ring  ->  tcgen05.mma  ->  TMEM.
+//   16-byte asynchronous row copies  ->  swizzled shared-memory ring  ->  tcgen05.mma  ->  accumulator in TMEM.
 //
 // Same decomposition as the FMA kernel (grid = column tiles x S, the S CTAs of a tile form a cluster and split the
 // input channels by interleaved 32-channel chunks, cluster exchange of the partial tiles at the end), but one CTA
@@ -7,17 +7,21 @@
 //   prologue   all 8 warps: d = x - m, |d| >= tau, union over the batch, ballot compaction (ascending kept list),
 //              and the pruned values split exactly into parts of the weight dtype (bf16: hi+mid+lo, fp16: hi+lo)
 //              written as the A operand: row (part * Bp + b), K-major core matrices of 8 rows x 16 bytes;
-//   warp 0     producer: per block of 16 kept rows, 16 gather4 copies (4 rows x 64 columns each, 128-byte swizzle)
-//              fill one 8 KB stage laid out as the MN-major B operand (N = 256 columns of W);
-//   warp 1     one lane issues tcgen05.mma M=128 N=256 K=16 per block (all parts of all batch rows at once, rows
-//              beyond parts * Bp read whatever follows in shared memory and produce accumulator rows nobody reads)
-//              and commits to the stage's "empty" barrier; the accumulator (128 lanes x 256 fp32 columns) stays in
-//              TMEM across blocks and fills;
+//   7 warps    producers: a warp moves one kept row (512 bytes of the tile) per instruction with 16-byte
+//              asynchronous copies (cp.async) straight into the row's place in a ring stage of 64 rows = four
+//              8 KB blocks, each laid out as the MN-major, 128-byte-swizzled B operand (N = 256 columns of W,
+//              K = 16 rows); an asynchronous arrival per lane and stage fires when the copies have landed, so
+//              producers never wait for data and the whole ring is the in-flight buffer;
+//   warp 1     one lane waits per stage and issues tcgen05.mma M=128 N=256 K=16 per block of 16 rows (all parts of all batch rows at
+//              once; rows of M beyond parts * Bp read whatever follows in shared memory and produce accumulator
+//              rows nobody reads) and commits to the stage's "empty" barrier; the accumulator (128 lanes x 256
+//              fp32 columns) stays in TMEM across blocks and fills;
 //   epilogue   warps 0-1 read the accumulator rows, the parts are added smallest first, and the cluster exchange
 //              and bias / SwiGLU epilogue are those of the other variants.
+// (A TMA row gather - cp.async.bulk.tensor tile::gather4, four rows x 128 bytes per instruction - was measured
+// first and was no faster on this access pattern.)
 // Every wait on an mbarrier is bounded; a wait that runs out sets a device status word, the CTA stops issuing work,
 // still passes every cluster barrier and frees its TMEM.
-#include <cuda.h>
 #include <string.h>
 
 #include "scap_fc.cuh"
@@ -25,8 +29,10 @@
 namespace scap {
 
 constexpr int TC_TN = 256;                          // columns per CTA
-constexpr int TC_STAGE = 16 * TC_TN * 2;            // bytes of one block of 16 kept rows
-constexpr int TC_NST = 16;                          // ring stages (128 KB in flight per SM)
+constexpr int TC_KB = 16 * TC_TN * 2;               // bytes of one block of 16 kept rows (one MMA)
+constexpr int TC_SROWS = 64;                        // kept rows per ring stage (4 blocks)
+constexpr int TC_STAGE = TC_SROWS * TC_TN * 2;      // 32 KB
+constexpr int TC_NST = 4;                           // ring stages (128 KB per SM)
 constexpr int TC_CAP = 1408;                        // most kept channels per fill (44 chunks)
 constexpr int TC_PLANE = TC_CAP * 48 + 2048;        // A-operand bytes: 48 per channel (3 parts x 8 rows x 2) + read slack
 constexpr int TC_PU = 6;                            // chunks per warp per fill, at most
@@ -60,8 +66,8 @@ __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)_
 __device__ __forceinline__ void mbar_init(unsigned long long *bar, int count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
 }
-__device__ __forceinline__ void mbar_expect_tx(unsigned long long *bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+__device__ __forceinline__ void mbar_arrive(unsigned long long *bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 __device__ __forceinline__ bool mbar_test(unsigned long long *bar, uint32_t parity) {
     uint32_t ok;
@@ -79,15 +85,6 @@ __device__ __forceinline__ bool mbar_wait(unsigned long long *bar, uint32_t pari
     atomicCAS(&g_tc_status, 0, code);
     *abort_flag = 1;
     return false;
-}
-
-__device__ __forceinline__ void tma_gather4(const CUtensorMap *tmap, unsigned long long *bar, void *dst, int x, int y0, int y1,
-                                            int y2, int y3) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.tile::gather4.mbarrier::complete_tx::bytes"
-        " [%0], [%1, {%3, %4, %5, %6, %7}], [%2];" ::"r"(smem_u32(dst)),
-        "l"(reinterpret_cast<uint64_t>(tmap)), "r"(smem_u32(bar)), "r"(x), "r"(y0), "r"(y1), "r"(y2), "r"(y3)
-        : "memory");
 }
 
 __device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
@@ -110,7 +107,7 @@ __device__ __forceinline__ uint64_t tc_desc(uint32_t addr, uint32_t lbo, uint32_
 }
 
 template <bool BF16, int MODE, typename XT, int EPI>
-__global__ void __launch_bounds__(FC_THREADS, 1) fc_tc_kernel(const FcArgs a, const __grid_constant__ CUtensorMap tmap) {
+__global__ void __launch_bounds__(FC_THREADS, 1) fc_tc_kernel(const FcArgs a) {
     constexpr int TNT = TC_TN, HALF = TNT / 2, NSPLIT = mma_nsplit(BF16);
     extern __shared__ unsigned char smem_raw[];
     unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -133,7 +130,7 @@ __global__ void __launch_bounds__(FC_THREADS, 1) fc_tc_kernel(const FcArgs a, co
 
     if (tid == 0) {
         for (int i = 0; i < TC_NST; ++i) {
-            mbar_init(&misc->full[i], 1);
+            mbar_init(&misc->full[i], (FC_WARPS - 1) * 32);  // one arrival per producer lane
             mbar_init(&misc->empty[i], 1);
         }
         mbar_init(&misc->fill_done, 1);
@@ -163,7 +160,7 @@ __global__ void __launch_bounds__(FC_THREADS, 1) fc_tc_kernel(const FcArgs a, co
     tc_fence_after();
     const uint32_t tmem = misc->tmem_base;
 
-    uint32_t blocks_done = 0;  // blocks streamed so far by this CTA (ring position), the same in every thread
+    uint32_t stages_done = 0;  // ring stages streamed so far by this CTA, the same in every thread
     int fills_done = 0;
     const uint32_t idesc = (1u << 4) | ((BF16 ? 1u : 0u) << 7) | ((BF16 ? 1u : 0u) << 10) | (0u << 15) | (1u << 16) |
                            ((uint32_t)(TNT >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
@@ -272,41 +269,60 @@ __global__ void __launch_bounds__(FC_THREADS, 1) fc_tc_kernel(const FcArgs a, co
         __syncthreads();
 
         const uint32_t nblk = (uint32_t)cnt_pad >> 4;
-        if (warp == 0) {
-            // ---- producer: block q goes to ring stage (blocks_done + q) % TC_NST
-            for (uint32_t q = 0; q < nblk; ++q) {
-                const uint32_t it = blocks_done + q, st = it % TC_NST, n = it / TC_NST;
+        const uint32_t nstg = ((uint32_t)cnt_pad + TC_SROWS - 1) / TC_SROWS;  // ring stages of this fill (the last may be short)
+        if (warp != 1) {
+            // ---- producers: stage sq of the fill holds kept rows 64 sq .. 64 sq + 63 and goes to ring slot
+            // (stages_done + sq) % TC_NST; inside a stage, warp pw takes rows pw, pw + 7, ...  A row moves with one
+            // 16-byte asynchronous copy per lane (global -> swizzled place in the stage, no registers in between);
+            // after its rows of a stage a lane posts one asynchronous arrival on the stage's "full" barrier, which
+            // fires when its copies have landed.  Producers never wait for data: the ring is the in-flight buffer.
+            constexpr int P = FC_WARPS - 1;
+            const int pw = warp == 0 ? 0 : warp - 1;
+            int col;
+            if constexpr (EPI == EPI_GLU) col = (lane >> 4) * a.Nh + tile * HALF + (lane & 15) * 8;
+            else col = tile * TNT + lane * 8;
+            const bool col_ok = EPI == EPI_GLU ? (tile * HALF + (lane & 15) * 8 < a.Nh) : (col < a.Nh);
+            const unsigned char *Wb = reinterpret_cast<const unsigned char *>(a.W) + (col_ok ? (size_t)col * 2 : 0);
+            const uint32_t src_bytes = col_ok ? 16u : 0u;  // 0: the copy writes zeros
+            const size_t row_bytes = (size_t)a.ldw * 2;
+            const uint32_t ring = smem_u32(s_ring) + (uint32_t)(lane >> 3) * 1024;  // + this lane's 64-column quarter
+            for (uint32_t sq = 0; sq < nstg; ++sq) {
+                const uint32_t it = stages_done + sq, st = it % TC_NST;
                 bool ok = true;
-                if (lane == 0) {
-                    ok = mbar_wait(&misc->empty[st], (n & 1u) ^ 1u, 1, abort_flag);
-                    if (ok) mbar_expect_tx(&misc->full[st], TC_STAGE);
-                }
+                if (lane == 0) ok = mbar_wait(&misc->empty[st], ((it / TC_NST) & 1u) ^ 1u, 1, abort_flag);
                 ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
                 if (!ok) break;
-                if (lane < 16) {  // lane = (column quarter, row quad): 4 rows x 64 columns = 512 bytes each
-                    const int nh = lane >> 2, rq = lane & 3;
-                    int xc;
-                    if constexpr (EPI == EPI_GLU) xc = (nh >> 1) * a.Nh + tile * HALF + (nh & 1) * 64;
-                    else xc = tile * TNT + nh * 64;
-                    const uint32_t *rows = s_k + q * 16 + rq * 4;
-                    unsigned char *dst = s_ring + st * TC_STAGE + (rq >> 1) * 4096 + nh * 1024 + (rq & 1) * 512;
-                    tma_gather4(&tmap, &misc->full[st], dst, xc, (int)rows[0], (int)rows[1], (int)rows[2], (int)rows[3]);
+                const int rows_here = min(TC_SROWS, cnt_pad - (int)sq * TC_SROWS);
+                const uint32_t base = ring + st * TC_STAGE;
+#pragma unroll
+                for (int u = 0; u < (TC_SROWS + P - 1) / P; ++u) {
+                    const int lr = pw + P * u;  // row inside the stage: block lr / 16, K half (lr / 8) & 1, row lr & 7
+                    if (lr < rows_here) {
+                        const uint32_t r = (uint32_t)lr & 7;
+                        const uint32_t dst = base + ((uint32_t)lr >> 4) * TC_KB + (((uint32_t)lr >> 3) & 1) * 4096 + r * 128 + (((uint32_t)lane & 7) ^ r) * 16;
+                        const unsigned char *src = Wb + (size_t)s_k[sq * TC_SROWS + lr] * row_bytes;
+                        asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+                    }
                 }
-                __syncwarp();
+                asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(smem_u32(&misc->full[st])) : "memory");
             }
-        } else if (warp == 1) {
-            // ---- MMA issuer
-            for (uint32_t q = 0; q < nblk; ++q) {
-                const uint32_t it = blocks_done + q, st = it % TC_NST, n = it / TC_NST;
+        } else {
+            // ---- MMA issuer: one wait per stage, then one MMA per block of 16 rows in it
+            for (uint32_t sq = 0; sq < nstg; ++sq) {
+                const uint32_t it = stages_done + sq, st = it % TC_NST;
                 bool ok = true;
                 if (lane == 0) {
-                    ok = mbar_wait(&misc->full[st], n & 1u, 2, abort_flag);
+                    ok = mbar_wait(&misc->full[st], (it / TC_NST) & 1u, 2, abort_flag);
                     if (ok) {
+                        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // copied rows -> tensor-core proxy
                         tc_fence_after();
-                        const uint64_t da = tc_desc(smem_u32(s_plane) + q * BLK, LBO, 128, 0);
-                        const uint64_t db = tc_desc(smem_u32(s_ring) + st * TC_STAGE, 1024, 4096, 2);
-                        tc_mma(tmem, da, db, idesc, it > 0 ? 1u : 0u);
-                        tc_commit(&misc->empty[st]);  // arrives once the MMA has read the stage
+                        const uint32_t kb_n = min(4u, nblk - sq * 4);
+                        for (uint32_t kb = 0; kb < kb_n; ++kb) {
+                            const uint64_t da = tc_desc(smem_u32(s_plane) + (sq * 4 + kb) * BLK, LBO, 128, 0);
+                            const uint64_t db = tc_desc(smem_u32(s_ring) + st * TC_STAGE + kb * TC_KB, 1024, 4096, 2);
+                            tc_mma(tmem, da, db, idesc, (it > 0 || kb > 0) ? 1u : 0u);
+                        }
+                        tc_commit(&misc->empty[st]);  // arrives once the MMAs have read the stage
                     }
                 }
                 ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
@@ -320,15 +336,16 @@ __global__ void __launch_bounds__(FC_THREADS, 1) fc_tc_kernel(const FcArgs a, co
             mbar_wait(&misc->fill_done, (uint32_t)fills_done & 1u, 3, abort_flag);
             ++fills_done;
         }
-        blocks_done += nblk;
+        stages_done += nstg;
         tc_fence_before();
         __syncthreads();
         tc_fence_after();
         if (*abort_flag) break;
     }
 
+    asm volatile("cp.async.wait_all;" ::: "memory");
     // ---- accumulator rows -> shared memory (the ring is idle now), parts added smallest first
-    const bool have_acc = blocks_done > 0 && !*abort_flag;
+    const bool have_acc = stages_done > 0 && !*abort_flag;
     const int acc_rows = NSPLIT * Bp;
     if (have_acc && warp * 32 < acc_rows && warp < 2) {
 #pragma unroll 1
@@ -406,59 +423,8 @@ __global__ void __launch_bounds__(FC_THREADS, 1) fc_tc_kernel(const FcArgs a, co
 
 // ---- host side ------------------------------------------------------------------------------------------------
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
-                                  const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-static EncodeTiledFn encode_fn() {
-    static EncodeTiledFn fn = nullptr;
-    static bool tried = false;
-    if (!tried) {
-        tried = true;
-        void *p = nullptr;
-        cudaDriverEntryPointQueryResult qr;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qr) == cudaSuccess &&
-            qr == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(p);
-        else
-            cudaGetLastError();
-    }
-    return fn;
-}
-
-// Tensor map of W[K, ldw] for row gathers: box = 64 columns x 1 row, 128-byte swizzle, zero fill outside.
-static bool make_map(const void *W, int K, int ldw, bool bf16, CUtensorMap *out) {
-    struct Key { const void *W; int K, ldw, bf16; };
-    struct Slot { Key k; CUtensorMap m; bool used; };
-    static Slot cache[64];
-    static int next = 0;
-    for (int i = 0; i < 64; ++i)
-        if (cache[i].used && cache[i].k.W == W && cache[i].k.K == K && cache[i].k.ldw == ldw && cache[i].k.bf16 == (int)bf16) {
-            *out = cache[i].m;
-            return true;
-        }
-    EncodeTiledFn fn = encode_fn();
-    if (!fn) return false;
-    const cuuint64_t dims[2] = {(cuuint64_t)ldw, (cuuint64_t)K};
-    const cuuint64_t strides[1] = {(cuuint64_t)ldw * 2};
-    const cuuint32_t box[2] = {64, 1};
-    const cuuint32_t estr[2] = {1, 1};
-    CUtensorMap m;
-    if (fn(&m, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void *>(W), dims, strides, box,
-           estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-        return false;
-    Slot &sl = cache[next];
-    next = (next + 1) % 64;
-    sl.k = Key{W, K, ldw, (int)bf16};
-    sl.m = m;
-    sl.used = true;
-    *out = m;
-    return true;
-}
-
 template <bool BF16, int MODE, typename XT, int EPI>
-static cudaError_t launch_tc_t(const FcArgs &a, const CUtensorMap &map, cudaStream_t st) {
+static cudaError_t launch_tc_t(const FcArgs &a, cudaStream_t st) {
     static bool attr_done = false;
     auto kern = fc_tc_kernel<BF16, MODE, XT, EPI>;
     if (!attr_done) {
@@ -466,20 +432,20 @@ static cudaError_t launch_tc_t(const FcArgs &a, const CUtensorMap &map, cudaStre
         if (e != cudaSuccess) return e;
         attr_done = true;
     }
-    return launch_cluster(kern, dim3(fc_tiles(a.Nh, EPI, TC_TN), a.S), dim3(FC_THREADS), TC_SMEM, a.S, st, g_tune.pdl != 0, a, map);
+    return launch_cluster(kern, dim3(fc_tiles(a.Nh, EPI, TC_TN), a.S), dim3(FC_THREADS), TC_SMEM, a.S, st, g_tune.pdl != 0, a);
 }
 
 template <bool BF16, int MODE, typename XT>
-static cudaError_t launch_tc_e(int epi, const FcArgs &a, const CUtensorMap &map, cudaStream_t st) {
-    return epi == EPI_GLU ? launch_tc_t<BF16, MODE, XT, EPI_GLU>(a, map, st) : launch_tc_t<BF16, MODE, XT, EPI_BIAS>(a, map, st);
+static cudaError_t launch_tc_e(int epi, const FcArgs &a, cudaStream_t st) {
+    return epi == EPI_GLU ? launch_tc_t<BF16, MODE, XT, EPI_GLU>(a, st) : launch_tc_t<BF16, MODE, XT, EPI_BIAS>(a, st);
 }
 
 template <bool BF16>
-static cudaError_t launch_tc_w(int mode, int xkind, int epi, const FcArgs &a, const CUtensorMap &map, cudaStream_t st) {
+static cudaError_t launch_tc_w(int mode, int xkind, int epi, const FcArgs &a, cudaStream_t st) {
     using ST = typename std::conditional<BF16, __nv_bfloat16, __half>::type;
     if (mode == MODE_DENSE)
-        return xkind == 2 ? launch_tc_e<BF16, MODE_DENSE, float>(epi, a, map, st) : launch_tc_e<BF16, MODE_DENSE, ST>(epi, a, map, st);
-    return xkind == 2 ? launch_tc_e<BF16, MODE_GATHER, float>(epi, a, map, st) : launch_tc_e<BF16, MODE_GATHER, ST>(epi, a, map, st);
+        return xkind == 2 ? launch_tc_e<BF16, MODE_DENSE, float>(epi, a, st) : launch_tc_e<BF16, MODE_DENSE, ST>(epi, a, st);
+    return xkind == 2 ? launch_tc_e<BF16, MODE_GATHER, float>(epi, a, st) : launch_tc_e<BF16, MODE_GATHER, ST>(epi, a, st);
 }
 
 // CTAs of clusters of size S resident at once with one CTA per SM.
@@ -511,7 +477,7 @@ static int tc_resident(int S) {
 
 bool tc_applicable(const FcArgs &a, int xkind) {
     (void)xkind;
-    return g_tune.tc != 0 && a.B >= 3 && a.B <= 16 && a.ldw % 8 == 0 && aligned16(a.W) && !a.hold_dependents && encode_fn() != nullptr;
+    return g_tune.tc != 0 && a.B >= 3 && a.B <= 16 && a.ldw % 8 == 0 && aligned16(a.W) && !a.hold_dependents;
 }
 
 // Split-K factor for the tensor-core kernel (tile width is fixed at 256): most CTAs that are all resident with
@@ -537,9 +503,7 @@ int tc_choose_split(int K, int Nh, int epi, int B, bool bf16) {
 }
 
 cudaError_t launch_fc_tc(bool bf16, int mode, int xkind, int epi, const FcArgs &a, cudaStream_t st) {
-    CUtensorMap map;
-    if (!make_map(a.W, a.K, a.ldw, bf16, &map)) return cudaErrorNotSupported;
-    return bf16 ? launch_tc_w<true>(mode, xkind, epi, a, map, st) : launch_tc_w<false>(mode, xkind, epi, a, map, st);
+    return bf16 ? launch_tc_w<true>(mode, xkind, epi, a, st) : launch_tc_w<false>(mode, xkind, epi, a, st);
 }
 
 // Reads and clears the status word of the bounded waits (synchronises the device).
