@@ -385,8 +385,15 @@ def main():
     ap.add_argument("--copies", type=int, default=0,
                     help="number of weight copies to rotate (default: enough for the cold-HBM rule); a small value keeps "
                          "device memory low for a profiler capture and is recorded in config.l2_policy")
+    ap.add_argument("--tune", action="append", default=[], metavar="KEY=VALUE",
+                    help="library tuning knob passed to scap_tune before anything runs, e.g. --tune tcgen05=0 --tune split_k=7")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.tune and args.impl == "ours":
+        import paper_2412_07174_b200 as _scap
+        for kv in args.tune:
+            key, _, value = kv.partition("=")
+            _scap.scap_tune(key, int(value))
 
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))

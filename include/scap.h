@@ -77,8 +77,9 @@ int scap_version(void);
 /* Process-wide tuning knobs (plain ints, not thread-safe against concurrent calls):
  *   "split_k"  cap the split-K factor (thread-block cluster size) of the FC kernel: 0 = automatic, else 1..8
  *   "pdl"      1 = launch dependent kernels with programmatic dependent launch (default), 0 = off
- *   "tcgen05"  1 = batch 3..16 calls of the FC and SwiGLU entry points run the TMA-gather + tcgen05
- *              kernel, 0 = the mma.sync variants
+ *   "tcgen05"  batch 3..16 calls of the FC and SwiGLU entry points: 0 = always the mma.sync variants,
+ *              1 = the tcgen05 (TMEM accumulator) kernel where its shared-memory operand region holds
+ *              the call's kept channels in one pass, else mma.sync (default), 2 = always tcgen05
  * Unknown keys return SCAP_ERR_INVALID_ARG.  Tuning never changes what is computed; split_k
  * changes the (fixed) summation order and therefore the last bits of y.  Query workspace sizes
  * after tuning.                                                                               */

@@ -6,7 +6,7 @@
 
 namespace scap {
 
-Tuning g_tune = {0, 1, 0};
+Tuning g_tune = {0, 1, 1};
 
 scap_status check_device() {
     static int cached[64];  // 0 unknown, 1 ok, 2 unsupported
@@ -42,7 +42,7 @@ int sm_count() {
 // needs S SMs of one GPC with a free CTA slot, so the figure depends on how the device's SMs are grouped and is a
 // little below 2 * SMs for S > 1).  Queried once per size for the batch-1 kernel, which has the launch shape of
 // all variants (256 threads, two CTAs per SM); 2 * SMs where the query is not possible.
-static int resident_ctas(int S) {
+int resident_ctas(int S) {
     static int cached[MAX_CLUSTER + 1];
     if (cached[S]) return cached[S];
     int n = 2 * sm_count();
@@ -134,7 +134,7 @@ static cudaError_t launch_fc_w(int mode, int xkind, int epi, const FcArgs &a, cu
 }
 
 cudaError_t launch_fc(bool bf16, int mode, int xkind, int epi, const FcArgs &a, cudaStream_t st) {
-    if (tc_applicable(a, xkind)) {
+    if (tc_applicable(a, epi, bf16)) {
         FcArgs t = a;
         t.tn = 256;
         t.S = tc_choose_split(a.K, a.Nh, epi, a.B, bf16);
@@ -265,7 +265,8 @@ scap_status scap_tune(const char *key, int value) {
         return SCAP_OK;
     }
     if (!strcmp(key, "tcgen05")) {
-        g_tune.tc = value != 0;
+        if (value < 0 || value > 2) return SCAP_ERR_INVALID_ARG;
+        g_tune.tc = value;
         return SCAP_OK;
     }
     return SCAP_ERR_INVALID_ARG;

@@ -795,10 +795,11 @@ inline int fc_tiles(int Nh, int epi, int tn) { return epi == EPI_GLU ? (Nh + tn 
 // Tile width (256 or 128 columns) and split-K factor (cluster size) for an FC with Nh columns per half and
 // `groups` concurrently active groups (experts): the pair with the most CTAs that are still all co-resident.
 void choose_config(int K, int Nh, int epi, int groups, int B, int *tn, int *S);
+int resident_ctas(int S);  // CTAs of clusters of size S resident at once (256 threads, two CTAs per SM)
 
 // tcgen05 kernel for batch 3..16 (scap_fc_tc.cu): whether it can take this call, its split-K factor, its launch,
 // and the status word of its bounded waits (0 = none ran out; reading synchronises the device and clears it).
-bool tc_applicable(const FcArgs &a, int xkind);
+bool tc_applicable(const FcArgs &a, int epi, bool bf16);
 int tc_choose_split(int K, int Nh, int epi, int B, bool bf16);
 cudaError_t launch_fc_tc(bool bf16, int mode, int xkind, int epi, const FcArgs &a, cudaStream_t st);
 int tc_take_status();

@@ -1,21 +1,21 @@
 // Batch 3..16 on the 5th-generation tensor cores: the sparse FC of Eq. 2-3 / Eq. 6 / Alg. 3 as
 //   16-byte asynchronous row copies  ->  swizzled shared-memory ring  ->  tcgen05.mma  ->  accumulator in TMEM.
 //
-// Same decomposition as the FMA kernel (grid = column tiles x S, the S CTAs of a tile form a cluster and split the
-// input channels by interleaved 32-channel chunks, cluster exchange of the partial tiles at the end), but one CTA
-// per SM with a deep ring:
+// Same decomposition as the FMA kernel (grid = 128-column tiles x S, the S CTAs of a tile form a cluster and split
+// the input channels by interleaved 32-channel chunks, cluster exchange of the partial tiles at the end, two CTAs
+// per SM):
 //   prologue   all 8 warps: d = x - m, |d| >= tau, union over the batch, ballot compaction (ascending kept list),
 //              and the pruned values split exactly into parts of the weight dtype (bf16: hi+mid+lo, fp16: hi+lo)
-//              written as the A operand: row (part * Bp + b), K-major core matrices of 8 rows x 16 bytes;
-//   7 warps    producers: a warp moves one kept row (512 bytes of the tile) per instruction with 16-byte
-//              asynchronous copies (cp.async) straight into the row's place in a ring stage of 64 rows = four
-//              8 KB blocks, each laid out as the MN-major, 128-byte-swizzled B operand (N = 256 columns of W,
+//              written as the A operand: row (part * B + b), K-major core matrices of 8 rows x 16 bytes;
+//   7 warps    producers: a warp moves two kept rows (256 bytes of the tile each) per instruction with 16-byte
+//              asynchronous copies (cp.async) straight into the rows' places in a ring stage of 64 rows = four
+//              4 KB blocks, each laid out as the MN-major, 128-byte-swizzled B operand (N = 128 columns of W,
 //              K = 16 rows); an asynchronous arrival per lane and stage fires when the copies have landed, so
 //              producers never wait for data and the whole ring is the in-flight buffer;
-//   warp 1     one lane waits per stage and issues tcgen05.mma M=128 N=256 K=16 per block of 16 rows (all parts of all batch rows at
-//              once; rows of M beyond parts * Bp read whatever follows in shared memory and produce accumulator
-//              rows nobody reads) and commits to the stage's "empty" barrier; the accumulator (128 lanes x 256
-//              fp32 columns) stays in TMEM across blocks and fills;
+//   warp 1     one lane waits per stage and issues tcgen05.mma M=128 N=128 K=16 per block of 16 rows (all parts
+//              of all batch rows at once; rows of M beyond parts * B read whatever follows in shared memory and
+//              produce accumulator rows nobody reads) and commits to the stage's "empty" barrier; the accumulator
+//              (128 lanes x 128 fp32 columns) stays in TMEM across blocks and fills;
 //   epilogue   warps 0-1 read the accumulator rows, the parts are added smallest first, and the cluster exchange
 //              and bias / SwiGLU epilogue are those of the other variants.
 // (A TMA row gather - cp.async.bulk.tensor tile::gather4, four rows x 128 bytes per instruction - was measured
@@ -28,26 +28,33 @@
 
 namespace scap {
 
-constexpr int TC_TN = 256;                          // columns per CTA
-constexpr int TC_KB = 16 * TC_TN * 2;               // bytes of one block of 16 kept rows (one MMA)
+constexpr int TC_TN = 128;                          // columns per CTA
+constexpr int TC_KB = 16 * TC_TN * 2;               // bytes of one block of 16 kept rows (one MMA): 4 KB
 constexpr int TC_SROWS = 64;                        // kept rows per ring stage (4 blocks)
-constexpr int TC_STAGE = TC_SROWS * TC_TN * 2;      // 32 KB
-constexpr int TC_NST = 4;                           // ring stages (128 KB per SM)
+constexpr int TC_STAGE = TC_SROWS * TC_TN * 2;      // 16 KB
+constexpr int TC_NST = 3;                           // ring stages (48 KB per CTA, two CTAs per SM)
 constexpr int TC_CAP = 1408;                        // most kept channels per fill (44 chunks)
-constexpr int TC_PLANE = TC_CAP * 48 + 2048;        // A-operand bytes: 48 per channel (3 parts x 8 rows x 2) + read slack
-constexpr int TC_PU = 6;                            // chunks per warp per fill, at most
-constexpr int TC_PART_LD = 257;                     // row pitch of the accumulator copy (conflict-free)
+constexpr int TC_PLANE_DATA = TC_CAP * 32;          // A-operand bytes: 16 per channel and 8-row group, two groups at full capacity
+constexpr int TC_PLANE = TC_PLANE_DATA + 2048;      // + slack for the rows of M that nobody uses
+constexpr int TC_PART_LD = TC_TN + 1;               // row pitch of the accumulator copy (conflict-free)
 constexpr uint32_t TC_SPIN = 1u << 20;              // polls before a wait gives up (tens of milliseconds)
+__host__ __device__ constexpr int tc_pu(int ROWS) { return ROWS == 8 ? 6 : 3; }  // chunks per warp per fill, at most
+// 8-row groups of the A operand for B batch rows (parts stacked densely: row = part * B + b), and the chunks of 32
+// channels that fit in the A-operand region with that many groups
+__host__ __device__ constexpr int tc_groups(int B, int nsplit) { return (nsplit * B + 7) / 8; }
+__host__ __device__ constexpr int tc_cap_chunks(int groups) {
+    return TC_PLANE_DATA / (groups * 16) / 32 < TC_CAP / 32 ? TC_PLANE_DATA / (groups * 16) / 32 : TC_CAP / 32;
+}
 
 // shared-memory map (offsets from a 1024-byte aligned base)
 constexpr int TC_OFF_RING = 0;
 constexpr int TC_OFF_PLANE = TC_OFF_RING + TC_NST * TC_STAGE;
 constexpr int TC_OFF_K = TC_OFF_PLANE + TC_PLANE;
 constexpr int TC_OFF_GATHER = TC_OFF_K + TC_CAP * 4;
-constexpr int TC_OFF_MISC = TC_OFF_GATHER + 16 * GATHER_LD * 4;
+constexpr int TC_OFF_MISC = TC_OFF_GATHER + 16 * TC_TN * 4;
 constexpr int TC_SMEM = TC_OFF_MISC + 1024 + 1024;  // misc block + alignment slack
 static_assert(48 * TC_PART_LD * 4 <= TC_NST * TC_STAGE, "accumulator copy must fit in the ring");
-static_assert(TC_SMEM <= 232448, "exceeds the shared memory of an SM");
+static_assert(2 * (TC_SMEM + 1024) <= 233472, "two CTAs must fit in the shared memory of an SM");
 
 __device__ int g_tc_status;  // 0, or the code of the first bounded wait that ran out
 
@@ -106,9 +113,9 @@ __device__ __forceinline__ uint64_t tc_desc(uint32_t addr, uint32_t lbo, uint32_
            ((uint64_t)((sbo >> 4) & 0x3fffu) << 32) | (1ull << 46) | ((uint64_t)layout << 61);
 }
 
-template <bool BF16, int MODE, typename XT, int EPI>
-__global__ void __launch_bounds__(FC_THREADS, 1) fc_tc_kernel(const FcArgs a) {
-    constexpr int TNT = TC_TN, HALF = TNT / 2, NSPLIT = mma_nsplit(BF16);
+template <bool BF16, int ROWS, int MODE, typename XT, int EPI>
+__global__ void __launch_bounds__(FC_THREADS, 2) fc_tc_kernel(const FcArgs a) {
+    constexpr int TNT = TC_TN, HALF = TNT / 2, NSPLIT = mma_nsplit(BF16), PU = tc_pu(ROWS);
     extern __shared__ unsigned char smem_raw[];
     unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     unsigned char *s_ring = smem + TC_OFF_RING;
@@ -122,10 +129,10 @@ __global__ void __launch_bounds__(FC_THREADS, 1) fc_tc_kernel(const FcArgs a) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int tile = blockIdx.x, s = blockIdx.y;
     const int B = a.B, S = a.S, K = a.K;
-    const int Bp = B <= 8 ? 8 : 16;            // batch rows per part in the A operand
-    const int G = NSPLIT * Bp / 8;             // 8-row groups of the A operand in use
+    const int racc = NSPLIT * B;               // rows of the A operand (and of the accumulator) in use: part * B + b
+    const int G = tc_groups(B, NSPLIT);        // 8-row groups that hold them
     const uint32_t LBO = G * 128, BLK = 2 * LBO;  // bytes: between the two K halves of a block, and per block
-    const int cap_chunks = min(TC_CAP / 32, (TC_CAP * 48) / (NSPLIT * Bp * 2) / 32);
+    const int cap_chunks = tc_cap_chunks(G);
     const XT *xg = reinterpret_cast<const XT *>(a.x);
 
     if (tid == 0) {
@@ -137,8 +144,8 @@ __global__ void __launch_bounds__(FC_THREADS, 1) fc_tc_kernel(const FcArgs a) {
         misc->abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 0) {  // the accumulator: 256 TMEM columns, allocated by warp 0 and freed by it at the end
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&misc->tmem_base)), "r"(256)
+    if (warp == 0) {  // the accumulator: 128 TMEM columns, allocated by warp 0 and freed by it at the end
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&misc->tmem_base)), "r"(TNT)
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
@@ -169,37 +176,37 @@ __global__ void __launch_bounds__(FC_THREADS, 1) fc_tc_kernel(const FcArgs a) {
         const int nj = min(cap_chunks, my_chunks - j0);
         const int pu = (nj + FC_WARPS - 1) / FC_WARPS;  // consecutive chunks per warp
         // ---- keep masks: all activation loads of a lane in flight together, values kept in registers
-        float mk[TC_PU];
-        XT xraw[TC_PU][16];
-        uint32_t km[TC_PU];
-        unsigned bal[TC_PU];
+        float mk[PU];
+        XT xraw[PU][ROWS];
+        uint32_t km[PU];
+        unsigned bal[PU];
 #pragma unroll
-        for (int p = 0; p < TC_PU; ++p) {
+        for (int p = 0; p < PU; ++p) {
             const int j = warp * pu + p;
             const int k = (s + S * (j0 + j)) * 32 + lane;
             mk[p] = a.m ? ld_nc_if(a.m + k, p < pu && j < nj && k < K) : 0.0f;
         }
 #pragma unroll
-        for (int p = 0; p < TC_PU; ++p) {
+        for (int p = 0; p < PU; ++p) {
             const int j = warp * pu + p;
             const int k = (s + S * (j0 + j)) * 32 + lane;
             const bool ok = p < pu && j < nj && k < K;
 #pragma unroll
-            for (int b = 0; b < 16; ++b) {
+            for (int b = 0; b < ROWS; ++b) {
                 const int row = a.in_rows ? misc->rows[b] : b;
                 xraw[p][b] = ld_act_if(xg + (size_t)row * a.x_ld + k, ok && b < B);
             }
         }
-        int my_off[TC_PU], wtotal = 0;
+        int my_off[PU], wtotal = 0;
 #pragma unroll
-        for (int p = 0; p < TC_PU; ++p) {
+        for (int p = 0; p < PU; ++p) {
             const int j = warp * pu + p;
             const int k = (s + S * (j0 + j)) * 32 + lane;
             const bool ok = p < pu && j < nj && k < K;
             uint32_t m_ = 0;
             if constexpr (MODE == MODE_GATHER) {
 #pragma unroll
-                for (int b = 0; b < 16; ++b) {
+                for (int b = 0; b < ROWS; ++b) {
                     const float xv = widen1(xraw[p][b]);
                     const float dv = a.m ? __fsub_rn(xv, mk[p]) : xv;
                     m_ |= (ok && b < B && fabsf(dv) >= tau) ? (1u << b) : 0u;
@@ -216,7 +223,7 @@ __global__ void __launch_bounds__(FC_THREADS, 1) fc_tc_kernel(const FcArgs a) {
         if (MODE == MODE_GATHER && a.bits && tile == 0) {
             unsigned mine = 0;
 #pragma unroll
-            for (int p = 0; p < TC_PU; ++p) mine = lane == p ? bal[p] : mine;
+            for (int p = 0; p < PU; ++p) mine = lane == p ? bal[p] : mine;
             const int j = warp * pu + lane;
             if (lane < pu && j < nj) a.bits[s + S * (j0 + j)] = mine;
         }
@@ -228,10 +235,10 @@ __global__ void __launch_bounds__(FC_THREADS, 1) fc_tc_kernel(const FcArgs a) {
             cnt += c;
             wbase += w < warp ? c : 0;
         }
-        // ---- kept list and A operand.  Element (row r = part * Bp + b, kept position pos): block pos / 16,
+        // ---- kept list and A operand.  Element (row r = part * B + b, kept position pos): block pos / 16,
         // K half (pos / 8) & 1, 8-row group r / 8, then 16 bytes per row of the group, 2 bytes per position.
 #pragma unroll
-        for (int p = 0; p < TC_PU; ++p) {
+        for (int p = 0; p < PU; ++p) {
             if (km[p]) {
                 const int j = warp * pu + p;
                 const int k = (s + S * (j0 + j)) * 32 + lane;
@@ -239,16 +246,16 @@ __global__ void __launch_bounds__(FC_THREADS, 1) fc_tc_kernel(const FcArgs a) {
                 s_k[pos] = (uint32_t)k;
                 unsigned char *blk = s_plane + (size_t)(pos >> 4) * BLK + ((pos >> 3) & 1) * LBO + (pos & 7) * 2;
 #pragma unroll
-                for (int b = 0; b < 16; ++b) {
-                    if (b < Bp) {
+                for (int b = 0; b < ROWS; ++b) {
+                    if (b < B) {
                         const float xv = widen1(xraw[p][b]);
                         const float dv = (MODE == MODE_GATHER && a.m) ? __fsub_rn(xv, mk[p]) : xv;
-                        const bool kept = MODE == MODE_DENSE ? (b < B) : (((km[p] >> b) & 1u) != 0);
+                        const bool kept = MODE == MODE_DENSE || (((km[p] >> b) & 1u) != 0);
                         unsigned short part[3];
                         split_parts<BF16>(kept ? dv : 0.0f, part);
 #pragma unroll
                         for (int q = 0; q < NSPLIT; ++q) {
-                            const int r = q * Bp + b;
+                            const int r = q * B + b;
                             *reinterpret_cast<unsigned short *>(blk + (r >> 3) * 128 + (r & 7) * 16) = part[q];
                         }
                     }
@@ -263,7 +270,7 @@ __global__ void __launch_bounds__(FC_THREADS, 1) fc_tc_kernel(const FcArgs a) {
             const int pos = cnt + tid;
             s_k[pos] = s_k[cnt - 1];
             unsigned char *blk = s_plane + (size_t)(pos >> 4) * BLK + ((pos >> 3) & 1) * LBO + (pos & 7) * 2;
-            for (int r = 0; r < NSPLIT * Bp; ++r) *reinterpret_cast<unsigned short *>(blk + (r >> 3) * 128 + (r & 7) * 16) = 0;
+            for (int r = 0; r < racc; ++r) *reinterpret_cast<unsigned short *>(blk + (r >> 3) * 128 + (r & 7) * 16) = 0;
         }
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes -> visible to the tensor core
         __syncthreads();
@@ -278,14 +285,15 @@ __global__ void __launch_bounds__(FC_THREADS, 1) fc_tc_kernel(const FcArgs a) {
             // fires when its copies have landed.  Producers never wait for data: the ring is the in-flight buffer.
             constexpr int P = FC_WARPS - 1;
             const int pw = warp == 0 ? 0 : warp - 1;
+            const int l16 = lane & 15;  // a row of the tile is 256 bytes = 16 lanes; a warp moves two rows at once
             int col;
-            if constexpr (EPI == EPI_GLU) col = (lane >> 4) * a.Nh + tile * HALF + (lane & 15) * 8;
-            else col = tile * TNT + lane * 8;
-            const bool col_ok = EPI == EPI_GLU ? (tile * HALF + (lane & 15) * 8 < a.Nh) : (col < a.Nh);
+            if constexpr (EPI == EPI_GLU) col = (l16 >> 3) * a.Nh + tile * HALF + (l16 & 7) * 8;
+            else col = tile * TNT + l16 * 8;
+            const bool col_ok = EPI == EPI_GLU ? (tile * HALF + (l16 & 7) * 8 < a.Nh) : (col < a.Nh);
             const unsigned char *Wb = reinterpret_cast<const unsigned char *>(a.W) + (col_ok ? (size_t)col * 2 : 0);
             const uint32_t src_bytes = col_ok ? 16u : 0u;  // 0: the copy writes zeros
             const size_t row_bytes = (size_t)a.ldw * 2;
-            const uint32_t ring = smem_u32(s_ring) + (uint32_t)(lane >> 3) * 1024;  // + this lane's 64-column quarter
+            const uint32_t ring = smem_u32(s_ring) + (uint32_t)(l16 >> 3) * 1024;  // + this lane's 64-column half
             for (uint32_t sq = 0; sq < nstg; ++sq) {
                 const uint32_t it = stages_done + sq, st = it % TC_NST;
                 bool ok = true;
@@ -295,11 +303,11 @@ __global__ void __launch_bounds__(FC_THREADS, 1) fc_tc_kernel(const FcArgs a) {
                 const int rows_here = min(TC_SROWS, cnt_pad - (int)sq * TC_SROWS);
                 const uint32_t base = ring + st * TC_STAGE;
 #pragma unroll
-                for (int u = 0; u < (TC_SROWS + P - 1) / P; ++u) {
-                    const int lr = pw + P * u;  // row inside the stage: block lr / 16, K half (lr / 8) & 1, row lr & 7
+                for (int u = 0; u < (TC_SROWS / 2 + P - 1) / P; ++u) {
+                    const int lr = 2 * (pw + P * u) + (lane >> 4);  // row inside the stage: block lr / 16, K half (lr / 8) & 1, row lr & 7
                     if (lr < rows_here) {
                         const uint32_t r = (uint32_t)lr & 7;
-                        const uint32_t dst = base + ((uint32_t)lr >> 4) * TC_KB + (((uint32_t)lr >> 3) & 1) * 4096 + r * 128 + (((uint32_t)lane & 7) ^ r) * 16;
+                        const uint32_t dst = base + ((uint32_t)lr >> 4) * TC_KB + (((uint32_t)lr >> 3) & 1) * 2048 + r * 128 + (((uint32_t)l16 & 7) ^ r) * 16;
                         const unsigned char *src = Wb + (size_t)s_k[sq * TC_SROWS + lr] * row_bytes;
                         asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
                     }
@@ -319,7 +327,7 @@ __global__ void __launch_bounds__(FC_THREADS, 1) fc_tc_kernel(const FcArgs a) {
                         const uint32_t kb_n = min(4u, nblk - sq * 4);
                         for (uint32_t kb = 0; kb < kb_n; ++kb) {
                             const uint64_t da = tc_desc(smem_u32(s_plane) + (sq * 4 + kb) * BLK, LBO, 128, 0);
-                            const uint64_t db = tc_desc(smem_u32(s_ring) + st * TC_STAGE + kb * TC_KB, 1024, 4096, 2);
+                            const uint64_t db = tc_desc(smem_u32(s_ring) + st * TC_STAGE + kb * TC_KB, 1024, 2048, 2);
                             tc_mma(tmem, da, db, idesc, (it > 0 || kb > 0) ? 1u : 0u);
                         }
                         tc_commit(&misc->empty[st]);  // arrives once the MMAs have read the stage
@@ -346,7 +354,7 @@ __global__ void __launch_bounds__(FC_THREADS, 1) fc_tc_kernel(const FcArgs a) {
     asm volatile("cp.async.wait_all;" ::: "memory");
     // ---- accumulator rows -> shared memory (the ring is idle now), parts added smallest first
     const bool have_acc = stages_done > 0 && !*abort_flag;
-    const int acc_rows = NSPLIT * Bp;
+    const int acc_rows = racc;
     if (have_acc && warp * 32 < acc_rows && warp < 2) {
 #pragma unroll 1
         for (int c0 = 0; c0 < TNT; c0 += 32) {
@@ -370,13 +378,13 @@ __global__ void __launch_bounds__(FC_THREADS, 1) fc_tc_kernel(const FcArgs a) {
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(256) : "memory");
+    if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TNT) : "memory");
     for (int i = tid; i < 16 * TNT; i += FC_THREADS) {
         const int b = i / TNT, c = i - b * TNT;
         float v = 0.0f;
-        if (have_acc && b < Bp) {
+        if (have_acc && b < B) {
 #pragma unroll
-            for (int q = NSPLIT - 1; q >= 0; --q) v += s_part[(q * Bp + b) * TC_PART_LD + c];
+            for (int q = NSPLIT - 1; q >= 0; --q) v += s_part[(q * B + b) * TC_PART_LD + c];
         }
         s_gather[i] = v;
     }
@@ -423,16 +431,21 @@ __global__ void __launch_bounds__(FC_THREADS, 1) fc_tc_kernel(const FcArgs a) {
 
 // ---- host side ------------------------------------------------------------------------------------------------
 
-template <bool BF16, int MODE, typename XT, int EPI>
-static cudaError_t launch_tc_t(const FcArgs &a, cudaStream_t st) {
+template <bool BF16, int ROWS, int MODE, typename XT, int EPI>
+static cudaError_t launch_tc_r(const FcArgs &a, cudaStream_t st) {
     static bool attr_done = false;
-    auto kern = fc_tc_kernel<BF16, MODE, XT, EPI>;
+    auto kern = fc_tc_kernel<BF16, ROWS, MODE, XT, EPI>;
     if (!attr_done) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM);
         if (e != cudaSuccess) return e;
         attr_done = true;
     }
     return launch_cluster(kern, dim3(fc_tiles(a.Nh, EPI, TC_TN), a.S), dim3(FC_THREADS), TC_SMEM, a.S, st, g_tune.pdl != 0, a);
+}
+
+template <bool BF16, int MODE, typename XT, int EPI>
+static cudaError_t launch_tc_t(const FcArgs &a, cudaStream_t st) {
+    return a.B <= 8 ? launch_tc_r<BF16, 8, MODE, XT, EPI>(a, st) : launch_tc_r<BF16, 16, MODE, XT, EPI>(a, st);
 }
 
 template <bool BF16, int MODE, typename XT>
@@ -448,46 +461,30 @@ static cudaError_t launch_tc_w(int mode, int xkind, int epi, const FcArgs &a, cu
     return xkind == 2 ? launch_tc_e<BF16, MODE_GATHER, float>(epi, a, st) : launch_tc_e<BF16, MODE_GATHER, ST>(epi, a, st);
 }
 
-// CTAs of clusters of size S resident at once with one CTA per SM.
-static int tc_resident(int S) {
-    static int cached[MAX_CLUSTER + 1];
-    if (cached[S]) return cached[S];
-    int n = sm_count();
-    if (S > 1) {
-        auto kern = fc_tc_kernel<true, MODE_GATHER, __nv_bfloat16, EPI_BIAS>;
-        cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM);
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(1, S);
-        cfg.blockDim = dim3(FC_THREADS);
-        cfg.dynamicSmemBytes = TC_SMEM;
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeClusterDimension;
-        attr[0].val.clusterDim.x = 1;
-        attr[0].val.clusterDim.y = S;
-        attr[0].val.clusterDim.z = 1;
-        cfg.attrs = attr;
-        cfg.numAttrs = 1;
-        int clusters = 0;
-        if (cudaOccupancyMaxActiveClusters(&clusters, kern, &cfg) == cudaSuccess && clusters > 0) n = clusters * S;
-        else { cudaGetLastError(); n = (sm_count() / S - 2) * S; }
-    }
-    cached[S] = n;
-    return n;
+// Resident CTAs: the occupancy queries count a kernel that allocates TMEM as one CTA per SM, but two CTAs with 128
+// TMEM columns each do share an SM (measured), so the budget is the one of the FMA kernel, which has the same
+// threads, registers and CTAs per SM.
+static int tc_resident(int S) { return resident_ctas(S); }
+
+static int tc_fills(int K, int S, int B, bool bf16) {
+    const int cap_chunks = tc_cap_chunks(tc_groups(B, bf16 ? 3 : 2));
+    return (((K + 31) / 32 + S - 1) / S + cap_chunks - 1) / cap_chunks;
 }
 
-bool tc_applicable(const FcArgs &a, int xkind) {
-    (void)xkind;
-    return g_tune.tc != 0 && a.B >= 3 && a.B <= 16 && a.ldw % 8 == 0 && aligned16(a.W) && !a.hold_dependents;
+// tune value 1 (default): calls whose kept channels fit the A-operand region in one fill per CTA - every further fill
+// drains and refills the ring, and the mma.sync variants are then faster; 2: every batch 3..16 call.
+bool tc_applicable(const FcArgs &a, int epi, bool bf16) {
+    if (g_tune.tc == 0 || a.B < 3 || a.B > 16 || a.ldw % 8 != 0 || !aligned16(a.W) || a.hold_dependents) return false;
+    if (g_tune.tc >= 2) return true;
+    return tc_fills(a.K, tc_choose_split(a.K, a.Nh, epi, a.B, bf16), a.B, bf16) == 1;
 }
 
-// Split-K factor for the tensor-core kernel (tile width is fixed at 256): most CTAs that are all resident with
-// one CTA per SM; ties: fewer fills, then the smaller cluster.
+// Split-K factor for the tensor-core kernel (tile width is fixed at 128): most CTAs that are all resident at
+// once; ties: fewer fills of the A-operand region, then the smaller cluster.
 int tc_choose_split(int K, int Nh, int epi, int B, bool bf16) {
     const int tiles = fc_tiles(Nh, epi, TC_TN);
     const int nchunks = (K + 31) / 32;
-    const int bp = B <= 8 ? 8 : 16, nsplit = bf16 ? 3 : 2;
-    int cap_chunks = (TC_CAP * 48) / (nsplit * bp * 2) / 32;
-    if (cap_chunks > TC_CAP / 32) cap_chunks = TC_CAP / 32;
+    const int cap_chunks = tc_cap_chunks(tc_groups(B, bf16 ? 3 : 2));
     int best_S = 1;
     long long best = -1;
     for (int S = 1; S <= MAX_CLUSTER; ++S) {
@@ -496,7 +493,8 @@ int tc_choose_split(int K, int Nh, int epi, int B, bool bf16) {
         const long long ctas = (long long)tiles * S;
         if (S > 1 && ctas > tc_resident(S)) continue;
         const int fills = ((nchunks + S - 1) / S + cap_chunks - 1) / cap_chunks;
-        const long long score = (ctas > sm_count() ? 0 : ctas * 64) + (63 - (fills < 63 ? fills : 63));
+        // one more fill costs about as much as a tenth of the CTAs: prefer a single fill over the last few CTAs
+        const long long score = (ctas > 2 * sm_count() ? 0 : ctas * 64) - (long long)(fills - 1) * 64 * 26;
         if (score > best) { best = score; best_S = S; }
     }
     return best_S;

@@ -258,3 +258,35 @@ def test_host_buffer_variant_matches_device_variant(S):
     torch.cuda.synchronize()
     assert ws.intact()
     assert np.array_equal(yh.numpy(), y_dev)
+
+
+# ---------------------------------------------------------------- batch 3..16 on the tcgen05 kernel (forced)
+
+@pytest.mark.parametrize("K,N,B,dt,split", [
+    (1500, 520, 3, si.BF16, 0), (1500, 520, 4, si.BF16, 3), (2048, 1024, 8, si.BF16, 0), (4100, 264, 5, si.F16, 0),
+    (1024, 136, 12, si.F16, 2), (3000, 640, 16, si.BF16, 0), (96, 8, 7, si.BF16, 1), (6000, 256, 9, si.BF16, 1),
+])
+def test_tcgen05_kernel_matches_the_oracle(S, K, N, B, dt, split):
+    # several fills of the operand region (6000 channels in one CTA), ragged tiles, both dtypes, all row groupings
+    d = si.laplace_fc(4, K, N, dt, 16, B)
+    try:
+        S.scap_tune("tcgen05", 2)
+        S.scap_tune("split_k", split)
+        check_fc(S, d, d["m_true"], 0.25)
+        check_fc(S, d, None, 0.4, with_bias=False)
+        S.scap_device_status()
+    finally:
+        S.scap_tune("tcgen05", 1)
+        S.scap_tune("split_k", 0)
+
+
+def test_tcgen05_and_mma_sync_paths_agree_closely(S):
+    d = si.laplace_fc(4, 2048, 512, si.BF16, 16, 6)
+    ys = []
+    for mode in (0, 2):
+        try:
+            S.scap_tune("tcgen05", mode)
+            ys.append(run_sparse(S, d, d["m_true"], 0.3, None)[0])
+        finally:
+            S.scap_tune("tcgen05", 1)
+    assert rel_l2_rows(ys[1], ys[0].astype(np.float64)) <= 1e-6

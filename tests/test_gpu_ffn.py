@@ -98,6 +98,18 @@ def test_glu_cluster_sizes_that_do_not_divide_the_tile(S, split, B):
         S.scap_tune("split_k", 0)
 
 
+@pytest.mark.parametrize("D,F,B", [(520, 1000, 3), (1024, 776, 8), (2048, 520, 16)])
+def test_glu_on_the_tcgen05_kernel(S, D, F, B):
+    g = si.glu_block(2, D, F, si.BF16, 64, B)
+    c = calibrate_glu(g, 0.4, 0.7)
+    try:
+        S.scap_tune("tcgen05", 2)
+        check_glu(S, g, c)
+        S.scap_device_status()
+    finally:
+        S.scap_tune("tcgen05", 1)
+
+
 def test_glu_fp16_and_no_centring(S):
     g = si.glu_block(2, 256, 520, si.F16, 64, 2)
     c = calibrate_glu(g, 0.3, 0.6, centre2=False)
