@@ -26,6 +26,23 @@ __device__ __forceinline__ void widen8(const uint4 &v, float (&f)[8]) {
     widen2<BF16>(v.w, f[6], f[7]);
 }
 
+// Rows t0, t0 + CAL_ROWS, ... (CAL_U of them) of this thread's 8 channels, all loads in flight together; rows at or
+// beyond T are skipped (their slots keep zeros and `valid` says how many are real).
+constexpr int CAL_U = 8;
+__device__ __forceinline__ int load_rows(const uint16_t *xp, int K, int T, int t0, uint4 (&v)[CAL_U]) {
+    int valid = 0;
+#pragma unroll
+    for (int u = 0; u < CAL_U; ++u) {
+        const int t = t0 + u * CAL_ROWS;
+        v[u] = make_uint4(0, 0, 0, 0);
+        if (t < T) {
+            v[u] = __ldg(reinterpret_cast<const uint4 *>(xp + (size_t)t * K));
+            valid = u + 1;
+        }
+    }
+    return valid;
+}
+
 // One CTA per strip of CW channels: min/max, histogram, arg-max -> m; then the first radix histogram
 // (bits 30..20 of |x - m|) of the strip is added to hist_a.
 template <bool BF16>
@@ -46,11 +63,18 @@ __global__ void __launch_bounds__(CAL_THREADS) mode_kernel(const uint16_t *__res
 #pragma unroll
         for (int j = 0; j < 8; ++j) { lo[j] = INFINITY; hi[j] = -INFINITY; }
         if (ok)
-            for (int t = rl; t < T; t += CAL_ROWS) {
-                float f[8];
-                widen8<BF16>(__ldg(reinterpret_cast<const uint4 *>(xp + (size_t)t * K)), f);
+            for (int t0 = rl; t0 < T; t0 += CAL_ROWS * CAL_U) {
+                uint4 v[CAL_U];
+                const int nv = load_rows(xp, K, T, t0, v);
 #pragma unroll
-                for (int j = 0; j < 8; ++j) { lo[j] = fminf(lo[j], f[j]); hi[j] = fmaxf(hi[j], f[j]); }
+                for (int u = 0; u < CAL_U; ++u) {
+                    if (u < nv) {
+                        float f[8];
+                        widen8<BF16>(v[u], f);
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) { lo[j] = fminf(lo[j], f[j]); hi[j] = fmaxf(hi[j], f[j]); }
+                    }
+                }
             }
         float *s_mm = reinterpret_cast<float *>(smem);  // [2][CAL_ROWS][CW]
 #pragma unroll
@@ -78,15 +102,22 @@ __global__ void __launch_bounds__(CAL_THREADS) mode_kernel(const uint16_t *__res
         }
         __syncthreads();
         if (ok)
-            for (int t = rl; t < T; t += CAL_ROWS) {
-                float f[8];
-                widen8<BF16>(__ldg(reinterpret_cast<const uint4 *>(xp + (size_t)t * K)), f);
+            for (int t0 = rl; t0 < T; t0 += CAL_ROWS * CAL_U) {
+                uint4 v[CAL_U];
+                const int nv = load_rows(xp, K, T, t0, v);
 #pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    if (hi[j] != lo[j]) {
-                        int i = (int)floorf(__fmul_rn(__fsub_rn(f[j], lo[j]), scale[j]));
-                        i = min(max(i, 0), nbins - 1);
-                        atomicAdd(&smem[(q * 8 + j) * HW + (i >> 1)], 1u << ((i & 1) * 16));
+                for (int u = 0; u < CAL_U; ++u) {
+                    if (u < nv) {
+                        float f[8];
+                        widen8<BF16>(v[u], f);
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            if (hi[j] != lo[j]) {
+                                int i = (int)floorf(__fmul_rn(__fsub_rn(f[j], lo[j]), scale[j]));
+                                i = min(max(i, 0), nbins - 1);
+                                atomicAdd(&smem[(q * 8 + j) * HW + (i >> 1)], 1u << ((i & 1) * 16));
+                            }
+                        }
                     }
                 }
             }
@@ -133,13 +164,20 @@ __global__ void __launch_bounds__(CAL_THREADS) mode_kernel(const uint16_t *__res
     for (int j = 0; j < 8; ++j) mk[j] = s_m[q * 8 + j];
     __syncthreads();
     if (ok)
-        for (int t = rl; t < T; t += CAL_ROWS) {
-            float f[8];
-            widen8<BF16>(__ldg(reinterpret_cast<const uint4 *>(xp + (size_t)t * K)), f);
+        for (int t0 = rl; t0 < T; t0 += CAL_ROWS * CAL_U) {
+            uint4 v[CAL_U];
+            const int nv = load_rows(xp, K, T, t0, v);
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                const uint32_t key = __float_as_uint(__fsub_rn(f[j], mk[j])) & 0x7fffffffu;
-                atomicAdd(&smem[key >> 20], 1u);
+            for (int u = 0; u < CAL_U; ++u) {
+                if (u < nv) {
+                    float f[8];
+                    widen8<BF16>(v[u], f);
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const uint32_t key = __float_as_uint(__fsub_rn(f[j], mk[j])) & 0x7fffffffu;
+                        atomicAdd(&smem[key >> 20], 1u);
+                    }
+                }
             }
         }
     __syncthreads();
@@ -158,20 +196,38 @@ __global__ void __launch_bounds__(256) radix_pass_kernel(const uint16_t *__restr
     const uint32_t p0 = st->prefix[0], p1 = st->prefix[1];
     const uint32_t mask = (1u << width) - 1u;
     __syncthreads();
-    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < M8; i += (long long)gridDim.x * blockDim.x) {
-        float f[8];
-        widen8<BF16>(__ldg(reinterpret_cast<const uint4 *>(x) + i), f);
-        const int kc = (int)((i * 8) % K);
-        const float4 ma = __ldg(reinterpret_cast<const float4 *>(m + kc));
-        const float4 mb = __ldg(reinterpret_cast<const float4 *>(m + kc + 4));
-        const float mk[8] = {ma.x, ma.y, ma.z, ma.w, mb.x, mb.y, mb.z, mb.w};
+    constexpr int RU = 4;  // 16-byte loads in flight per thread
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    for (long long i0 = (long long)blockIdx.x * blockDim.x + threadIdx.x; i0 < M8; i0 += stride * RU) {
+        uint4 v[RU];
+        float4 ma[RU], mb[RU];
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            const uint32_t key = __float_as_uint(__fsub_rn(f[j], mk[j])) & 0x7fffffffu;
-            const uint32_t hi = key >> (shift + width);
-            const uint32_t b = (key >> shift) & mask;
-            if (hi == p0) atomicAdd(&s_h[0][b], 1u);
-            if (hi == p1) atomicAdd(&s_h[1][b], 1u);
+        for (int u = 0; u < RU; ++u) {
+            const long long i = i0 + stride * u;
+            v[u] = make_uint4(0, 0, 0, 0);
+            ma[u] = mb[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (i < M8) {
+                v[u] = __ldg(reinterpret_cast<const uint4 *>(x) + i);
+                const int kc = (int)((i * 8) % K);
+                ma[u] = __ldg(reinterpret_cast<const float4 *>(m + kc));
+                mb[u] = __ldg(reinterpret_cast<const float4 *>(m + kc + 4));
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < RU; ++u) {
+            if (i0 + stride * u < M8) {
+                float f[8];
+                widen8<BF16>(v[u], f);
+                const float mk[8] = {ma[u].x, ma[u].y, ma[u].z, ma[u].w, mb[u].x, mb[u].y, mb[u].z, mb[u].w};
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const uint32_t key = __float_as_uint(__fsub_rn(f[j], mk[j])) & 0x7fffffffu;
+                    const uint32_t hi = key >> (shift + width);
+                    const uint32_t b = (key >> shift) & mask;
+                    if (hi == p0) atomicAdd(&s_h[0][b], 1u);
+                    if (hi == p1) atomicAdd(&s_h[1][b], 1u);
+                }
+            }
         }
     }
     __syncthreads();
@@ -187,8 +243,14 @@ __global__ void __launch_bounds__(256) radix_pass_kernel(const uint16_t *__restr
 __global__ void select_kernel(const uint32_t *__restrict__ hist, int nb, int width, int first, int last, uint32_t j,
                               uint32_t j1, double frac, SelState *__restrict__ st, float *__restrict__ tau_out) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    __shared__ uint32_t s_cnt[2][RADIX_BINS];  // the counts, fetched with all loads in flight (the scan below is serial)
+    for (int i = threadIdx.x; i < 2 * nb; i += blockDim.x) {
+        const int w = i / nb, b = i - w * nb;
+        s_cnt[w][b] = hist[(first ? 0 : w * RADIX_BINS) + b];
+    }
+    __syncthreads();
     if (warp < 2) {
-        const uint32_t *h = hist + (first ? 0 : warp * RADIX_BINS);
+        const uint32_t *h = s_cnt[warp];
         const uint32_t rank = first ? (warp == 0 ? j : j1) : st->rank[warp];
         const uint32_t prefix = first ? 0u : st->prefix[warp];
         uint32_t carry = 0, found_b = 0, found_r = 0;
@@ -270,19 +332,19 @@ static scap_status calibrate_t(const uint16_t *x, int T, int K, double sparsity,
     const long long j1 = j + 1 < M ? j + 1 : M - 1;
     const int grid = sm_count() * 4;
     // pass A (bits 30..20) was accumulated by mode_kernel
-    e = launch(select_kernel, dim3(1), dim3(64), 0, st, false, (const uint32_t *)hist, RADIX_BINS, 11, 1, 0, (uint32_t)j,
+    e = launch(select_kernel, dim3(1), dim3(256), 0, st, false, (const uint32_t *)hist, RADIX_BINS, 11, 1, 0, (uint32_t)j,
                (uint32_t)j1, frac, state, tau_out);
     if (e != cudaSuccess) return cuda_status(e);
     e = launch(radix_pass_kernel<BF16>, dim3(grid), dim3(256), 0, st, false, x, (const float *)m_out, M / 8, K,
                (const SelState *)state, 9, 11, hist + 2 * RADIX_BINS);
     if (e != cudaSuccess) return cuda_status(e);
-    e = launch(select_kernel, dim3(1), dim3(64), 0, st, false, (const uint32_t *)(hist + 2 * RADIX_BINS), RADIX_BINS, 11, 0, 0,
+    e = launch(select_kernel, dim3(1), dim3(256), 0, st, false, (const uint32_t *)(hist + 2 * RADIX_BINS), RADIX_BINS, 11, 0, 0,
                0u, 0u, frac, state, tau_out);
     if (e != cudaSuccess) return cuda_status(e);
     e = launch(radix_pass_kernel<BF16>, dim3(grid), dim3(256), 0, st, false, x, (const float *)m_out, M / 8, K,
                (const SelState *)state, 0, 9, hist + 4 * RADIX_BINS);
     if (e != cudaSuccess) return cuda_status(e);
-    e = launch(select_kernel, dim3(1), dim3(64), 0, st, false, (const uint32_t *)(hist + 4 * RADIX_BINS), 512, 9, 0, 1, 0u, 0u,
+    e = launch(select_kernel, dim3(1), dim3(256), 0, st, false, (const uint32_t *)(hist + 4 * RADIX_BINS), 512, 9, 0, 1, 0u, 0u,
                frac, state, tau_out);
     return cuda_status(e);
 }

@@ -64,6 +64,7 @@ struct FcArgs {
     float *z_copy;        // EPI_GLU: optional second copy of z, [B, F] dense rows
     uint32_t *bits;       // optional [ceil(K/32)]: union keep mask, one word per 32-channel chunk
     int hold_dependents;  // 1: do not let the next kernel start before this grid completes (it writes parameters)
+    int no_tc;            // 1: keep this call off the tcgen05 kernel
 };
 
 template <bool BF16, int BT, int CAP>

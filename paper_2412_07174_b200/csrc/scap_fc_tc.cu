@@ -474,7 +474,7 @@ static int tc_fills(int K, int S, int B, bool bf16) {
 // tune value 1 (default): calls whose kept channels fit the A-operand region in one fill per CTA - every further fill
 // drains and refills the ring, and the mma.sync variants are then faster; 2: every batch 3..16 call.
 bool tc_applicable(const FcArgs &a, int epi, bool bf16) {
-    if (g_tune.tc == 0 || a.B < 3 || a.B > 16 || a.ldw % 8 != 0 || !aligned16(a.W) || a.hold_dependents) return false;
+    if (g_tune.tc == 0 || a.no_tc || a.B < 3 || a.B > 16 || a.ldw % 8 != 0 || !aligned16(a.W) || a.hold_dependents) return false;
     if (g_tune.tc >= 2) return true;
     return tc_fills(a.K, tc_choose_split(a.K, a.Nh, epi, a.B, bf16), a.B, bf16) == 1;
 }

@@ -59,15 +59,18 @@ scap_status scap_glu_ffn(const void *h, const void *Wgu, const void *Wd, const f
     a.x = h; a.x_ld = D; a.m = m1; a.tau = tau1; a.bias = bgu_fused;
     a.y = z; a.y_ld = F; a.z_copy = z_out;
     if (idx1_out || nnz1_out) a.bits = reinterpret_cast<uint32_t *>(w + G.bits1);
-    cudaError_t e = launch_fc(bf16, MODE_GATHER, bf16 ? 1 : 0, EPI_GLU, a, st);
-    if (e != cudaSuccess) return cuda_status(e);
-
     FcArgs d;
     memset(&d, 0, sizeof(d));
     d.W = Wd; d.K = F; d.ldw = D; d.Nh = D; d.B = B;
     choose_config(F, D, EPI_BIAS, 1, B, &d.tn, &d.S);
     d.x = z; d.x_ld = F; d.m = m2; d.tau = tau2; d.bias = bd_fused; d.y = y; d.y_ld = D;
     if (idx2_out || nnz2_out) d.bits = reinterpret_cast<uint32_t *>(w + G.bits2);
+    // The two stages run back to back: either both take the tcgen05 kernel or neither does (measured: a stage on
+    // it between two mma.sync stages loses more at the kernel boundaries than it gains).
+    if (!(tc_applicable(a, EPI_GLU, bf16) && tc_applicable(d, EPI_BIAS, bf16))) a.no_tc = d.no_tc = 1;
+
+    cudaError_t e = launch_fc(bf16, MODE_GATHER, bf16 ? 1 : 0, EPI_GLU, a, st);
+    if (e != cudaSuccess) return cuda_status(e);
     e = launch_fc(bf16, MODE_GATHER, 2, EPI_BIAS, d, st);
     if (e != cudaSuccess) return cuda_status(e);
 
