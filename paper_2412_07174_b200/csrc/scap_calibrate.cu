@@ -9,7 +9,7 @@
 namespace scap {
 
 constexpr int CW = 32;             // channels per CTA strip: 4 threads x 8 channels (16 B) per row
-constexpr int CAL_THREADS = 256;   // 64 rows per sweep
+constexpr int CAL_THREADS = 512;   // 128 rows per sweep
 constexpr int CAL_ROWS = CAL_THREADS / 4;
 constexpr int RADIX_BINS = 2048;   // 11 bits per pass; passes take bits 30..20, 19..9, 8..0
 
@@ -28,7 +28,7 @@ __device__ __forceinline__ void widen8(const uint4 &v, float (&f)[8]) {
 
 // Rows t0, t0 + CAL_ROWS, ... (CAL_U of them) of this thread's 8 channels, all loads in flight together; rows at or
 // beyond T are skipped (their slots keep zeros and `valid` says how many are real).
-constexpr int CAL_U = 8;
+constexpr int CAL_U = 16;  // with 128 rows per sweep: 2048 rows of a strip live in registers at once
 __device__ __forceinline__ int load_rows(const uint16_t *xp, int K, int T, int t0, uint4 (&v)[CAL_U]) {
     int valid = 0;
 #pragma unroll
@@ -56,6 +56,12 @@ __global__ void __launch_bounds__(CAL_THREADS) mode_kernel(const uint16_t *__res
     const int kc = k0 + q * 8;
     const bool ok = kc < K;  // K is a multiple of 8
     const uint16_t *xp = x + kc;
+    // Up to CAL_ROWS * CAL_U = 2048 rows: the strip is read once, all loads in flight together, and the three
+    // passes below run from registers; longer inputs are re-read per pass (from L2 when they fit).
+    const bool resident = T <= CAL_ROWS * CAL_U;
+    uint4 v[CAL_U];
+    int nv = 0;
+    if (resident && ok) nv = load_rows(xp, K, T, rl, v);
 
     if (nbins > 0) {
         // ---- pass 1: per-channel min / max
@@ -64,8 +70,7 @@ __global__ void __launch_bounds__(CAL_THREADS) mode_kernel(const uint16_t *__res
         for (int j = 0; j < 8; ++j) { lo[j] = INFINITY; hi[j] = -INFINITY; }
         if (ok)
             for (int t0 = rl; t0 < T; t0 += CAL_ROWS * CAL_U) {
-                uint4 v[CAL_U];
-                const int nv = load_rows(xp, K, T, t0, v);
+                if (!resident) nv = load_rows(xp, K, T, t0, v);
 #pragma unroll
                 for (int u = 0; u < CAL_U; ++u) {
                     if (u < nv) {
@@ -103,8 +108,7 @@ __global__ void __launch_bounds__(CAL_THREADS) mode_kernel(const uint16_t *__res
         __syncthreads();
         if (ok)
             for (int t0 = rl; t0 < T; t0 += CAL_ROWS * CAL_U) {
-                uint4 v[CAL_U];
-                const int nv = load_rows(xp, K, T, t0, v);
+                if (!resident) nv = load_rows(xp, K, T, t0, v);
 #pragma unroll
                 for (int u = 0; u < CAL_U; ++u) {
                     if (u < nv) {
@@ -122,9 +126,9 @@ __global__ void __launch_bounds__(CAL_THREADS) mode_kernel(const uint16_t *__res
                 }
             }
         __syncthreads();
-        // ---- arg-max: lowest bin with the largest count; warp w takes channels 4w .. 4w+3
+        // ---- arg-max: lowest bin with the largest count; warp w takes channels 2w, 2w+1
         const int lane = tid & 31, warp = tid >> 5;
-        for (int c = warp * (CW / 8); c < (warp + 1) * (CW / 8); ++c) {
+        for (int c = warp * (CW / (CAL_THREADS / 32)); c < (warp + 1) * (CW / (CAL_THREADS / 32)); ++c) {
             uint32_t best_cnt = 0;
             int best_i = 0;
             for (int i = lane; i < nbins; i += 32) {
@@ -165,8 +169,7 @@ __global__ void __launch_bounds__(CAL_THREADS) mode_kernel(const uint16_t *__res
     __syncthreads();
     if (ok)
         for (int t0 = rl; t0 < T; t0 += CAL_ROWS * CAL_U) {
-            uint4 v[CAL_U];
-            const int nv = load_rows(xp, K, T, t0, v);
+            if (!resident) nv = load_rows(xp, K, T, t0, v);
 #pragma unroll
             for (int u = 0; u < CAL_U; ++u) {
                 if (u < nv) {
