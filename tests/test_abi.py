@@ -64,6 +64,10 @@ def test_argument_validation_returns_codes(L):
     assert L.scap_tune(b"no_such_key", 1) == 1
     assert L.scap_tune(b"split_k", 9) == 1
     assert L.scap_tune(b"split_k", 0) == 0
+    assert L.scap_tune(b"tcgen05", 3) == 1
+    assert L.scap_tune(b"tcgen05", -1) == 1
+    for v in (0, 2, 1):  # leaves the default
+        assert L.scap_tune(b"tcgen05", v) == 0
     assert L.scap_calibrate(P, 16, 12, 1, 0.5, 16, P, P, P, 1 << 20, None) == 4   # K not a multiple of 8
     assert L.scap_calibrate(P, 16, 16, 1, 1.5, 16, P, P, P, 1 << 20, None) == 1   # sparsity outside [0, 1)
     assert L.scap_glu_ffn(P, P, P, None, P, None, None, P, None, P, 1, 64, 60, 1, None, None, None, None, None, P,
