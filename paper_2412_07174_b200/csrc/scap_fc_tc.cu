@@ -476,7 +476,10 @@ static int tc_fills(int K, int S, int B, bool bf16) {
 bool tc_applicable(const FcArgs &a, int epi, bool bf16) {
     if (g_tune.tc == 0 || a.no_tc || a.B < 3 || a.B > 16 || a.ldw % 8 != 0 || !aligned16(a.W) || a.hold_dependents) return false;
     if (g_tune.tc >= 2) return true;
-    return tc_fills(a.K, tc_choose_split(a.K, a.Nh, epi, a.B, bf16), a.B, bf16) == 1;
+    // ... and whose CTAs stream at least 32 chunks each: on shorter streams the heavier set-up (TMEM, barriers,
+    // operand staging) of this kernel outweighs its gain (measured at K = N = 4096)
+    const int S = tc_choose_split(a.K, a.Nh, epi, a.B, bf16);
+    return tc_fills(a.K, S, a.B, bf16) == 1 && ((a.K + 31) / 32 + S - 1) / S >= 32;
 }
 
 // Split-K factor for the tensor-core kernel (tile width is fixed at 128): most CTAs that are all resident at
