@@ -134,6 +134,22 @@ def oracle_calibration(d):
     return cal
 
 
+def max_over_ranks(value, world, device):
+    """The slowest rank's time: replicas are independent, so the job is as slow as its slowest replica."""
+    if world <= 1:
+        return float(value)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_gbs(bytes_per_rank, world, seconds):
+    """Aggregate GB/s of `world` replicas that each touch bytes_per_rank in `seconds` (weak scaling)."""
+    return world * bytes_per_rank / seconds / 1e9
+
+
 def run_reference(args, rank):
     """CPU oracle arm: the same metric on a bounded sample per step, on the host cores."""
     if rank != 0:
@@ -535,12 +551,9 @@ def main():
     barrier()
     clocks = sampler.stop() if rank == 0 else None
     ms = e0.elapsed_time(e1)
-    if world > 1:
-        t = torch.tensor([ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = max_over_ranks(ms, world, "cuda")
     ms_per_step = ms / args.steps
-    value = world * step_bytes / (ms_per_step * 1e-3) / 1e9
+    value = whole_job_gbs(step_bytes, world, ms_per_step * 1e-3)
 
     # ------------------------------------------------------------------ per-sparsity and dense detail (rank 0 reports)
     detail = {}
@@ -579,11 +592,8 @@ def main():
         host_step(ctr)
     barrier()
     e2e_s = time.perf_counter() - t0
-    if world > 1:
-        t = torch.tensor([e2e_s], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_s = float(t.item())
-    e2e_value = world * step_bytes * e2e_steps / e2e_s / 1e9
+    e2e_s = max_over_ranks(e2e_s, world, "cuda")
+    e2e_value = whole_job_gbs(step_bytes * e2e_steps, world, e2e_s)
 
     if rank != 0:
         if world > 1:
