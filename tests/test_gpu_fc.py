@@ -86,18 +86,45 @@ def test_sparsity_levels(S, s):
 
 # ---------------------------------------------------------------- degenerate cases
 
-def test_tau_zero_is_dense_and_tau_inf_returns_bias(S):
+@pytest.mark.parametrize("tc_mode", [1, 2])                        # 2: the batch-3 call runs on the tcgen05 kernel
+def test_tau_zero_is_dense_and_tau_inf_returns_bias(S, tc_mode):
     d = si.laplace_fc(4, 640, 264, si.BF16, 8, 3)
     dt = d["dt"]
     bf = np.linspace(-1, 1, 264).astype(np.float32)
-    y, idx, n = run_sparse(S, d, None, 0.0, bf)
-    assert n == 640 and np.array_equal(idx, np.arange(640, dtype=np.uint32))
-    y64 = oracle.dense_fc(si.to_f32(d["x"], dt), d["W"], dt, bf)
+    try:
+        S.scap_tune("tcgen05", tc_mode)
+        y, idx, n = run_sparse(S, d, None, 0.0, bf)
+        assert n == 640 and np.array_equal(idx, np.arange(640, dtype=np.uint32))
+        y64 = oracle.dense_fc(si.to_f32(d["x"], dt), d["W"], dt, bf)
+        assert rel_l2_rows(y, y64) <= REL_L2_TOL
+        y, idx, n = run_sparse(S, d, d["m_true"], np.inf, bf)
+        assert n == 0 and np.array_equal(y, np.tile(bf, (3, 1)))   # nnz = 0: y == b_fused exactly
+        y, idx, n = run_sparse(S, d, d["m_true"], np.inf, None)
+        assert n == 0 and not y.any()
+        S.scap_device_status()
+    finally:
+        S.scap_tune("tcgen05", 1)
+
+
+@pytest.mark.parametrize("tc_mode", [0, 2])
+def test_nan_and_threshold_ties_in_a_batch_of_three(S, tc_mode):
+    K, N = 72, 24
+    d = si.laplace_fc(4, K, N, si.BF16, 8, 3)
+    x = np.zeros((3, K))
+    x[0, 0], x[0, 1], x[0, 2], x[0, 4] = 0.5, -0.5, 0.49, -0.0
+    x[1, 5], x[1, 6] = 2.0, -0.25
+    x[2, 40], x[2, 71] = -3.0, 0.5
+    xb = si.to_bits(x, si.BF16)
+    xb[:, 3] = 0x7FC0                                              # bf16 NaN in every row: dropped, never multiplied
+    y64, keep, idx = oracle_fc(d, None, 0.5, None, x_bits=xb)
+    assert idx.tolist() == [0, 1, 5, 40, 71]
+    try:
+        S.scap_tune("tcgen05", tc_mode)
+        y, gidx, n = run_sparse(S, d, None, 0.5, None, x_bits=xb)
+    finally:
+        S.scap_tune("tcgen05", 1)
+    assert gidx.tolist() == [0, 1, 5, 40, 71] and np.isfinite(y).all()
     assert rel_l2_rows(y, y64) <= REL_L2_TOL
-    y, idx, n = run_sparse(S, d, d["m_true"], np.inf, bf)
-    assert n == 0 and np.array_equal(y, np.tile(bf, (3, 1)))       # nnz = 0: y == b_fused exactly
-    y, idx, n = run_sparse(S, d, d["m_true"], np.inf, None)
-    assert n == 0 and not y.any()
 
 
 def test_ties_signed_zero_and_nan(S):
