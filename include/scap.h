@@ -80,6 +80,8 @@ int scap_version(void);
  *   "tcgen05"  batch 3..16 calls of the FC and SwiGLU entry points: 0 = always the mma.sync variants,
  *              1 = the tcgen05 (TMEM accumulator) kernel where its shared-memory operand region holds
  *              the call's kept channels in one pass, else mma.sync (default), 2 = always tcgen05
+ *   "host_direct"  scap_sparse_fc_host: 1 = when x_host and y_host are page-locked and addressable by the
+ *              device, a kernel pulls x and the FC kernel writes y to host memory (default), 0 = always copies
  * Unknown keys return SCAP_ERR_INVALID_ARG.  Tuning never changes what is computed; split_k
  * changes the (fixed) summation order and therefore the last bits of y.  Query workspace sizes
  * after tuning.                                                                               */
@@ -142,6 +144,9 @@ scap_status scap_dense_fc(const void *x, const void *W, const float *b, float *y
 /* scap_sparse_fc for a caller whose activations live in HOST memory: copies x_host[B,K]
  * (dtype dt; pinned memory recommended) to the device, runs the sparse FC, and copies y back to
  * y_host[B,N] (fp32), all enqueued on `stream`; y_host is valid once the stream has drained.
+ * If both buffers are page-locked and addressable by the device (cudaHostAlloc, cudaHostRegister), the
+ * transfers are done by the library's kernels instead of copy operations (a small kernel pulls x into
+ * the workspace, the FC kernel stores y to host memory); x_host must stay unchanged until then.
  * W, m, tau, b_fused stay device-resident.  Needs scap_fc_host_workspace(B, K, N) bytes.        */
 size_t scap_fc_host_workspace(int B, int K, int N);
 scap_status scap_sparse_fc_host(const void *x_host, const void *W, const float *m, const float *tau,

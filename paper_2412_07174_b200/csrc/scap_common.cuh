@@ -18,6 +18,7 @@ struct Tuning {
     int split_k;  // 0 = automatic
     int pdl;      // programmatic dependent launch between the kernels of one call
     int tc;       // batch 3..16 on the tcgen05 kernel (0: the mma.sync variants)
+    int host_direct;  // scap_sparse_fc_host moves device-addressable pinned host buffers with its own kernels
 };
 extern Tuning g_tune;
 

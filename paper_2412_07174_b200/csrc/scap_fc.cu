@@ -6,7 +6,7 @@
 
 namespace scap {
 
-Tuning g_tune = {0, 1, 1};
+Tuning g_tune = {0, 1, 1, 1};
 
 scap_status check_device() {
     static int cached[64];  // 0 unknown, 1 ok, 2 unsupported
@@ -143,6 +143,14 @@ cudaError_t launch_fc(bool bf16, int mode, int xkind, int epi, const FcArgs &a, 
     return bf16 ? launch_fc_w<true>(mode, xkind, epi, a, st) : launch_fc_w<false>(mode, xkind, epi, a, st);
 }
 
+// Copies n16 16-byte words from device-addressable host memory into device memory (one word per thread).
+__global__ void __launch_bounds__(256) pull_host_kernel(const uint4 *__restrict__ src, uint4 *__restrict__ dst, long long n16) {
+    griddep_wait();               // the previous kernel in the stream may still read dst
+    griddep_launch_dependents();  // the FC kernel that follows waits for this grid before it reads dst
+    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n16) dst[i] = src[i];
+}
+
 // One CTA of 1024 threads: popcount prefix over the mask words, then every word's thread writes its set bits.
 __global__ void __launch_bounds__(1024) expand_bits_kernel(const uint32_t *__restrict__ bits, int K,
                                                           uint32_t *__restrict__ idx_out, int *__restrict__ nnz_out) {
@@ -264,6 +272,10 @@ scap_status scap_tune(const char *key, int value) {
         g_tune.pdl = value != 0;
         return SCAP_OK;
     }
+    if (!strcmp(key, "host_direct")) {
+        g_tune.host_direct = value != 0;
+        return SCAP_OK;
+    }
     if (!strcmp(key, "tcgen05")) {
         if (value < 0 || value > 2) return SCAP_ERR_INVALID_ARG;
         g_tune.tc = value;
@@ -336,6 +348,25 @@ scap_status scap_sparse_fc_host(const void *x_host, const void *W, const float *
     unsigned char *x_dev = w + fc;
     float *y_dev = reinterpret_cast<float *>(w + fc + align_up((size_t)B * K * 2, 256));
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    // Page-locked buffers that the device can address (cudaHostAlloc / cudaHostRegister memory under unified
+    // addressing): a small kernel pulls x across the bus once into the workspace, and the FC kernel writes each
+    // element of y straight to host memory - two launches instead of copy, launch, copy.  (Reading x in place from
+    // the FC kernel would fetch it once per column tile over the bus; measured slower.)  Anything else goes
+    // through the staging copies below.
+    if (g_tune.host_direct) {
+        cudaPointerAttributes ax, ay;
+        const bool okx = cudaPointerGetAttributes(&ax, x_host) == cudaSuccess && ax.type == cudaMemoryTypeHost && ax.devicePointer;
+        const bool oky = okx && cudaPointerGetAttributes(&ay, y_host) == cudaSuccess && ay.type == cudaMemoryTypeHost && ay.devicePointer;
+        if (!okx || !oky) cudaGetLastError();
+        if (okx && oky && aligned16(ax.devicePointer) && aligned16(ay.devicePointer) && ((size_t)B * K * 2) % 16 == 0) {
+            const long long n16 = (long long)B * K * 2 / 16;
+            const int blocks = (int)((n16 + 255) / 256);
+            cudaError_t e = launch(pull_host_kernel, dim3(blocks), dim3(256), 0, s, g_tune.pdl != 0,
+                                   static_cast<const uint4 *>(ax.devicePointer), reinterpret_cast<uint4 *>(x_dev), n16);
+            if (e != cudaSuccess) return cuda_status(e);
+            return sparse_fc_impl(x_dev, W, m, tau, b_fused, static_cast<float *>(ay.devicePointer), B, K, N, dt, nullptr, nullptr, w, s);
+        }
+    }
     cudaError_t e = cudaMemcpyAsync(x_dev, x_host, (size_t)B * K * 2, cudaMemcpyHostToDevice, s);
     if (e != cudaSuccess) return cuda_status(e);
     st = sparse_fc_impl(x_dev, W, m, tau, b_fused, y_dev, B, K, N, dt, nullptr, nullptr, w, s);

@@ -273,16 +273,25 @@ def test_fold_bias(S, K, N, dt, bias):
     assert np.linalg.norm(got - want) / np.linalg.norm(want) <= 1e-6
 
 
-def test_host_buffer_variant_matches_device_variant(S):
-    d = si.laplace_fc(4, 1024, 520, si.BF16, 16, 4)
+@pytest.mark.parametrize("pinned,direct", [(True, 1), (True, 0), (False, 1)])
+@pytest.mark.parametrize("B", [1, 4])
+def test_host_buffer_variant_matches_device_variant(S, pinned, direct, B):
+    # pinned + direct: the library's kernels pull x from and store y to host memory; otherwise staging copies
+    d = si.laplace_fc(4, 1024, 520, si.BF16, 16, B)
     dt = d["dt"]
     y_dev, _, _ = run_sparse(S, d, d["m_true"], 0.3, None, want_idx=False)
     W, m, tau = dev(d["W"], dt), f32(d["m_true"]), f32([0.3])
-    xh = si.as_torch(d["x"], dt).pin_memory()
-    yh = torch.zeros((4, 520), dtype=torch.float32).pin_memory()
-    ws = workspace(S.scap_fc_host_workspace(4, 1024, 520))
-    S.scap_sparse_fc_host(xh, W, m, tau, None, yh, ws.payload)
-    torch.cuda.synchronize()
+    xh = si.as_torch(d["x"], dt)
+    yh = torch.zeros((B, 520), dtype=torch.float32)
+    if pinned:
+        xh, yh = xh.pin_memory(), yh.pin_memory()
+    ws = workspace(S.scap_fc_host_workspace(B, 1024, 520))
+    try:
+        S.scap_tune("host_direct", direct)
+        S.scap_sparse_fc_host(xh, W, m, tau, None, yh, ws.payload)
+        torch.cuda.synchronize()
+    finally:
+        S.scap_tune("host_direct", 1)
     assert ws.intact()
     assert np.array_equal(yh.numpy(), y_dev)
 
