@@ -56,6 +56,12 @@ def lib():
         L.scap_oracle_fold_bias.restype = None
         L.scap_oracle_mode.argtypes = [vp, i, i, i, vp]
         L.scap_oracle_mode.restype = None
+        L.scap_oracle_mean.argtypes = [vp, i, i, vp]
+        L.scap_oracle_mean.restype = None
+        L.scap_oracle_median.argtypes = [vp, i, i, vp]
+        L.scap_oracle_median.restype = None
+        L.scap_oracle_eta_mean.argtypes = [vp, i, i]
+        L.scap_oracle_eta_mean.restype = f
         L.scap_oracle_tau.argtypes = [vp, i, i, vp, d, vp, vp]
         L.scap_oracle_tau.restype = f
         L.scap_oracle_glu_ffn.argtypes = [vp, vp, vp, i, vp, f, vp, vp, f, vp, i, i, i, vp, vp, vp]
@@ -173,6 +179,40 @@ def mode(xf_calib, nbins: int = 2048):
     m = np.empty(K, np.float32)
     lib().scap_oracle_mode(_p(xf), T, K, nbins, _p(m))
     return m
+
+
+HISTOGRAM, MEAN, MEDIAN = 0, 1, 2      # mode estimators (Section 3, "Determination of mode value")
+PER_CHANNEL, SCALAR = 0, 1             # one mode per input channel, or the paper's single eta per FC
+
+
+def mode_estimate(xf_calib, estimator: int = HISTOGRAM, scope: int = PER_CHANNEL, nbins: int = 2048):
+    """m[K] by the chosen estimator; with scope SCALAR the single eta of the pooled tensor, broadcast to K entries."""
+    xf = _f32(np.atleast_2d(xf_calib))
+    T, K = xf.shape
+    if scope == PER_CHANNEL:
+        if estimator == HISTOGRAM:
+            return mode(xf, nbins)
+        m = np.empty(K, np.float32)
+        (lib().scap_oracle_mean if estimator == MEAN else lib().scap_oracle_median)(_p(xf), T, K, _p(m))
+        return m
+    if estimator == MEAN:
+        eta = np.float32(lib().scap_oracle_eta_mean(_p(xf), T, K))
+    else:
+        flat = np.ascontiguousarray(xf.reshape(T * K, 1))
+        one = np.empty(1, np.float32)
+        if estimator == HISTOGRAM:
+            lib().scap_oracle_mode(_p(flat), T * K, 1, nbins, _p(one))
+        else:
+            lib().scap_oracle_median(_p(flat), T * K, 1, _p(one))
+        eta = one[0]
+    return np.full(K, eta, np.float32)
+
+
+def calibrate_ex(xf_calib, s: float, estimator: int = HISTOGRAM, scope: int = PER_CHANNEL, nbins: int = 2048):
+    """Mode by the chosen estimator and scope, then the threshold on the centred importance."""
+    xf = _f32(np.atleast_2d(xf_calib))
+    m = mode_estimate(xf, estimator, scope, nbins)
+    return m, tau(xf, m, s)
 
 
 def tau(xf_calib, m, s: float, want_neighbours=False):

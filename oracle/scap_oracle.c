@@ -214,6 +214,47 @@ static int cmp_float(const void *a, const void *b) {
     return (x > y) - (x < y);
 }
 
+/* ---------------------------------------------------------------- mode by mean or median
+ * Section 3 ("Determination of mode value"): a fast estimate of the mode is the empirical mean or
+ * the median of the calibration activations.  Per channel k:
+ *   mean:    m[k] = ( sum_{t = 0 .. T-1, in this order} x[t,k] ) / T   in binary64, rounded once to binary32;
+ *   median:  v = the column sorted ascending, m[k] = ( v[(T-1)/2] + v[T/2] ) / 2 in binary64, rounded once
+ *            (the middle value for odd T, the mean of the two middle values for even T).
+ * A result of -0 is returned as +0.                                                             */
+void scap_oracle_mean(const float *xf /*[T,K]*/, int T, int K, float *m_out) {
+    for (int k = 0; k < K; ++k) {
+        double acc = 0.0;
+        for (int t = 0; t < T; ++t) acc += (double)xf[(long)t * K + k];
+        m_out[k] = (float)(acc / (double)T) + 0.0f;
+    }
+}
+
+void scap_oracle_median(const float *xf /*[T,K]*/, int T, int K, float *m_out) {
+    float *v = (float *)malloc(sizeof(float) * (size_t)T);
+    for (int k = 0; k < K; ++k) {
+        for (int t = 0; t < T; ++t) v[t] = xf[(long)t * K + k];
+        qsort(v, (size_t)T, sizeof(float), cmp_float);
+        volatile double mid = ((double)v[(T - 1) / 2] + (double)v[T / 2]) / 2.0;
+        m_out[k] = (float)mid + 0.0f;
+    }
+    free(v);
+}
+
+/* Scalar eta for the whole FC input (the paper's eta is one scalar per layer), from all T*K values:
+ *   mean:    the per-channel sums above (each over t in order), added over k = 0 .. K-1 in this order in
+ *            binary64, divided by T*K, rounded once to binary32;
+ *   median and histogram mode: the per-channel definitions applied to the tensor read as one channel of
+ *            T*K values (callers pass T*K, 1).                                                   */
+float scap_oracle_eta_mean(const float *xf /*[T,K]*/, int T, int K) {
+    double total = 0.0;
+    for (int k = 0; k < K; ++k) {
+        double acc = 0.0;
+        for (int t = 0; t < T; ++t) acc += (double)xf[(long)t * K + k];
+        total += acc;
+    }
+    return (float)(total / ((double)T * (double)K)) + 0.0f;
+}
+
 float scap_oracle_tau(const float *xf /*[T,K]*/, int T, int K, const float *m, double s,
                       float *vj_out, float *vj1_out) {
     long M = (long)T * K;

@@ -406,3 +406,75 @@ def test_ffn_sparsity_reproduces_printed_rows():
         assert abs(got - float(ffn)) <= 0.1 + 1e-9, (up, gate, down, ffn, got)
     # the shared-input form printed in Appendix B: 2/3 s_x + 1/3 s_gated
     assert abs(oracle.ffn_sparsity(42.0, 42.0, 61.7) - (2 / 3 * 42.0 + 1 / 3 * 61.7)) < 1e-12
+
+
+# ---------------------------------------------------------------- mean / median estimators, scalar eta (Section 3)
+
+def test_mean_and_median_agree_with_library_routines_and_closed_forms():
+    rng = np.random.default_rng(7)
+    for T, K in ((1, 3), (2, 5), (101, 7), (256, 4)):
+        x = rng.standard_normal((T, K)).astype(np.float32)
+        x[:, 0] = 1.5                                              # constant channel
+        mean = oracle.mode_estimate(x, oracle.MEAN)
+        med = oracle.mode_estimate(x, oracle.MEDIAN)
+        # library mean differs from the in-order sum by rounding order only: one ulp of binary32 at most
+        ref_mean = x.astype(np.float64).mean(axis=0)
+        assert np.all(np.abs(mean - ref_mean) <= np.spacing(np.abs(ref_mean).astype(np.float32)))
+        assert np.array_equal(med, np.median(x.astype(np.float64), axis=0).astype(np.float32))
+        assert mean[0] == np.float32(1.5) and med[0] == np.float32(1.5)
+    # closed forms: arithmetic progression (mean = median = midpoint), exact in binary64
+    x = np.arange(1, 1001, dtype=np.float32).reshape(-1, 1)[::-1].copy()
+    assert oracle.mode_estimate(x, oracle.MEAN)[0] == np.float32(500.5)
+    assert oracle.mode_estimate(x, oracle.MEDIAN)[0] == np.float32(500.5)
+    # odd count: the middle element itself; even: the mean of the two middle ones
+    assert oracle.mode_estimate(np.float32([[5], [1], [9]]), oracle.MEDIAN)[0] == np.float32(5)
+    assert oracle.mode_estimate(np.float32([[5], [1], [9], [6]]), oracle.MEDIAN)[0] == np.float32(5.5)
+
+
+def test_mean_is_a_sum_in_row_order_in_binary64():
+    # 2^20 + 2^-30 is exact in binary64 (50 bits apart) but not in binary32: the accumulator is binary64
+    x = np.float32([[2.0 ** 20], [2.0 ** -30], [-(2.0 ** 20)]])
+    assert oracle.mode_estimate(x, oracle.MEAN)[0] == np.float32((2.0 ** -30) / 3.0)
+    # ... and rows are added in order: here the small term is absorbed before the large ones cancel
+    x = np.float32([[2.0 ** 60], [2.0 ** -30], [-(2.0 ** 60)]])   # absorbed: 2^60 + 2^-30 == 2^60 in binary64
+    assert oracle.mode_estimate(x, oracle.MEAN)[0] == np.float32(0.0)
+
+
+def test_signed_zero_results_are_returned_as_plus_zero():
+    x = np.float32([[-0.0], [-0.0]])
+    for est in (oracle.MEAN, oracle.MEDIAN):
+        m = oracle.mode_estimate(x, est)
+        assert m[0] == 0 and not np.signbit(m[0])
+
+
+def test_scalar_eta_pools_the_whole_tensor_and_is_broadcast():
+    rng = np.random.default_rng(11)
+    x = (rng.standard_normal((64, 9)) + np.linspace(-2, 2, 9)[None, :]).astype(np.float32)
+    for est in (oracle.HISTOGRAM, oracle.MEAN, oracle.MEDIAN):
+        m = oracle.mode_estimate(x, est, oracle.SCALAR, nbins=32)
+        assert m.shape == (9,) and np.all(m == m[0])
+    eta_mean = oracle.mode_estimate(x, oracle.MEAN, oracle.SCALAR)[0]
+    ref = x.astype(np.float64).mean()
+    assert abs(eta_mean - ref) <= np.spacing(np.float32(abs(ref)))
+    assert oracle.mode_estimate(x, oracle.MEDIAN, oracle.SCALAR)[0] == np.float32(np.median(x.astype(np.float64)))
+    # pooled histogram mode == per-channel definition on the flattened tensor
+    flat = x.reshape(-1, 1)
+    assert oracle.mode_estimate(x, oracle.HISTOGRAM, oracle.SCALAR, nbins=32)[0] == oracle.mode(flat, 32)[0]
+    # one channel: scalar and per-channel coincide
+    one = x[:, :1].copy()
+    for est in (oracle.HISTOGRAM, oracle.MEAN, oracle.MEDIAN):
+        assert np.array_equal(oracle.mode_estimate(one, est, oracle.SCALAR, 32), oracle.mode_estimate(one, est, oracle.PER_CHANNEL, 32))
+
+
+def test_estimators_rank_as_expected_on_a_skewed_distribution():
+    # exponential-like (GELU-output-like) data: mode < median < mean; centring by a better mode estimate prunes more at fixed tau
+    rng = np.random.default_rng(3)
+    x = rng.exponential(1.0, size=(4096, 2)).astype(np.float32)
+    hist = oracle.mode_estimate(x, oracle.HISTOGRAM, nbins=64)
+    med = oracle.mode_estimate(x, oracle.MEDIAN)
+    mean = oracle.mode_estimate(x, oracle.MEAN)
+    assert np.all(hist < med) and np.all(med < mean)
+    assert np.all(np.abs(med - math.log(2.0)) < 0.05) and np.all(np.abs(mean - 1.0) < 0.05)
+    tau = np.float32(0.25)
+    frac = [float(np.mean(np.abs(x - m[None, :]) < tau)) for m in (hist, med, mean)]
+    assert frac[0] > frac[1] > frac[2]
