@@ -271,6 +271,32 @@ def suite_calibrate(torch, scap, out):
          "compulsory_bytes": T * Kk * 2, "gbs_on_compulsory_bytes": round(T * Kk * 2 / t / 1e3, 1), "passes_over_input": 3 if T <= 2048 else 5,
          "l2": "flushed before each run"})
 
+    # The paper's other estimators of the mode (mean, median) and its scalar eta, on the same tensor and on a skewed
+    # one (|N(0,1)|^1.5, GELU-output-like): time per call, and the sparsity each centring induces at one fixed tau.
+    names = {0: "histogram", 1: "mean", 2: "median"}
+    skew = si.to_bits(np.abs(si.normal(si.stream_seed(4, 9), T * Kk).reshape(T, Kk)) ** 1.5, si.BF16)
+    xs = si.as_torch(skew, si.BF16).cuda()
+    for scope in (0, 1):
+        for est in (0, 1, 2):
+            times = []
+            for _ in range(6):
+                flush.fill_(1)
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                torch.cuda.synchronize()
+                e0.record()
+                scap.scap_calibrate_ex(xc, 0.6, est, scope, NBINS, m, tau, cws)
+                e1.record()
+                torch.cuda.synchronize()
+                times.append(e0.elapsed_time(e1) * 1e3)
+            scap.scap_calibrate_ex(xs, 0.6, est, scope, NBINS, m, tau, cws)
+            torch.cuda.synchronize()
+            fixed_tau = 0.15
+            pruned = float(((xs.float() - m[None, :]).abs() < fixed_tau).float().mean().item())
+            out({"suite": "calibrate_ex", "T": T, "K": Kk, "estimator": names[est], "scope": "scalar" if scope else "per_channel",
+                 "us": round(float(np.median(times[2:])), 1), "skewed_input": "|N(0,1)|^1.5 in bf16",
+                 "sparsity_at_tau_%.2f_on_skewed_input" % fixed_tau: round(pruned, 4),
+                 "tau_for_60pct_on_skewed_input": round(float(tau.item()), 5)})
+
 
 def suite_glu(torch, scap, peak, out):
     """Config 2: full Llama-2-7B-shaped SwiGLU block, batch 1 / 4 / 8, 40 % / 70 % targets."""

@@ -109,6 +109,24 @@ size_t scap_calibrate_workspace(int T, int K, int nbins);
 scap_status scap_calibrate(const void *x_calib, int T, int K, scap_dtype dt, double sparsity, int nbins,
                            float *m_out, float *tau_out, void *ws, size_t ws_bytes, scap_stream_t stream);
 
+/* Section 3, "Determination of mode value": the paper names the empirical mean and the median as fast
+ * estimates of the mode, and its eta is one scalar per FC.  scap_calibrate_ex is scap_calibrate with the
+ * estimator and the scope chosen by the caller (same workspace query, same tau computation on |x - m|):
+ *   SCAP_MODE_HISTOGRAM  arg-max bin centre as in scap_calibrate
+ *   SCAP_MODE_MEAN       per channel: the column added in row order in binary64, divided by T, rounded once
+ *   SCAP_MODE_MEDIAN     per channel: the middle value, or the mean of the two middle values (binary64,
+ *                        rounded once) for even T
+ *   SCAP_ETA_PER_CHANNEL one value per input channel in m_out[K]
+ *   SCAP_ETA_SCALAR      one value for the whole tensor, written to all K entries of m_out: the estimator
+ *                        applied to all T*K values as one sample (mean: the column sums of the per-channel
+ *                        form added in channel order, divided by T*K)
+ * A result of -0 is returned as +0.  Inputs must be finite.                                            */
+typedef enum { SCAP_MODE_HISTOGRAM = 0, SCAP_MODE_MEAN = 1, SCAP_MODE_MEDIAN = 2 } scap_mode_estimator;
+typedef enum { SCAP_ETA_PER_CHANNEL = 0, SCAP_ETA_SCALAR = 1 } scap_eta_scope;
+scap_status scap_calibrate_ex(const void *x_calib, int T, int K, scap_dtype dt, double sparsity,
+                              scap_mode_estimator estimator, scap_eta_scope scope, int nbins, float *m_out,
+                              float *tau_out, void *ws, size_t ws_bytes, scap_stream_t stream);
+
 /* Eq. 5-6: b_fused[n] = b[n] + sum_k m[k] W[k,n].  b is in the weight dtype and may be NULL
  * (zero bias).  Run once per layer after calibration.                                          */
 size_t scap_fold_bias_workspace(int K, int N);

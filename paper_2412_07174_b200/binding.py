@@ -8,7 +8,8 @@ import torch
 
 __all__ = [
     "SCAP_F16", "SCAP_BF16", "ScapError", "lib", "lib_path", "status_string", "scap_version", "scap_tune", "scap_device_status",
-    "scap_calibrate_workspace", "scap_calibrate", "scap_fold_bias_workspace", "scap_fold_bias",
+    "scap_calibrate_workspace", "scap_calibrate", "scap_calibrate_ex", "SCAP_MODE_HISTOGRAM", "SCAP_MODE_MEAN", "SCAP_MODE_MEDIAN",
+    "SCAP_ETA_PER_CHANNEL", "SCAP_ETA_SCALAR", "scap_fold_bias_workspace", "scap_fold_bias",
     "scap_fc_workspace", "scap_sparse_fc", "scap_dense_fc", "scap_fc_host_workspace", "scap_sparse_fc_host",
     "scap_glu_workspace", "scap_glu_ffn", "scap_glu_static_capacity", "scap_glu_ffn_static", "scap_moe_workspace",
     "scap_moe_ffn", "ScapExpert", "dtype_of", "EXPORTS",
@@ -20,7 +21,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 # every symbol include/scap.h declares
 EXPORTS = [
     "scap_status_string", "scap_version", "scap_tune", "scap_device_status", "scap_calibrate_workspace", "scap_calibrate",
-    "scap_fold_bias_workspace", "scap_fold_bias", "scap_fc_workspace", "scap_sparse_fc", "scap_dense_fc",
+    "scap_calibrate_ex", "scap_fold_bias_workspace", "scap_fold_bias", "scap_fc_workspace", "scap_sparse_fc", "scap_dense_fc",
     "scap_fc_host_workspace", "scap_sparse_fc_host", "scap_glu_workspace", "scap_glu_ffn",
     "scap_glu_static_capacity", "scap_glu_ffn_static", "scap_moe_workspace", "scap_moe_ffn",
 ]
@@ -66,6 +67,8 @@ def lib():
     L.scap_calibrate_workspace.restype = sz
     L.scap_calibrate.argtypes = [vp, i, i, i, d, i, vp, vp, vp, sz, vp]
     L.scap_calibrate.restype = i
+    L.scap_calibrate_ex.argtypes = [vp, i, i, i, d, i, i, i, vp, vp, vp, sz, vp]
+    L.scap_calibrate_ex.restype = i
     L.scap_fold_bias_workspace.argtypes = [i, i]
     L.scap_fold_bias_workspace.restype = sz
     L.scap_fold_bias.argtypes = [vp, vp, vp, i, i, i, vp, vp, sz, vp]
@@ -156,6 +159,17 @@ def scap_calibrate(x_calib, sparsity: float, nbins: int, m_out, tau_out, ws, str
     p, n = _ws(ws)
     _check(lib().scap_calibrate(_ptr(x_calib), T, K, dtype_of(x_calib), float(sparsity), nbins, _ptr(m_out), _ptr(tau_out),
                                 p, n, _stream(stream)), "scap_calibrate")
+
+
+SCAP_MODE_HISTOGRAM, SCAP_MODE_MEAN, SCAP_MODE_MEDIAN = 0, 1, 2
+SCAP_ETA_PER_CHANNEL, SCAP_ETA_SCALAR = 0, 1
+
+
+def scap_calibrate_ex(x_calib, sparsity: float, estimator: int, scope: int, nbins: int, m_out, tau_out, ws, stream=None) -> None:
+    T, K = x_calib.shape
+    p, n = _ws(ws)
+    _check(lib().scap_calibrate_ex(_ptr(x_calib), T, K, dtype_of(x_calib), float(sparsity), int(estimator), int(scope), nbins,
+                                   _ptr(m_out), _ptr(tau_out), p, n, _stream(stream)), "scap_calibrate_ex")
 
 
 def scap_fold_bias_workspace(K: int, N: int) -> int:

@@ -48,7 +48,7 @@ __device__ __forceinline__ int load_rows(const uint16_t *xp, int K, int T, int t
 template <bool BF16>
 __global__ void __launch_bounds__(CAL_THREADS) mode_kernel(const uint16_t *__restrict__ x, int T, int K, int nbins,
                                                            float *__restrict__ m_out, uint32_t *__restrict__ hist_a,
-                                                           int want_hist) {
+                                                           int want_hist, const float *__restrict__ m_given) {
     extern __shared__ __align__(16) uint32_t smem[];
     __shared__ float s_lo[CW], s_hi[CW], s_m[CW];
     const int tid = threadIdx.x, q = tid & 3, rl = tid >> 2;
@@ -63,7 +63,10 @@ __global__ void __launch_bounds__(CAL_THREADS) mode_kernel(const uint16_t *__res
     int nv = 0;
     if (resident && ok) nv = load_rows(xp, K, T, rl, v);
 
-    if (nbins > 0) {
+    if (m_given) {  // the mode was estimated by another kernel: only the radix histogram below is wanted
+        if (tid < CW) s_m[tid] = k0 + tid < K ? __ldcg(m_given + k0 + tid) : 0.0f;
+        __syncthreads();
+    } else if (nbins > 0) {
         // ---- pass 1: per-channel min / max
         float lo[8], hi[8];
 #pragma unroll
@@ -292,27 +295,404 @@ __global__ void select_kernel(const uint32_t *__restrict__ hist, int nb, int wid
 
 __global__ void set_float_kernel(float *p, float v) { *p = v; }
 
-struct CalLayout {
-    size_t hist, state, total;  // hist: 3 passes x 2 x RADIX_BINS counters
+
+// ---------------------------------------------------------------------------------------------------------
+// Other estimators of the mode (Section 3, "Determination of mode value": mean, median) and the paper's scalar
+// eta (one value for the whole FC input instead of one per channel).
+// ---------------------------------------------------------------------------------------------------------
+
+template <bool BF16>
+__device__ __forceinline__ float widen16(uint16_t u) {
+    if constexpr (BF16) return __uint_as_float((uint32_t)u << 16);
+    else return __half2float(__ushort_as_half(u));
+}
+
+// Monotone 16-bit key of a 16-bit float pattern (ascending values <-> ascending keys) and its inverse.
+__device__ __forceinline__ uint32_t key16(uint16_t u) { return (u & 0x8000u) ? (uint32_t)(uint16_t)~u : (uint32_t)(u | 0x8000u); }
+__device__ __forceinline__ uint16_t unkey16(uint32_t k) { return (k & 0x8000u) ? (uint16_t)(k & 0x7fffu) : (uint16_t)~k; }
+
+// Mean: a CTA owns 32 channels.  All threads stage tiles of 64 rows in shared memory (16-byte loads, the next tile
+// in flight while the current one is consumed); thread c < 32 adds column c of each tile in row order in binary64
+// (the definition fixes the order).  Writes the rounded mean and, for the scalar form, the unrounded column sum.
+template <bool BF16>
+__global__ void __launch_bounds__(256) mean_kernel(const uint16_t *__restrict__ x, int T, int K, float *__restrict__ m_out,
+                                                   double *__restrict__ col_sum) {
+    __shared__ __align__(16) uint16_t s_t[2][64][32];
+    const int tid = threadIdx.x, row = tid >> 2, q = tid & 3;
+    const int k0 = blockIdx.x * 32, kc = k0 + q * 8;
+    const bool ok = kc < K;  // K is a multiple of 8
+    const uint16_t *xp = x + kc;
+    const int ntiles = (T + 63) / 64;
+    auto fetch = [&](int i) {
+        const int t = i * 64 + row;
+        return (ok && t < T) ? __ldg(reinterpret_cast<const uint4 *>(xp + (size_t)t * K)) : make_uint4(0, 0, 0, 0);
+    };
+    uint4 r = fetch(0);
+    *reinterpret_cast<uint4 *>(&s_t[0][row][q * 8]) = r;
+    __syncthreads();
+    double acc = 0.0;
+    for (int i = 0; i < ntiles; ++i) {
+        if (i + 1 < ntiles) r = fetch(i + 1);
+        if (tid < 32) {
+            const int n = min(64, T - i * 64);
+#pragma unroll 8
+            for (int j = 0; j < n; ++j) acc = __dadd_rn(acc, (double)widen16<BF16>(s_t[i & 1][j][tid]));
+        }
+        if (i + 1 < ntiles) *reinterpret_cast<uint4 *>(&s_t[(i + 1) & 1][row][q * 8]) = r;
+        __syncthreads();
+    }
+    if (tid < 32 && k0 + tid < K) {
+        if (m_out) m_out[k0 + tid] = __fadd_rn((float)__ddiv_rn(acc, (double)T), 0.0f);
+        if (col_sum) col_sum[k0 + tid] = acc;
+    }
+}
+
+// One CTA: the sums are staged in shared memory 2048 at a time (all threads), thread 0 adds them in order.
+__global__ void __launch_bounds__(256) eta_mean_kernel(const double *__restrict__ col_sum, int T, int K, float *__restrict__ eta) {
+    __shared__ double s_v[2048];
+    double total = 0.0;
+    for (int k0 = 0; k0 < K; k0 += 2048) {
+        const int n = min(2048, K - k0);
+        for (int i = threadIdx.x; i < n; i += blockDim.x) s_v[i] = __ldcg(col_sum + k0 + i);
+        __syncthreads();
+        if (threadIdx.x == 0)
+            for (int i = 0; i < n; ++i) total = __dadd_rn(total, s_v[i]);
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) *eta = __fadd_rn((float)__ddiv_rn(total, __dmul_rn((double)T, (double)K)), 0.0f);
+}
+
+__global__ void broadcast_kernel(float *__restrict__ m_out, int K, const float *__restrict__ eta) {
+    const int k = blockIdx.x * blockDim.x + threadIdx.x;
+    if (k < K) m_out[k] = __ldcg(eta);
+}
+
+// Finds, in a 256-bin histogram h, the bin that holds rank r (0-based) and the rank inside that bin.  One warp.
+__device__ __forceinline__ void find_rank256(const uint32_t *h, uint32_t r, int lane, uint32_t &bin, uint32_t &inner) {
+    uint32_t c[8], tot = 0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) { c[i] = h[lane * 8 + i]; tot += c[i]; }
+    uint32_t incl = tot;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += t;
+    }
+    uint32_t excl = incl - tot;
+    const unsigned hit = __ballot_sync(0xffffffffu, r >= excl && r < incl);
+    const int src = hit ? __ffs(hit) - 1 : 31;
+    uint32_t b = 0, in = 0;
+    if (lane == src) {
+        uint32_t run = excl;
+        b = 7; in = 0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            if (r >= run && r < run + c[i]) { b = (uint32_t)i; in = r - run; }
+            run += c[i];
+        }
+        b += (uint32_t)lane * 8;
+    }
+    bin = __shfl_sync(0xffffffffu, b, src);
+    inner = __shfl_sync(0xffffffffu, in, src);
+}
+
+// Median per channel: two 8-bit radix passes over the 16-bit keys of a strip of CW channels, from registers.
+// Shared memory: hi[CW][256] | lo[2][CW][256] counters | per-channel bucket state.
+template <bool BF16>
+__global__ void __launch_bounds__(CAL_THREADS) median_kernel(const uint16_t *__restrict__ x, int T, int K, float *__restrict__ m_out) {
+    extern __shared__ __align__(16) uint32_t smem[];
+    uint32_t *s_hi = smem, *s_lo = smem + CW * 256;
+    __shared__ uint32_t s_bucket[2][CW], s_inner[2][CW];
+    const int tid = threadIdx.x, q = tid & 3, rl = tid >> 2, lane = tid & 31, warp = tid >> 5;
+    const int k0 = blockIdx.x * CW, kc = k0 + q * 8;
+    const bool ok = kc < K;
+    const uint16_t *xp = x + kc;
+    const bool resident = T <= CAL_ROWS * CAL_U;
+    uint4 v[CAL_U];
+    int nv = 0;
+    if (resident && ok) nv = load_rows(xp, K, T, rl, v);
+    for (int i = tid; i < 3 * CW * 256; i += CAL_THREADS) smem[i] = 0;
+    __syncthreads();
+    // pass A: high byte
+    if (ok)
+        for (int t0 = rl; t0 < T; t0 += CAL_ROWS * CAL_U) {
+            if (!resident) nv = load_rows(xp, K, T, t0, v);
+#pragma unroll
+            for (int u = 0; u < CAL_U; ++u) {
+                if (u < nv) {
+                    const uint32_t w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const uint32_t key = key16((uint16_t)(w[j >> 1] >> ((j & 1) * 16)));
+                        atomicAdd(&s_hi[(q * 8 + j) * 256 + (key >> 8)], 1u);
+                    }
+                }
+            }
+        }
+    __syncthreads();
+    const uint32_t r0 = (uint32_t)(T - 1) / 2, r1 = (uint32_t)T / 2;
+    for (int c = warp * (CW / (CAL_THREADS / 32)); c < (warp + 1) * (CW / (CAL_THREADS / 32)); ++c) {
+        uint32_t b, in;
+        find_rank256(s_hi + c * 256, r0, lane, b, in);
+        if (lane == 0) { s_bucket[0][c] = b; s_inner[0][c] = in; }
+        find_rank256(s_hi + c * 256, r1, lane, b, in);
+        if (lane == 0) { s_bucket[1][c] = b; s_inner[1][c] = in; }
+    }
+    __syncthreads();
+    // pass B: low byte inside the two buckets
+    if (ok)
+        for (int t0 = rl; t0 < T; t0 += CAL_ROWS * CAL_U) {
+            if (!resident) nv = load_rows(xp, K, T, t0, v);
+#pragma unroll
+            for (int u = 0; u < CAL_U; ++u) {
+                if (u < nv) {
+                    const uint32_t w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const int c = q * 8 + j;
+                        const uint32_t key = key16((uint16_t)(w[j >> 1] >> ((j & 1) * 16)));
+                        if ((key >> 8) == s_bucket[0][c]) atomicAdd(&s_lo[c * 256 + (key & 255u)], 1u);
+                        if ((key >> 8) == s_bucket[1][c]) atomicAdd(&s_lo[(CW + c) * 256 + (key & 255u)], 1u);
+                    }
+                }
+            }
+        }
+    __syncthreads();
+    for (int c = warp * (CW / (CAL_THREADS / 32)); c < (warp + 1) * (CW / (CAL_THREADS / 32)); ++c) {
+        uint32_t b0, b1, in;
+        find_rank256(s_lo + c * 256, s_inner[0][c], lane, b0, in);
+        find_rank256(s_lo + (CW + c) * 256, s_inner[1][c], lane, b1, in);
+        if (lane == 0 && k0 + c < K) {
+            const double lo = (double)widen16<BF16>(unkey16((s_bucket[0][c] << 8) | b0));
+            const double hi = (double)widen16<BF16>(unkey16((s_bucket[1][c] << 8) | b1));
+            m_out[k0 + c] = __fadd_rn((float)__ddiv_rn(__dadd_rn(lo, hi), 2.0), 0.0f);
+        }
+    }
+}
+
+// Pooled (whole-tensor) statistics for the scalar eta.
+struct PoolState {
+    uint32_t bucket[2], inner[2];  // median: high-byte bucket and rank inside it, for the two middle ranks
+    int lo_key, hi_key;            // histogram mode: ordered-integer images of the minimum and the maximum
+    float eta;
 };
-static CalLayout cal_layout() {
-    CalLayout L;
-    L.hist = 0;
-    L.state = align_up(sizeof(uint32_t) * 3 * 2 * RADIX_BINS, 256);
-    L.total = L.state + 256;
-    return L;
+
+__device__ __forceinline__ int ordered_int(float f) { const int i = __float_as_int(f); return i >= 0 ? i : i ^ 0x7fffffff; }
+__device__ __forceinline__ float from_ordered_int(int i) { return __int_as_float(i >= 0 ? i : i ^ 0x7fffffff); }
+
+// pass 0: histogram of the high key byte; pass 1: of the low byte inside the two buckets found after pass 0.
+template <bool BF16>
+__global__ void __launch_bounds__(256) pooled_key_hist_kernel(const uint16_t *__restrict__ x, long long M8, int pass,
+                                                              const PoolState *__restrict__ st, uint32_t *__restrict__ hist) {
+    __shared__ uint32_t s_h[2][256];
+    for (int i = threadIdx.x; i < 512; i += blockDim.x) (&s_h[0][0])[i] = 0;
+    const uint32_t bk0 = pass ? st->bucket[0] : 0u, bk1 = pass ? st->bucket[1] : 0u;
+    __syncthreads();
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < M8; i += stride) {
+        const uint4 v = __ldg(reinterpret_cast<const uint4 *>(x) + i);
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const uint32_t key = key16((uint16_t)(w[j >> 1] >> ((j & 1) * 16)));
+            if (pass == 0) {
+                atomicAdd(&s_h[0][key >> 8], 1u);
+            } else {
+                if ((key >> 8) == bk0) atomicAdd(&s_h[0][key & 255u], 1u);
+                if ((key >> 8) == bk1) atomicAdd(&s_h[1][key & 255u], 1u);
+            }
+        }
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < 512; i += blockDim.x) {
+        const uint32_t c = (&s_h[0][0])[i];
+        if (c) atomicAdd(&hist[i], c);
+    }
+}
+
+// One warp.  pass 0: locate the buckets of the two middle ranks; pass 1: locate the low bytes and form eta.
+template <bool BF16>
+__global__ void pooled_median_select_kernel(const uint32_t *__restrict__ hist, int pass, uint32_t r0, uint32_t r1,
+                                            PoolState *__restrict__ st) {
+    const int lane = threadIdx.x & 31;
+    if (threadIdx.x >= 32) return;
+    uint32_t b0, in0, b1, in1;
+    if (pass == 0) {
+        find_rank256(hist, r0, lane, b0, in0);
+        find_rank256(hist, r1, lane, b1, in1);
+        if (lane == 0) { st->bucket[0] = b0; st->inner[0] = in0; st->bucket[1] = b1; st->inner[1] = in1; }
+    } else {
+        find_rank256(hist, st->inner[0], lane, b0, in0);
+        find_rank256(hist + 256, st->inner[1], lane, b1, in1);
+        if (lane == 0) {
+            const double lo = (double)widen16<BF16>(unkey16((st->bucket[0] << 8) | b0));
+            const double hi = (double)widen16<BF16>(unkey16((st->bucket[1] << 8) | b1));
+            st->eta = __fadd_rn((float)__ddiv_rn(__dadd_rn(lo, hi), 2.0), 0.0f);
+        }
+    }
 }
 
 template <bool BF16>
-static scap_status calibrate_t(const uint16_t *x, int T, int K, double sparsity, int nbins, float *m_out, float *tau_out,
-                               unsigned char *ws, cudaStream_t st) {
-    const CalLayout L = cal_layout();
+__global__ void __launch_bounds__(256) pooled_minmax_kernel(const uint16_t *__restrict__ x, long long M8, PoolState *__restrict__ st) {
+    float lo = INFINITY, hi = -INFINITY;
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < M8; i += stride) {
+        float f[8];
+        widen8<BF16>(__ldg(reinterpret_cast<const uint4 *>(x) + i), f);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) { lo = fminf(lo, f[j]); hi = fmaxf(hi, f[j]); }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        lo = fminf(lo, __shfl_xor_sync(0xffffffffu, lo, o));
+        hi = fmaxf(hi, __shfl_xor_sync(0xffffffffu, hi, o));
+    }
+    if ((threadIdx.x & 31) == 0) {
+        atomicMin(&st->lo_key, ordered_int(lo));
+        atomicMax(&st->hi_key, ordered_int(hi));
+    }
+}
+
+// Pooled histogram with the per-channel bin arithmetic (binary32, every operation rounded separately).
+template <bool BF16>
+__global__ void __launch_bounds__(256) pooled_hist_kernel(const uint16_t *__restrict__ x, long long M8, int nbins,
+                                                          const PoolState *__restrict__ st, uint32_t *__restrict__ hist) {
+    __shared__ uint32_t s_h[2048];
+    for (int i = threadIdx.x; i < nbins; i += blockDim.x) s_h[i] = 0;
+    const float lo = from_ordered_int(st->lo_key), hi = from_ordered_int(st->hi_key);
+    const float scale = hi != lo ? __fdiv_rn((float)nbins, __fsub_rn(hi, lo)) : 0.0f;
+    __syncthreads();
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    if (hi != lo)
+        for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < M8; i += stride) {
+            float f[8];
+            widen8<BF16>(__ldg(reinterpret_cast<const uint4 *>(x) + i), f);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                int b = (int)floorf(__fmul_rn(__fsub_rn(f[j], lo), scale));
+                b = min(max(b, 0), nbins - 1);
+                atomicAdd(&s_h[b], 1u);
+            }
+        }
+    __syncthreads();
+    for (int i = threadIdx.x; i < nbins; i += blockDim.x)
+        if (s_h[i]) atomicAdd(&hist[i], s_h[i]);
+}
+
+// One warp: lowest bin with the largest count -> eta = lo + (i + 1/2) * (hi - lo) / nbins.
+__global__ void pooled_argmax_kernel(const uint32_t *__restrict__ hist, int nbins, PoolState *__restrict__ st) {
+    const int lane = threadIdx.x & 31;
+    if (threadIdx.x >= 32) return;
+    uint32_t best_cnt = 0;
+    int best_i = 0;
+    for (int i = lane; i < nbins; i += 32) {
+        const uint32_t c = hist[i];
+        if (c > best_cnt) { best_cnt = c; best_i = i; }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const uint32_t oc = __shfl_xor_sync(0xffffffffu, best_cnt, o);
+        const int oi = __shfl_xor_sync(0xffffffffu, best_i, o);
+        if (oc > best_cnt || (oc == best_cnt && oi < best_i)) { best_cnt = oc; best_i = oi; }
+    }
+    if (lane == 0) {
+        const float lo = from_ordered_int(st->lo_key), hi = from_ordered_int(st->hi_key);
+        float mv = lo;
+        if (hi != lo) {
+            const float w = __fmul_rn(__fsub_rn(hi, lo), __fdiv_rn(1.0f, (float)nbins));
+            mv = __fadd_rn(lo, __fmul_rn(__fadd_rn((float)best_i, 0.5f), w));
+        }
+        st->eta = mv;
+    }
+}
+
+__global__ void init_pool_state_kernel(PoolState *st) {
+    st->lo_key = 0x7fffffff;
+    st->hi_key = (int)0x80000000;
+    st->eta = 0.0f;
+}
+
+struct CalLayout {
+    size_t hist, state, pool, pool_hist, zeroed, col_sum, total;  // hist: 3 passes x 2 x RADIX_BINS counters
+};
+static CalLayout cal_layout(int K) {
+    CalLayout L;
+    L.hist = 0;
+    L.state = align_up(sizeof(uint32_t) * 3 * 2 * RADIX_BINS, 256);
+    L.pool = L.state + 256;                                   // PoolState
+    L.pool_hist = L.pool + 256;                               // 2048 bins, then 256 + 512 key counters
+    L.zeroed = L.pool_hist + sizeof(uint32_t) * (2048 + 768);  // everything before this is cleared per call
+    L.col_sum = align_up(L.zeroed, 256);                      // K column sums (binary64)
+    L.total = L.col_sum + align_up(sizeof(double) * (size_t)K, 256);
+    return L;
+}
+
+// m_out by an estimator other than the per-channel histogram (estimator: 0 histogram, 1 mean, 2 median; scalar: one
+// eta from the pooled tensor, broadcast to the K entries of m_out).
+template <bool BF16>
+static cudaError_t estimate_mode(const uint16_t *x, int T, int K, int estimator, bool scalar, int nbins, float *m_out,
+                                 unsigned char *ws, const CalLayout &L, cudaStream_t st) {
+    PoolState *pool = reinterpret_cast<PoolState *>(ws + L.pool);
+    uint32_t *phist = reinterpret_cast<uint32_t *>(ws + L.pool_hist);
+    double *col_sum = reinterpret_cast<double *>(ws + L.col_sum);
+    const long long M = (long long)T * K, M8 = M / 8;
+    const int grid = sm_count() * 4;
+    cudaError_t e = cudaSuccess;
+    if (!scalar) {
+        if (estimator == 1) return launch(mean_kernel<BF16>, dim3((K + 31) / 32), dim3(256), 0, st, false, x, T, K, m_out, (double *)nullptr);
+        static bool attr_set[2] = {false, false};
+        const size_t smem = (size_t)3 * CW * 256 * 4;
+        if (!attr_set[BF16]) {
+            e = cudaFuncSetAttribute(median_kernel<BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            if (e != cudaSuccess) return e;
+            attr_set[BF16] = true;
+        }
+        return launch(median_kernel<BF16>, dim3((K + CW - 1) / CW), dim3(CAL_THREADS), smem, st, false, x, T, K, m_out);
+    }
+    if (estimator == 1) {
+        e = launch(mean_kernel<BF16>, dim3((K + 31) / 32), dim3(256), 0, st, false, x, T, K, (float *)nullptr, col_sum);
+        if (e != cudaSuccess) return e;
+        e = launch(eta_mean_kernel, dim3(1), dim3(256), 0, st, false, (const double *)col_sum, T, K, &pool->eta);
+    } else if (estimator == 2) {
+        const uint32_t r0 = (uint32_t)((M - 1) / 2), r1 = (uint32_t)(M / 2);
+        e = launch(pooled_key_hist_kernel<BF16>, dim3(grid), dim3(256), 0, st, false, x, M8, 0, (const PoolState *)pool, phist + 2048);
+        if (e != cudaSuccess) return e;
+        e = launch(pooled_median_select_kernel<BF16>, dim3(1), dim3(32), 0, st, false, (const uint32_t *)(phist + 2048), 0, r0, r1, pool);
+        if (e != cudaSuccess) return e;
+        e = launch(pooled_key_hist_kernel<BF16>, dim3(grid), dim3(256), 0, st, false, x, M8, 1, (const PoolState *)pool, phist + 2048 + 256);
+        if (e != cudaSuccess) return e;
+        e = launch(pooled_median_select_kernel<BF16>, dim3(1), dim3(32), 0, st, false, (const uint32_t *)(phist + 2048 + 256), 1, r0, r1, pool);
+    } else {
+        e = launch(init_pool_state_kernel, dim3(1), dim3(1), 0, st, false, pool);
+        if (e != cudaSuccess) return e;
+        if (nbins > 0) {
+            e = launch(pooled_minmax_kernel<BF16>, dim3(grid), dim3(256), 0, st, false, x, M8, pool);
+            if (e != cudaSuccess) return e;
+            e = launch(pooled_hist_kernel<BF16>, dim3(grid), dim3(256), 0, st, false, x, M8, nbins, (const PoolState *)pool, phist);
+            if (e != cudaSuccess) return e;
+            e = launch(pooled_argmax_kernel, dim3(1), dim3(32), 0, st, false, (const uint32_t *)phist, nbins, pool);
+        }
+    }
+    if (e != cudaSuccess) return e;
+    return launch(broadcast_kernel, dim3((K + 255) / 256), dim3(256), 0, st, false, m_out, K, (const float *)&pool->eta);
+}
+
+template <bool BF16>
+static scap_status calibrate_t(const uint16_t *x, int T, int K, double sparsity, int estimator, bool scalar, int nbins,
+                               float *m_out, float *tau_out, unsigned char *ws, cudaStream_t st) {
+    const CalLayout L = cal_layout(K);
     uint32_t *hist = reinterpret_cast<uint32_t *>(ws + L.hist);
     SelState *state = reinterpret_cast<SelState *>(ws + L.state);
     const long long M = (long long)T * K;
     const bool want_tau = sparsity > 0.0;
-    cudaError_t e = cudaMemsetAsync(ws, 0, L.total, st);
+    cudaError_t e = cudaMemsetAsync(ws, 0, L.zeroed, st);
     if (e != cudaSuccess) return cuda_status(e);
+    const bool own_mode = estimator == 0 && !scalar;  // the strip kernel estimates the per-channel histogram mode itself
+    if (!own_mode) {
+        e = estimate_mode<BF16>(x, T, K, estimator, scalar, nbins, m_out, ws, L, st);
+        if (e != cudaSuccess) return cuda_status(e);
+        if (!want_tau) return cuda_status(launch(set_float_kernel, dim3(1), dim3(1), 0, st, false, tau_out, 0.0f));
+    }
     const int HW = (nbins + 1) / 2;
     size_t smem = (size_t)CW * HW * 4;
     if (smem < (size_t)2 * CAL_ROWS * CW * 4) smem = (size_t)2 * CAL_ROWS * CW * 4;
@@ -324,7 +704,7 @@ static scap_status calibrate_t(const uint16_t *x, int T, int K, double sparsity,
         attr_set[BF16] = true;
     }
     e = launch(mode_kernel<BF16>, dim3((K + CW - 1) / CW), dim3(CAL_THREADS), smem, st, false, x, T, K, nbins, m_out, hist,
-               want_tau ? 1 : 0);
+               want_tau ? 1 : 0, own_mode ? (const float *)nullptr : (const float *)m_out);
     if (e != cudaSuccess) return cuda_status(e);
     if (!want_tau) return cuda_status(launch(set_float_kernel, dim3(1), dim3(1), 0, st, false, tau_out, 0.0f));
 
@@ -360,7 +740,27 @@ extern "C" {
 
 size_t scap_calibrate_workspace(int T, int K, int nbins) {
     if (T < 1 || K < 1 || nbins < 0 || nbins > 2048) return 0;
-    return cal_layout().total;
+    return cal_layout(K).total;
+}
+
+scap_status scap_calibrate_ex(const void *x_calib, int T, int K, scap_dtype dt, double sparsity, scap_mode_estimator estimator,
+                              scap_eta_scope scope, int nbins, float *m_out, float *tau_out, void *ws, size_t ws_bytes,
+                              scap_stream_t stream) {
+    if (!x_calib || !m_out || !tau_out || !ws) return SCAP_ERR_INVALID_ARG;
+    if (dt != SCAP_F16 && dt != SCAP_BF16) return SCAP_ERR_DTYPE;
+    if (T < 1 || T > 65535 || K < 1 || (long long)T * K >= (1ll << 31)) return SCAP_ERR_SHAPE;
+    if (nbins < 0 || nbins > 2048 || !(sparsity < 1.0)) return SCAP_ERR_INVALID_ARG;
+    if ((int)estimator < 0 || (int)estimator > 2 || (int)scope < 0 || (int)scope > 1) return SCAP_ERR_INVALID_ARG;
+    if (K % 8 != 0 || !aligned16(x_calib) || !aligned16(m_out) || !aligned16(ws)) return SCAP_ERR_ALIGN;
+    if (ws_bytes < scap_calibrate_workspace(T, K, nbins)) return SCAP_ERR_WORKSPACE;
+    scap_status st = check_device();
+    if (st != SCAP_OK) return st;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    unsigned char *w = static_cast<unsigned char *>(ws);
+    const uint16_t *x = static_cast<const uint16_t *>(x_calib);
+    const bool scalar = scope == SCAP_ETA_SCALAR;
+    return dt == SCAP_BF16 ? calibrate_t<true>(x, T, K, sparsity, (int)estimator, scalar, nbins, m_out, tau_out, w, s)
+                           : calibrate_t<false>(x, T, K, sparsity, (int)estimator, scalar, nbins, m_out, tau_out, w, s);
 }
 
 scap_status scap_calibrate(const void *x_calib, int T, int K, scap_dtype dt, double sparsity, int nbins, float *m_out,
@@ -376,8 +776,8 @@ scap_status scap_calibrate(const void *x_calib, int T, int K, scap_dtype dt, dou
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
     unsigned char *w = static_cast<unsigned char *>(ws);
     const uint16_t *x = static_cast<const uint16_t *>(x_calib);
-    return dt == SCAP_BF16 ? calibrate_t<true>(x, T, K, sparsity, nbins, m_out, tau_out, w, s)
-                           : calibrate_t<false>(x, T, K, sparsity, nbins, m_out, tau_out, w, s);
+    return dt == SCAP_BF16 ? calibrate_t<true>(x, T, K, sparsity, 0, false, nbins, m_out, tau_out, w, s)
+                           : calibrate_t<false>(x, T, K, sparsity, 0, false, nbins, m_out, tau_out, w, s);
 }
 
 }  // extern "C"

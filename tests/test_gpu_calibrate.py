@@ -83,3 +83,59 @@ def test_config4_calibration_size(S):
     assert np.array_equal(m_g, m_o) and tau_g == tau_o
     keep = oracle.mask(xf[:64], m_o, tau_o)[0]
     assert abs((1 - keep.mean()) - 0.6) < 0.01
+
+
+# ---------------------------------------------------------------- mean / median estimators and the scalar eta
+
+def run_calibrate_ex(S, xbits, dt, s, estimator, scope, nbins):
+    x = dev(xbits, dt)
+    T, K = x.shape
+    ws = workspace(S.scap_calibrate_workspace(T, K, nbins))
+    mg = workspace(K * 4)
+    tg = workspace(4)
+    m = mg.view(torch.float32, (K,))
+    tau = tg.view(torch.float32, (1,))
+    S.scap_calibrate_ex(x, s, estimator, scope, nbins, m, tau, ws.payload)
+    torch.cuda.synchronize()
+    assert ws.intact() and mg.intact() and tg.intact()
+    return m.cpu().numpy().copy(), np.float32(tau.item())
+
+
+@pytest.mark.parametrize("scope", [oracle.PER_CHANNEL, oracle.SCALAR])
+@pytest.mark.parametrize("estimator", [oracle.HISTOGRAM, oracle.MEAN, oracle.MEDIAN])
+@pytest.mark.parametrize("T,K,dt,nbins,s", [
+    (256, 1024, si.F16, 2048, 0.5),
+    (64, 40, si.BF16, 16, 0.3),           # one partial strip
+    (101, 264, si.BF16, 333, 0.65),       # odd row count: the median is the middle element
+    (2500, 72, si.F16, 64, 0.8),          # more rows than a strip keeps in registers
+    (1, 8, si.BF16, 4, 0.2),
+])
+def test_estimators_and_scopes_bit_exact(S, estimator, scope, T, K, dt, nbins, s):
+    d = si.laplace_fc(0 if dt == si.F16 else 4, K, 8, dt, T, 1)
+    xf = si.to_f32(d["x_calib"], dt)
+    m_o, tau_o = oracle.calibrate_ex(xf, s, estimator, scope, nbins)
+    m_g, tau_g = run_calibrate_ex(S, d["x_calib"], dt, s, estimator, scope, nbins)
+    assert np.array_equal(m_g.view(np.uint32), m_o.view(np.uint32))
+    assert tau_g.view(np.uint32) == np.float32(tau_o).view(np.uint32)
+
+
+def test_skewed_inputs_median_and_mean_differ_from_the_histogram_mode(S):
+    # GELU-output-like skew: the three estimators disagree, each matches its oracle, and the better mode prunes more
+    rng_bits = si.to_bits(np.abs(si.normal(si.stream_seed(4, 9), 512 * 64).reshape(512, 64)) ** 1.5, si.BF16)
+    xf = si.to_f32(rng_bits, si.BF16)
+    kept = []
+    for est in (oracle.HISTOGRAM, oracle.MEDIAN, oracle.MEAN):
+        m_g, _ = run_calibrate_ex(S, rng_bits, si.BF16, 0.5, est, oracle.PER_CHANNEL, 64)
+        assert np.array_equal(m_g, oracle.mode_estimate(xf, est, oracle.PER_CHANNEL, 64))
+        kept.append(float(np.mean(np.abs(xf - m_g[None, :]) >= np.float32(0.2))))
+    assert kept[0] < kept[1] < kept[2]
+
+
+def test_calibrate_ex_rejects_unknown_estimator_and_scope(S):
+    x = dev(si.laplace_fc(4, 64, 8, si.BF16, 16, 1)["x_calib"], si.BF16)
+    ws = workspace(S.scap_calibrate_workspace(16, 64, 8))
+    m = torch.zeros(64, device="cuda")
+    tau = torch.zeros(1, device="cuda")
+    for est, scope in ((3, 0), (-1, 0), (0, 2)):
+        with pytest.raises(S.ScapError):
+            S.scap_calibrate_ex(x, 0.5, est, scope, 8, m, tau, ws.payload)
