@@ -66,6 +66,8 @@ def lib():
         L.scap_oracle_tau.restype = f
         L.scap_oracle_glu_ffn.argtypes = [vp, vp, vp, i, vp, f, vp, vp, f, vp, i, i, i, vp, vp, vp]
         L.scap_oracle_glu_ffn.restype = None
+        L.scap_oracle_gelu_ffn.argtypes = [vp, vp, vp, i, vp, f, vp, vp, f, vp, i, i, i, vp, vp, vp]
+        L.scap_oracle_gelu_ffn.restype = None
         L.scap_oracle_router.argtypes = [vp, i, i, i, vp, vp]
         L.scap_oracle_router.restype = None
         L.scap_oracle_ffn_sparsity.argtypes = [d, d, d]
@@ -245,6 +247,21 @@ def glu_ffn(hf, Wgu, Wd, dt, m1, tau1, bgu_fused, m2, tau2, bd_fused, z_in=None)
     zin = None if z_in is None else _f32(z_in)
     lib().scap_oracle_glu_ffn(_p(hf), _p(Wgu), _p(Wd), dt, _p(_f32(m1)), float(np.float32(tau1)), _p(_f32(bgu_fused)),
                               _p(_f32(m2)), float(np.float32(tau2)), _p(_f32(bd_fused)), B, D, F, _p(zin), _p(y), _p(z))
+    return y, z
+
+
+def gelu_ffn(hf, Wu, Wd, dt, m1, tau1, bu_fused, m2, tau2, bd_fused, z_in=None):
+    """Non-GLU FFN (up -> exact GELU -> mode-centred sparse down).  Returns (y[B,D] float64, z32[B,F] float32)."""
+    hf = _f32(np.atleast_2d(hf))
+    B, D = hf.shape
+    Wu, Wd = _u16(Wu), _u16(Wd)
+    F = Wd.shape[0]
+    assert Wu.shape == (D, F) and Wd.shape == (F, D)
+    y = np.empty((B, D), np.float64)
+    z = np.empty((B, F), np.float32)
+    zin = None if z_in is None else _f32(z_in)
+    lib().scap_oracle_gelu_ffn(_p(hf), _p(Wu), _p(Wd), dt, _p(_f32(m1)), float(np.float32(tau1)), _p(_f32(bu_fused)),
+                               _p(_f32(m2)), float(np.float32(tau2)), _p(_f32(bd_fused)), B, D, F, _p(zin), _p(y), _p(z))
     return y, z
 
 

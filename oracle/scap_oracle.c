@@ -312,6 +312,29 @@ void scap_oracle_glu_ffn(const float *hf /*[B,D]*/, const uint16_t *Wgu, const u
     free(z32);
 }
 
+/* ---------------------------------------------------------------- non-GLU FFN (Section 4.3, ablation of mode centring)
+ * Falcon / MPT-style block: u = sparse_fc(h; Wu, m1, tau1, bu_fused) [B,F]; z = gelu(u) with the exact
+ * GELU, gelu(v) = v/2 (1 + erf(v / sqrt 2)), in binary64; the down projection reads z stored as binary32
+ * and prunes it with (m2, tau2) - the input whose mode centring the paper's ablation is about.  z_in, if
+ * non-NULL, replaces the computed z (teacher forcing for a stage-wise comparison).                     */
+void scap_oracle_gelu_ffn(const float *hf /*[B,D]*/, const uint16_t *Wu /*[D,F]*/, const uint16_t *Wd /*[F,D]*/, int dt,
+                          const float *m1, float tau1, const float *bu_fused /*[F] nullable*/,
+                          const float *m2, float tau2, const float *bd_fused /*[D] nullable*/,
+                          int B, int D, int F, const float *z_in, double *y, float *z_out) {
+    float *z32 = (float *)malloc(sizeof(float) * (size_t)B * F);
+    if (z_in) {
+        memcpy(z32, z_in, sizeof(float) * (size_t)B * F);
+    } else {
+        double *u = (double *)malloc(sizeof(double) * (size_t)B * F);
+        scap_oracle_sparse_fc(hf, Wu, dt, m1, tau1, bu_fused, B, D, F, u);
+        for (long i = 0; i < (long)B * F; ++i) z32[i] = (float)(0.5 * u[i] * (1.0 + erf(u[i] / sqrt(2.0))));
+        free(u);
+    }
+    if (z_out) memcpy(z_out, z32, sizeof(float) * (size_t)B * F);
+    scap_oracle_sparse_fc(z32, Wd, dt, m2, tau2, bd_fused, B, F, D, y);
+    free(z32);
+}
+
 /* ---------------------------------------------------------------- MoE router (convention: see header)
  * p = softmax(logits[b, 0..E-1]) in binary64; the top_k largest p (ties -> lower index) are
  * selected and their weights renormalised to sum to one.                                     */

@@ -478,3 +478,49 @@ def test_estimators_rank_as_expected_on_a_skewed_distribution():
     tau = np.float32(0.25)
     frac = [float(np.mean(np.abs(x - m[None, :]) < tau)) for m in (hist, med, mean)]
     assert frac[0] > frac[1] > frac[2]
+
+
+# ---------------------------------------------------------------- non-GLU FFN (up -> GELU -> sparse down)
+
+def _gelu64(v):
+    return np.array([0.5 * t * (1.0 + math.erf(t / math.sqrt(2.0))) for t in np.ravel(v)]).reshape(np.shape(v))
+
+
+def test_gelu_ffn_tau_zero_is_the_dense_mlp_and_gelu_has_its_textbook_values():
+    g = si.glu_block(2, 48, 40, si.BF16, 8, 3)
+    Wu = g["Wgu"][:, :40].copy()                                   # any [D, F] weight will do
+    h = si.to_f32(g["h"], si.BF16)
+    bu = np.linspace(-0.5, 0.5, 40).astype(np.float32)
+    y, z = oracle.gelu_ffn(h, Wu, g["Wd"], si.BF16, None, 0.0, bu, None, 0.0, None)
+    Wuf, Wdf = si.to_f32(Wu, si.BF16).astype(np.float64), si.to_f32(g["Wd"], si.BF16).astype(np.float64)
+    u = h.astype(np.float64) @ Wuf + bu
+    z_ref = _gelu64(u)
+    assert np.allclose(z, z_ref, rtol=1e-6, atol=1e-9)
+    assert np.allclose(y, z.astype(np.float64) @ Wdf, rtol=1e-12, atol=1e-12)
+    # textbook values of the exact GELU through the same code path: one-channel "network" with unit weights
+    one = si.to_bits(np.ones((1, 1)), si.BF16)
+    for v, want in ((0.0, 0.0), (1.0, 0.8413447460685429), (-1.0, -0.15865525393145707), (6.0, 5.999999994080277), (-6.0, -5.919723e-09)):
+        _, zz = oracle.gelu_ffn(np.float32([[v]]), one, one, si.BF16, None, 0.0, None, None, 0.0, None)
+        assert abs(float(zz[0, 0]) - want) <= 1e-6 * max(1.0, abs(want)) + 1e-12
+
+
+def test_gelu_ffn_is_the_composition_of_its_stages_and_honours_teacher_forcing():
+    g = si.glu_block(2, 64, 56, si.BF16, 32, 2)
+    Wu = g["Wgu"][:, 56:].copy()
+    h = si.to_f32(g["h"], si.BF16)
+    hc = si.to_f32(g["h_calib"], si.BF16)
+    m1, tau1 = oracle.calibrate(hc, 0.3, 64)
+    b1 = oracle.fold_bias(Wu, si.BF16, m1, None)
+    _, zc = oracle.gelu_ffn(hc, Wu, g["Wd"], si.BF16, m1, tau1, b1, None, 0.0, None)
+    m2, tau2 = oracle.calibrate(zc, 0.6, 64)
+    b2 = oracle.fold_bias(g["Wd"], si.BF16, m2, None)
+    y, z = oracle.gelu_ffn(h, Wu, g["Wd"], si.BF16, m1, tau1, b1, m2, tau2, b2)
+    u = oracle.sparse_fc(h, Wu, si.BF16, m1, tau1, b1)
+    assert np.array_equal(z, _gelu64(u).astype(np.float32))
+    assert np.array_equal(y, oracle.sparse_fc(z, g["Wd"], si.BF16, m2, tau2, b2))
+    z2 = z + np.float32(0.25)
+    y2, z2o = oracle.gelu_ffn(h, Wu, g["Wd"], si.BF16, m1, tau1, b1, m2, tau2, b2, z_in=z2)
+    assert np.array_equal(z2o, z2) and np.array_equal(y2, oracle.sparse_fc(z2, g["Wd"], si.BF16, m2, tau2, b2))
+    # GELU output is skewed (bounded below near -0.17): the centred threshold prunes the target, the uncentred one less
+    kept_c = float(np.mean(np.abs(zc - m2[None, :]) >= tau2))
+    assert abs(kept_c - 0.4) < 0.02
