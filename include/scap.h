@@ -189,6 +189,19 @@ scap_status scap_glu_ffn(const void *h, const void *Wgu, const void *Wd, const f
                          int *nnz1_out, uint32_t *idx2_out, int *nnz2_out, void *ws, size_t ws_bytes,
                          scap_stream_t stream);
 
+/* Non-GLU FFN block (Section 4.3, the Falcon / MPT ablation of mode centring): up projection, exact GELU,
+ * mode-centred sparse down projection.
+ *   u = scap_sparse_fc(h; Wu[D,F], m1, tau1, bu_fused)      (tau1 = 0 runs the up projection on every channel)
+ *   z = gelu(u) = u/2 (1 + erf(u / sqrt 2))                 fp32, formed in the epilogue of the first kernel
+ *   y = scap_sparse_fc(z; Wd[F,D], m2, tau2, bd_fused)      z in fp32, never leaves L2
+ * Arguments, optional outputs (z_out[B,F], idx1_out .. nnz2_out), workspace rules and errors as scap_glu_ffn; the workspace
+ * query returns the same size as scap_glu_workspace.                                                           */
+size_t scap_gelu_ffn_workspace(int B, int D, int F);
+scap_status scap_gelu_ffn(const void *h, const void *Wu, const void *Wd, const float *m1, const float *tau1,
+                          const float *bu_fused, const float *m2, const float *tau2, const float *bd_fused, float *y,
+                          int B, int D, int F, scap_dtype dt, float *z_out, uint32_t *idx1_out, int *nnz1_out,
+                          uint32_t *idx2_out, int *nnz2_out, void *ws, size_t ws_bytes, scap_stream_t stream);
+
 /* scap_glu_ffn without a workspace argument (the paper has no counterpart; this is a deployment aid).
  *
  * Some callers must not allocate device memory on the decode path: a serving process that handed all

@@ -11,7 +11,7 @@ __all__ = [
     "scap_calibrate_workspace", "scap_calibrate", "scap_calibrate_ex", "SCAP_MODE_HISTOGRAM", "SCAP_MODE_MEAN", "SCAP_MODE_MEDIAN",
     "SCAP_ETA_PER_CHANNEL", "SCAP_ETA_SCALAR", "scap_fold_bias_workspace", "scap_fold_bias",
     "scap_fc_workspace", "scap_sparse_fc", "scap_dense_fc", "scap_fc_host_workspace", "scap_sparse_fc_host",
-    "scap_glu_workspace", "scap_glu_ffn", "scap_glu_static_capacity", "scap_glu_ffn_static", "scap_moe_workspace",
+    "scap_glu_workspace", "scap_glu_ffn", "scap_gelu_ffn_workspace", "scap_gelu_ffn", "scap_glu_static_capacity", "scap_glu_ffn_static", "scap_moe_workspace",
     "scap_moe_ffn", "ScapExpert", "dtype_of", "EXPORTS",
 ]
 
@@ -22,8 +22,8 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 EXPORTS = [
     "scap_status_string", "scap_version", "scap_tune", "scap_device_status", "scap_calibrate_workspace", "scap_calibrate",
     "scap_calibrate_ex", "scap_fold_bias_workspace", "scap_fold_bias", "scap_fc_workspace", "scap_sparse_fc", "scap_dense_fc",
-    "scap_fc_host_workspace", "scap_sparse_fc_host", "scap_glu_workspace", "scap_glu_ffn",
-    "scap_glu_static_capacity", "scap_glu_ffn_static", "scap_moe_workspace", "scap_moe_ffn",
+    "scap_fc_host_workspace", "scap_sparse_fc_host", "scap_glu_workspace", "scap_glu_ffn", "scap_gelu_ffn_workspace",
+    "scap_gelu_ffn", "scap_glu_static_capacity", "scap_glu_ffn_static", "scap_moe_workspace", "scap_moe_ffn",
 ]
 
 
@@ -87,6 +87,10 @@ def lib():
     L.scap_glu_workspace.restype = sz
     L.scap_glu_ffn.argtypes = [vp] * 10 + [i, i, i, i] + [vp] * 5 + [vp, sz, vp]
     L.scap_glu_ffn.restype = i
+    L.scap_gelu_ffn_workspace.argtypes = [i, i, i]
+    L.scap_gelu_ffn_workspace.restype = sz
+    L.scap_gelu_ffn.argtypes = [vp] * 10 + [i, i, i, i] + [vp] * 5 + [vp, sz, vp]
+    L.scap_gelu_ffn.restype = i
     L.scap_glu_static_capacity.argtypes = []
     L.scap_glu_static_capacity.restype = sz
     L.scap_glu_ffn_static.argtypes = [vp] * 10 + [i, i, i, i] + [vp, vp]
@@ -228,6 +232,20 @@ def scap_glu_ffn(h, Wgu, Wd, m1, tau1, bgu_fused, m2, tau2, bd_fused, y, ws, z_o
     _check(lib().scap_glu_ffn(_ptr(h), _ptr(Wgu), _ptr(Wd), _ptr(m1), _ptr(tau1), _ptr(bgu_fused), _ptr(m2), _ptr(tau2),
                               _ptr(bd_fused), _ptr(y), B, D, F, dtype_of(Wgu), _ptr(z_out), _ptr(idx1_out), _ptr(nnz1_out),
                               _ptr(idx2_out), _ptr(nnz2_out), p, n, _stream(stream)), "scap_glu_ffn")
+
+
+def scap_gelu_ffn_workspace(B: int, D: int, F: int) -> int:
+    return lib().scap_gelu_ffn_workspace(B, D, F)
+
+
+def scap_gelu_ffn(h, Wu, Wd, m1, tau1, bu_fused, m2, tau2, bd_fused, y, ws, z_out=None, idx1_out=None, nnz1_out=None,
+                  idx2_out=None, nnz2_out=None, stream=None) -> None:
+    B, D = h.shape
+    F = Wd.shape[0]
+    p, n = _ws(ws)
+    _check(lib().scap_gelu_ffn(_ptr(h), _ptr(Wu), _ptr(Wd), _ptr(m1), _ptr(tau1), _ptr(bu_fused), _ptr(m2), _ptr(tau2),
+                               _ptr(bd_fused), _ptr(y), B, D, F, dtype_of(Wu), _ptr(z_out), _ptr(idx1_out), _ptr(nnz1_out),
+                               _ptr(idx2_out), _ptr(nnz2_out), p, n, _stream(stream)), "scap_gelu_ffn")
 
 
 def scap_glu_static_capacity() -> int:

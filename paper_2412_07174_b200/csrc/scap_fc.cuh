@@ -65,6 +65,7 @@ struct FcArgs {
     uint32_t *bits;       // optional [ceil(K/32)]: union keep mask, one word per 32-channel chunk
     int hold_dependents;  // 1: do not let the next kernel start before this grid completes (it writes parameters)
     int no_tc;            // 1: keep this call off the tcgen05 kernel
+    int act;              // EPI_BIAS: 1 = the exact GELU is applied to the biased result (z_copy then gets a copy)
 };
 
 template <bool BF16, int BT, int CAP>
@@ -80,6 +81,16 @@ __device__ __forceinline__ void fma_row(float (&acc)[BT][8], const uint4 &v, con
 #pragma unroll
         for (int j = 0; j < 8; ++j) acc[b][j] = fmaf(xv, w[j], acc[b][j]);
     }
+}
+
+// Exact GELU, gelu(v) = v/2 (1 + erf(v / sqrt 2)), binary32.
+__device__ __forceinline__ float gelu_exact(float v) { return 0.5f * v * (1.0f + erff(v * 0.70710678118654752f)); }
+
+// Stores one finished EPI_BIAS result (activation applied first, if any).
+__device__ __forceinline__ void store_result(const FcArgs &a, int row, int b, int n, float v) {
+    if (a.act == 1) v = gelu_exact(v);
+    a.y[(size_t)row * a.y_ld + n] = v;
+    if (a.z_copy) a.z_copy[(size_t)b * a.Nh + n] = v;
 }
 
 template <bool BF16>
@@ -137,7 +148,7 @@ __device__ __forceinline__ void finish_columns(const FcArgs &a, int tile, int s,
 #pragma unroll
                 for (int q = 0; q < MAX_CLUSTER; ++q)
                     if (q < S) v += s_gather[(q * BT + b) * per + c];
-                a.y[(size_t)row * a.y_ld + n] = v;
+                store_result(a, row, b, n, v);
             }
         } else {
             const int F = a.Nh, f = tile * HALF + s * per + c;
@@ -748,7 +759,7 @@ __device__ __forceinline__ void fc_body_mma(const FcArgs &a, const int tile, con
 #pragma unroll
                 for (int q = 0; q < MAX_CLUSTER; ++q)
                     if (q < S) v += part[q];
-                a.y[(size_t)row * a.y_ld + n] = v;
+                store_result(a, row, b, n, v);
             }
         } else {
             const int F = a.Nh, f = tile * HALF + s * per + c;

@@ -407,7 +407,7 @@ __global__ void __launch_bounds__(FC_THREADS, 2) fc_tc_kernel(const FcArgs a) {
 #pragma unroll
                 for (int q = 0; q < MAX_CLUSTER; ++q)
                     if (q < S) v += peer[q][b * TNT + s * per + c];
-                a.y[(size_t)row * a.y_ld + n] = v;
+                store_result(a, row, b, n, v);
             }
         } else {
             const int F = a.Nh, f = tile * HALF + s * per + c;

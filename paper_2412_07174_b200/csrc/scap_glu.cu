@@ -31,10 +31,12 @@ size_t scap_glu_workspace(int B, int D, int F) {
     return glu_layout(B, D, F).total;
 }
 
-scap_status scap_glu_ffn(const void *h, const void *Wgu, const void *Wd, const float *m1, const float *tau1,
-                         const float *bgu_fused, const float *m2, const float *tau2, const float *bd_fused, float *y, int B,
-                         int D, int F, scap_dtype dt, float *z_out, uint32_t *idx1_out, int *nnz1_out, uint32_t *idx2_out,
-                         int *nnz2_out, void *ws, size_t ws_bytes, scap_stream_t stream) {
+// Both two-stage FFN blocks: gated (packed gate|up weight [D, 2F], z = up * silu(gate)) or plain (up weight [D, F],
+// z = gelu(up)); the second stage is the sparse down projection on z in either case.
+static scap_status ffn_impl(bool gated, const void *h, const void *Wgu, const void *Wd, const float *m1, const float *tau1,
+                            const float *bgu_fused, const float *m2, const float *tau2, const float *bd_fused, float *y, int B,
+                            int D, int F, scap_dtype dt, float *z_out, uint32_t *idx1_out, int *nnz1_out, uint32_t *idx2_out,
+                            int *nnz2_out, void *ws, size_t ws_bytes, scap_stream_t stream) {
     if (!h || !Wgu || !Wd || !tau1 || !tau2 || !y || !ws) return SCAP_ERR_INVALID_ARG;
     if (dt != SCAP_F16 && dt != SCAP_BF16) return SCAP_ERR_DTYPE;
     if (B < 1 || B > SCAP_MAX_BATCH || D < 1 || F < 1 || D > SCAP_MAX_K || F > SCAP_MAX_K) return SCAP_ERR_SHAPE;
@@ -54,8 +56,10 @@ scap_status scap_glu_ffn(const void *h, const void *Wgu, const void *Wd, const f
 
     FcArgs a;
     memset(&a, 0, sizeof(a));
-    a.W = Wgu; a.K = D; a.ldw = 2 * F; a.Nh = F; a.B = B;
-    choose_config(D, F, EPI_GLU, 1, B, &a.tn, &a.S);
+    const int epi1 = gated ? EPI_GLU : EPI_BIAS;
+    a.W = Wgu; a.K = D; a.ldw = gated ? 2 * F : F; a.Nh = F; a.B = B;
+    a.act = gated ? 0 : 1;
+    choose_config(D, F, epi1, 1, B, &a.tn, &a.S);
     a.x = h; a.x_ld = D; a.m = m1; a.tau = tau1; a.bias = bgu_fused;
     a.y = z; a.y_ld = F; a.z_copy = z_out;
     if (idx1_out || nnz1_out) a.bits = reinterpret_cast<uint32_t *>(w + G.bits1);
@@ -67,9 +71,9 @@ scap_status scap_glu_ffn(const void *h, const void *Wgu, const void *Wd, const f
     if (idx2_out || nnz2_out) d.bits = reinterpret_cast<uint32_t *>(w + G.bits2);
     // The two stages run back to back: either both take the tcgen05 kernel or neither does (measured: a stage on
     // it between two mma.sync stages loses more at the kernel boundaries than it gains).
-    if (!(tc_applicable(a, EPI_GLU, bf16) && tc_applicable(d, EPI_BIAS, bf16))) a.no_tc = d.no_tc = 1;
+    if (!(tc_applicable(a, epi1, bf16) && tc_applicable(d, EPI_BIAS, bf16))) a.no_tc = d.no_tc = 1;
 
-    cudaError_t e = launch_fc(bf16, MODE_GATHER, bf16 ? 1 : 0, EPI_GLU, a, st);
+    cudaError_t e = launch_fc(bf16, MODE_GATHER, bf16 ? 1 : 0, epi1, a, st);
     if (e != cudaSuccess) return cuda_status(e);
     e = launch_fc(bf16, MODE_GATHER, 2, EPI_BIAS, d, st);
     if (e != cudaSuccess) return cuda_status(e);
@@ -83,6 +87,24 @@ scap_status scap_glu_ffn(const void *h, const void *Wgu, const void *Wd, const f
         if (e != cudaSuccess) return cuda_status(e);
     }
     return SCAP_OK;
+}
+
+scap_status scap_glu_ffn(const void *h, const void *Wgu, const void *Wd, const float *m1, const float *tau1,
+                         const float *bgu_fused, const float *m2, const float *tau2, const float *bd_fused, float *y, int B,
+                         int D, int F, scap_dtype dt, float *z_out, uint32_t *idx1_out, int *nnz1_out, uint32_t *idx2_out,
+                         int *nnz2_out, void *ws, size_t ws_bytes, scap_stream_t stream) {
+    return ffn_impl(true, h, Wgu, Wd, m1, tau1, bgu_fused, m2, tau2, bd_fused, y, B, D, F, dt, z_out, idx1_out, nnz1_out, idx2_out,
+                    nnz2_out, ws, ws_bytes, stream);
+}
+
+size_t scap_gelu_ffn_workspace(int B, int D, int F) { return scap_glu_workspace(B, D, F); }
+
+scap_status scap_gelu_ffn(const void *h, const void *Wu, const void *Wd, const float *m1, const float *tau1,
+                          const float *bu_fused, const float *m2, const float *tau2, const float *bd_fused, float *y, int B,
+                          int D, int F, scap_dtype dt, float *z_out, uint32_t *idx1_out, int *nnz1_out, uint32_t *idx2_out,
+                          int *nnz2_out, void *ws, size_t ws_bytes, scap_stream_t stream) {
+    return ffn_impl(false, h, Wu, Wd, m1, tau1, bu_fused, m2, tau2, bd_fused, y, B, D, F, dt, z_out, idx1_out, nnz1_out, idx2_out,
+                    nnz2_out, ws, ws_bytes, stream);
 }
 
 }  // extern "C"

@@ -179,3 +179,78 @@ def test_moe_small(S, D, F, E, B, top_k):
     assert np.array_equal(ex, ex_o)
     assert np.allclose(w, w_o, rtol=1e-6, atol=0)
     assert rel_l2_rows(y, y64) <= REL_L2_TOL
+
+
+# ---------------------------------------------------------------- non-GLU FFN (up -> exact GELU -> centred sparse down)
+
+def gelu_block(D, F, B, dt=si.BF16, T=64):
+    """A [D, F] up weight (the up half of the packed recipe), the down weight and inputs of the SwiGLU recipe."""
+    g = si.glu_block(2, D, F, dt, T, B)
+    g["Wu"] = np.ascontiguousarray(g["Wgu"][:, F:])
+    return g
+
+
+def calibrate_gelu(g, s1, s2, nbins=64):
+    dt = g["dt"]
+    hc = si.to_f32(g["h_calib"], dt)
+    m1, tau1 = oracle.calibrate(hc, s1, nbins)
+    b1 = oracle.fold_bias(g["Wu"], dt, m1, None).astype(np.float32)
+    _, zc = oracle.gelu_ffn(hc, g["Wu"], g["Wd"], dt, m1, tau1, b1, None, 0.0, None)
+    m2, tau2 = oracle.calibrate(zc, s2, nbins)
+    b2 = oracle.fold_bias(g["Wd"], dt, m2, None).astype(np.float32)
+    return dict(m1=m1, tau1=tau1, b1=b1, m2=m2, tau2=tau2, b2=b2)
+
+
+def check_gelu(S, g, c):
+    dt = g["dt"]
+    hf = si.to_f32(g["h"], dt)
+    h, Wu, Wd = dev(g["h"], dt), dev(g["Wu"], dt), dev(g["Wd"], dt)
+    B, D = h.shape
+    F = g["F"]
+    ws = workspace(S.scap_gelu_ffn_workspace(B, D, F))
+    yg, zg = workspace(B * D * 4), workspace(B * F * 4)
+    y, z = yg.view(torch.float32, (B, D)), zg.view(torch.float32, (B, F))
+    idx1 = torch.full((D,), -1, dtype=torch.int32, device="cuda")
+    idx2 = torch.full((F,), -1, dtype=torch.int32, device="cuda")
+    n1 = torch.zeros(1, dtype=torch.int32, device="cuda")
+    n2 = torch.zeros(1, dtype=torch.int32, device="cuda")
+    S.scap_gelu_ffn(h, Wu, Wd, f32(c["m1"]), f32([c["tau1"]]), f32(c["b1"]), f32(c["m2"]), f32([c["tau2"]]), f32(c["b2"]),
+                    y, ws.payload, z_out=z, idx1_out=idx1, nnz1_out=n1, idx2_out=idx2, nnz2_out=n2)
+    torch.cuda.synchronize()
+    assert ws.intact() and yg.intact() and zg.intact()
+    y, z = y.cpu().numpy().copy(), z.cpu().numpy().copy()
+    idx1, idx2 = idx1[: int(n1)].cpu().numpy().astype(np.uint32), idx2[: int(n2)].cpu().numpy().astype(np.uint32)
+    assert np.array_equal(idx1, oracle.mask(hf, c["m1"], c["tau1"])[2])                      # stage-1 mask: bit-exact
+    y64, z_o = oracle.gelu_ffn(hf, g["Wu"], g["Wd"], dt, c["m1"], c["tau1"], c["b1"], c["m2"], c["tau2"], c["b2"])
+    assert np.max(np.abs(z - z_o)) <= 2e-6 * max(1.0, float(np.max(np.abs(z_o))))          # erff vs erf, fp32 accumulation
+    keep2, _, idx2_o = oracle.mask(z, c["m2"], c["tau2"])                                    # stage-2 mask from the GPU's z
+    assert np.array_equal(idx2, idx2_o)
+    y_tf, _ = oracle.gelu_ffn(hf, g["Wu"], g["Wd"], dt, c["m1"], c["tau1"], c["b1"], c["m2"], c["tau2"], c["b2"], z_in=z)
+    assert rel_l2_rows(y, y_tf) <= REL_L2_TOL
+    assert rel_l2_rows(y, y64) <= REL_L2_TOL
+    keep2_o = oracle.mask(z_o, c["m2"], c["tau2"])[0]
+    flips = keep2 != keep2_o
+    if flips.any():
+        dz = np.abs(z_o - c["m2"][None, :])
+        assert np.all(np.abs(dz[flips] - c["tau2"]) <= 1e-5 * np.maximum(c["tau2"], dz[flips]))
+    return keep2.mean()
+
+
+@pytest.mark.parametrize("tc_mode", [1, 2])
+@pytest.mark.parametrize("D,F,B", [(256, 512, 1), (200, 264, 3), (512, 1000, 8), (64, 8, 2), (1024, 776, 16)])
+def test_gelu_ffn_small_shapes(S, D, F, B, tc_mode):
+    g = gelu_block(D, F, B)
+    c = calibrate_gelu(g, 0.3, 0.5)
+    try:
+        S.scap_tune("tcgen05", tc_mode)
+        kept2 = check_gelu(S, g, c)
+    finally:
+        S.scap_tune("tcgen05", 1)
+    assert kept2 < 0.95
+
+
+def test_gelu_ffn_dense_up_projection_and_fp16(S):
+    g = gelu_block(264, 520, 4, dt=si.F16)
+    c = calibrate_gelu(g, 0.3, 0.5)
+    c["tau1"] = np.float32(0.0)                                   # every input channel of the up projection kept
+    check_gelu(S, g, c)
