@@ -345,6 +345,74 @@ def suite_glu(torch, scap, peak, out):
              "ffn_sparsity_paper_accounting": round(1 - (2 * np.mean(k1) / D + np.mean(k2) / F) / 3, 4), "weight_copies": R, "kernels_per_call": 2})
 
 
+def suite_gelu(torch, scap, peak, out):
+    """Non-GLU FFN (MPT-7B shape: D = 4096, F = 16384, bf16): dense up projection, exact GELU, down projection pruned at 50 %
+    on the mode-centred GELU output; the same block with the centring switched off (m2 = 0) needs a smaller tau for the same
+    sparsity.  Plus the fused QKV projection with its shared-input mask (one sparse FC with N = 3 D)."""
+    D, F = 4096, 16384
+    dt = si.BF16
+    stream = torch.cuda.Stream()
+    l2 = torch.cuda.get_device_properties(0).L2_cache_size
+    g = si.glu_block(5, D, F // 2, dt, 512, 64)          # reuse the recipe's generators: h, h_calib, a [D, F] and a [F/2, D] weight
+    Wu0 = si.as_torch(g["Wgu"], dt).cuda()               # [D, 2 * F/2] = [D, F]
+    Wd0 = (torch.randn(F, D, device="cuda", generator=torch.Generator(device="cuda").manual_seed(2412)) * 0.02).to(torch.bfloat16)
+    hc, hs = si.as_torch(g["h_calib"], dt).cuda(), si.as_torch(g["h"], dt).cuda()
+    ws = torch.empty(max(scap.scap_gelu_ffn_workspace(16, D, F), scap.scap_calibrate_workspace(512, F, NBINS)), dtype=torch.uint8, device="cuda")
+    tau1 = torch.zeros(1, dtype=torch.float32, device="cuda")   # dense up projection
+    m2 = torch.empty(F, dtype=torch.float32, device="cuda")
+    tau2 = torch.zeros(1, dtype=torch.float32, device="cuda")
+    b2 = torch.empty(D, dtype=torch.float32, device="cuda")
+    zc = torch.empty((512, F), dtype=torch.float32, device="cuda")
+    ytmp = torch.empty((16, D), dtype=torch.float32, device="cuda")
+    for i in range(0, 512, 16):
+        scap.scap_gelu_ffn(hc[i:i + 16], Wu0, Wd0, None, tau1, None, None, tau2, None, ytmp, ws, z_out=zc[i:i + 16])
+    zc16 = zc.to(torch.bfloat16)
+    R = max(2, int(np.ceil(4 * l2 / (D * F * 2 + 0.5 * F * D * 2))))
+    Wus = [Wu0] + [Wu0.clone() for _ in range(R - 1)]
+    Wds = [Wd0] + [Wd0.clone() for _ in range(R - 1)]
+    n2 = torch.zeros(1, dtype=torch.int32, device="cuda")
+    for centred in (True, False):
+        scap.scap_calibrate(zc16, 0.5, NBINS if centred else 0, m2, tau2, ws)
+        scap.scap_fold_bias(Wd0, m2, None, b2, ws)
+        for B in (1, 4):
+            y = torch.empty((B, D), dtype=torch.float32, device="cuda")
+            hb = [hs[i * 8:i * 8 + B] for i in range(8)]
+            k2 = []
+            for i in range(8):
+                scap.scap_gelu_ffn(hb[i], Wu0, Wd0, None, tau1, None, m2, tau2, b2, y, ws, nnz2_out=n2)
+                k2.append(int(n2.item()))
+            t = _time_graph(torch, stream, lambda: [scap.scap_gelu_ffn(hb[r % 8], Wus[r], Wds[r], None, tau1, None, m2, tau2, b2, y, ws) for r in range(R)]) / R
+            nb = D * F * 2 + np.mean(k2) * D * 2 + B * D * 2 + 4 * F + 4 * D + 4 * B * D + 8
+            out({"suite": "gelu_ffn", "D": D, "F": F, "B": B, "down_target": 0.5, "mode_centred": centred, "tau2": round(float(tau2.item()), 5),
+                 "kept_fraction_down": round(float(np.mean(k2)) / F, 4), "us_per_call": round(t, 2), "gbs": round(nb / t / 1e3, 1),
+                 "frac_of_measured_peak": round(nb / t / 1e3 / peak, 3), "weight_copies": R, "kernels_per_call": 2})
+    # fused QKV: one mask for the three projections because they share their input
+    N3 = 3 * D
+    Wq0 = (torch.randn(D, N3, device="cuda", generator=torch.Generator(device="cuda").manual_seed(2413)) * 0.02).to(torch.bfloat16)
+    R = max(2, int(np.ceil(4 * l2 / (0.5 * D * N3 * 2))))
+    Wqs = [Wq0] + [Wq0.clone() for _ in range(R - 1)]
+    m1 = torch.empty(D, dtype=torch.float32, device="cuda")
+    bq = torch.empty(N3, dtype=torch.float32, device="cuda")
+    scap.scap_calibrate(hc, 0.5, NBINS, m1, tau1, ws)
+    scap.scap_fold_bias(Wq0, m1, None, bq, ws)
+    fws = torch.empty(scap.scap_fc_workspace(16, D, N3), dtype=torch.uint8, device="cuda")
+    nn = torch.zeros(1, dtype=torch.int32, device="cuda")
+    idx = torch.empty(D, dtype=torch.int32, device="cuda")
+    for B in (1, 4):
+        y = torch.empty((B, N3), dtype=torch.float32, device="cuda")
+        hb = [hs[i * 8:i * 8 + B] for i in range(8)]
+        ks = []
+        for i in range(8):
+            scap.scap_sparse_fc(hb[i], Wq0, m1, tau1, bq, y, fws, idx_out=idx, nnz_out=nn)
+            ks.append(int(nn.item()))
+        t = _time_graph(torch, stream, lambda: [scap.scap_sparse_fc(hb[r % 8], Wqs[r], m1, tau1, bq, y, fws) for r in range(R)]) / R
+        td = _time_graph(torch, stream, lambda: [scap.scap_dense_fc(hb[r % 8], Wqs[r], None, y, fws) for r in range(R)]) / R
+        nb = np.mean(ks) * N3 * 2 + B * D * 2 + 4 * D + 4 * N3 + 4 * B * N3 + 4
+        out({"suite": "fused_qkv", "K": D, "N": N3, "B": B, "target": 0.5, "kept_fraction": round(float(np.mean(ks)) / D, 4),
+             "us_per_call": round(t, 2), "dense_us": round(td, 2), "speedup_vs_dense": round(td / t, 3), "gbs": round(nb / t / 1e3, 1),
+             "frac_of_measured_peak": round(nb / t / 1e3 / peak, 3), "weight_copies": R})
+
+
 def suite_moe(torch, scap, peak, out):
     """Config 3: Mixtral-8x7B-shaped MoE layer, 8 experts, top-2, batch 1..4, 40 % / 60 % targets."""
     D, F, E = 4096, 14336, 8
@@ -397,6 +465,8 @@ def run_suite(args):
         suite_calibrate(torch, scap, out)
     if which in ("glu", "all"):
         suite_glu(torch, scap, peak, out)
+    if which in ("gelu", "all"):
+        suite_gelu(torch, scap, peak, out)
     if which in ("sweep", "all", "sweep-small"):
         shapes = [(4096, 4096), (4096, 11008), (11008, 4096), (14336, 4096)]
         if which == "sweep-small":
@@ -422,7 +492,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--detail", action="store_true", help="also print a per-sparsity table to stderr")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--suite", default="", choices=["", "calibrate", "glu", "moe", "sweep", "sweep-small", "all"],
+    ap.add_argument("--suite", default="", choices=["", "calibrate", "glu", "gelu", "moe", "sweep", "sweep-small", "all"],
                     help="run the other workload descriptions instead of the headline line (one JSON object per line)")
     ap.add_argument("--copies", type=int, default=0,
                     help="number of weight copies to rotate (default: enough for the cold-HBM rule); a small value keeps "
