@@ -68,6 +68,10 @@ def lib():
         L.scap_oracle_glu_ffn.restype = None
         L.scap_oracle_gelu_ffn.argtypes = [vp, vp, vp, i, vp, f, vp, vp, f, vp, i, i, i, vp, vp, vp]
         L.scap_oracle_gelu_ffn.restype = None
+        L.scap_oracle_sparse_fc_q8.argtypes = [vp, vp, vp, vp, f, vp, i, i, i, vp]
+        L.scap_oracle_sparse_fc_q8.restype = None
+        L.scap_oracle_fold_bias_q8.argtypes = [vp, vp, vp, vp, i, i, vp]
+        L.scap_oracle_fold_bias_q8.restype = None
         L.scap_oracle_router.argtypes = [vp, i, i, i, vp, vp]
         L.scap_oracle_router.restype = None
         L.scap_oracle_ffn_sparsity.argtypes = [d, d, d]
@@ -233,6 +237,25 @@ def calibrate(xf_calib, s: float, nbins: int = 2048):
     xf = _f32(np.atleast_2d(xf_calib))
     m = mode(xf, nbins) if nbins > 0 else np.zeros(xf.shape[1], np.float32)
     return m, tau(xf, m, s)
+
+
+def sparse_fc_q8(xf, Wq, scale, m, tau, b_fused):
+    """Sparse FC on 8-bit weights: W[k,n] = scale[k] * Wq[k,n] (signed 8-bit, one scale per input channel)."""
+    xf = _f32(np.atleast_2d(xf))
+    B, K = xf.shape
+    Wq = np.ascontiguousarray(Wq, np.int8)
+    N = Wq.shape[1]
+    y = np.empty((B, N), np.float64)
+    lib().scap_oracle_sparse_fc_q8(_p(xf), _p(Wq), _p(_f32(scale)), _p(_f32(m)), float(np.float32(tau)), _p(_f32(b_fused)), B, K, N, _p(y))
+    return y
+
+
+def fold_bias_q8(Wq, scale, m, b):
+    Wq = np.ascontiguousarray(Wq, np.int8)
+    K, N = Wq.shape
+    out = np.empty(N, np.float64)
+    lib().scap_oracle_fold_bias_q8(_p(Wq), _p(_f32(scale)), _p(_f32(m)), _p(_f32(b)), K, N, _p(out))
+    return out
 
 
 def glu_ffn(hf, Wgu, Wd, dt, m1, tau1, bgu_fused, m2, tau2, bd_fused, z_in=None):

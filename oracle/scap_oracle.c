@@ -282,6 +282,32 @@ float scap_oracle_tau(const float *xf /*[T,K]*/, int T, int K, const float *m, d
     return (float)t64;
 }
 
+/* ---------------------------------------------------------------- 8-bit weights (Table 4 applies SCAP to 8-bit models)
+ * Storage reading: Wq[K,N] signed 8-bit, one binary32 scale per input channel, W[k,n] = scale[k] * Wq[k,n]
+ * (symmetric, no zero point).  The sparse FC and the bias folding are Eq. 2-3 and Eq. 5-6 on that W, in binary64. */
+void scap_oracle_sparse_fc_q8(const float *xf, const signed char *Wq, const float *scale, const float *m, float tau,
+                              const float *b_fused, int B, int K, int N, double *y) {
+    for (int b = 0; b < B; ++b)
+        for (int n = 0; n < N; ++n) {
+            double acc = b_fused ? (double)b_fused[n] : 0.0;
+            for (int k = 0; k < K; ++k) {
+                volatile float d = m ? xf[(long)b * K + k] - m[k] : xf[(long)b * K + k];   /* the decision: binary32 */
+                double xc = (double)xf[(long)b * K + k] - (m ? (double)m[k] : 0.0);      /* the product: exact difference */
+                if (fabsf(d) >= tau) acc += xc * ((double)scale[k] * (double)Wq[(long)k * N + n]);
+            }
+            y[(long)b * N + n] = acc;
+        }
+}
+
+void scap_oracle_fold_bias_q8(const signed char *Wq, const float *scale, const float *m, const float *b /*[N] nullable*/,
+                              int K, int N, double *b_fused) {
+    for (int n = 0; n < N; ++n) {
+        double acc = b ? (double)b[n] : 0.0;
+        for (int k = 0; k < K; ++k) acc += (double)m[k] * ((double)scale[k] * (double)Wq[(long)k * N + n]);
+        b_fused[n] = acc;
+    }
+}
+
 /* ---------------------------------------------------------------- Alg. 2: SwiGLU block
  * Wgu[D,2F]: columns 0..F-1 are the gate projection, F..2F-1 the up projection; both read the
  * same pruned input (one tau_x, one mask).  z = up * silu(gate), silu(g) = g / (1 + exp(-g)),

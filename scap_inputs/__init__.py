@@ -265,3 +265,13 @@ def config3(B: int = 1) -> dict:
 
 def config4_fc(K: int, N: int, B: int, T_calib: int = 2048) -> dict:
     return laplace_fc(4, K, N, BF16, T_calib, B, with_bias=False)
+
+
+def quantise_q8(W_bits: np.ndarray, dt: int):
+    """Symmetric 8-bit quantisation of a 16-bit weight, one scale per input channel (row): scale = max|row| / 127
+    (1 for an all-zero row), q = round-half-even(W / scale) clipped to [-127, 127].  Returns (int8 [K,N], float32 [K])."""
+    Wf = to_f32(W_bits, dt).astype(np.float64)
+    amax = np.abs(Wf).max(axis=1)
+    scale = np.where(amax > 0, amax / 127.0, 1.0).astype(np.float32)
+    q = np.clip(np.rint(Wf / scale.astype(np.float64)[:, None]), -127, 127).astype(np.int8)
+    return q, scale

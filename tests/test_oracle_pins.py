@@ -524,3 +524,34 @@ def test_gelu_ffn_is_the_composition_of_its_stages_and_honours_teacher_forcing()
     # GELU output is skewed (bounded below near -0.17): the centred threshold prunes the target, the uncentred one less
     kept_c = float(np.mean(np.abs(zc - m2[None, :]) >= tau2))
     assert abs(kept_c - 0.4) < 0.02
+
+
+# ---------------------------------------------------------------- 8-bit weights
+
+def test_q8_oracle_reduces_to_the_16_bit_oracle_when_the_products_are_representable():
+    # scale a power of two and |q| <= 127: scale * q is exact in fp16, so both oracles see the same real matrix
+    rng = np.random.default_rng(5)
+    K, N, B = 96, 24, 3
+    q = rng.integers(-127, 128, size=(K, N)).astype(np.int8)
+    scale = (2.0 ** rng.integers(-9, -5, size=K)).astype(np.float32)
+    W16 = si.to_bits(scale[:, None].astype(np.float64) * q.astype(np.float64), si.F16)
+    assert np.array_equal(si.to_f32(W16, si.F16), scale[:, None] * q.astype(np.float32))
+    d = si.laplace_fc(4, K, N, si.F16, 8, B)
+    xf = si.to_f32(d["x"], si.F16)
+    m, bf = d["m_true"], np.linspace(-1, 1, N).astype(np.float32)
+    for tau in (0.0, 0.2, 5.0):
+        assert np.array_equal(oracle.sparse_fc_q8(xf, q, scale, m, tau, bf), oracle.sparse_fc(xf, W16, si.F16, m, tau, bf))
+    assert np.array_equal(oracle.fold_bias_q8(q, scale, m, None), oracle.fold_bias(W16, si.F16, m, None))
+
+
+def test_q8_brute_force_on_a_tiny_case_and_quantiser_properties():
+    q = np.int8([[1, -2], [3, 4], [-128 + 1, 127]])
+    scale = np.float32([0.5, 0.25, 2.0])
+    x = np.float32([[1.0, -3.0, 0.1]])
+    y = oracle.sparse_fc_q8(x, q, scale, None, 0.5, np.float32([10, 20]))
+    assert np.array_equal(y, [[10 + 1.0 * 0.5 * 1 - 3.0 * 0.25 * 3, 20 + 1.0 * 0.5 * -2 - 3.0 * 0.25 * 4]])  # channel 2 pruned
+    W = si.weight(4, 64, 40, si.BF16)
+    qq, ss = si.quantise_q8(W, si.BF16)
+    Wf = si.to_f32(W, si.BF16)
+    assert qq.dtype == np.int8 and np.abs(qq).max() == 127 and np.all(np.abs(qq).max(axis=1) == 127)
+    assert np.all(np.abs(ss[:, None] * qq - Wf) <= 0.5 * ss[:, None] * (1 + 1e-3))
