@@ -159,6 +159,20 @@ scap_status scap_sparse_fc(const void *x, const void *W, const float *m, const f
 scap_status scap_dense_fc(const void *x, const void *W, const float *b, float *y, int B, int K, int N,
                           scap_dtype dt, void *ws, size_t ws_bytes, scap_stream_t stream);
 
+/* 8-bit weights (Table 4 applies SCAP to 8-bit models).  Storage: Wq[K,N] signed 8-bit, row-major like W, and
+ * wscale[K] fp32, one scale per input channel: W[k,n] = wscale[k] * Wq[k,n] (symmetric, no zero point).  x has
+ * dtype xdt (fp16 or bf16); everything else as in scap_sparse_fc / scap_dense_fc / scap_fold_bias, with these
+ * differences: N must be a multiple of 16; the bias b of the dense call and of the folding is fp32 [N] or
+ * NULL; batches of more than two rows are processed two rows at a time (results per row as in scap_sparse_fc;
+ * idx_out / nnz_out are only available for B <= 2, else SCAP_ERR_SHAPE).  Workspace: scap_fc_workspace(B, K, N). */
+scap_status scap_sparse_fc_q8(const void *x, scap_dtype xdt, const signed char *Wq, const float *wscale, const float *m,
+                              const float *tau, const float *b_fused, float *y, int B, int K, int N, uint32_t *idx_out,
+                              int *nnz_out, void *ws, size_t ws_bytes, scap_stream_t stream);
+scap_status scap_dense_fc_q8(const void *x, scap_dtype xdt, const signed char *Wq, const float *wscale, const float *b,
+                             float *y, int B, int K, int N, void *ws, size_t ws_bytes, scap_stream_t stream);
+scap_status scap_fold_bias_q8(const signed char *Wq, const float *wscale, const float *m, const float *b, int K, int N,
+                              float *b_fused, void *ws, size_t ws_bytes, scap_stream_t stream);
+
 /* scap_sparse_fc for a caller whose activations live in HOST memory: copies x_host[B,K]
  * (dtype dt; pinned memory recommended) to the device, runs the sparse FC, and copies y back to
  * y_host[B,N] (fp32), all enqueued on `stream`; y_host is valid once the stream has drained.

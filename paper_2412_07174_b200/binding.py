@@ -10,7 +10,8 @@ __all__ = [
     "SCAP_F16", "SCAP_BF16", "ScapError", "lib", "lib_path", "status_string", "scap_version", "scap_tune", "scap_device_status",
     "scap_calibrate_workspace", "scap_calibrate", "scap_calibrate_ex", "SCAP_MODE_HISTOGRAM", "SCAP_MODE_MEAN", "SCAP_MODE_MEDIAN",
     "SCAP_ETA_PER_CHANNEL", "SCAP_ETA_SCALAR", "scap_fold_bias_workspace", "scap_fold_bias",
-    "scap_fc_workspace", "scap_sparse_fc", "scap_dense_fc", "scap_fc_host_workspace", "scap_sparse_fc_host",
+    "scap_fc_workspace", "scap_sparse_fc", "scap_dense_fc", "scap_sparse_fc_q8", "scap_dense_fc_q8", "scap_fold_bias_q8",
+    "scap_fc_host_workspace", "scap_sparse_fc_host",
     "scap_glu_workspace", "scap_glu_ffn", "scap_gelu_ffn_workspace", "scap_gelu_ffn", "scap_glu_static_capacity", "scap_glu_ffn_static", "scap_moe_workspace",
     "scap_moe_ffn", "ScapExpert", "dtype_of", "EXPORTS",
 ]
@@ -22,7 +23,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 EXPORTS = [
     "scap_status_string", "scap_version", "scap_tune", "scap_device_status", "scap_calibrate_workspace", "scap_calibrate",
     "scap_calibrate_ex", "scap_fold_bias_workspace", "scap_fold_bias", "scap_fc_workspace", "scap_sparse_fc", "scap_dense_fc",
-    "scap_fc_host_workspace", "scap_sparse_fc_host", "scap_glu_workspace", "scap_glu_ffn", "scap_gelu_ffn_workspace",
+    "scap_sparse_fc_q8", "scap_dense_fc_q8", "scap_fold_bias_q8", "scap_fc_host_workspace", "scap_sparse_fc_host", "scap_glu_workspace", "scap_glu_ffn", "scap_gelu_ffn_workspace",
     "scap_gelu_ffn", "scap_glu_static_capacity", "scap_glu_ffn_static", "scap_moe_workspace", "scap_moe_ffn",
 ]
 
@@ -79,6 +80,12 @@ def lib():
     L.scap_sparse_fc.restype = i
     L.scap_dense_fc.argtypes = [vp, vp, vp, vp, i, i, i, i, vp, sz, vp]
     L.scap_dense_fc.restype = i
+    L.scap_sparse_fc_q8.argtypes = [vp, i, vp, vp, vp, vp, vp, vp, i, i, i, vp, vp, vp, sz, vp]
+    L.scap_sparse_fc_q8.restype = i
+    L.scap_dense_fc_q8.argtypes = [vp, i, vp, vp, vp, vp, i, i, i, vp, sz, vp]
+    L.scap_dense_fc_q8.restype = i
+    L.scap_fold_bias_q8.argtypes = [vp, vp, vp, vp, i, i, vp, vp, sz, vp]
+    L.scap_fold_bias_q8.restype = i
     L.scap_fc_host_workspace.argtypes = [i, i, i]
     L.scap_fc_host_workspace.restype = sz
     L.scap_sparse_fc_host.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, vp, sz, vp]
@@ -205,6 +212,30 @@ def scap_dense_fc(x, W, b, y, ws, stream=None) -> None:
     p, n = _ws(ws)
     _check(lib().scap_dense_fc(_ptr(x), _ptr(W), _ptr(b), _ptr(y), B, K, N, dtype_of(W), p, n, _stream(stream)),
            "scap_dense_fc")
+
+
+def scap_sparse_fc_q8(x, Wq, wscale, m, tau, b_fused, y, ws, idx_out=None, nnz_out=None, stream=None) -> None:
+    """Sparse FC on 8-bit weights: Wq int8 [K, N], wscale fp32 [K] (one scale per input channel)."""
+    B, K = x.shape
+    N = Wq.shape[1]
+    p, n = _ws(ws)
+    _check(lib().scap_sparse_fc_q8(_ptr(x), dtype_of(x), _ptr(Wq), _ptr(wscale), _ptr(m), _ptr(tau), _ptr(b_fused), _ptr(y), B, K, N,
+                                   _ptr(idx_out), _ptr(nnz_out), p, n, _stream(stream)), "scap_sparse_fc_q8")
+
+
+def scap_dense_fc_q8(x, Wq, wscale, b, y, ws, stream=None) -> None:
+    B, K = x.shape
+    N = Wq.shape[1]
+    p, n = _ws(ws)
+    _check(lib().scap_dense_fc_q8(_ptr(x), dtype_of(x), _ptr(Wq), _ptr(wscale), _ptr(b), _ptr(y), B, K, N, p, n, _stream(stream)),
+           "scap_dense_fc_q8")
+
+
+def scap_fold_bias_q8(Wq, wscale, m, b, b_fused, ws, stream=None) -> None:
+    K, N = Wq.shape
+    p, n = _ws(ws)
+    _check(lib().scap_fold_bias_q8(_ptr(Wq), _ptr(wscale), _ptr(m), _ptr(b), K, N, _ptr(b_fused), p, n, _stream(stream)),
+           "scap_fold_bias_q8")
 
 
 def scap_fc_host_workspace(B: int, K: int, N: int) -> int:

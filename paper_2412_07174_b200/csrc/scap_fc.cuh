@@ -66,6 +66,7 @@ struct FcArgs {
     int hold_dependents;  // 1: do not let the next kernel start before this grid completes (it writes parameters)
     int no_tc;            // 1: keep this call off the tcgen05 kernel
     int act;              // EPI_BIAS: 1 = the exact GELU is applied to the biased result (z_copy then gets a copy)
+    const float *wscale;  // 8-bit weights only: one scale per input channel, W[k,n] = wscale[k] * Wq[k,n]
 };
 
 template <bool BF16, int BT, int CAP>
