@@ -247,6 +247,55 @@ def suite_sweep(torch, scap, peak, shapes, sparsities, batches, out):
         torch.cuda.empty_cache()
 
 
+def suite_q8(torch, scap, peak, out):
+    """8-bit weights (per-input-channel scales) at the bench shape, batch 1 and 2: the weight bytes halve, the fixed latencies
+    of a call do not, so this is the harder roofline; next to the bf16 call on the same inputs."""
+    stream = torch.cuda.Stream()
+    l2 = torch.cuda.get_device_properties(0).L2_cache_size
+    Kk, Nn = 11008, 4096
+    d = si.config4_fc(Kk, Nn, 16 * 8, T_calib=2048)
+    q, sc = si.quantise_q8(d["W"], si.BF16)
+    W0 = si.as_torch(d["W"], si.BF16).cuda()
+    Q0 = torch.from_numpy(q).cuda()
+    scl = torch.from_numpy(sc).cuda()
+    xc = si.as_torch(d["x_calib"], si.BF16).cuda()
+    xs = si.as_torch(d["x"], si.BF16).cuda()
+    Rmax = int(np.ceil(4 * l2 / (0.2 * Kk * Nn)))
+    Qs = [Q0] + [Q0.clone() for _ in range(Rmax - 1)]
+    Ws = [W0] + [W0.clone() for _ in range(Rmax // 2)]
+    cws = torch.empty(scap.scap_calibrate_workspace(2048, Kk, NBINS), dtype=torch.uint8, device="cuda")
+    m = torch.empty(Kk, dtype=torch.float32, device="cuda")
+    bf = torch.empty(Nn, dtype=torch.float32, device="cuda")
+    bq = torch.empty(Nn, dtype=torch.float32, device="cuda")
+    nnz = torch.zeros(1, dtype=torch.int32, device="cuda")
+    idx = torch.empty(Kk, dtype=torch.int32, device="cuda")
+    for B in (1, 2):
+        ws = torch.empty(scap.scap_fc_workspace(B, Kk, Nn), dtype=torch.uint8, device="cuda")
+        y = torch.empty((B, Nn), dtype=torch.float32, device="cuda")
+        xb = [xs[i * 16:i * 16 + B] for i in range(8)]
+        Rd = max(2, int(np.ceil(4 * l2 / (Kk * Nn))))
+        t_dense = _time_graph(torch, stream, lambda: [scap.scap_dense_fc_q8(xb[r % 8], Qs[r], scl, None, y, ws) for r in range(Rd)]) / Rd
+        for s in (0.0, 0.5, 0.65, 0.8):
+            tau = torch.empty(1, dtype=torch.float32, device="cuda")
+            scap.scap_calibrate(xc, s, NBINS, m, tau, cws)
+            scap.scap_fold_bias(W0, m, None, bf, ws)
+            scap.scap_fold_bias_q8(Q0, scl, m, None, bq, ws)
+            kept = []
+            for i in range(8):
+                scap.scap_sparse_fc_q8(xb[i], Q0, scl, m, tau, bq, y, ws, idx_out=idx, nnz_out=nnz)
+                kept.append(int(nnz.item()))
+            rho = float(np.mean(kept)) / Kk
+            R = max(2, min(Rmax, int(np.ceil(4 * l2 / (max(rho, 0.2) * Kk * Nn)))))
+            t = _time_graph(torch, stream, lambda: [scap.scap_sparse_fc_q8(xb[r % 8], Qs[r], scl, m, tau, bq, y, ws) for r in range(R)]) / R
+            R16 = max(2, min(len(Ws), int(np.ceil(4 * l2 / (max(rho, 0.2) * Kk * Nn * 2)))))
+            t16 = _time_graph(torch, stream, lambda: [scap.scap_sparse_fc(xb[r % 8], Ws[r], m, tau, bf, y, ws) for r in range(R16)]) / R16
+            nb = float(np.mean(kept)) * Nn + B * Kk * 2 + 4 * Kk + 4 * Kk + 4 + 4 * Nn + 4 * B * Nn
+            out({"suite": "q8", "K": Kk, "N": Nn, "B": B, "sparsity_target": s, "union_kept_fraction": round(rho, 4), "us_per_call": round(t, 3),
+                 "gbs": round(nb / t / 1e3, 1), "frac_of_measured_peak": round(nb / t / 1e3 / peak, 3), "dense_q8_us": round(t_dense, 3),
+                 "speedup_vs_dense_q8": round(t_dense / t, 3), "bf16_sparse_us": round(t16, 3), "speedup_vs_bf16_sparse": round(t16 / t, 3),
+                 "weight_copies": R})
+
+
 def suite_calibrate(torch, scap, out):
     """Config 4's timed calibration: 2048 tokens x 14336 channels, 2048 bins, plus the tau quantile."""
     T, Kk = 2048, 14336
@@ -467,6 +516,8 @@ def run_suite(args):
         suite_glu(torch, scap, peak, out)
     if which in ("gelu", "all"):
         suite_gelu(torch, scap, peak, out)
+    if which in ("q8", "all"):
+        suite_q8(torch, scap, peak, out)
     if which in ("sweep", "all", "sweep-small"):
         shapes = [(4096, 4096), (4096, 11008), (11008, 4096), (14336, 4096)]
         if which == "sweep-small":
@@ -492,7 +543,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--detail", action="store_true", help="also print a per-sparsity table to stderr")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--suite", default="", choices=["", "calibrate", "glu", "gelu", "moe", "sweep", "sweep-small", "all"],
+    ap.add_argument("--suite", default="", choices=["", "calibrate", "glu", "gelu", "q8", "moe", "sweep", "sweep-small", "all"],
                     help="run the other workload descriptions instead of the headline line (one JSON object per line)")
     ap.add_argument("--copies", type=int, default=0,
                     help="number of weight copies to rotate (default: enough for the cold-HBM rule); a small value keeps "
