@@ -683,20 +683,45 @@ __device__ __forceinline__ void fc_body_mma(const FcArgs &a, const int tile, con
                     b1[2 * i + 1] = __byte_perm(r2[i], r3[i], 0x7632);
                 }
                 const int w0 = 8 * (rw + NRW * q) + t;  // pair index of kept rows (2t, 2t+1) of this block
+                if constexpr (ROWS == 8) {
+                    // The 16 rows of M hold two parts of the 8 batch rows: the last part (bf16: lo) goes alone, with a
+                    // zero upper half; then hi in rows 0-7 and the second part in rows 8-15 of one MMA.  Accumulator
+                    // rows g hold hi (+ lo), rows g + 8 the second part; they are added when the fragments are stored.
+                    if constexpr (NSPLIT == 3) {
+                        const uint32_t *pl = s_xp + 2 * BT * XLD2;
+                        uint32_t af[4] = {0u, 0u, 0u, 0u};
+                        if (g < Bp) {
+                            af[0] = pl[g * XLD2 + w0];
+                            af[2] = pl[g * XLD2 + w0 + 4];
+                        }
 #pragma unroll
-                for (int qs = NSPLIT - 1; qs >= 0; --qs) {  // smallest part first
-                    const uint32_t *pl = s_xp + qs * BT * XLD2;
+                        for (int i = 0; i < 8; ++i) mma_k16<BF16>(acc[i], af, b0[i], b1[i]);
+                    }
                     uint32_t af[4] = {0u, 0u, 0u, 0u};
                     if (g < Bp) {
-                        af[0] = pl[g * XLD2 + w0];
-                        af[2] = pl[g * XLD2 + w0 + 4];
-                    }
-                    if (ROWS == 16 && g + 8 < Bp) {
-                        af[1] = pl[(g + 8) * XLD2 + w0];
-                        af[3] = pl[(g + 8) * XLD2 + w0 + 4];
+                        af[0] = s_xp[g * XLD2 + w0];
+                        af[2] = s_xp[g * XLD2 + w0 + 4];
+                        af[1] = s_xp[(BT + g) * XLD2 + w0];
+                        af[3] = s_xp[(BT + g) * XLD2 + w0 + 4];
                     }
 #pragma unroll
                     for (int i = 0; i < 8; ++i) mma_k16<BF16>(acc[i], af, b0[i], b1[i]);
+                } else {
+#pragma unroll
+                    for (int qs = NSPLIT - 1; qs >= 0; --qs) {  // smallest part first
+                        const uint32_t *pl = s_xp + qs * BT * XLD2;
+                        uint32_t af[4] = {0u, 0u, 0u, 0u};
+                        if (g < Bp) {
+                            af[0] = pl[g * XLD2 + w0];
+                            af[2] = pl[g * XLD2 + w0 + 4];
+                        }
+                        if (g + 8 < Bp) {
+                            af[1] = pl[(g + 8) * XLD2 + w0];
+                            af[3] = pl[(g + 8) * XLD2 + w0 + 4];
+                        }
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) mma_k16<BF16>(acc[i], af, b0[i], b1[i]);
+                    }
                 }
             };
 #pragma unroll
@@ -722,11 +747,14 @@ __device__ __forceinline__ void fc_body_mma(const FcArgs &a, const int tile, con
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
         const int c0 = cw * 64 + 8 * (2 * t) + i, c1 = c0 + 8;
-        s_red[(rw * BT + g) * TNT + c0] = acc[i][0];
-        s_red[(rw * BT + g) * TNT + c1] = acc[i][1];
         if constexpr (ROWS == 16) {
+            s_red[(rw * BT + g) * TNT + c0] = acc[i][0];
+            s_red[(rw * BT + g) * TNT + c1] = acc[i][1];
             s_red[(rw * BT + g + 8) * TNT + c0] = acc[i][2];
             s_red[(rw * BT + g + 8) * TNT + c1] = acc[i][3];
+        } else {  // rows g + 8 of the accumulator hold the second part of batch row g
+            s_red[(rw * BT + g) * TNT + c0] = acc[i][0] + acc[i][2];
+            s_red[(rw * BT + g) * TNT + c1] = acc[i][1] + acc[i][3];
         }
     }
     __syncthreads();
