@@ -640,13 +640,10 @@ static cudaError_t estimate_mode(const uint16_t *x, int T, int K, int estimator,
     cudaError_t e = cudaSuccess;
     if (!scalar) {
         if (estimator == 1) return launch(mean_kernel<BF16>, dim3((K + 31) / 32), dim3(256), 0, st, false, x, T, K, m_out, (double *)nullptr);
-        static bool attr_set[2] = {false, false};
+        static SmemOptIn opt_in;
         const size_t smem = (size_t)3 * CW * 256 * 4;
-        if (!attr_set[BF16]) {
-            e = cudaFuncSetAttribute(median_kernel<BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-            if (e != cudaSuccess) return e;
-            attr_set[BF16] = true;
-        }
+        e = ensure_dynamic_smem(median_kernel<BF16>, (int)smem, opt_in);
+        if (e != cudaSuccess) return e;
         return launch(median_kernel<BF16>, dim3((K + CW - 1) / CW), dim3(CAL_THREADS), smem, st, false, x, T, K, m_out);
     }
     if (estimator == 1) {
@@ -697,12 +694,9 @@ static scap_status calibrate_t(const uint16_t *x, int T, int K, double sparsity,
     size_t smem = (size_t)CW * HW * 4;
     if (smem < (size_t)2 * CAL_ROWS * CW * 4) smem = (size_t)2 * CAL_ROWS * CW * 4;
     if (smem < (size_t)RADIX_BINS * 4) smem = (size_t)RADIX_BINS * 4;
-    static bool attr_set[2] = {false, false};
-    if (!attr_set[BF16]) {
-        e = cudaFuncSetAttribute(mode_kernel<BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 2048 / 2 * CW * 4);
-        if (e != cudaSuccess) return cuda_status(e);
-        attr_set[BF16] = true;
-    }
+    static SmemOptIn opt_in;
+    e = ensure_dynamic_smem(mode_kernel<BF16>, 2048 / 2 * CW * 4, opt_in);
+    if (e != cudaSuccess) return cuda_status(e);
     e = launch(mode_kernel<BF16>, dim3((K + CW - 1) / CW), dim3(CAL_THREADS), smem, st, false, x, T, K, nbins, m_out, hist,
                want_tau ? 1 : 0, own_mode ? (const float *)nullptr : (const float *)m_out);
     if (e != cudaSuccess) return cuda_status(e);

@@ -35,6 +35,22 @@ inline scap_status cuda_status(cudaError_t e) {
     return SCAP_ERR_CUDA;
 }
 
+// Opt-in to more than 48 KB of dynamic shared memory, once per kernel and device (the attribute belongs to the
+// device's copy of the function, so a process that drives several devices sets it on each).
+struct SmemOptIn {
+    unsigned long long done = 0;  // bit d: set on device d (devices beyond 63 are set every time)
+};
+template <typename Kern>
+inline cudaError_t ensure_dynamic_smem(Kern kern, int bytes, SmemOptIn &state) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev >= 0 && dev < 64 && ((state.done >> dev) & 1ull)) return cudaSuccess;
+    e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e == cudaSuccess && dev >= 0 && dev < 64) state.done |= 1ull << dev;
+    return e;
+}
+
 // ---- programmatic dependent launch ----------------------------------------------------------
 // wait: blocks until every kernel this grid depends on has finished and its writes are visible
 // (returns at once when the launch carried no programmatic dependency).

@@ -95,13 +95,10 @@ void choose_config(int K, int Nh, int epi, int groups, int B, int *tn_out, int *
 
 template <bool BF16, int BT, int MODE, typename XT, int EPI, int TNT>
 static cudaError_t launch_fc_tn(const FcArgs &a, cudaStream_t st) {
-    static bool attr_done = false;
+    static SmemOptIn opt_in;
     auto kern = fc_kernel<BF16, BT, MODE, XT, EPI, TNT>;
-    if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, fc_smem_for(BT));
-        if (e != cudaSuccess) return e;
-        attr_done = true;
-    }
+    cudaError_t e0 = ensure_dynamic_smem(kern, fc_smem_for(BT), opt_in);
+    if (e0 != cudaSuccess) return e0;
     return launch_cluster(kern, dim3(fc_tiles(a.Nh, EPI, TNT), a.S), dim3(FC_THREADS), fc_smem_for(BT), a.S, st,
                           g_tune.pdl != 0, a);
 }

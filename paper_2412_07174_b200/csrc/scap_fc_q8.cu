@@ -243,13 +243,10 @@ static int q8_split(int K, int N) {
 
 template <int BT, int MODE, typename XT>
 static cudaError_t launch_q8_t(const FcArgs &a, cudaStream_t st) {
-    static bool attr_done = false;
+    static SmemOptIn opt_in;
     auto kern = fc_q8_kernel<BT, MODE, XT>;
-    if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, fc_smem_bytes(BT));
-        if (e != cudaSuccess) return e;
-        attr_done = true;
-    }
+    cudaError_t e0 = ensure_dynamic_smem(kern, fc_smem_bytes(BT), opt_in);
+    if (e0 != cudaSuccess) return e0;
     return launch_cluster(kern, dim3((a.Nh + Q8_TN - 1) / Q8_TN, a.S), dim3(FC_THREADS), fc_smem_bytes(BT), a.S, st, g_tune.pdl != 0, a);
 }
 

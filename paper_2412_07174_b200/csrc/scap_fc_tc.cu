@@ -433,13 +433,10 @@ __global__ void __launch_bounds__(FC_THREADS, 2) fc_tc_kernel(const FcArgs a) {
 
 template <bool BF16, int ROWS, int MODE, typename XT, int EPI>
 static cudaError_t launch_tc_r(const FcArgs &a, cudaStream_t st) {
-    static bool attr_done = false;
+    static SmemOptIn opt_in;
     auto kern = fc_tc_kernel<BF16, ROWS, MODE, XT, EPI>;
-    if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM);
-        if (e != cudaSuccess) return e;
-        attr_done = true;
-    }
+    cudaError_t e0 = ensure_dynamic_smem(kern, TC_SMEM, opt_in);
+    if (e0 != cudaSuccess) return e0;
     return launch_cluster(kern, dim3(fc_tiles(a.Nh, EPI, TC_TN), a.S), dim3(FC_THREADS), TC_SMEM, a.S, st, g_tune.pdl != 0, a);
 }
 

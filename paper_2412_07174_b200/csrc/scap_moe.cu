@@ -144,13 +144,10 @@ static MoeLayout moe_layout(int B, int D, int F, int E, int top_k) {
 
 template <bool BF16, int BT, int STAGE, int TNT>
 static cudaError_t launch_moe_fc_tn(const MoeArgs &a, int tiles, int S, cudaStream_t st) {
-    static bool attr_done = false;
+    static SmemOptIn opt_in;
     auto kern = moe_fc_kernel<BF16, BT, STAGE, TNT>;
-    if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, fc_smem_for(BT));
-        if (e != cudaSuccess) return e;
-        attr_done = true;
-    }
+    cudaError_t e0 = ensure_dynamic_smem(kern, fc_smem_for(BT), opt_in);
+    if (e0 != cudaSuccess) return e0;
     return launch_cluster(kern, dim3(tiles, S, a.E), dim3(FC_THREADS), fc_smem_for(BT), S, st, g_tune.pdl != 0, a);
 }
 
