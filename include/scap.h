@@ -77,7 +77,9 @@ int scap_version(void);
 /* Process-wide tuning knobs (plain ints, not thread-safe against concurrent calls):
  *   "split_k"  cap the split-K factor (thread-block cluster size) of the FC kernel: 0 = automatic, else 1..8
  *   "pdl"      1 = launch dependent kernels with programmatic dependent launch (default), 0 = off
- *   "tcgen05"  batch 3..16 calls of the FC and SwiGLU entry points: 0 = always the mma.sync variants,
+ *   "fma_rows" largest batch that runs on the fp32-FMA form of the FC kernel: 4 (default) or 2; larger
+ *              batches (up to 16) run on a tensor-core form
+ *   "tcgen05"  tensor-core batches of the FC and SwiGLU entry points: 0 = always the mma.sync variants,
  *              1 = the tcgen05 (TMEM accumulator) kernel where its shared-memory operand region holds
  *              the call's kept channels in one pass, else mma.sync (default), 2 = always tcgen05
  *   "host_direct"  scap_sparse_fc_host: 1 = when x_host and y_host are page-locked and addressable by the

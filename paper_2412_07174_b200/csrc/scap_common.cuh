@@ -19,6 +19,7 @@ struct Tuning {
     int pdl;      // programmatic dependent launch between the kernels of one call
     int tc;       // batch 3..16 on the tcgen05 kernel (0: the mma.sync variants)
     int host_direct;  // scap_sparse_fc_host moves device-addressable pinned host buffers with its own kernels
+    int fma_rows;     // largest batch that takes the fp32-FMA body (2 or 4); larger batches take a tensor-core variant
 };
 extern Tuning g_tune;
 

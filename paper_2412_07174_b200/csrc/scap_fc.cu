@@ -6,7 +6,7 @@
 
 namespace scap {
 
-Tuning g_tune = {0, 1, 1, 1};
+Tuning g_tune = {0, 1, 1, 1, 4};
 
 scap_status check_device() {
     static int cached[64];  // 0 unknown, 1 ok, 2 unsupported
@@ -72,7 +72,7 @@ int resident_ctas(int S) {
 // Ties: fewer fills of the kept-channel stage per CTA (B decides the stage capacity), then the narrower tile (its
 // smaller cluster exchanges less), then the larger cluster.
 void choose_config(int K, int Nh, int epi, int groups, int B, int *tn_out, int *S_out) {
-    const int bt = batch_tile(B), cap = is_mma(bt) ? mma_cap(bt) : fc_cap(bt);
+    const int bt = fc_batch_tile(B), cap = is_mma(bt) ? mma_cap(bt) : fc_cap(bt);
     const int nchunks = (K + 31) / 32;
     int best_tn = 256, best_S = 1;
     long long best = -1;
@@ -110,9 +110,10 @@ static cudaError_t launch_fc_t(const FcArgs &a, cudaStream_t st) {
 
 template <bool BF16, int MODE, typename XT, int EPI>
 static cudaError_t launch_fc_bt(const FcArgs &a, cudaStream_t st) {
-    switch (batch_tile(a.B)) {
+    switch (fc_batch_tile(a.B)) {
         case 1: return launch_fc_t<BF16, 1, MODE, XT, EPI>(a, st);
         case 2: return launch_fc_t<BF16, 2, MODE, XT, EPI>(a, st);
+        case 4: return launch_fc_t<BF16, 4, MODE, XT, EPI>(a, st);
         case 8: return launch_fc_t<BF16, 8, MODE, XT, EPI>(a, st);
         default: return launch_fc_t<BF16, 16, MODE, XT, EPI>(a, st);
     }
@@ -271,6 +272,11 @@ scap_status scap_tune(const char *key, int value) {
     }
     if (!strcmp(key, "host_direct")) {
         g_tune.host_direct = value != 0;
+        return SCAP_OK;
+    }
+    if (!strcmp(key, "fma_rows")) {
+        if (value != 2 && value != 4) return SCAP_ERR_INVALID_ARG;
+        g_tune.fma_rows = value;
         return SCAP_OK;
     }
     if (!strcmp(key, "tcgen05")) {

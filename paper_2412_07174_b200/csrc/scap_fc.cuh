@@ -28,7 +28,7 @@ constexpr int FC_THREADS = 256;  // 8 warps; two CTAs fit on an SM, so every clu
 constexpr int FC_WARPS = FC_THREADS / 32;
 __host__ __device__ constexpr int fc_min_blocks(int BT) { return 2; }
 // chunks (of 32 channels) each warp thresholds per fill; their centred values stay in registers
-__host__ __device__ constexpr int fc_pu(int BT) { return BT <= 2 ? 8 : BT <= 4 ? 4 : BT <= 8 ? 2 : 1; }
+__host__ __device__ constexpr int fc_pu(int BT) { return BT <= 2 ? 8 : BT <= 4 ? 6 : BT <= 8 ? 2 : 1; }
 __host__ __device__ constexpr int fc_cap(int BT) { return FC_WARPS * fc_pu(BT) * 32; }  // channels staged per fill
 __host__ __device__ constexpr int fc_rb(int BT) { return BT < 4 ? BT : 4; }              // batch rows per cross-warp round
 __host__ __device__ constexpr int fc_unroll(int BT) { return BT <= 1 ? 16 : BT <= 4 ? 8 : 4; }  // row loads in flight per thread
@@ -257,6 +257,7 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
     }
     for (int j0 = 0; j0 < my_chunks; j0 += CAPC) {
         const int nj = min(CAPC, my_chunks - j0);
+        const int pw = (nj + FC_WARPS - 1) / FC_WARPS;  // chunks per warp this fill: warp w owns chunks w * pw .. w * pw + pw - 1
         // ---- A: every warp loads PU chunks at once, centres and thresholds them (Alg. 3: one binary32
         // subtraction, one compare per element) and keeps the values in registers.  Loads of unused slots are
         // predicated off (no branch) and nothing consumes a value inside the load loops, so the PU * (BT + 1)
@@ -265,18 +266,18 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
         float xv[PU][BT], mk[PU];
 #pragma unroll
         for (int p = 0; p < PU; ++p) {
-            const int j = warp * PU + p;
+            const int j = warp * pw + p;
             const int k = (s + S * (j0 + j)) * 32 + lane;
-            mk[p] = a.m ? ld_nc_if(a.m + k, j < nj && k < K) : 0.0f;
+            mk[p] = a.m ? ld_nc_if(a.m + k, p < pw && j < nj && k < K) : 0.0f;
         }
         if (wait_inside && j0 == 0 && !a.in_rows) {
             // Pull this CTA's slice of x towards L2 while the previous kernel drains.  L2 is the coherence point,
             // so a line the previous kernel still writes stays correct; the values are only read after the wait.
 #pragma unroll
             for (int p = 0; p < PU; ++p) {
-                const int j = warp * PU + p;
+                const int j = warp * pw + p;
                 const int k = (s + S * j) * 32 + lane;
-                if (j < nj && k < K) {
+                if (p < pw && j < nj && k < K) {
 #pragma unroll
                     for (int b = 0; b < BT; ++b)
                         if (b < B) prefetch_l2(xg + (size_t)b * a.x_ld + k);
@@ -287,9 +288,9 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
         }
 #pragma unroll
         for (int p = 0; p < PU; ++p) {
-            const int j = warp * PU + p;
+            const int j = warp * pw + p;
             const int k = (s + S * (j0 + j)) * 32 + lane;
-            const bool ok = j < nj && k < K;
+            const bool ok = p < pw && j < nj && k < K;
 #pragma unroll
             for (int b = 0; b < BT; ++b) {
                 const int bb = b < B ? b : 0;
@@ -305,9 +306,9 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
         unsigned bal[PU];
 #pragma unroll
         for (int p = 0; p < PU; ++p) {
-            const int j = warp * PU + p;
+            const int j = warp * pw + p;
             const int k = (s + S * (j0 + j)) * 32 + lane;
-            const bool ok = j < nj && k < K;
+            const bool ok = p < pw && j < nj && k < K;
             uint32_t m_ = 0;
 #pragma unroll
             for (int b = 0; b < BT; ++b) {
@@ -335,8 +336,8 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
             unsigned mine = 0;
 #pragma unroll
             for (int p = 0; p < PU; ++p) mine = lane == p ? bal[p] : mine;
-            const int j = warp * PU + lane;
-            if (lane < PU && j < nj) a.bits[s + S * (j0 + j)] = mine;
+            const int j = warp * pw + lane;
+            if (lane < pw && j < nj) a.bits[s + S * (j0 + j)] = mine;
         }
         __syncthreads();
         int cnt = 0, wbase = 0;
@@ -350,7 +351,7 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
 #pragma unroll
         for (int p = 0; p < PU; ++p) {
             if (km[p]) {
-                const int j = warp * PU + p;
+                const int j = warp * pw + p;
                 const int pos = wbase + my_off[p] + __popc(bal[p] & ((1u << lane) - 1u));
                 s_k[pos] = (uint32_t)((s + S * (j0 + j)) * 32 + lane);
 #pragma unroll
@@ -831,6 +832,8 @@ __global__ void __launch_bounds__(FC_THREADS, fc_min_blocks(BT)) fc_kernel(const
 // ---- host-side plumbing shared by the entry points ------------------------------------------------
 
 inline int batch_tile(int B) { return B <= 1 ? 1 : B <= 2 ? 2 : B <= 8 ? 8 : 16; }  // 3..16 rows: tensor-core variants
+// Batch tile of the plain FC and FFN calls: batches up to the tuned limit stay on the fp32-FMA body.
+inline int fc_batch_tile(int B) { return (B > 2 && B <= g_tune.fma_rows) ? 4 : batch_tile(B); }
 inline int fc_tiles(int Nh, int epi, int tn) { return epi == EPI_GLU ? (Nh + tn / 2 - 1) / (tn / 2) : (Nh + tn - 1) / tn; }
 
 // Tile width (256 or 128 columns) and split-K factor (cluster size) for an FC with Nh columns per half and

@@ -473,6 +473,7 @@ static int tc_fills(int K, int S, int B, bool bf16) {
 bool tc_applicable(const FcArgs &a, int epi, bool bf16) {
     if (g_tune.tc == 0 || a.no_tc || a.B < 3 || a.B > 16 || a.ldw % 8 != 0 || !aligned16(a.W) || a.hold_dependents) return false;
     if (g_tune.tc >= 2) return true;
+    if (a.B <= g_tune.fma_rows) return false;
     // ... and whose CTAs stream at least 32 chunks each: on shorter streams the heavier set-up (TMEM, barriers,
     // operand staging) of this kernel outweighs its gain (measured at K = N = 4096)
     const int S = tc_choose_split(a.K, a.Nh, epi, a.B, bf16);

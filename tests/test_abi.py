@@ -64,6 +64,9 @@ def test_argument_validation_returns_codes(L):
     assert L.scap_tune(b"no_such_key", 1) == 1
     assert L.scap_tune(b"split_k", 9) == 1
     assert L.scap_tune(b"split_k", 0) == 0
+    assert L.scap_tune(b"fma_rows", 3) == 1
+    assert L.scap_tune(b"fma_rows", 2) == 0
+    assert L.scap_tune(b"fma_rows", 4) == 0
     assert L.scap_tune(b"tcgen05", 3) == 1
     assert L.scap_tune(b"tcgen05", -1) == 1
     for v in (0, 2, 1):  # leaves the default

@@ -86,13 +86,28 @@ def test_sparsity_levels(S, s):
 
 # ---------------------------------------------------------------- degenerate cases
 
-@pytest.mark.parametrize("tc_mode", [1, 2])                        # 2: the batch-3 call runs on the tcgen05 kernel
-def test_tau_zero_is_dense_and_tau_inf_returns_bias(S, tc_mode):
+# the three forms of the kernel a batch of three can run on: (fma_rows, tcgen05) tune values
+ROUTES = {"fma": (4, 0), "mma_sync": (2, 0), "tcgen05": (2, 2)}
+
+
+def set_route(S, route):
+    rows, tc = ROUTES[route]
+    S.scap_tune("fma_rows", rows)
+    S.scap_tune("tcgen05", tc)
+
+
+def reset_route(S):
+    S.scap_tune("fma_rows", 4)
+    S.scap_tune("tcgen05", 1)
+
+
+@pytest.mark.parametrize("route", sorted(ROUTES))
+def test_tau_zero_is_dense_and_tau_inf_returns_bias(S, route):
     d = si.laplace_fc(4, 640, 264, si.BF16, 8, 3)
     dt = d["dt"]
     bf = np.linspace(-1, 1, 264).astype(np.float32)
     try:
-        S.scap_tune("tcgen05", tc_mode)
+        set_route(S, route)
         y, idx, n = run_sparse(S, d, None, 0.0, bf)
         assert n == 640 and np.array_equal(idx, np.arange(640, dtype=np.uint32))
         y64 = oracle.dense_fc(si.to_f32(d["x"], dt), d["W"], dt, bf)
@@ -103,11 +118,11 @@ def test_tau_zero_is_dense_and_tau_inf_returns_bias(S, tc_mode):
         assert n == 0 and not y.any()
         S.scap_device_status()
     finally:
-        S.scap_tune("tcgen05", 1)
+        reset_route(S)
 
 
-@pytest.mark.parametrize("tc_mode", [0, 2])
-def test_nan_and_threshold_ties_in_a_batch_of_three(S, tc_mode):
+@pytest.mark.parametrize("route", sorted(ROUTES))
+def test_nan_and_threshold_ties_in_a_batch_of_three(S, route):
     K, N = 72, 24
     d = si.laplace_fc(4, K, N, si.BF16, 8, 3)
     x = np.zeros((3, K))
@@ -119,10 +134,10 @@ def test_nan_and_threshold_ties_in_a_batch_of_three(S, tc_mode):
     y64, keep, idx = oracle_fc(d, None, 0.5, None, x_bits=xb)
     assert idx.tolist() == [0, 1, 5, 40, 71]
     try:
-        S.scap_tune("tcgen05", tc_mode)
+        set_route(S, route)
         y, gidx, n = run_sparse(S, d, None, 0.5, None, x_bits=xb)
     finally:
-        S.scap_tune("tcgen05", 1)
+        reset_route(S)
     assert gidx.tolist() == [0, 1, 5, 40, 71] and np.isfinite(y).all()
     assert rel_l2_rows(y, y64) <= REL_L2_TOL
 
@@ -174,7 +189,7 @@ def test_bitwise_determinism_and_row_independence(S):
         assert rel_l2_rows(y1[b:b + 1], y64) <= REL_L2_TOL
 
 
-@pytest.mark.parametrize("B", [1, 3, 12])
+@pytest.mark.parametrize("B", [1, 3, 6, 12])                       # FMA body with 1 and 4 rows, mma.sync with 8 and 16
 @pytest.mark.parametrize("split", [1, 2, 3, 4, 5, 6, 7, 8])
 def test_any_split_k_gives_the_same_answer(S, split, B):
     # cluster sizes that do not divide the column tile leave the last rank with fewer columns
@@ -314,6 +329,17 @@ def test_tcgen05_kernel_matches_the_oracle(S, K, N, B, dt, split):
     finally:
         S.scap_tune("tcgen05", 1)
         S.scap_tune("split_k", 0)
+
+
+@pytest.mark.parametrize("K,N,B,dt", [(777, 520, 3, si.BF16), (300, 4096, 4, si.BF16), (2048, 1032, 4, si.F16), (33, 8, 3, si.F16)])
+def test_batch_three_and_four_on_the_mma_sync_route(S, K, N, B, dt):
+    d = si.laplace_fc(4, K, N, dt, 32, B)
+    tau = oracle.tau(si.to_f32(d["x_calib"], dt), d["m_true"], 0.6)
+    try:
+        set_route(S, "mma_sync")
+        check_fc(S, d, d["m_true"], tau)
+    finally:
+        reset_route(S)
 
 
 def test_tcgen05_and_mma_sync_paths_agree_closely(S):

@@ -78,7 +78,7 @@ def check_glu(S, g, c, B=None):
     return keep2.mean()
 
 
-@pytest.mark.parametrize("D,F,B", [(256, 512, 1), (200, 264, 3), (512, 1000, 8), (64, 8, 2), (1024, 776, 16)])
+@pytest.mark.parametrize("D,F,B", [(256, 512, 1), (200, 264, 3), (304, 520, 4), (512, 1000, 8), (64, 8, 2), (1024, 776, 16)])
 def test_glu_small_shapes(S, D, F, B):
     g = si.glu_block(2, D, F, si.BF16, 64, B)
     c = calibrate_glu(g, 0.4, 0.7)
