@@ -463,12 +463,12 @@ def suite_gelu(torch, scap, peak, out):
 
 
 def suite_moe(torch, scap, peak, out):
-    """Config 3: Mixtral-8x7B-shaped MoE layer, 8 experts, top-2, batch 1..4, 40 % / 60 % targets."""
+    """Config 3: Mixtral-8x7B-shaped MoE layer, 8 experts, top-2, batch 1..8, 40 % / 60 % targets."""
     D, F, E = 4096, 14336, 8
     dt = si.BF16
     stream = torch.cuda.Stream()
-    mo = si.moe_layer(3, D, F, E, dt, 2048, 64)
-    ws = torch.empty(max(scap.scap_moe_workspace(4, D, F, E, 2), scap.scap_glu_workspace(16, D, F),
+    mo = si.moe_layer(3, D, F, E, dt, 2048, 128)
+    ws = torch.empty(max(scap.scap_moe_workspace(8, D, F, E, 2), scap.scap_glu_workspace(16, D, F),
                          scap.scap_calibrate_workspace(2048, F, NBINS)), dtype=torch.uint8, device="cuda")
     experts = []
     ytmp = torch.empty((16, D), dtype=torch.float32, device="cuda")
@@ -488,10 +488,10 @@ def suite_moe(torch, scap, peak, out):
         experts.append(t)
     hs = si.as_torch(mo["h"], dt).cuda()
     logits = torch.from_numpy(mo["logits"]).cuda()
-    for B in (1, 2, 4):
+    for B in (1, 2, 4, 8):
         y = torch.empty((B, D), dtype=torch.float32, device="cuda")
-        hb = [hs[i * 4:i * 4 + B] for i in range(16)]
-        lb = [logits[i * 4:i * 4 + B].contiguous() for i in range(16)]
+        hb = [hs[i * 8:i * 8 + B] for i in range(16)]
+        lb = [logits[i * 8:i * 8 + B].contiguous() for i in range(16)]
         t = _time_graph(torch, stream, lambda: [scap.scap_moe_ffn(hb[r], lb[r], experts, 2, y, ws) for r in range(16)]) / 16
         sel = [len(set(torch.topk(lb[r], 2, dim=1).indices.flatten().tolist())) for r in range(16)]
         out({"suite": "moe", "D": D, "F": F, "E": E, "top_k": 2, "B": B, "targets": [0.4, 0.6], "us_per_call": round(t, 2),

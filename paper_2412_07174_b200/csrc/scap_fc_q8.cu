@@ -84,14 +84,15 @@ __global__ void __launch_bounds__(FC_THREADS, 2) fc_q8_kernel(const FcArgs a) {
     }
     for (int j0 = 0; j0 < my_chunks; j0 += CAPC) {
         const int nj = min(CAPC, my_chunks - j0);
+        const int pw = (nj + FC_WARPS - 1) / FC_WARPS;  // chunks per warp this fill: warp w owns chunks w * pw .. w * pw + pw - 1
         XT xraw[PU][BT];
         float xv[PU][BT], mk[PU], sc[PU];
 #pragma unroll
         for (int p = 0; p < PU; ++p) {
-            const int j = warp * PU + p;
+            const int j = warp * pw + p;
             const int k = (s + S * (j0 + j)) * 32 + lane;
-            mk[p] = a.m ? ld_nc_if(a.m + k, j < nj && k < K) : 0.0f;
-            sc[p] = ld_nc_if(a.wscale + k, j < nj && k < K);
+            mk[p] = a.m ? ld_nc_if(a.m + k, p < pw && j < nj && k < K) : 0.0f;
+            sc[p] = ld_nc_if(a.wscale + k, p < pw && j < nj && k < K);
         }
         if (j0 == 0 && !a.hold_dependents) {
             griddep_wait();
@@ -99,9 +100,9 @@ __global__ void __launch_bounds__(FC_THREADS, 2) fc_q8_kernel(const FcArgs a) {
         }
 #pragma unroll
         for (int p = 0; p < PU; ++p) {
-            const int j = warp * PU + p;
+            const int j = warp * pw + p;
             const int k = (s + S * (j0 + j)) * 32 + lane;
-            const bool ok = j < nj && k < K;
+            const bool ok = p < pw && j < nj && k < K;
 #pragma unroll
             for (int b = 0; b < BT; ++b) xraw[p][b] = ld_act_if(xg + (size_t)(b < B ? b : 0) * a.x_ld + k, ok && b < B);
         }
@@ -113,9 +114,9 @@ __global__ void __launch_bounds__(FC_THREADS, 2) fc_q8_kernel(const FcArgs a) {
         unsigned bal[PU];
 #pragma unroll
         for (int p = 0; p < PU; ++p) {
-            const int j = warp * PU + p;
+            const int j = warp * pw + p;
             const int k = (s + S * (j0 + j)) * 32 + lane;
-            const bool ok = j < nj && k < K;
+            const bool ok = p < pw && j < nj && k < K;
             uint32_t m_ = 0;
 #pragma unroll
             for (int b = 0; b < BT; ++b) {
@@ -141,8 +142,8 @@ __global__ void __launch_bounds__(FC_THREADS, 2) fc_q8_kernel(const FcArgs a) {
             unsigned mine = 0;
 #pragma unroll
             for (int p = 0; p < PU; ++p) mine = lane == p ? bal[p] : mine;
-            const int j = warp * PU + lane;
-            if (lane < PU && j < nj) a.bits[s + S * (j0 + j)] = mine;
+            const int j = warp * pw + lane;
+            if (lane < pw && j < nj) a.bits[s + S * (j0 + j)] = mine;
         }
         __syncthreads();
         int cnt = 0, wbase = 0;
@@ -156,7 +157,7 @@ __global__ void __launch_bounds__(FC_THREADS, 2) fc_q8_kernel(const FcArgs a) {
 #pragma unroll
         for (int p = 0; p < PU; ++p) {
             if (km[p]) {
-                const int j = warp * PU + p;
+                const int j = warp * pw + p;
                 const int pos = wbase + my_off[p] + __popc(bal[p] & ((1u << lane) - 1u));
                 s_k[pos] = (uint32_t)((s + S * (j0 + j)) * 32 + lane);
 #pragma unroll

@@ -79,6 +79,7 @@ __global__ void __launch_bounds__(64) moe_route_kernel(const float *__restrict__
 template <bool BF16, int BT, int STAGE, int TNT>
 __global__ void __launch_bounds__(FC_THREADS, fc_min_blocks(BT)) moe_fc_kernel(const MoeArgs a) {
     using ST = typename std::conditional<BF16, __nv_bfloat16, __half>::type;
+    static_assert(fc_smem_for(BT) >= fc_smem_bytes(BT <= 4 ? BT : 4), "the FMA bodies for small experts use the kernel's shared memory");
     griddep_wait();
     griddep_launch_dependents();
     const int e = blockIdx.z;
@@ -95,9 +96,10 @@ __global__ void __launch_bounds__(FC_THREADS, fc_min_blocks(BT)) moe_fc_kernel(c
         g.x = a.h; g.x_ld = a.D; g.in_rows = a.route->rows[e];
         g.m = a.ex[e].m1; g.tau = a.ex[e].tau1; g.bias = a.ex[e].bgu_fused;
         g.y = z; g.y_ld = a.F;
-        // an expert that got one or two rows of a larger batch takes the FMA body (cluster-uniform choice)
+        // an expert that got up to four rows of a larger batch takes the FMA body (cluster-uniform choice)
         if constexpr (is_mma(BT)) {
             if (nb <= 2) fc_body<BF16, 2, MODE_GATHER, ST, EPI_GLU, TNT>(g, blockIdx.x, blockIdx.y, false);
+            else if (nb <= 4) fc_body<BF16, 4, MODE_GATHER, ST, EPI_GLU, TNT>(g, blockIdx.x, blockIdx.y, false);
             else fc_body_mma<BF16, BT, MODE_GATHER, ST, EPI_GLU, TNT>(g, blockIdx.x, blockIdx.y, false);
         } else {
             fc_body<BF16, BT, MODE_GATHER, ST, EPI_GLU, TNT>(g, blockIdx.x, blockIdx.y, false);
@@ -109,6 +111,7 @@ __global__ void __launch_bounds__(FC_THREADS, fc_min_blocks(BT)) moe_fc_kernel(c
         g.y = a.yslot; g.y_ld = a.D; g.out_rows = a.route->slots[e];
         if constexpr (is_mma(BT)) {
             if (nb <= 2) fc_body<BF16, 2, MODE_GATHER, float, EPI_BIAS, TNT>(g, blockIdx.x, blockIdx.y, false);
+            else if (nb <= 4) fc_body<BF16, 4, MODE_GATHER, float, EPI_BIAS, TNT>(g, blockIdx.x, blockIdx.y, false);
             else fc_body_mma<BF16, BT, MODE_GATHER, float, EPI_BIAS, TNT>(g, blockIdx.x, blockIdx.y, false);
         } else {
             fc_body<BF16, BT, MODE_GATHER, float, EPI_BIAS, TNT>(g, blockIdx.x, blockIdx.y, false);
