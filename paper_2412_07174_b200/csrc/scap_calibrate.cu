@@ -193,53 +193,68 @@ __global__ void __launch_bounds__(CAL_THREADS) mode_kernel(const uint16_t *__res
 
 // Later radix passes: histogram of the next `width` key bits over the elements whose higher bits equal
 // the prefix of order statistic j (hist[0]) or j+1 (hist[1]).
+// A CTA owns a block of 256 channels (32 lanes x 8 channels: a warp reads 512 contiguous bytes of a row) and the
+// rows blockIdx.y * 8 + ty, stepping by 8 * gridDim.y; the modes of a thread's 8 channels stay in registers.
+// With t = key - (prefix << (shift + width)) as unsigned, the higher bits match iff t < 2^(shift + width), and
+// t >> shift is then the bucket.  The two order statistics are neighbours and nearly always share their prefix:
+// then one histogram is counted and added to both outputs.
+constexpr int RP_U = 8;  // 16-byte loads in flight per thread
 template <bool BF16>
-__global__ void __launch_bounds__(256) radix_pass_kernel(const uint16_t *__restrict__ x, const float *__restrict__ m, long long M8,
+__global__ void __launch_bounds__(256) radix_pass_kernel(const uint16_t *__restrict__ x, const float *__restrict__ m, int T,
                                                          int K, const SelState *__restrict__ st, int shift, int width,
                                                          uint32_t *__restrict__ hist) {
     __shared__ uint32_t s_h[2][RADIX_BINS];
     for (int i = threadIdx.x; i < 2 * RADIX_BINS; i += blockDim.x) (&s_h[0][0])[i] = 0;
+    const int sh = shift + width;
     const uint32_t p0 = st->prefix[0], p1 = st->prefix[1];
-    const uint32_t mask = (1u << width) - 1u;
+    const uint32_t base0 = p0 << sh, base1 = p1 << sh, span = 1u << sh;
+    const bool same = p0 == p1;
+    const int kc = (blockIdx.x * 32 + (threadIdx.x & 31)) * 8;
+    const int ty = threadIdx.x >> 5;
+    float mk[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) mk[j] = 0.0f;
+    if (kc < K) {
+        const float4 ma = __ldg(reinterpret_cast<const float4 *>(m + kc)), mb = __ldg(reinterpret_cast<const float4 *>(m + kc + 4));
+        mk[0] = ma.x; mk[1] = ma.y; mk[2] = ma.z; mk[3] = ma.w;
+        mk[4] = mb.x; mk[5] = mb.y; mk[6] = mb.z; mk[7] = mb.w;
+    }
     __syncthreads();
-    constexpr int RU = 4;  // 16-byte loads in flight per thread
-    const long long stride = (long long)gridDim.x * blockDim.x;
-    for (long long i0 = (long long)blockIdx.x * blockDim.x + threadIdx.x; i0 < M8; i0 += stride * RU) {
-        uint4 v[RU];
-        float4 ma[RU], mb[RU];
+    if (kc < K) {
+        const int step = 8 * gridDim.y;
+        const uint16_t *xp = x + kc;
+        for (int t0 = blockIdx.y * 8 + ty; t0 < T; t0 += step * RP_U) {
+            uint4 v[RP_U];
 #pragma unroll
-        for (int u = 0; u < RU; ++u) {
-            const long long i = i0 + stride * u;
-            v[u] = make_uint4(0, 0, 0, 0);
-            ma[u] = mb[u] = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (i < M8) {
-                v[u] = __ldg(reinterpret_cast<const uint4 *>(x) + i);
-                const int kc = (int)((i * 8) % K);
-                ma[u] = __ldg(reinterpret_cast<const float4 *>(m + kc));
-                mb[u] = __ldg(reinterpret_cast<const float4 *>(m + kc + 4));
+            for (int u = 0; u < RP_U; ++u) {
+                const int t = t0 + step * u;
+                v[u] = make_uint4(0, 0, 0, 0);
+                if (t < T) v[u] = __ldg(reinterpret_cast<const uint4 *>(xp + (size_t)t * K));
             }
-        }
 #pragma unroll
-        for (int u = 0; u < RU; ++u) {
-            if (i0 + stride * u < M8) {
-                float f[8];
-                widen8<BF16>(v[u], f);
-                const float mk[8] = {ma[u].x, ma[u].y, ma[u].z, ma[u].w, mb[u].x, mb[u].y, mb[u].z, mb[u].w};
+            for (int u = 0; u < RP_U; ++u) {
+                if (t0 + step * u < T) {
+                    float f[8];
+                    widen8<BF16>(v[u], f);
 #pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    const uint32_t key = __float_as_uint(__fsub_rn(f[j], mk[j])) & 0x7fffffffu;
-                    const uint32_t hi = key >> (shift + width);
-                    const uint32_t b = (key >> shift) & mask;
-                    if (hi == p0) atomicAdd(&s_h[0][b], 1u);
-                    if (hi == p1) atomicAdd(&s_h[1][b], 1u);
+                    for (int j = 0; j < 8; ++j) {
+                        const uint32_t key = __float_as_uint(__fsub_rn(f[j], mk[j])) & 0x7fffffffu;
+                        const uint32_t d0 = key - base0;
+                        if (d0 < span) atomicAdd(&s_h[0][d0 >> shift], 1u);
+                        if (!same) {
+                            const uint32_t d1 = key - base1;
+                            if (d1 < span) atomicAdd(&s_h[1][d1 >> shift], 1u);
+                        }
+                    }
                 }
             }
         }
     }
     __syncthreads();
-    for (int i = threadIdx.x; i < 2 * RADIX_BINS; i += blockDim.x) {
-        const uint32_t v = (&s_h[0][0])[i];
-        if (v) atomicAdd(&hist[i], v);
+    for (int i = threadIdx.x; i < RADIX_BINS; i += blockDim.x) {
+        const uint32_t c0 = s_h[0][i], c1 = same ? c0 : s_h[1][i];
+        if (c0) atomicAdd(&hist[i], c0);
+        if (c1) atomicAdd(&hist[RADIX_BINS + i], c1);
     }
 }
 
@@ -636,7 +651,11 @@ static cudaError_t estimate_mode(const uint16_t *x, int T, int K, int estimator,
     uint32_t *phist = reinterpret_cast<uint32_t *>(ws + L.pool_hist);
     double *col_sum = reinterpret_cast<double *>(ws + L.col_sum);
     const long long M = (long long)T * K, M8 = M / 8;
-    const int grid = sm_count() * 4;
+    // radix passes: 256 channels per CTA column, enough row slabs for about four CTAs per SM
+    const int gx = (K + 255) / 256;
+    int gy = (sm_count() * 4 + gx - 1) / gx;
+    if (gy > (T + 7) / 8) gy = (T + 7) / 8;
+    const dim3 grid(gx, gy < 1 ? 1 : gy);
     cudaError_t e = cudaSuccess;
     if (!scalar) {
         if (estimator == 1) return launch(mean_kernel<BF16>, dim3((K + 31) / 32), dim3(256), 0, st, false, x, T, K, m_out, (double *)nullptr);
@@ -707,18 +726,22 @@ static scap_status calibrate_t(const uint16_t *x, int T, int K, double sparsity,
     if (j > M - 1) j = M - 1;
     const double frac = pos - (double)j;
     const long long j1 = j + 1 < M ? j + 1 : M - 1;
-    const int grid = sm_count() * 4;
+    // radix passes: 256 channels per CTA column, enough row slabs for about four CTAs per SM
+    const int gx = (K + 255) / 256;
+    int gy = (sm_count() * 4 + gx - 1) / gx;
+    if (gy > (T + 7) / 8) gy = (T + 7) / 8;
+    const dim3 grid(gx, gy < 1 ? 1 : gy);
     // pass A (bits 30..20) was accumulated by mode_kernel
     e = launch(select_kernel, dim3(1), dim3(256), 0, st, false, (const uint32_t *)hist, RADIX_BINS, 11, 1, 0, (uint32_t)j,
                (uint32_t)j1, frac, state, tau_out);
     if (e != cudaSuccess) return cuda_status(e);
-    e = launch(radix_pass_kernel<BF16>, dim3(grid), dim3(256), 0, st, false, x, (const float *)m_out, M / 8, K,
+    e = launch(radix_pass_kernel<BF16>, grid, dim3(256), 0, st, false, x, (const float *)m_out, T, K,
                (const SelState *)state, 9, 11, hist + 2 * RADIX_BINS);
     if (e != cudaSuccess) return cuda_status(e);
     e = launch(select_kernel, dim3(1), dim3(256), 0, st, false, (const uint32_t *)(hist + 2 * RADIX_BINS), RADIX_BINS, 11, 0, 0,
                0u, 0u, frac, state, tau_out);
     if (e != cudaSuccess) return cuda_status(e);
-    e = launch(radix_pass_kernel<BF16>, dim3(grid), dim3(256), 0, st, false, x, (const float *)m_out, M / 8, K,
+    e = launch(radix_pass_kernel<BF16>, grid, dim3(256), 0, st, false, x, (const float *)m_out, T, K,
                (const SelState *)state, 0, 9, hist + 4 * RADIX_BINS);
     if (e != cudaSuccess) return cuda_status(e);
     e = launch(select_kernel, dim3(1), dim3(256), 0, st, false, (const uint32_t *)(hist + 4 * RADIX_BINS), 512, 9, 0, 1, 0u, 0u,
