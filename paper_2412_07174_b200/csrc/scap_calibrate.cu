@@ -43,15 +43,46 @@ __device__ __forceinline__ int load_rows(const uint16_t *xp, int K, int T, int t
     return valid;
 }
 
+// Rotates the 8 channels of a 16-byte row piece by r places: channel i of the result is channel (i + r) mod 8 of v.
+// Branch-free (r differs between the lanes of a warp).
+__device__ __forceinline__ uint4 rotate_channels(const uint4 &v, int r) {
+    uint32_t w0 = v.x, w1 = v.y, w2 = v.z, w3 = v.w;
+    {
+        const bool on = (r & 1) != 0;  // one channel = 16 bits
+        const uint32_t t0 = __funnelshift_r(w0, w1, 16), t1 = __funnelshift_r(w1, w2, 16);
+        const uint32_t t2 = __funnelshift_r(w2, w3, 16), t3 = __funnelshift_r(w3, w0, 16);
+        w0 = on ? t0 : w0; w1 = on ? t1 : w1; w2 = on ? t2 : w2; w3 = on ? t3 : w3;
+    }
+    {
+        const bool on = (r & 2) != 0;  // two channels = one word
+        const uint32_t t0 = w1, t1 = w2, t2 = w3, t3 = w0;
+        w0 = on ? t0 : w0; w1 = on ? t1 : w1; w2 = on ? t2 : w2; w3 = on ? t3 : w3;
+    }
+    {
+        const bool on = (r & 4) != 0;  // four channels = two words
+        const uint32_t t0 = w2, t1 = w3, t2 = w0, t3 = w1;
+        w0 = on ? t0 : w0; w1 = on ? t1 : w1; w2 = on ? t2 : w2; w3 = on ? t3 : w3;
+    }
+    return make_uint4(w0, w1, w2, w3);
+}
+
 // One CTA per strip of CW channels: min/max, histogram, arg-max -> m; then the first radix histogram
 // (bits 30..20 of |x - m|) of the strip is added to hist_a.
+//
+// Histogram layout: the two 16-bit counters of bins 2h and 2h+1 of channel c share word h * CW + c, so the bank of
+// a counter is its channel.  A warp holds 8 rows x 4 pieces of 8 channels; each lane rotates its 8 channels by its
+// row number, so that in every step of the unrolled loop the 32 lanes of a warp update 32 different channels:
+// no two lanes ever meet in a bank, whatever the bins.
 template <bool BF16>
 __global__ void __launch_bounds__(CAL_THREADS) mode_kernel(const uint16_t *__restrict__ x, int T, int K, int nbins,
                                                            float *__restrict__ m_out, uint32_t *__restrict__ hist_a,
                                                            int want_hist, const float *__restrict__ m_given) {
+    constexpr int NW = CAL_THREADS / 32;
     extern __shared__ __align__(16) uint32_t smem[];
     __shared__ float s_lo[CW], s_hi[CW], s_m[CW];
+    __shared__ float s_wlo[NW][CW], s_whi[NW][CW];  // per-warp partial min / max, later partial arg-max (count, bin)
     const int tid = threadIdx.x, q = tid & 3, rl = tid >> 2;
+    const int lane = tid & 31, warp = tid >> 5, r = lane >> 2;
     const int k0 = blockIdx.x * CW;
     const int kc = k0 + q * 8;
     const bool ok = kc < K;  // K is a multiple of 8
@@ -67,7 +98,7 @@ __global__ void __launch_bounds__(CAL_THREADS) mode_kernel(const uint16_t *__res
         if (tid < CW) s_m[tid] = k0 + tid < K ? __ldcg(m_given + k0 + tid) : 0.0f;
         __syncthreads();
     } else if (nbins > 0) {
-        // ---- pass 1: per-channel min / max
+        // ---- pass 1: per-channel min / max (thread -> 8 rows of the warp by shuffles -> warps through shared memory)
         float lo[8], hi[8];
 #pragma unroll
         for (int j = 0; j < 8; ++j) { lo[j] = INFINITY; hi[j] = -INFINITY; }
@@ -84,31 +115,42 @@ __global__ void __launch_bounds__(CAL_THREADS) mode_kernel(const uint16_t *__res
                     }
                 }
             }
-        float *s_mm = reinterpret_cast<float *>(smem);  // [2][CAL_ROWS][CW]
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            s_mm[rl * CW + q * 8 + j] = lo[j];
-            s_mm[(CAL_ROWS + rl) * CW + q * 8 + j] = hi[j];
+        for (int o = 4; o < 32; o <<= 1)
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                lo[j] = fminf(lo[j], __shfl_xor_sync(0xffffffffu, lo[j], o));
+                hi[j] = fmaxf(hi[j], __shfl_xor_sync(0xffffffffu, hi[j], o));
+            }
+        if (lane < 4) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                s_wlo[warp][q * 8 + j] = lo[j];
+                s_whi[warp][q * 8 + j] = hi[j];
+            }
         }
         __syncthreads();
         if (tid < CW) {
             float l = INFINITY, h = -INFINITY;
-            for (int r = 0; r < CAL_ROWS; ++r) { l = fminf(l, s_mm[r * CW + tid]); h = fmaxf(h, s_mm[(CAL_ROWS + r) * CW + tid]); }
+#pragma unroll
+            for (int w = 0; w < NW; ++w) { l = fminf(l, s_wlo[w][tid]); h = fmaxf(h, s_whi[w][tid]); }
             s_lo[tid] = l;
             s_hi[tid] = h;
         }
-        __syncthreads();
         // ---- pass 2: histogram; two 16-bit counters per word (a count never exceeds T <= 65535)
         const int HW = (nbins + 1) / 2;
         for (int i = tid; i < CW * HW; i += CAL_THREADS) smem[i] = 0;
-        float scale[8];
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            lo[j] = s_lo[q * 8 + j];
-            hi[j] = s_hi[q * 8 + j];
-            scale[j] = hi[j] != lo[j] ? __fdiv_rn((float)nbins, __fsub_rn(hi[j], lo[j])) : 0.0f;
-        }
         __syncthreads();
+        // this lane's channels in rotated order: slot i holds channel q * 8 + (i + r) mod 8
+        float scale[8];
+        int cidx[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            cidx[i] = q * 8 + ((i + r) & 7);
+            lo[i] = s_lo[cidx[i]];
+            hi[i] = s_hi[cidx[i]];
+            scale[i] = hi[i] != lo[i] ? __fdiv_rn((float)nbins, __fsub_rn(hi[i], lo[i])) : 0.0f;
+        }
         if (ok)
             for (int t0 = rl; t0 < T; t0 += CAL_ROWS * CAL_U) {
                 if (!resident) nv = load_rows(xp, K, T, t0, v);
@@ -116,44 +158,51 @@ __global__ void __launch_bounds__(CAL_THREADS) mode_kernel(const uint16_t *__res
                 for (int u = 0; u < CAL_U; ++u) {
                     if (u < nv) {
                         float f[8];
-                        widen8<BF16>(v[u], f);
+                        widen8<BF16>(rotate_channels(v[u], r), f);
 #pragma unroll
-                        for (int j = 0; j < 8; ++j) {
-                            if (hi[j] != lo[j]) {
-                                int i = (int)floorf(__fmul_rn(__fsub_rn(f[j], lo[j]), scale[j]));
-                                i = min(max(i, 0), nbins - 1);
-                                atomicAdd(&smem[(q * 8 + j) * HW + (i >> 1)], 1u << ((i & 1) * 16));
+                        for (int i = 0; i < 8; ++i) {
+                            if (hi[i] != lo[i]) {
+                                int b = (int)floorf(__fmul_rn(__fsub_rn(f[i], lo[i]), scale[i]));
+                                b = min(max(b, 0), nbins - 1);
+                                atomicAdd(&smem[(b >> 1) * CW + cidx[i]], 1u << ((b & 1) * 16));
                             }
                         }
                     }
                 }
             }
         __syncthreads();
-        // ---- arg-max: lowest bin with the largest count; warp w takes channels 2w, 2w+1
-        const int lane = tid & 31, warp = tid >> 5;
-        for (int c = warp * (CW / (CAL_THREADS / 32)); c < (warp + 1) * (CW / (CAL_THREADS / 32)); ++c) {
+        // ---- arg-max: lowest bin with the largest count.  Lane = channel; warp w scans its share of the bin pairs
+        // in ascending order, then thread c combines the warps in ascending order (strict >: the first maximum stays).
+        {
+            const int per = (HW + NW - 1) / NW;
             uint32_t best_cnt = 0;
             int best_i = 0;
-            for (int i = lane; i < nbins; i += 32) {
-                const uint32_t cnt = (smem[c * HW + (i >> 1)] >> ((i & 1) * 16)) & 0xffffu;
-                if (cnt > best_cnt) { best_cnt = cnt; best_i = i; }  // ascending i: first maximum kept
+            for (int h = warp * per; h < min(HW, (warp + 1) * per); ++h) {
+                const uint32_t wv = smem[h * CW + lane];
+                const uint32_t c0 = wv & 0xffffu, c1 = wv >> 16;  // bin 2h + 1 beyond nbins was never counted
+                if (c0 > best_cnt) { best_cnt = c0; best_i = 2 * h; }
+                if (c1 > best_cnt) { best_cnt = c1; best_i = 2 * h + 1; }
             }
+            s_wlo[warp][lane] = __uint_as_float(best_cnt);
+            s_whi[warp][lane] = __int_as_float(best_i);
+        }
+        __syncthreads();
+        if (tid < CW) {
+            uint32_t best_cnt = 0;
+            int best_i = 0;
 #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) {
-                const uint32_t oc = __shfl_xor_sync(0xffffffffu, best_cnt, o);
-                const int oi = __shfl_xor_sync(0xffffffffu, best_i, o);
-                if (oc > best_cnt || (oc == best_cnt && oi < best_i)) { best_cnt = oc; best_i = oi; }
+            for (int w = 0; w < NW; ++w) {
+                const uint32_t c = __float_as_uint(s_wlo[w][tid]);
+                if (c > best_cnt) { best_cnt = c; best_i = __float_as_int(s_whi[w][tid]); }
             }
-            if (lane == 0) {
-                const float l = s_lo[c], h = s_hi[c];
-                float mv = l;
-                if (h != l) {
-                    const float w = __fmul_rn(__fsub_rn(h, l), __fdiv_rn(1.0f, (float)nbins));
-                    mv = __fadd_rn(l, __fmul_rn(__fadd_rn((float)best_i, 0.5f), w));
-                }
-                s_m[c] = mv;
-                if (k0 + c < K) m_out[k0 + c] = mv;
+            const float l = s_lo[tid], h = s_hi[tid];
+            float mv = l;
+            if (h != l) {
+                const float w = __fmul_rn(__fsub_rn(h, l), __fdiv_rn(1.0f, (float)nbins));
+                mv = __fadd_rn(l, __fmul_rn(__fadd_rn((float)best_i, 0.5f), w));
             }
+            s_m[tid] = mv;
+            if (k0 + tid < K) m_out[k0 + tid] = mv;
         }
         __syncthreads();
     } else {
@@ -164,12 +213,15 @@ __global__ void __launch_bounds__(CAL_THREADS) mode_kernel(const uint16_t *__res
         __syncthreads();
     }
     if (!want_hist) return;
-    // ---- pass 3: first radix histogram of the importance |x - m|
-    for (int i = tid; i < RADIX_BINS; i += CAL_THREADS) smem[i] = 0;
+    // ---- pass 3: first radix histogram of the importance |x - m|.  The keys crowd into a few dozen buckets (the
+    // top 11 bits are the exponent and three mantissa bits), so the four lanes that share a row count into four
+    // copies of the histogram, each shifted by 8 banks against the previous one.
+    for (int i = tid; i < 4 * RADIX_BINS; i += CAL_THREADS) smem[i] = 0;
     float mk[8];
 #pragma unroll
     for (int j = 0; j < 8; ++j) mk[j] = s_m[q * 8 + j];
     __syncthreads();
+    uint32_t *hq = smem + q * RADIX_BINS;
     if (ok)
         for (int t0 = rl; t0 < T; t0 += CAL_ROWS * CAL_U) {
             if (!resident) nv = load_rows(xp, K, T, t0, v);
@@ -181,18 +233,82 @@ __global__ void __launch_bounds__(CAL_THREADS) mode_kernel(const uint16_t *__res
 #pragma unroll
                     for (int j = 0; j < 8; ++j) {
                         const uint32_t key = __float_as_uint(__fsub_rn(f[j], mk[j])) & 0x7fffffffu;
-                        atomicAdd(&smem[key >> 20], 1u);
+                        atomicAdd(&hq[((key >> 20) + 8 * q) & (RADIX_BINS - 1)], 1u);
                     }
                 }
             }
         }
     __syncthreads();
-    for (int i = tid; i < RADIX_BINS; i += CAL_THREADS)
-        if (smem[i]) atomicAdd(&hist_a[i], smem[i]);
+    for (int i = tid; i < RADIX_BINS; i += CAL_THREADS) {
+        uint32_t c = 0;
+#pragma unroll
+        for (int qq = 0; qq < 4; ++qq) c += smem[qq * RADIX_BINS + ((i + 8 * qq) & (RADIX_BINS - 1))];
+        if (c) atomicAdd(&hist_a[i], c);
+    }
 }
 
-// Later radix passes: histogram of the next `width` key bits over the elements whose higher bits equal
+// Block-wide bucket search (256 threads): for the order statistics w = 0, 1, finds in the nb counters h[w] (nb a
+// multiple of 256, at most 2048) the bucket that holds rank[w] (0-based among the counted keys) and rebases the rank
+// to that bucket.  Every thread returns both results.  Thread t adds its nb / 256 consecutive counters, the block
+// scans the 256 sums, and the one thread whose stretch contains the rank walks its own counters.
+struct SelPick {
+    uint32_t bucket[2], rank[2];
+};
+__device__ __forceinline__ SelPick block_select(const uint32_t *const (&h)[2], int nb, const uint32_t (&rank)[2]) {
+    __shared__ uint32_t s_wsum[2][8];
+    __shared__ uint32_t s_pick[2][2];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int per = nb >> 8;  // 1 .. 8
+    uint32_t cnt[2][8], incl[2];
+#pragma unroll
+    for (int w = 0; w < 2; ++w) {
+        uint32_t sum = 0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            cnt[w][i] = i < per ? __ldcg(h[w] + tid * per + i) : 0u;
+            sum += cnt[w][i];
+        }
+        uint32_t v = sum;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t t = __shfl_up_sync(0xffffffffu, v, o);
+            if (lane >= o) v += t;
+        }
+        incl[w] = v;
+        if (lane == 31) s_wsum[w][warp] = v;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int w = 0; w < 2; ++w) {
+        uint32_t before = 0;
+#pragma unroll
+        for (int q = 0; q < 8; ++q) before += q < warp ? s_wsum[w][q] : 0u;
+        uint32_t sum = 0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) sum += cnt[w][i];
+        uint32_t lo = before + incl[w] - sum;  // keys in the buckets before this thread's stretch
+        if (rank[w] >= lo && rank[w] < lo + sum) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                if (rank[w] >= lo && rank[w] < lo + cnt[w][i]) {
+                    s_pick[w][0] = (uint32_t)(tid * per + i);
+                    s_pick[w][1] = rank[w] - lo;
+                }
+                lo += cnt[w][i];
+            }
+        }
+    }
+    __syncthreads();
+    SelPick r;
+    r.bucket[0] = s_pick[0][0]; r.rank[0] = s_pick[0][1];
+    r.bucket[1] = s_pick[1][0]; r.rank[1] = s_pick[1][1];
+    return r;
+}
+
+// Radix passes after the first: histogram of the next `width` key bits over the elements whose higher bits equal
 // the prefix of order statistic j (hist[0]) or j+1 (hist[1]).
+// Each CTA first extends the two prefixes itself from the previous pass's counters (block_select: every CTA gets
+// the same answer, so no separate one-CTA kernel sits between two passes); CTA (0, 0) records them in st_out.
 // A CTA owns a block of 256 channels (32 lanes x 8 channels: a warp reads 512 contiguous bytes of a row) and the
 // rows blockIdx.y * 8 + ty, stepping by 8 * gridDim.y; the modes of a thread's 8 channels stay in registers.
 // With t = key - (prefix << (shift + width)) as unsigned, the higher bits match iff t < 2^(shift + width), and
@@ -201,19 +317,30 @@ __global__ void __launch_bounds__(CAL_THREADS) mode_kernel(const uint16_t *__res
 constexpr int RP_U = 8;  // 16-byte loads in flight per thread
 template <bool BF16>
 __global__ void __launch_bounds__(256) radix_pass_kernel(const uint16_t *__restrict__ x, const float *__restrict__ m, int T,
-                                                         int K, const SelState *__restrict__ st, int shift, int width,
+                                                         int K, const uint32_t *__restrict__ prev_hist, int prev_two,
+                                                         int prev_width, const SelState *__restrict__ st_in, uint32_t j,
+                                                         uint32_t j1, SelState *__restrict__ st_out, int shift, int width,
                                                          uint32_t *__restrict__ hist) {
     __shared__ uint32_t s_h[2][RADIX_BINS];
     for (int i = threadIdx.x; i < 2 * RADIX_BINS; i += blockDim.x) (&s_h[0][0])[i] = 0;
     const int sh = shift + width;
-    const uint32_t p0 = st->prefix[0], p1 = st->prefix[1];
+    // previous pass: one shared histogram (the first pass) or one per order statistic
+    const uint32_t *const ph[2] = {prev_hist, prev_two ? prev_hist + RADIX_BINS : prev_hist};
+    const uint32_t rk[2] = {st_in ? st_in->rank[0] : j, st_in ? st_in->rank[1] : j1};
+    const SelPick pick = block_select(ph, RADIX_BINS, rk);
+    const uint32_t p0 = ((st_in ? st_in->prefix[0] : 0u) << prev_width) | pick.bucket[0];
+    const uint32_t p1 = ((st_in ? st_in->prefix[1] : 0u) << prev_width) | pick.bucket[1];
+    if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) {
+        st_out->prefix[0] = p0; st_out->prefix[1] = p1;
+        st_out->rank[0] = pick.rank[0]; st_out->rank[1] = pick.rank[1];
+    }
     const uint32_t base0 = p0 << sh, base1 = p1 << sh, span = 1u << sh;
     const bool same = p0 == p1;
     const int kc = (blockIdx.x * 32 + (threadIdx.x & 31)) * 8;
     const int ty = threadIdx.x >> 5;
     float mk[8];
 #pragma unroll
-    for (int j = 0; j < 8; ++j) mk[j] = 0.0f;
+    for (int jj = 0; jj < 8; ++jj) mk[jj] = 0.0f;
     if (kc < K) {
         const float4 ma = __ldg(reinterpret_cast<const float4 *>(m + kc)), mb = __ldg(reinterpret_cast<const float4 *>(m + kc + 4));
         mk[0] = ma.x; mk[1] = ma.y; mk[2] = ma.z; mk[3] = ma.w;
@@ -237,8 +364,8 @@ __global__ void __launch_bounds__(256) radix_pass_kernel(const uint16_t *__restr
                     float f[8];
                     widen8<BF16>(v[u], f);
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        const uint32_t key = __float_as_uint(__fsub_rn(f[j], mk[j])) & 0x7fffffffu;
+                    for (int jj = 0; jj < 8; ++jj) {
+                        const uint32_t key = __float_as_uint(__fsub_rn(f[jj], mk[jj])) & 0x7fffffffu;
                         const uint32_t d0 = key - base0;
                         if (d0 < span) atomicAdd(&s_h[0][d0 >> shift], 1u);
                         if (!same) {
@@ -258,51 +385,18 @@ __global__ void __launch_bounds__(256) radix_pass_kernel(const uint16_t *__restr
     }
 }
 
-// One CTA.  Warp w (0 or 1) finds the bucket holding its order statistic in hist[first ? 0 : w], extends
-// the prefix by `width` bits and rebases the rank.  After the last pass thread 0 interpolates:
+// One CTA of 256 threads, after the last pass: finds the last `width` key bits of both order statistics in
+// hist[0] / hist[1] (nb counters each) and interpolates
 // tau = v_j + frac * (v_j1 - v_j) in binary64, each operation rounded once, then rounded to binary32.
-__global__ void select_kernel(const uint32_t *__restrict__ hist, int nb, int width, int first, int last, uint32_t j,
-                              uint32_t j1, double frac, SelState *__restrict__ st, float *__restrict__ tau_out) {
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    __shared__ uint32_t s_cnt[2][RADIX_BINS];  // the counts, fetched with all loads in flight (the scan below is serial)
-    for (int i = threadIdx.x; i < 2 * nb; i += blockDim.x) {
-        const int w = i / nb, b = i - w * nb;
-        s_cnt[w][b] = hist[(first ? 0 : w * RADIX_BINS) + b];
-    }
-    __syncthreads();
-    if (warp < 2) {
-        const uint32_t *h = s_cnt[warp];
-        const uint32_t rank = first ? (warp == 0 ? j : j1) : st->rank[warp];
-        const uint32_t prefix = first ? 0u : st->prefix[warp];
-        uint32_t carry = 0, found_b = 0, found_r = 0;
-        bool found = false;
-        for (int c0 = 0; c0 < nb && !found; c0 += 32) {
-            const uint32_t cnt = (c0 + lane < nb) ? h[c0 + lane] : 0u;
-            uint32_t v = cnt;
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const uint32_t t = __shfl_up_sync(0xffffffffu, v, o);
-                if (lane >= o) v += t;
-            }
-            const uint32_t incl = carry + v, excl = incl - cnt;
-            const unsigned hit = __ballot_sync(0xffffffffu, rank >= excl && rank < incl);
-            if (hit) {
-                const int src = __ffs(hit) - 1;
-                found_b = (uint32_t)(c0 + src);
-                found_r = rank - __shfl_sync(0xffffffffu, excl, src);
-                found = true;
-            }
-            carry = __shfl_sync(0xffffffffu, incl, 31);
-        }
-        if (lane == 0) {
-            st->prefix[warp] = (prefix << width) | found_b;
-            st->rank[warp] = found_r;
-        }
-    }
-    __syncthreads();
-    if (last && threadIdx.x == 0) {
-        const double vj = (double)__uint_as_float(st->prefix[0]);
-        const double vj1 = (double)__uint_as_float(st->prefix[1]);
+__global__ void __launch_bounds__(256) select_kernel(const uint32_t *__restrict__ hist, int nb, int width,
+                                                     const SelState *__restrict__ st_in, double frac,
+                                                     float *__restrict__ tau_out) {
+    const uint32_t *const ph[2] = {hist, hist + RADIX_BINS};
+    const uint32_t rk[2] = {st_in->rank[0], st_in->rank[1]};
+    const SelPick pick = block_select(ph, nb, rk);
+    if (threadIdx.x == 0) {
+        const double vj = (double)__uint_as_float((st_in->prefix[0] << width) | pick.bucket[0]);
+        const double vj1 = (double)__uint_as_float((st_in->prefix[1] << width) | pick.bucket[1]);
         const double t64 = __dadd_rn(vj, __dmul_rn(frac, __dsub_rn(vj1, vj)));
         *tau_out = (float)t64;
     }
@@ -651,11 +745,7 @@ static cudaError_t estimate_mode(const uint16_t *x, int T, int K, int estimator,
     uint32_t *phist = reinterpret_cast<uint32_t *>(ws + L.pool_hist);
     double *col_sum = reinterpret_cast<double *>(ws + L.col_sum);
     const long long M = (long long)T * K, M8 = M / 8;
-    // radix passes: 256 channels per CTA column, enough row slabs for about four CTAs per SM
-    const int gx = (K + 255) / 256;
-    int gy = (sm_count() * 4 + gx - 1) / gx;
-    if (gy > (T + 7) / 8) gy = (T + 7) / 8;
-    const dim3 grid(gx, gy < 1 ? 1 : gy);
+    const int grid = sm_count() * 4;
     cudaError_t e = cudaSuccess;
     if (!scalar) {
         if (estimator == 1) return launch(mean_kernel<BF16>, dim3((K + 31) / 32), dim3(256), 0, st, false, x, T, K, m_out, (double *)nullptr);
@@ -711,8 +801,7 @@ static scap_status calibrate_t(const uint16_t *x, int T, int K, double sparsity,
     }
     const int HW = (nbins + 1) / 2;
     size_t smem = (size_t)CW * HW * 4;
-    if (smem < (size_t)2 * CAL_ROWS * CW * 4) smem = (size_t)2 * CAL_ROWS * CW * 4;
-    if (smem < (size_t)RADIX_BINS * 4) smem = (size_t)RADIX_BINS * 4;
+    if (smem < (size_t)4 * RADIX_BINS * 4) smem = (size_t)4 * RADIX_BINS * 4;  // the four copies of the first radix histogram
     static SmemOptIn opt_in;
     e = ensure_dynamic_smem(mode_kernel<BF16>, 2048 / 2 * CW * 4, opt_in);
     if (e != cudaSuccess) return cuda_status(e);
@@ -731,21 +820,17 @@ static scap_status calibrate_t(const uint16_t *x, int T, int K, double sparsity,
     int gy = (sm_count() * 4 + gx - 1) / gx;
     if (gy > (T + 7) / 8) gy = (T + 7) / 8;
     const dim3 grid(gx, gy < 1 ? 1 : gy);
-    // pass A (bits 30..20) was accumulated by mode_kernel
-    e = launch(select_kernel, dim3(1), dim3(256), 0, st, false, (const uint32_t *)hist, RADIX_BINS, 11, 1, 0, (uint32_t)j,
-               (uint32_t)j1, frac, state, tau_out);
+    // pass A (bits 30..20) was accumulated by mode_kernel; each later pass first extends the prefixes from the
+    // counters of the pass before it
+    e = launch(radix_pass_kernel<BF16>, grid, dim3(256), 0, st, false, x, (const float *)m_out, T, K, (const uint32_t *)hist, 0,
+               11, (const SelState *)nullptr, (uint32_t)j, (uint32_t)j1, state, 9, 11, hist + 2 * RADIX_BINS);
     if (e != cudaSuccess) return cuda_status(e);
     e = launch(radix_pass_kernel<BF16>, grid, dim3(256), 0, st, false, x, (const float *)m_out, T, K,
-               (const SelState *)state, 9, 11, hist + 2 * RADIX_BINS);
+               (const uint32_t *)(hist + 2 * RADIX_BINS), 1, 11, (const SelState *)state, 0u, 0u, state + 1, 0, 9,
+               hist + 4 * RADIX_BINS);
     if (e != cudaSuccess) return cuda_status(e);
-    e = launch(select_kernel, dim3(1), dim3(256), 0, st, false, (const uint32_t *)(hist + 2 * RADIX_BINS), RADIX_BINS, 11, 0, 0,
-               0u, 0u, frac, state, tau_out);
-    if (e != cudaSuccess) return cuda_status(e);
-    e = launch(radix_pass_kernel<BF16>, grid, dim3(256), 0, st, false, x, (const float *)m_out, T, K,
-               (const SelState *)state, 0, 9, hist + 4 * RADIX_BINS);
-    if (e != cudaSuccess) return cuda_status(e);
-    e = launch(select_kernel, dim3(1), dim3(256), 0, st, false, (const uint32_t *)(hist + 4 * RADIX_BINS), 512, 9, 0, 1, 0u, 0u,
-               frac, state, tau_out);
+    e = launch(select_kernel, dim3(1), dim3(256), 0, st, false, (const uint32_t *)(hist + 4 * RADIX_BINS), 512, 9,
+               (const SelState *)(state + 1), frac, tau_out);
     return cuda_status(e);
 }
 
