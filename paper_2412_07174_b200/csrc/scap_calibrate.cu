@@ -161,11 +161,13 @@ __global__ void __launch_bounds__(CAL_THREADS) mode_kernel(const uint16_t *__res
                         widen8<BF16>(rotate_channels(v[u], r), f);
 #pragma unroll
                         for (int i = 0; i < 8; ++i) {
-                            if (hi[i] != lo[i]) {
-                                int b = (int)floorf(__fmul_rn(__fsub_rn(f[i], lo[i]), scale[i]));
-                                b = min(max(b, 0), nbins - 1);
-                                atomicAdd(&smem[(b >> 1) * CW + cidx[i]], 1u << ((b & 1) * 16));
-                            }
+                            // floor of the non-negative product without a conversion instruction: adding 2^23
+                            // rounding down leaves floor(v) in the mantissa (exact for 0 <= v < 2^23).  A constant
+                            // channel has scale 0 and counts into bin 0; its mode is set from lo below.
+                            const float vb = __fmul_rn(__fsub_rn(f[i], lo[i]), scale[i]);
+                            int b = __float_as_int(__fadd_rd(vb, 8388608.0f)) & 0x7fffff;
+                            b = min(b, nbins - 1);
+                            atomicAdd(&smem[(b >> 1) * CW + cidx[i]], 1u << ((b & 1) * 16));
                         }
                     }
                 }
@@ -177,11 +179,17 @@ __global__ void __launch_bounds__(CAL_THREADS) mode_kernel(const uint16_t *__res
             const int per = (HW + NW - 1) / NW;
             uint32_t best_cnt = 0;
             int best_i = 0;
-            for (int h = warp * per; h < min(HW, (warp + 1) * per); ++h) {
-                const uint32_t wv = smem[h * CW + lane];
-                const uint32_t c0 = wv & 0xffffu, c1 = wv >> 16;  // bin 2h + 1 beyond nbins was never counted
-                if (c0 > best_cnt) { best_cnt = c0; best_i = 2 * h; }
-                if (c1 > best_cnt) { best_cnt = c1; best_i = 2 * h + 1; }
+            const int h_end = min(HW, (warp + 1) * per);
+            for (int h0 = warp * per; h0 < h_end; h0 += 8) {
+                uint32_t wv[8];  // eight independent loads, then the ordered compares
+#pragma unroll
+                for (int e = 0; e < 8; ++e) wv[e] = h0 + e < h_end ? smem[(h0 + e) * CW + lane] : 0u;
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    const uint32_t c0 = wv[e] & 0xffffu, c1 = wv[e] >> 16;  // bin 2h + 1 beyond nbins was never counted
+                    if (c0 > best_cnt) { best_cnt = c0; best_i = 2 * (h0 + e); }
+                    if (c1 > best_cnt) { best_cnt = c1; best_i = 2 * (h0 + e) + 1; }
+                }
             }
             s_wlo[warp][lane] = __uint_as_float(best_cnt);
             s_whi[warp][lane] = __int_as_float(best_i);
