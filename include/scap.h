@@ -84,6 +84,8 @@ int scap_version(void);
  *              the call's kept channels in one pass, else mma.sync (default), 2 = always tcgen05
  *   "host_direct"  scap_sparse_fc_host: 1 = when x_host and y_host are page-locked and addressable by the
  *              device, a kernel pulls x and the FC kernel writes y to host memory (default), 0 = always copies
+ *   "cal_strip"  scap_calibrate: channels per CTA of the per-channel histogram kernel, 16 (default: 256 threads,
+ *              two CTAs per SM) or 32 (512 threads, one CTA per SM)
  * Unknown keys return SCAP_ERR_INVALID_ARG.  Tuning never changes what is computed; split_k
  * changes the (fixed) summation order and therefore the last bits of y.  Query workspace sizes
  * after tuning.                                                                               */

@@ -66,24 +66,30 @@ __device__ __forceinline__ uint4 rotate_channels(const uint4 &v, int r) {
     return make_uint4(w0, w1, w2, w3);
 }
 
-// One CTA per strip of CW channels: min/max, histogram, arg-max -> m; then the first radix histogram
+// One CTA per strip of CWT channels (32: 512 threads, one CTA per SM; 16: 256 threads, two CTAs per SM, finer
+// strips that spread better over the SMs): min/max, histogram, arg-max -> m; then the first radix histogram
 // (bits 30..20 of |x - m|) of the strip is added to hist_a.
 //
 // Histogram layout: the two 16-bit counters of bins 2h and 2h+1 of channel c share word h * CW + c, so the bank of
-// a counter is its channel.  A warp holds 8 rows x 4 pieces of 8 channels; each lane rotates its 8 channels by its
-// row number, so that in every step of the unrolled loop the 32 lanes of a warp update 32 different channels:
-// no two lanes ever meet in a bank, whatever the bins.
-template <bool BF16>
-__global__ void __launch_bounds__(CAL_THREADS) mode_kernel(const uint16_t *__restrict__ x, int T, int K, int nbins,
+// a counter is its channel (CWT = 32; with 16 channels two bin pairs share a row of banks).  A warp holds 8 rows x 4
+// pieces (16 rows x 2 pieces) of 8 channels; each lane rotates its 8 channels by its row number, so that in every
+// step of the unrolled loop the lanes of a warp update CWT different channels: with 32 channels no two lanes ever
+// meet in a bank, whatever the bins; with 16 channels two lanes can.
+template <bool BF16, int CWT>
+__global__ void __launch_bounds__(CWT * 16, CWT == 16 ? 2 : 1) mode_kernel(const uint16_t *__restrict__ x, int T, int K, int nbins,
                                                            float *__restrict__ m_out, uint32_t *__restrict__ hist_a,
                                                            int want_hist, const float *__restrict__ m_given) {
-    constexpr int NW = CAL_THREADS / 32;
+    griddep_wait();               // m_given and the cleared counters come from earlier work on the stream
+    griddep_launch_dependents();  // the next pass may become resident early; it waits for this grid itself
+    constexpr int QN = CWT / 8;        // 16-byte pieces per row of the strip
+    constexpr int NTH = QN * CAL_ROWS;  // threads: 128 rows per sweep
+    constexpr int NW = NTH / 32;
     extern __shared__ __align__(16) uint32_t smem[];
-    __shared__ float s_lo[CW], s_hi[CW], s_m[CW];
-    __shared__ float s_wlo[NW][CW], s_whi[NW][CW];  // per-warp partial min / max, later partial arg-max (count, bin)
-    const int tid = threadIdx.x, q = tid & 3, rl = tid >> 2;
-    const int lane = tid & 31, warp = tid >> 5, r = lane >> 2;
-    const int k0 = blockIdx.x * CW;
+    __shared__ float s_lo[CWT], s_hi[CWT], s_m[CWT];
+    __shared__ float s_wlo[NW][CWT], s_whi[NW][CWT];  // per-warp partial min / max, later partial arg-max (count, bin)
+    const int tid = threadIdx.x, q = tid % QN, rl = tid / QN;
+    const int lane = tid & 31, warp = tid >> 5, r = (lane / QN) & 7;
+    const int k0 = blockIdx.x * CWT;
     const int kc = k0 + q * 8;
     const bool ok = kc < K;  // K is a multiple of 8
     const uint16_t *xp = x + kc;
@@ -95,7 +101,7 @@ __global__ void __launch_bounds__(CAL_THREADS) mode_kernel(const uint16_t *__res
     if (resident && ok) nv = load_rows(xp, K, T, rl, v);
 
     if (m_given) {  // the mode was estimated by another kernel: only the radix histogram below is wanted
-        if (tid < CW) s_m[tid] = k0 + tid < K ? __ldcg(m_given + k0 + tid) : 0.0f;
+        if (tid < CWT) s_m[tid] = k0 + tid < K ? __ldcg(m_given + k0 + tid) : 0.0f;
         __syncthreads();
     } else if (nbins > 0) {
         // ---- pass 1: per-channel min / max (thread -> 8 rows of the warp by shuffles -> warps through shared memory)
@@ -116,13 +122,13 @@ __global__ void __launch_bounds__(CAL_THREADS) mode_kernel(const uint16_t *__res
                 }
             }
 #pragma unroll
-        for (int o = 4; o < 32; o <<= 1)
+        for (int o = QN; o < 32; o <<= 1)
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
                 lo[j] = fminf(lo[j], __shfl_xor_sync(0xffffffffu, lo[j], o));
                 hi[j] = fmaxf(hi[j], __shfl_xor_sync(0xffffffffu, hi[j], o));
             }
-        if (lane < 4) {
+        if (lane < QN) {
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
                 s_wlo[warp][q * 8 + j] = lo[j];
@@ -130,7 +136,7 @@ __global__ void __launch_bounds__(CAL_THREADS) mode_kernel(const uint16_t *__res
             }
         }
         __syncthreads();
-        if (tid < CW) {
+        if (tid < CWT) {
             float l = INFINITY, h = -INFINITY;
 #pragma unroll
             for (int w = 0; w < NW; ++w) { l = fminf(l, s_wlo[w][tid]); h = fmaxf(h, s_whi[w][tid]); }
@@ -139,7 +145,7 @@ __global__ void __launch_bounds__(CAL_THREADS) mode_kernel(const uint16_t *__res
         }
         // ---- pass 2: histogram; two 16-bit counters per word (a count never exceeds T <= 65535)
         const int HW = (nbins + 1) / 2;
-        for (int i = tid; i < CW * HW; i += CAL_THREADS) smem[i] = 0;
+        for (int i = tid; i < CWT * HW; i += NTH) smem[i] = 0;
         __syncthreads();
         // this lane's channels in rotated order: slot i holds channel q * 8 + (i + r) mod 8
         float scale[8];
@@ -167,35 +173,45 @@ __global__ void __launch_bounds__(CAL_THREADS) mode_kernel(const uint16_t *__res
                             const float vb = __fmul_rn(__fsub_rn(f[i], lo[i]), scale[i]);
                             int b = __float_as_int(__fadd_rd(vb, 8388608.0f)) & 0x7fffff;
                             b = min(b, nbins - 1);
-                            atomicAdd(&smem[(b >> 1) * CW + cidx[i]], 1u << ((b & 1) * 16));
+                            atomicAdd(&smem[(b >> 1) * CWT + cidx[i]], 1u << ((b & 1) * 16));
                         }
                     }
                 }
             }
         __syncthreads();
-        // ---- arg-max: lowest bin with the largest count.  Lane = channel; warp w scans its share of the bin pairs
-        // in ascending order, then thread c combines the warps in ascending order (strict >: the first maximum stays).
+        // ---- arg-max: lowest bin with the largest count.  A lane scans bin pairs of channel lane mod CWT in ascending
+        // order (strict >: the first maximum stays); with 16 channels the two half-warps take alternate pairs and
+        // are merged by (count, then lower bin).  Thread c then combines the warps in ascending order.
         {
+            constexpr int LS = 32 / CWT;  // lanes per channel in a warp
             const int per = (HW + NW - 1) / NW;
+            const int sub = lane / CWT, ch = lane % CWT;
             uint32_t best_cnt = 0;
             int best_i = 0;
             const int h_end = min(HW, (warp + 1) * per);
-            for (int h0 = warp * per; h0 < h_end; h0 += 8) {
+            for (int h0 = warp * per + sub; h0 < h_end; h0 += 8 * LS) {
                 uint32_t wv[8];  // eight independent loads, then the ordered compares
 #pragma unroll
-                for (int e = 0; e < 8; ++e) wv[e] = h0 + e < h_end ? smem[(h0 + e) * CW + lane] : 0u;
+                for (int e = 0; e < 8; ++e) wv[e] = h0 + e * LS < h_end ? smem[(h0 + e * LS) * CWT + ch] : 0u;
 #pragma unroll
                 for (int e = 0; e < 8; ++e) {
                     const uint32_t c0 = wv[e] & 0xffffu, c1 = wv[e] >> 16;  // bin 2h + 1 beyond nbins was never counted
-                    if (c0 > best_cnt) { best_cnt = c0; best_i = 2 * (h0 + e); }
-                    if (c1 > best_cnt) { best_cnt = c1; best_i = 2 * (h0 + e) + 1; }
+                    if (c0 > best_cnt) { best_cnt = c0; best_i = 2 * (h0 + e * LS); }
+                    if (c1 > best_cnt) { best_cnt = c1; best_i = 2 * (h0 + e * LS) + 1; }
                 }
             }
-            s_wlo[warp][lane] = __uint_as_float(best_cnt);
-            s_whi[warp][lane] = __int_as_float(best_i);
+            if constexpr (LS == 2) {
+                const uint32_t oc = __shfl_xor_sync(0xffffffffu, best_cnt, 16);
+                const int oi = __shfl_xor_sync(0xffffffffu, best_i, 16);
+                if (oc > best_cnt || (oc == best_cnt && oi < best_i)) { best_cnt = oc; best_i = oi; }
+            }
+            if (sub == 0) {
+                s_wlo[warp][ch] = __uint_as_float(best_cnt);
+                s_whi[warp][ch] = __int_as_float(best_i);
+            }
         }
         __syncthreads();
-        if (tid < CW) {
+        if (tid < CWT) {
             uint32_t best_cnt = 0;
             int best_i = 0;
 #pragma unroll
@@ -214,7 +230,7 @@ __global__ void __launch_bounds__(CAL_THREADS) mode_kernel(const uint16_t *__res
         }
         __syncthreads();
     } else {
-        if (tid < CW) {
+        if (tid < CWT) {
             s_m[tid] = 0.0f;
             if (k0 + tid < K) m_out[k0 + tid] = 0.0f;
         }
@@ -222,14 +238,15 @@ __global__ void __launch_bounds__(CAL_THREADS) mode_kernel(const uint16_t *__res
     }
     if (!want_hist) return;
     // ---- pass 3: first radix histogram of the importance |x - m|.  The keys crowd into a few dozen buckets (the
-    // top 11 bits are the exponent and three mantissa bits), so the four lanes that share a row count into four
+    // top 11 bits are the exponent and three mantissa bits), so groups of four neighbouring lanes count into four
     // copies of the histogram, each shifted by 8 banks against the previous one.
-    for (int i = tid; i < 4 * RADIX_BINS; i += CAL_THREADS) smem[i] = 0;
+    for (int i = tid; i < 4 * RADIX_BINS; i += NTH) smem[i] = 0;
     float mk[8];
 #pragma unroll
     for (int j = 0; j < 8; ++j) mk[j] = s_m[q * 8 + j];
     __syncthreads();
-    uint32_t *hq = smem + q * RADIX_BINS;
+    const int cp = lane & 3;  // copy of this lane
+    uint32_t *hq = smem + cp * RADIX_BINS;
     if (ok)
         for (int t0 = rl; t0 < T; t0 += CAL_ROWS * CAL_U) {
             if (!resident) nv = load_rows(xp, K, T, t0, v);
@@ -241,13 +258,13 @@ __global__ void __launch_bounds__(CAL_THREADS) mode_kernel(const uint16_t *__res
 #pragma unroll
                     for (int j = 0; j < 8; ++j) {
                         const uint32_t key = __float_as_uint(__fsub_rn(f[j], mk[j])) & 0x7fffffffu;
-                        atomicAdd(&hq[((key >> 20) + 8 * q) & (RADIX_BINS - 1)], 1u);
+                        atomicAdd(&hq[((key >> 20) + 8 * cp) & (RADIX_BINS - 1)], 1u);
                     }
                 }
             }
         }
     __syncthreads();
-    for (int i = tid; i < RADIX_BINS; i += CAL_THREADS) {
+    for (int i = tid; i < RADIX_BINS; i += NTH) {
         uint32_t c = 0;
 #pragma unroll
         for (int qq = 0; qq < 4; ++qq) c += smem[qq * RADIX_BINS + ((i + 8 * qq) & (RADIX_BINS - 1))];
@@ -331,6 +348,8 @@ __global__ void __launch_bounds__(256) radix_pass_kernel(const uint16_t *__restr
                                                          uint32_t *__restrict__ hist) {
     __shared__ uint32_t s_h[2][RADIX_BINS];
     for (int i = threadIdx.x; i < 2 * RADIX_BINS; i += blockDim.x) (&s_h[0][0])[i] = 0;
+    griddep_wait();               // the previous pass's counters are complete
+    griddep_launch_dependents();
     const int sh = shift + width;
     // previous pass: one shared histogram (the first pass) or one per order statistic
     const uint32_t *const ph[2] = {prev_hist, prev_two ? prev_hist + RADIX_BINS : prev_hist};
@@ -399,6 +418,7 @@ __global__ void __launch_bounds__(256) radix_pass_kernel(const uint16_t *__restr
 __global__ void __launch_bounds__(256) select_kernel(const uint32_t *__restrict__ hist, int nb, int width,
                                                      const SelState *__restrict__ st_in, double frac,
                                                      float *__restrict__ tau_out) {
+    griddep_wait();
     const uint32_t *const ph[2] = {hist, hist + RADIX_BINS};
     const uint32_t rk[2] = {st_in->rank[0], st_in->rank[1]};
     const SelPick pick = block_select(ph, nb, rk);
@@ -799,6 +819,7 @@ static scap_status calibrate_t(const uint16_t *x, int T, int K, double sparsity,
     SelState *state = reinterpret_cast<SelState *>(ws + L.state);
     const long long M = (long long)T * K;
     const bool want_tau = sparsity > 0.0;
+    const bool pdl = g_tune.pdl != 0;
     cudaError_t e = cudaMemsetAsync(ws, 0, L.zeroed, st);
     if (e != cudaSuccess) return cuda_status(e);
     const bool own_mode = estimator == 0 && !scalar;  // the strip kernel estimates the per-channel histogram mode itself
@@ -808,13 +829,22 @@ static scap_status calibrate_t(const uint16_t *x, int T, int K, double sparsity,
         if (!want_tau) return cuda_status(launch(set_float_kernel, dim3(1), dim3(1), 0, st, false, tau_out, 0.0f));
     }
     const int HW = (nbins + 1) / 2;
-    size_t smem = (size_t)CW * HW * 4;
+    const int cw = g_tune.cal_strip;  // 16 or 32 channels per CTA
+    size_t smem = (size_t)cw * HW * 4;
     if (smem < (size_t)4 * RADIX_BINS * 4) smem = (size_t)4 * RADIX_BINS * 4;  // the four copies of the first radix histogram
-    static SmemOptIn opt_in;
-    e = ensure_dynamic_smem(mode_kernel<BF16>, 2048 / 2 * CW * 4, opt_in);
-    if (e != cudaSuccess) return cuda_status(e);
-    e = launch(mode_kernel<BF16>, dim3((K + CW - 1) / CW), dim3(CAL_THREADS), smem, st, false, x, T, K, nbins, m_out, hist,
-               want_tau ? 1 : 0, own_mode ? (const float *)nullptr : (const float *)m_out);
+    static SmemOptIn opt_in32, opt_in16;
+    const float *given = own_mode ? (const float *)nullptr : (const float *)m_out;
+    if (cw == 16) {
+        e = ensure_dynamic_smem(mode_kernel<BF16, 16>, 2048 / 2 * 16 * 4, opt_in16);
+        if (e != cudaSuccess) return cuda_status(e);
+        e = launch(mode_kernel<BF16, 16>, dim3((K + 15) / 16), dim3(256), smem, st, pdl, x, T, K, nbins, m_out, hist,
+                   want_tau ? 1 : 0, given);
+    } else {
+        e = ensure_dynamic_smem(mode_kernel<BF16, 32>, 2048 / 2 * 32 * 4, opt_in32);
+        if (e != cudaSuccess) return cuda_status(e);
+        e = launch(mode_kernel<BF16, 32>, dim3((K + 31) / 32), dim3(512), smem, st, pdl, x, T, K, nbins, m_out, hist,
+                   want_tau ? 1 : 0, given);
+    }
     if (e != cudaSuccess) return cuda_status(e);
     if (!want_tau) return cuda_status(launch(set_float_kernel, dim3(1), dim3(1), 0, st, false, tau_out, 0.0f));
 
@@ -830,14 +860,14 @@ static scap_status calibrate_t(const uint16_t *x, int T, int K, double sparsity,
     const dim3 grid(gx, gy < 1 ? 1 : gy);
     // pass A (bits 30..20) was accumulated by mode_kernel; each later pass first extends the prefixes from the
     // counters of the pass before it
-    e = launch(radix_pass_kernel<BF16>, grid, dim3(256), 0, st, false, x, (const float *)m_out, T, K, (const uint32_t *)hist, 0,
+    e = launch(radix_pass_kernel<BF16>, grid, dim3(256), 0, st, pdl, x, (const float *)m_out, T, K, (const uint32_t *)hist, 0,
                11, (const SelState *)nullptr, (uint32_t)j, (uint32_t)j1, state, 9, 11, hist + 2 * RADIX_BINS);
     if (e != cudaSuccess) return cuda_status(e);
-    e = launch(radix_pass_kernel<BF16>, grid, dim3(256), 0, st, false, x, (const float *)m_out, T, K,
+    e = launch(radix_pass_kernel<BF16>, grid, dim3(256), 0, st, pdl, x, (const float *)m_out, T, K,
                (const uint32_t *)(hist + 2 * RADIX_BINS), 1, 11, (const SelState *)state, 0u, 0u, state + 1, 0, 9,
                hist + 4 * RADIX_BINS);
     if (e != cudaSuccess) return cuda_status(e);
-    e = launch(select_kernel, dim3(1), dim3(256), 0, st, false, (const uint32_t *)(hist + 4 * RADIX_BINS), 512, 9,
+    e = launch(select_kernel, dim3(1), dim3(256), 0, st, pdl, (const uint32_t *)(hist + 4 * RADIX_BINS), 512, 9,
                (const SelState *)(state + 1), frac, tau_out);
     return cuda_status(e);
 }

@@ -20,6 +20,7 @@ struct Tuning {
     int tc;       // batch 3..16 on the tcgen05 kernel (0: the mma.sync variants)
     int host_direct;  // scap_sparse_fc_host moves device-addressable pinned host buffers with its own kernels
     int fma_rows;     // largest batch that takes the fp32-FMA body (2 or 4); larger batches take a tensor-core variant
+    int cal_strip;    // channels per CTA of the calibration histogram kernel: 16 or 32
 };
 extern Tuning g_tune;
 

@@ -6,7 +6,7 @@
 
 namespace scap {
 
-Tuning g_tune = {0, 1, 1, 1, 4};
+Tuning g_tune = {0, 1, 1, 1, 4, 16};
 
 scap_status check_device() {
     static int cached[64];  // 0 unknown, 1 ok, 2 unsupported
@@ -277,6 +277,11 @@ scap_status scap_tune(const char *key, int value) {
     if (!strcmp(key, "fma_rows")) {
         if (value != 2 && value != 4) return SCAP_ERR_INVALID_ARG;
         g_tune.fma_rows = value;
+        return SCAP_OK;
+    }
+    if (!strcmp(key, "cal_strip")) {
+        if (value != 16 && value != 32) return SCAP_ERR_INVALID_ARG;
+        g_tune.cal_strip = value;
         return SCAP_OK;
     }
     if (!strcmp(key, "tcgen05")) {

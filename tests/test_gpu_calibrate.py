@@ -49,6 +49,25 @@ def test_mode_and_tau_bit_exact(S, T, K, dt, nbins, s):
     assert tau_g.view(np.uint32) == np.float32(tau_o).view(np.uint32)
 
 
+@pytest.mark.parametrize("strip", [16, 32])
+@pytest.mark.parametrize("T,K,nbins,s", [
+    (2100, 72, 2048, 0.6),    # more rows than a strip keeps in registers: the passes re-read the input
+    (300, 520, 333, 0.8),
+    (64, 40, 16, 0.3),        # a partial strip for either width
+])
+def test_both_strip_widths_of_the_histogram_kernel(S, strip, T, K, nbins, s):
+    d = si.laplace_fc(4, K, 8, si.BF16, T, 1)
+    xf = si.to_f32(d["x_calib"], si.BF16)
+    m_o, tau_o = oracle.calibrate(xf, s, nbins)
+    S.scap_tune("cal_strip", strip)
+    try:
+        m_g, tau_g = run_calibrate(S, d["x_calib"], si.BF16, s, nbins)
+    finally:
+        S.scap_tune("cal_strip", 16)
+    assert np.array_equal(m_g, m_o)
+    assert tau_g.view(np.uint32) == np.float32(tau_o).view(np.uint32)
+
+
 def test_no_centring_and_zero_sparsity(S):
     d = si.laplace_fc(4, 128, 8, si.BF16, 200, 1)
     xf = si.to_f32(d["x_calib"], si.BF16)
