@@ -20,7 +20,8 @@
  * inputs, textbook special cases, library quantile/matmul cross-checks, the paper's printed
  * FFN-sparsity rows) EXCEPT the following, which are "parity unpinned" because the paper
  * prints nothing that fixes them:
- *   - the accuracy of the histogram mode estimator (its definition is pinned on hand-built cases);
+ *   - the accuracy of the histogram mode estimator (its definition is pinned on hand-built cases
+ *     and against a library histogram on samples away from bin edges);
  *   - the mixture-of-experts router convention (softmax, top-k, renormalise, ties to lower index).
  */
 #include <math.h>

@@ -281,6 +281,25 @@ def test_mode_is_translation_equivariant_on_exact_grid():
     assert np.array_equal(oracle.mode(x + np.float32(2.0), 16), oracle.mode(x, 16) + np.float32(2.0))
 
 
+def test_mode_matches_the_library_histogram_away_from_bin_edges():
+    # Samples at exact bin centres of [0, 64) plus the two range ends: every bin decision is exact in any arithmetic,
+    # so numpy.histogram (float64 edges) must count what the oracle counts, and the first arg-max bin centre is the mode.
+    rng = np.random.default_rng(17)
+    T, K, nbins = 500, 9, 64
+    bins = rng.integers(0, nbins, size=(T, K))
+    bins[:60, 3] = 41                       # a clear peak
+    bins[:40, 4] = 7
+    bins[40:80, 4] = 50                     # two tall peaks; whichever is taller (or the lower bin on a tie) must win
+    x = (bins + 0.5).astype(np.float32)
+    x[-1, :] = 0.0                          # range ends: lo = 0 (bin 0), hi = 64 (clamped into the last bin)
+    x[-2, :] = 64.0
+    m = oracle.mode(x, nbins)
+    for k in range(K):
+        counts, edges = np.histogram(x[:, k].astype(np.float64), bins=nbins, range=(0.0, 64.0))
+        i = int(np.argmax(counts))          # first maximum = lowest bin
+        assert m[k] == np.float32(0.5 * (edges[i] + edges[i + 1]))
+
+
 def test_calibrate_runs_mode_then_tau_on_centred_values():
     d = small_fc(K=64, N=8)
     xc = si.to_f32(d["x_calib"], d["dt"])
