@@ -459,17 +459,20 @@ __device__ __forceinline__ void mma_k16(float (&d)[4], const uint32_t (&a)[4], u
                      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
-// Splits v into NSPLIT values of the weight dtype whose sum is v to 2^-22 or better; part[0] is the leading one.
+// Splits v into NSPLIT values of the weight dtype whose sum is v (bf16: exactly, unless a part falls below the
+// binary32 normal range; fp16: to 2^-22); part[0] is the leading one.
 template <bool BF16>
 __device__ __forceinline__ void split_parts(float v, unsigned short (&part)[3]) {
     if constexpr (BF16) {
-        const __nv_bfloat16 h = __float2bfloat16_rn(v);
-        const float r1 = v - __bfloat162float(h);
-        const __nv_bfloat16 m = __float2bfloat16_rn(r1);
-        const __nv_bfloat16 l = __float2bfloat16_rn(r1 - __bfloat162float(m));
-        part[0] = __bfloat16_as_ushort(h);
-        part[1] = __bfloat16_as_ushort(m);
-        part[2] = __bfloat16_as_ushort(l);
+        // Truncation cuts the 24-bit significand into three consecutive 8-bit fields: hi = the upper half of the
+        // pattern, r1 = v - hi (exact), mid = the upper half of r1, lo = r1 - mid (exact, at most 8 bits: a bf16).
+        const uint32_t hb = __float_as_uint(v) & 0xffff0000u;
+        const float r1 = v - __uint_as_float(hb);
+        const uint32_t mb = __float_as_uint(r1) & 0xffff0000u;
+        const float r2 = r1 - __uint_as_float(mb);
+        part[0] = (unsigned short)(hb >> 16);
+        part[1] = (unsigned short)(mb >> 16);
+        part[2] = (unsigned short)(__float_as_uint(r2) >> 16);
     } else {
         const __half h = __float2half_rn(v);
         const __half l = __float2half_rn(v - __half2float(h));
