@@ -86,6 +86,9 @@ int scap_version(void);
  *              device, a kernel pulls x and the FC kernel writes y to host memory (default), 0 = always copies
  *   "cal_strip"  scap_calibrate: channels per CTA of the per-channel histogram kernel, 16 (default: 256 threads,
  *              two CTAs per SM) or 32 (512 threads, one CTA per SM)
+ *   "l2_hints"  batch 1..4 FC kernel: 1 = loads carry L2 eviction hints (default): activations and modes, which every
+ *              column tile of a call reads again, are kept (evict_last); weight rows, read once, go first
+ *              (evict_first); 0 = no hints
  * Unknown keys return SCAP_ERR_INVALID_ARG.  Tuning never changes what is computed; split_k
  * changes the (fixed) summation order and therefore the last bits of y.  Query workspace sizes
  * after tuning.                                                                               */

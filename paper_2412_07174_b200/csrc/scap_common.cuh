@@ -21,6 +21,7 @@ struct Tuning {
     int host_direct;  // scap_sparse_fc_host moves device-addressable pinned host buffers with its own kernels
     int fma_rows;     // largest batch that takes the fp32-FMA body (2 or 4); larger batches take a tensor-core variant
     int cal_strip;    // channels per CTA of the calibration histogram kernel: 16 or 32
+    int l2_hints;     // batch 1..4 FC kernel: L2 eviction hints (keep activations and modes, stream weights)
 };
 extern Tuning g_tune;
 
@@ -172,6 +173,51 @@ __device__ __forceinline__ unsigned short ld_act_if_u16(const void *p, bool on) 
 }
 __device__ __forceinline__ __nv_bfloat16 ld_act_if(const __nv_bfloat16 *p, bool on) { return __ushort_as_bfloat16(ld_act_if_u16(p, on)); }
 __device__ __forceinline__ __half ld_act_if(const __half *p, bool on) { return __ushort_as_half(ld_act_if_u16(p, on)); }
+
+// L2 eviction policies for loads that carry a cache hint.  keep: small data every column tile of a call reads again
+// (activations, modes); stream: weight rows, read once.
+__device__ __forceinline__ uint64_t l2_policy_keep() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ uint64_t l2_policy_stream() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ uint64_t l2_policy_normal() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_normal.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ uint4 ld_stream16(const void *p, uint64_t pol) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.L2::cache_hint.v4.u32 {%0,%1,%2,%3}, [%4], %5;"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p), "l"(pol));
+    return v;
+}
+__device__ __forceinline__ float ld_nc_if(const float *p, bool on, uint64_t pol) {
+    float v;
+    asm volatile("{ .reg .pred q; setp.ne.u32 q, %2, 0; mov.f32 %0, 0f00000000; @q ld.global.nc.L2::cache_hint.f32 %0, [%1], %3; }"
+                 : "=f"(v) : "l"(p), "r"((unsigned)on), "l"(pol));
+    return v;
+}
+__device__ __forceinline__ float ld_act_if(const float *p, bool on, uint64_t pol) {
+    float v;
+    asm volatile("{ .reg .pred q; setp.ne.u32 q, %2, 0; mov.f32 %0, 0f00000000; @q ld.global.cg.L2::cache_hint.f32 %0, [%1], %3; }"
+                 : "=f"(v) : "l"(p), "r"((unsigned)on), "l"(pol) : "memory");
+    return v;
+}
+__device__ __forceinline__ unsigned short ld_act_if_u16(const void *p, bool on, uint64_t pol) {
+    unsigned short v;
+    asm volatile("{ .reg .pred q; setp.ne.u32 q, %2, 0; mov.u16 %0, 0; @q ld.global.cg.L2::cache_hint.u16 %0, [%1], %3; }"
+                 : "=h"(v) : "l"(p), "r"((unsigned)on), "l"(pol) : "memory");
+    return v;
+}
+__device__ __forceinline__ __nv_bfloat16 ld_act_if(const __nv_bfloat16 *p, bool on, uint64_t pol) { return __ushort_as_bfloat16(ld_act_if_u16(p, on, pol)); }
+__device__ __forceinline__ __half ld_act_if(const __half *p, bool on, uint64_t pol) { return __ushort_as_half(ld_act_if_u16(p, on, pol)); }
 
 // Hint: bring the line that holds *p into L2 (no register result, no ordering effect).
 __device__ __forceinline__ void prefetch_l2(const void *p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }

@@ -6,7 +6,7 @@
 
 namespace scap {
 
-Tuning g_tune = {0, 1, 1, 1, 4, 16};
+Tuning g_tune = {0, 1, 1, 1, 4, 16, 1};
 
 scap_status check_device() {
     static int cached[64];  // 0 unknown, 1 ok, 2 unsupported
@@ -138,7 +138,9 @@ cudaError_t launch_fc(bool bf16, int mode, int xkind, int epi, const FcArgs &a, 
         t.S = tc_choose_split(a.K, a.Nh, epi, a.B, bf16);
         return launch_fc_tc(bf16, mode, xkind, epi, t, st);
     }
-    return bf16 ? launch_fc_w<true>(mode, xkind, epi, a, st) : launch_fc_w<false>(mode, xkind, epi, a, st);
+    FcArgs f = a;
+    f.l2_hints = g_tune.l2_hints;
+    return bf16 ? launch_fc_w<true>(mode, xkind, epi, f, st) : launch_fc_w<false>(mode, xkind, epi, f, st);
 }
 
 // Copies n16 16-byte words from device-addressable host memory into device memory (one word per thread).
@@ -282,6 +284,10 @@ scap_status scap_tune(const char *key, int value) {
     if (!strcmp(key, "cal_strip")) {
         if (value != 16 && value != 32) return SCAP_ERR_INVALID_ARG;
         g_tune.cal_strip = value;
+        return SCAP_OK;
+    }
+    if (!strcmp(key, "l2_hints")) {
+        g_tune.l2_hints = value != 0;
         return SCAP_OK;
     }
     if (!strcmp(key, "tcgen05")) {

@@ -67,6 +67,7 @@ struct FcArgs {
     int no_tc;            // 1: keep this call off the tcgen05 kernel
     int act;              // EPI_BIAS: 1 = the exact GELU is applied to the biased result (z_copy then gets a copy)
     const float *wscale;  // 8-bit weights only: one scale per input channel, W[k,n] = wscale[k] * Wq[k,n]
+    int l2_hints;         // fp32-FMA body: 1 = loads carry L2 eviction hints (keep x and m, stream W)
 };
 
 template <bool BF16, int BT, int CAP>
@@ -246,6 +247,10 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
     const int my_chunks = nchunks > s ? (nchunks - s + S - 1) / S : 0;  // chunks s, s+S, ...
     float tau = 0.0f;
     if constexpr (MODE == MODE_GATHER) tau = ld_nc(a.tau);
+    // x and m are read again by every column tile of the call (and m by every later call): ask L2 to keep them and
+    // to drop the weight rows, which are read once, first.
+    const uint64_t pol_keep = a.l2_hints ? l2_policy_keep() : l2_policy_normal();
+    const uint64_t pol_stream = a.l2_hints ? l2_policy_stream() : l2_policy_normal();
 
     if (wait_inside && (my_chunks == 0 || a.in_rows)) {
         griddep_wait();
@@ -268,7 +273,7 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
         for (int p = 0; p < PU; ++p) {
             const int j = warp * pw + p;
             const int k = (s + S * (j0 + j)) * 32 + lane;
-            mk[p] = a.m ? ld_nc_if(a.m + k, p < pw && j < nj && k < K) : 0.0f;
+            mk[p] = a.m ? ld_nc_if(a.m + k, p < pw && j < nj && k < K, pol_keep) : 0.0f;
         }
         if (wait_inside && j0 == 0 && !a.in_rows) {
             // Pull this CTA's slice of x towards L2 while the previous kernel drains.  L2 is the coherence point,
@@ -294,7 +299,7 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
 #pragma unroll
             for (int b = 0; b < BT; ++b) {
                 const int bb = b < B ? b : 0;
-                xraw[p][b] = ld_act_if(xg + (size_t)(a.in_rows ? s_rows[bb] : bb) * a.x_ld + k, ok && b < B);
+                xraw[p][b] = ld_act_if(xg + (size_t)(a.in_rows ? s_rows[bb] : bb) * a.x_ld + k, ok && b < B, pol_keep);
             }
         }
 #pragma unroll
@@ -369,23 +374,23 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
             uint4 ga[G], gb[G];
 #pragma unroll
             for (int u = 0; u < G; ++u)
-                if (u < nrows) ga[u] = ld_stream16(Wb + (size_t)s_k[rg + NR * u] * row_bytes);
+                if (u < nrows) ga[u] = ld_stream16(Wb + (size_t)s_k[rg + NR * u] * row_bytes, pol_stream);
 #pragma unroll
             for (int u = 0; u < G; ++u)
-                if (G + u < nrows) gb[u] = ld_stream16(Wb + (size_t)s_k[rg + NR * (G + u)] * row_bytes);
+                if (G + u < nrows) gb[u] = ld_stream16(Wb + (size_t)s_k[rg + NR * (G + u)] * row_bytes, pol_stream);
             for (int t0 = 0; t0 < nrows; t0 += 2 * G) {
 #pragma unroll
                 for (int u = 0; u < G; ++u)
                     if (t0 + u < nrows) fma_row<BF16, BT, CAP>(acc, ga[u], s_xs, rg + NR * (t0 + u));
 #pragma unroll
                 for (int u = 0; u < G; ++u)
-                    if (t0 + 2 * G + u < nrows) ga[u] = ld_stream16(Wb + (size_t)s_k[rg + NR * (t0 + 2 * G + u)] * row_bytes);
+                    if (t0 + 2 * G + u < nrows) ga[u] = ld_stream16(Wb + (size_t)s_k[rg + NR * (t0 + 2 * G + u)] * row_bytes, pol_stream);
 #pragma unroll
                 for (int u = 0; u < G; ++u)
                     if (t0 + G + u < nrows) fma_row<BF16, BT, CAP>(acc, gb[u], s_xs, rg + NR * (t0 + G + u));
 #pragma unroll
                 for (int u = 0; u < G; ++u)
-                    if (t0 + 3 * G + u < nrows) gb[u] = ld_stream16(Wb + (size_t)s_k[rg + NR * (t0 + 3 * G + u)] * row_bytes);
+                    if (t0 + 3 * G + u < nrows) gb[u] = ld_stream16(Wb + (size_t)s_k[rg + NR * (t0 + 3 * G + u)] * row_bytes, pol_stream);
             }
         }
         __syncthreads();

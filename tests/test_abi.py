@@ -67,6 +67,8 @@ def test_argument_validation_returns_codes(L):
     assert L.scap_tune(b"fma_rows", 3) == 1
     assert L.scap_tune(b"fma_rows", 2) == 0
     assert L.scap_tune(b"fma_rows", 4) == 0
+    assert L.scap_tune(b"l2_hints", 0) == 0
+    assert L.scap_tune(b"l2_hints", 1) == 0
     assert L.scap_tune(b"cal_strip", 24) == 1
     assert L.scap_tune(b"cal_strip", 32) == 0
     assert L.scap_tune(b"cal_strip", 16) == 0
