@@ -526,6 +526,11 @@ def run_suite(args):
             suite_sweep(torch, scap, peak, shapes, (0.0, 0.25, 0.5, 0.6, 0.7, 0.8, 0.9), (1, 2, 4, 8, 16), out)
     if which in ("moe", "all"):
         suite_moe(torch, scap, peak, out)
+    if which in ("mamba", "all"):
+        # Mamba2-2.7B projection shapes (d_model 2560, d_inner 5120, d_state 128, 80 heads): in_proj 2560 -> 10576 at the
+        # paper's 30 % input sparsity, out_proj 5120 -> 2560 at 60 % (Table 4); records carry "suite": "sweep"
+        suite_sweep(torch, scap, peak, [(2560, 10576)], (0.0, 0.3), (1, 4), out)
+        suite_sweep(torch, scap, peak, [(5120, 2560)], (0.0, 0.6), (1, 4), out)
 
 
 
@@ -543,7 +548,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--detail", action="store_true", help="also print a per-sparsity table to stderr")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--suite", default="", choices=["", "calibrate", "glu", "gelu", "q8", "moe", "sweep", "sweep-small", "all"],
+    ap.add_argument("--suite", default="", choices=["", "calibrate", "glu", "gelu", "q8", "moe", "mamba", "sweep", "sweep-small", "all"],
                     help="run the other workload descriptions instead of the headline line (one JSON object per line)")
     ap.add_argument("--copies", type=int, default=0,
                     help="number of weight copies to rotate (default: enough for the cold-HBM rule); a small value keeps "

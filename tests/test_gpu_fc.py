@@ -67,6 +67,7 @@ def test_config0_single_fc_fp16(S):
 @pytest.mark.parametrize("K,N,B,dt", [
     (1000, 264, 1, si.BF16), (33, 8, 3, si.F16), (1, 16, 2, si.BF16), (777, 520, 5, si.BF16),
     (2048, 1032, 16, si.F16), (300, 4096, 4, si.BF16), (5000, 256, 8, si.BF16), (256, 248, 2, si.F16),
+    (2560, 10576, 1, si.BF16), (5120, 2560, 4, si.BF16),     # Mamba2-2.7B in_proj / out_proj (N = 10576 ends in a ragged tile)
 ])
 def test_shapes_and_batches(S, K, N, B, dt):
     d = si.laplace_fc(4, K, N, dt, 32, B)
