@@ -60,6 +60,8 @@ def lib():
         L.scap_oracle_mean.restype = None
         L.scap_oracle_median.argtypes = [vp, i, i, vp]
         L.scap_oracle_median.restype = None
+        L.scap_oracle_kde.argtypes = [vp, i, i, i, vp, i, vp]
+        L.scap_oracle_kde.restype = None
         L.scap_oracle_eta_mean.argtypes = [vp, i, i]
         L.scap_oracle_eta_mean.restype = f
         L.scap_oracle_tau.argtypes = [vp, i, i, vp, d, vp, vp]
@@ -187,7 +189,7 @@ def mode(xf_calib, nbins: int = 2048):
     return m
 
 
-HISTOGRAM, MEAN, MEDIAN = 0, 1, 2      # mode estimators (Section 3, "Determination of mode value")
+HISTOGRAM, MEAN, MEDIAN, KDE = 0, 1, 2, 3   # mode estimators (Section 3, "Determination of mode value")
 PER_CHANNEL, SCALAR = 0, 1             # one mode per input channel, or the paper's single eta per FC
 
 
@@ -199,8 +201,13 @@ def mode_estimate(xf_calib, estimator: int = HISTOGRAM, scope: int = PER_CHANNEL
         if estimator == HISTOGRAM:
             return mode(xf, nbins)
         m = np.empty(K, np.float32)
+        if estimator == KDE:
+            lib().scap_oracle_kde(_p(xf), T, K, int(nbins), _p(m), -1, None)
+            return m
         (lib().scap_oracle_mean if estimator == MEAN else lib().scap_oracle_median)(_p(xf), T, K, _p(m))
         return m
+    if estimator == KDE:
+        raise ValueError("the KDE peak is defined per channel only")
     if estimator == MEAN:
         eta = np.float32(lib().scap_oracle_eta_mean(_p(xf), T, K))
     else:
@@ -212,6 +219,18 @@ def mode_estimate(xf_calib, estimator: int = HISTOGRAM, scope: int = PER_CHANNEL
             lib().scap_oracle_median(_p(flat), T * K, 1, _p(one))
         eta = one[0]
     return np.full(K, eta, np.float32)
+
+
+def kde_density(xf_calib, k: int, G: int):
+    """The G (unnormalised) densities of channel k on its grid, and the grid itself (binary64)."""
+    xf = _f32(np.atleast_2d(xf_calib))
+    T, K = xf.shape
+    m = np.empty(K, np.float32)
+    dens = np.empty(G, np.float64)
+    lib().scap_oracle_kde(_p(xf), T, K, int(G), _p(m), int(k), dens.ctypes.data_as(C.c_void_p))
+    lo, hi = np.float64(xf[:, k].min()), np.float64(xf[:, k].max())
+    grid = lo + np.arange(G, dtype=np.float64) * ((hi - lo) / (G - 1))
+    return dens, grid
 
 
 def calibrate_ex(xf_calib, s: float, estimator: int = HISTOGRAM, scope: int = PER_CHANNEL, nbins: int = 2048):

@@ -241,6 +241,54 @@ void scap_oracle_median(const float *xf /*[T,K]*/, int T, int K, float *m_out) {
     free(v);
 }
 
+/* Mode as the peak of a kernel density estimate (Section 3, "Determination of mode value", names KDE next to the
+ * mean and the median and leaves its parameters to a statistics package).  Reading taken, per channel, all in
+ * binary64: Gaussian kernel; bandwidth h = sigma * T^(-1/5) (Scott's rule) with sigma the sample standard
+ * deviation (divisor T - 1) about the mean, both summed in row order; the density is evaluated on G points
+ * g_i = lo + i (hi - lo) / (G - 1), i = 0 .. G-1, between the channel's smallest and largest value,
+ *   dens_i = sum_t exp( -((g_i - x_t) / h)^2 / 2 )      (the common factor 1 / (T h sqrt(2 pi)) is left out),
+ * and the mode is the first g_i of largest density, rounded once to binary32.  A constant channel returns its
+ * constant.  dens_out (optional) receives the G densities of channel k_dens.                           */
+void scap_oracle_kde(const float *xf /*[T,K]*/, int T, int K, int G, float *m_out, int k_dens, double *dens_out /*[G] or NULL*/) {
+    for (int k = 0; k < K; ++k) {
+        float lo = xf[k], hi = xf[k];
+        double sum = 0.0;
+        for (int t = 0; t < T; ++t) {
+            const float v = xf[(long)t * K + k];
+            if (v < lo) lo = v;
+            if (v > hi) hi = v;
+            sum += (double)v;
+        }
+        if (hi == lo) {
+            m_out[k] = lo + 0.0f;
+            if (dens_out && k == k_dens) for (int i = 0; i < G; ++i) dens_out[i] = (double)T;
+            continue;
+        }
+        const double mu = sum / (double)T;
+        double ss = 0.0;
+        for (int t = 0; t < T; ++t) {
+            const double d = (double)xf[(long)t * K + k] - mu;
+            ss += d * d;
+        }
+        const double sigma = sqrt(ss / (double)(T - 1));
+        const double h = sigma * pow((double)T, -0.2);
+        const double step = ((double)hi - (double)lo) / (double)(G - 1);
+        double best = -1.0;
+        int best_i = 0;
+        for (int i = 0; i < G; ++i) {
+            const double g = (double)lo + (double)i * step;
+            double dens = 0.0;
+            for (int t = 0; t < T; ++t) {
+                const double u = (g - (double)xf[(long)t * K + k]) / h;
+                dens += exp(-0.5 * (u * u));
+            }
+            if (dens_out && k == k_dens) dens_out[i] = dens;
+            if (dens > best) { best = dens; best_i = i; }
+        }
+        m_out[k] = (float)((double)lo + (double)best_i * step) + 0.0f;
+    }
+}
+
 /* Scalar eta for the whole FC input (the paper's eta is one scalar per layer), from all T*K values:
  *   mean:    the per-channel sums above (each over t in order), added over k = 0 .. K-1 in this order in
  *            binary64, divided by T*K, rounded once to binary32;

@@ -485,6 +485,31 @@ def test_scalar_eta_pools_the_whole_tensor_and_is_broadcast():
         assert np.array_equal(oracle.mode_estimate(one, est, oracle.SCALAR, 32), oracle.mode_estimate(one, est, oracle.PER_CHANNEL, 32))
 
 
+def test_kde_peak_agrees_with_the_library_kde_and_hand_cases():
+    from scipy.stats import gaussian_kde
+    rng = np.random.default_rng(23)
+    T, K, G = 300, 5, 129
+    x = np.stack([rng.normal(0.3, 1.0, T), rng.gamma(2.0, 1.0, T), rng.laplace(-1.0, 0.4, T),
+                  np.abs(rng.normal(0, 1, T)) ** 1.5, rng.uniform(-1, 1, T) ** 3], axis=1).astype(np.float32)
+    m = oracle.mode_estimate(x, oracle.KDE, oracle.PER_CHANNEL, G)
+    for k in range(K):
+        col = x[:, k].astype(np.float64)
+        grid = col.min() + np.arange(G) * ((col.max() - col.min()) / (G - 1))
+        lib_dens = gaussian_kde(col).evaluate(grid)        # Scott's factor T^(-1/5), covariance with divisor T - 1
+        assert m[k] == np.float32(grid[int(np.argmax(lib_dens))])
+        dens, g2 = oracle.kde_density(x, k, G)
+        assert np.array_equal(g2, grid)
+        norm = len(col) * np.std(col, ddof=1) * len(col) ** -0.2 * np.sqrt(2 * np.pi)
+        assert np.allclose(dens / norm, lib_dens, rtol=1e-9, atol=0)
+    # hand cases: a constant channel; a symmetric sample peaks at its centre; three of four points at the low end
+    h = np.array([[0.75, -2.0, 1.0], [0.75, -1.0, 1.0], [0.75, 0.0, 1.0], [0.75, 0.0, 9.0],
+                  [0.75, 0.0, 1.0], [0.75, 1.0, 1.0], [0.75, 2.0, 1.0]], np.float32)
+    mh = oracle.mode_estimate(h, oracle.KDE, oracle.PER_CHANNEL, 5)
+    assert mh[0] == np.float32(0.75) and mh[1] == np.float32(0.0) and mh[2] == np.float32(1.0)
+    # translation by an exactly representable amount moves the peak by that amount
+    assert np.array_equal(oracle.mode_estimate(h + np.float32(4.0), oracle.KDE, oracle.PER_CHANNEL, 5), mh + np.float32(4.0))
+
+
 def test_estimators_rank_as_expected_on_a_skewed_distribution():
     # exponential-like (GELU-output-like) data: mode < median < mean; centring by a better mode estimate prunes more at fixed tau
     rng = np.random.default_rng(3)
