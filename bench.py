@@ -322,27 +322,30 @@ def suite_calibrate(torch, scap, out):
 
     # The paper's other estimators of the mode (mean, median) and its scalar eta, on the same tensor and on a skewed
     # one (|N(0,1)|^1.5, GELU-output-like): time per call, and the sparsity each centring induces at one fixed tau.
-    names = {0: "histogram", 1: "mean", 2: "median"}
+    names = {0: "histogram", 1: "mean", 2: "median", 3: "kde_peak_512_points"}
     skew = si.to_bits(np.abs(si.normal(si.stream_seed(4, 9), T * Kk).reshape(T, Kk)) ** 1.5, si.BF16)
     xs = si.as_torch(skew, si.BF16).cuda()
     for scope in (0, 1):
-        for est in (0, 1, 2):
+        for est in (0, 1, 2, 3):
+            if est == 3 and scope == 1:
+                continue  # the KDE peak is defined per channel only
+            nb = 512 if est == 3 else NBINS  # KDE: grid points (T x 512 binary64 exponentials per channel)
             times = []
-            for _ in range(6):
+            for _ in range(3 if est == 3 else 6):
                 flush.fill_(1)
                 e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 torch.cuda.synchronize()
                 e0.record()
-                scap.scap_calibrate_ex(xc, 0.6, est, scope, NBINS, m, tau, cws)
+                scap.scap_calibrate_ex(xc, 0.6, est, scope, nb, m, tau, cws)
                 e1.record()
                 torch.cuda.synchronize()
                 times.append(e0.elapsed_time(e1) * 1e3)
-            scap.scap_calibrate_ex(xs, 0.6, est, scope, NBINS, m, tau, cws)
+            scap.scap_calibrate_ex(xs, 0.6, est, scope, nb, m, tau, cws)
             torch.cuda.synchronize()
             fixed_tau = 0.15
             pruned = float(((xs.float() - m[None, :]).abs() < fixed_tau).float().mean().item())
             out({"suite": "calibrate_ex", "T": T, "K": Kk, "estimator": names[est], "scope": "scalar" if scope else "per_channel",
-                 "us": round(float(np.median(times[2:])), 1), "skewed_input": "|N(0,1)|^1.5 in bf16",
+                 "us": round(float(np.median(times[1:] if est == 3 else times[2:])), 1), "skewed_input": "|N(0,1)|^1.5 in bf16",
                  "sparsity_at_tau_%.2f_on_skewed_input" % fixed_tau: round(pruned, 4),
                  "tau_for_60pct_on_skewed_input": round(float(tau.item()), 5)})
 

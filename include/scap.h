@@ -123,12 +123,17 @@ scap_status scap_calibrate(const void *x_calib, int T, int K, scap_dtype dt, dou
  *   SCAP_MODE_MEAN       per channel: the column added in row order in binary64, divided by T, rounded once
  *   SCAP_MODE_MEDIAN     per channel: the middle value, or the mean of the two middle values (binary64,
  *                        rounded once) for even T
+ *   SCAP_MODE_KDE        per channel only: peak of a Gaussian kernel density estimate, bandwidth sigma * T^(-1/5)
+ *                        (Scott's rule, sample standard deviation), evaluated in binary64 on nbins >= 2 grid points
+ *                        from the channel's minimum to its maximum; the first point of largest density.  T <= 4096
+ *                        (else SCAP_ERR_SHAPE); with SCAP_ETA_SCALAR or nbins < 2: SCAP_ERR_INVALID_ARG.  Where two
+ *                        grid points have densities equal to within rounding, either may be returned.
  *   SCAP_ETA_PER_CHANNEL one value per input channel in m_out[K]
  *   SCAP_ETA_SCALAR      one value for the whole tensor, written to all K entries of m_out: the estimator
  *                        applied to all T*K values as one sample (mean: the column sums of the per-channel
  *                        form added in channel order, divided by T*K)
  * A result of -0 is returned as +0.  Inputs must be finite.                                            */
-typedef enum { SCAP_MODE_HISTOGRAM = 0, SCAP_MODE_MEAN = 1, SCAP_MODE_MEDIAN = 2 } scap_mode_estimator;
+typedef enum { SCAP_MODE_HISTOGRAM = 0, SCAP_MODE_MEAN = 1, SCAP_MODE_MEDIAN = 2, SCAP_MODE_KDE = 3 } scap_mode_estimator;
 typedef enum { SCAP_ETA_PER_CHANNEL = 0, SCAP_ETA_SCALAR = 1 } scap_eta_scope;
 scap_status scap_calibrate_ex(const void *x_calib, int T, int K, scap_dtype dt, double sparsity,
                               scap_mode_estimator estimator, scap_eta_scope scope, int nbins, float *m_out,

@@ -8,7 +8,7 @@ import torch
 
 __all__ = [
     "SCAP_F16", "SCAP_BF16", "ScapError", "lib", "lib_path", "status_string", "scap_version", "scap_tune", "scap_device_status",
-    "scap_calibrate_workspace", "scap_calibrate", "scap_calibrate_ex", "SCAP_MODE_HISTOGRAM", "SCAP_MODE_MEAN", "SCAP_MODE_MEDIAN",
+    "scap_calibrate_workspace", "scap_calibrate", "scap_calibrate_ex", "SCAP_MODE_HISTOGRAM", "SCAP_MODE_MEAN", "SCAP_MODE_MEDIAN", "SCAP_MODE_KDE",
     "SCAP_ETA_PER_CHANNEL", "SCAP_ETA_SCALAR", "scap_fold_bias_workspace", "scap_fold_bias",
     "scap_fc_workspace", "scap_sparse_fc", "scap_dense_fc", "scap_sparse_fc_q8", "scap_dense_fc_q8", "scap_fold_bias_q8",
     "scap_fc_host_workspace", "scap_sparse_fc_host",
@@ -172,7 +172,7 @@ def scap_calibrate(x_calib, sparsity: float, nbins: int, m_out, tau_out, ws, str
                                 p, n, _stream(stream)), "scap_calibrate")
 
 
-SCAP_MODE_HISTOGRAM, SCAP_MODE_MEAN, SCAP_MODE_MEDIAN = 0, 1, 2
+SCAP_MODE_HISTOGRAM, SCAP_MODE_MEAN, SCAP_MODE_MEDIAN, SCAP_MODE_KDE = 0, 1, 2, 3
 SCAP_ETA_PER_CHANNEL, SCAP_ETA_SCALAR = 0, 1
 
 

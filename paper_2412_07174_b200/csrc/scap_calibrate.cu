@@ -607,6 +607,109 @@ __global__ void __launch_bounds__(CAL_THREADS) median_kernel(const uint16_t *__r
     }
 }
 
+// KDE peak per channel (Section 3 names the KDE next to the mean and the median): Gaussian kernel, bandwidth
+// h = sigma * T^(-1/5) with the sample standard deviation (divisor T - 1), density on G grid points between the
+// channel's minimum and maximum, first point of largest density.  All in binary64.
+// One CTA of 256 threads per strip of 8 channels: the strip is staged in shared memory as binary32 (exact for
+// 16-bit inputs), warp c computes the statistics of channel c, then for each channel every thread evaluates the
+// grid points tid, tid + 256, ... (all T samples each, read as shared-memory broadcasts) and the block keeps the
+// best (density, then lower index).
+constexpr int KDE_MAX_T = 4096;
+template <bool BF16>
+__global__ void __launch_bounds__(256) kde_kernel(const uint16_t *__restrict__ x, int T, int K, int G, float *__restrict__ m_out) {
+    extern __shared__ __align__(16) float s_x[];  // [8][T]
+    __shared__ float s_lo[8], s_hi[8];
+    __shared__ double s_h[8];
+    __shared__ double s_bd[8];
+    __shared__ int s_bi[8];
+    griddep_wait();
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int k0 = blockIdx.x * 8;  // K is a multiple of 8
+    for (int t = tid; t < T; t += 256) {
+        const uint4 v = __ldg(reinterpret_cast<const uint4 *>(x + (size_t)t * K + k0));
+        float f[8];
+        widen8<BF16>(v, f);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) s_x[j * T + t] = f[j];
+    }
+    __syncthreads();
+    {  // statistics of channel `warp`
+        const float *xc = s_x + warp * T;
+        float lo = INFINITY, hi = -INFINITY;
+        double sum = 0.0;
+        for (int t = lane; t < T; t += 32) {
+            const float v = xc[t];
+            lo = fminf(lo, v);
+            hi = fmaxf(hi, v);
+            sum += (double)v;
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            lo = fminf(lo, __shfl_xor_sync(0xffffffffu, lo, o));
+            hi = fmaxf(hi, __shfl_xor_sync(0xffffffffu, hi, o));
+            sum += __shfl_xor_sync(0xffffffffu, sum, o);
+        }
+        const double mu = sum / (double)T;
+        double ss = 0.0;
+        for (int t = lane; t < T; t += 32) {
+            const double d = (double)xc[t] - mu;
+            ss += d * d;
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+        if (lane == 0) {
+            s_lo[warp] = lo;
+            s_hi[warp] = hi;
+            s_h[warp] = T > 1 ? sqrt(ss / (double)(T - 1)) * pow((double)T, -0.2) : 0.0;
+        }
+    }
+    __syncthreads();
+    for (int c = 0; c < 8; ++c) {
+        const float lo = s_lo[c], hi = s_hi[c];
+        if (hi == lo) {  // constant channel (block-uniform)
+            if (tid == 0) m_out[k0 + c] = lo + 0.0f;
+            continue;
+        }
+        const float *xc = s_x + c * T;
+        const double inv_h = 1.0 / s_h[c];
+        const double step = ((double)hi - (double)lo) / (double)(G - 1);
+        double best = -1.0;
+        int best_i = 0x7fffffff;
+        for (int i = tid; i < G; i += 256) {
+            const double g = (double)lo + (double)i * step;
+            double d0 = 0.0, d1 = 0.0;
+            int t = 0;
+            for (; t + 1 < T; t += 2) {  // two independent chains
+                const double u0 = (g - (double)xc[t]) * inv_h, u1 = (g - (double)xc[t + 1]) * inv_h;
+                d0 += exp(-0.5 * (u0 * u0));
+                d1 += exp(-0.5 * (u1 * u1));
+            }
+            if (t < T) {
+                const double u0 = (g - (double)xc[t]) * inv_h;
+                d0 += exp(-0.5 * (u0 * u0));
+            }
+            const double dens = d0 + d1;
+            if (dens > best) { best = dens; best_i = i; }  // ascending i per thread: the first maximum stays
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const double od = __shfl_xor_sync(0xffffffffu, best, o);
+            const int oi = __shfl_xor_sync(0xffffffffu, best_i, o);
+            if (od > best || (od == best && oi < best_i)) { best = od; best_i = oi; }
+        }
+        if (lane == 0) { s_bd[warp] = best; s_bi[warp] = best_i; }
+        __syncthreads();
+        if (tid == 0) {
+            double bd = s_bd[0];
+            int bi = s_bi[0];
+            for (int w = 1; w < 8; ++w)
+                if (s_bd[w] > bd || (s_bd[w] == bd && s_bi[w] < bi)) { bd = s_bd[w]; bi = s_bi[w]; }
+            m_out[k0 + c] = (float)((double)lo + (double)bi * step) + 0.0f;
+        }
+        __syncthreads();
+    }
+}
+
 // Pooled (whole-tensor) statistics for the scalar eta.
 struct PoolState {
     uint32_t bucket[2], inner[2];  // median: high-byte bucket and rank inside it, for the two middle ranks
@@ -775,6 +878,12 @@ static cudaError_t estimate_mode(const uint16_t *x, int T, int K, int estimator,
     const long long M = (long long)T * K, M8 = M / 8;
     const int grid = sm_count() * 4;
     cudaError_t e = cudaSuccess;
+    if (!scalar && estimator == 3) {
+        static SmemOptIn opt_in_kde;
+        e = ensure_dynamic_smem(kde_kernel<BF16>, 8 * KDE_MAX_T * 4, opt_in_kde);
+        if (e != cudaSuccess) return e;
+        return launch(kde_kernel<BF16>, dim3(K / 8), dim3(256), (size_t)8 * T * 4, st, false, x, T, K, nbins, m_out);
+    }
     if (!scalar) {
         if (estimator == 1) return launch(mean_kernel<BF16>, dim3((K + 31) / 32), dim3(256), 0, st, false, x, T, K, m_out, (double *)nullptr);
         static SmemOptIn opt_in;
@@ -890,7 +999,11 @@ scap_status scap_calibrate_ex(const void *x_calib, int T, int K, scap_dtype dt, 
     if (dt != SCAP_F16 && dt != SCAP_BF16) return SCAP_ERR_DTYPE;
     if (T < 1 || T > 65535 || K < 1 || (long long)T * K >= (1ll << 31)) return SCAP_ERR_SHAPE;
     if (nbins < 0 || nbins > 2048 || !(sparsity < 1.0)) return SCAP_ERR_INVALID_ARG;
-    if ((int)estimator < 0 || (int)estimator > 2 || (int)scope < 0 || (int)scope > 1) return SCAP_ERR_INVALID_ARG;
+    if ((int)estimator < 0 || (int)estimator > 3 || (int)scope < 0 || (int)scope > 1) return SCAP_ERR_INVALID_ARG;
+    if (estimator == SCAP_MODE_KDE) {  // per channel only; the strip must fit in shared memory; nbins = grid points
+        if (scope != SCAP_ETA_PER_CHANNEL || nbins < 2) return SCAP_ERR_INVALID_ARG;
+        if (T > KDE_MAX_T) return SCAP_ERR_SHAPE;
+    }
     if (K % 8 != 0 || !aligned16(x_calib) || !aligned16(m_out) || !aligned16(ws)) return SCAP_ERR_ALIGN;
     if (ws_bytes < scap_calibrate_workspace(T, K, nbins)) return SCAP_ERR_WORKSPACE;
     scap_status st = check_device();

@@ -138,6 +138,40 @@ def test_estimators_and_scopes_bit_exact(S, estimator, scope, T, K, dt, nbins, s
     assert tau_g.view(np.uint32) == np.float32(tau_o).view(np.uint32)
 
 
+@pytest.mark.parametrize("T,K,dt,G,s", [
+    (256, 64, si.F16, 129, 0.5),
+    (300, 40, si.BF16, 64, 0.3),
+    (1000, 16, si.BF16, 2048, 0.7),
+    (3, 8, si.BF16, 2, 0.2),
+])
+def test_kde_peak_matches_the_oracle(S, T, K, dt, G, s):
+    # Both sides evaluate the densities in binary64 but with different exp routines and summation orders, so where
+    # two grid points are equally dense to within rounding either is right: the mode must be the oracle's, or a grid
+    # point whose oracle density is within 1e-9 (relative) of the oracle's maximum.  tau then follows bit for bit.
+    d = si.laplace_fc(0 if dt == si.F16 else 4, K, 8, dt, T, 1)
+    bits = d["x_calib"].copy()
+    bits[:, 3] = bits[0, 3]                               # a constant channel
+    xf = si.to_f32(bits, dt)
+    m_o = oracle.mode_estimate(xf, oracle.KDE, oracle.PER_CHANNEL, G)
+    m_g, tau_g = run_calibrate_ex(S, bits, dt, s, oracle.KDE, oracle.PER_CHANNEL, G)
+    differ = np.flatnonzero(m_g.view(np.uint32) != m_o.view(np.uint32))
+    assert len(differ) <= max(1, K // 8)
+    for k in differ:
+        dens, grid = oracle.kde_density(xf, int(k), G)
+        i = int(np.flatnonzero(grid.astype(np.float32) == m_g[k])[0])
+        assert dens[i] >= dens.max() * (1 - 1e-9)
+    assert m_g[3] == xf[0, 3]
+    assert tau_g.view(np.uint32) == np.float32(oracle.tau(xf, m_g, s)).view(np.uint32)
+
+
+def test_kde_rejects_scalar_scope_long_inputs_and_one_point_grids(S):
+    L = S.lib()
+    P = 0x10000  # never dereferenced: the argument checks come first
+    assert L.scap_calibrate_ex(P, 64, 8, 1, 0.5, 3, 1, 64, P, P, P, 1 << 30, None) == 1     # scalar scope: SCAP_ERR_INVALID_ARG
+    assert L.scap_calibrate_ex(P, 64, 8, 1, 0.5, 3, 0, 1, P, P, P, 1 << 30, None) == 1      # one grid point
+    assert L.scap_calibrate_ex(P, 5000, 8, 1, 0.5, 3, 0, 64, P, P, P, 1 << 30, None) == 2   # T > 4096: SCAP_ERR_SHAPE
+
+
 def test_skewed_inputs_median_and_mean_differ_from_the_histogram_mode(S):
     # GELU-output-like skew: the three estimators disagree, each matches its oracle, and the better mode prunes more
     rng_bits = si.to_bits(np.abs(si.normal(si.stream_seed(4, 9), 512 * 64).reshape(512, 64)) ** 1.5, si.BF16)
@@ -155,6 +189,6 @@ def test_calibrate_ex_rejects_unknown_estimator_and_scope(S):
     ws = workspace(S.scap_calibrate_workspace(16, 64, 8))
     m = torch.zeros(64, device="cuda")
     tau = torch.zeros(1, device="cuda")
-    for est, scope in ((3, 0), (-1, 0), (0, 2)):
+    for est, scope in ((4, 0), (-1, 0), (0, 2)):
         with pytest.raises(S.ScapError):
             S.scap_calibrate_ex(x, 0.5, est, scope, 8, m, tau, ws.payload)
