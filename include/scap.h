@@ -76,6 +76,7 @@ int scap_version(void);
 
 /* Process-wide tuning knobs (plain ints, not thread-safe against concurrent calls):
  *   "split_k"  cap the split-K factor (thread-block cluster size) of the FC kernel: 0 = automatic, else 1..8
+ *   "tile"     columns of the output a CTA of the FC kernel owns: 0 = automatic (default), else 128 or 256
  *   "pdl"      1 = launch dependent kernels with programmatic dependent launch (default), 0 = off
  *   "fma_rows" largest batch that runs on the fp32-FMA form of the FC kernel: 4 (default) or 2; larger
  *              batches (up to 16) run on a tensor-core form

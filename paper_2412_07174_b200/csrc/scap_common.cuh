@@ -22,6 +22,7 @@ struct Tuning {
     int fma_rows;     // largest batch that takes the fp32-FMA body (2 or 4); larger batches take a tensor-core variant
     int cal_strip;    // channels per CTA of the calibration histogram kernel: 16 or 32
     int l2_hints;     // batch 1..4 FC kernel: L2 eviction hints (keep activations and modes, stream weights)
+    int tile;         // columns per CTA of the FC kernel: 0 = automatic, else 128 or 256
 };
 extern Tuning g_tune;
 
@@ -103,6 +104,13 @@ template <bool BF16>
 __device__ __forceinline__ float widen_at(const void *p, size_t i) {
     if constexpr (BF16) return widen1(reinterpret_cast<const __nv_bfloat16 *>(p)[i]);
     else return widen1(reinterpret_cast<const __half *>(p)[i]);
+}
+
+// One 16-bit storage pattern -> float (exact).
+template <bool BF16>
+__device__ __forceinline__ float widen_bits(unsigned short u) {
+    if constexpr (BF16) return __uint_as_float((uint32_t)u << 16);
+    else return __half2float(__ushort_as_half(u));
 }
 
 // 16-byte streaming load of weights: read-only path, no L1 allocation (each byte is used once).
@@ -198,6 +206,16 @@ __device__ __forceinline__ uint4 ld_stream16(const void *p, uint64_t pol) {
                  : "l"(p), "l"(pol));
     return v;
 }
+// Predicated form: zeros where `on` does not hold (no request goes out).
+__device__ __forceinline__ uint4 ld_stream16_if(const void *p, bool on, uint64_t pol) {
+    uint4 v;
+    asm volatile(
+        "{ .reg .pred q; setp.ne.u32 q, %5, 0; mov.u32 %0, 0; mov.u32 %1, 0; mov.u32 %2, 0; mov.u32 %3, 0;"
+        " @q ld.global.nc.L1::no_allocate.L2::cache_hint.v4.u32 {%0,%1,%2,%3}, [%4], %6; }"
+        : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+        : "l"(p), "r"((unsigned)on), "l"(pol));
+    return v;
+}
 __device__ __forceinline__ float ld_nc_if(const float *p, bool on, uint64_t pol) {
     float v;
     asm volatile("{ .reg .pred q; setp.ne.u32 q, %2, 0; mov.f32 %0, 0f00000000; @q ld.global.nc.L2::cache_hint.f32 %0, [%1], %3; }"
@@ -218,6 +236,38 @@ __device__ __forceinline__ unsigned short ld_act_if_u16(const void *p, bool on, 
 }
 __device__ __forceinline__ __nv_bfloat16 ld_act_if(const __nv_bfloat16 *p, bool on, uint64_t pol) { return __ushort_as_bfloat16(ld_act_if_u16(p, on, pol)); }
 __device__ __forceinline__ __half ld_act_if(const __half *p, bool on, uint64_t pol) { return __ushort_as_half(ld_act_if_u16(p, on, pol)); }
+
+// ---- shared-memory barriers and cluster addressing (split-K exchange of the FC kernel) ---------------------
+__device__ __forceinline__ uint32_t smem_addr(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+// Address of the same shared-memory location in the CTA with rank `rank` of this cluster.
+__device__ __forceinline__ uint32_t cluster_addr(uint32_t local, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void mbarrier_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+// One arrival that also announces `bytes` of asynchronous stores still to land on the barrier.
+__device__ __forceinline__ void mbarrier_arrive_expect(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbarrier_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Asynchronous 4-byte store into another CTA of the cluster; the store itself counts 4 bytes down on that CTA's
+// barrier when it lands, so data and notification travel together (no acknowledgement, no cluster barrier).
+__device__ __forceinline__ void st_async_f32(uint32_t remote_addr, float v, uint32_t remote_bar) {
+    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.b32 [%0], %1, [%2];" ::"r"(remote_addr),
+                 "r"(__float_as_uint(v)), "r"(remote_bar) : "memory");
+}
+// Split cluster barrier: arrive early, wait where the guarantee is needed.
+__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
 
 // Hint: bring the line that holds *p into L2 (no register result, no ordering effect).
 __device__ __forceinline__ void prefetch_l2(const void *p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }

@@ -6,7 +6,7 @@
 
 namespace scap {
 
-Tuning g_tune = {0, 1, 1, 1, 4, 16, 1};
+Tuning g_tune = {0, 1, 1, 1, 4, 16, 1, 0};
 
 scap_status check_device() {
     static int cached[64];  // 0 unknown, 1 ok, 2 unsupported
@@ -74,16 +74,17 @@ int resident_ctas(int S) {
 void choose_config(int K, int Nh, int epi, int groups, int B, int *tn_out, int *S_out) {
     const int bt = fc_batch_tile(B), cap = is_mma(bt) ? mma_cap(bt) : fc_cap(bt);
     const int nchunks = (K + 31) / 32;
-    int best_tn = 256, best_S = 1;
+    int best_tn = g_tune.tile ? g_tune.tile : 256, best_S = 1;
     long long best = -1;
     for (int tn = 128; tn <= 256; tn <<= 1) {
+        if (g_tune.tile && tn != g_tune.tile) continue;
         const int tiles = fc_tiles(Nh, epi, tn);
         for (int S = MAX_CLUSTER; S >= 1; --S) {
             if (g_tune.split_k > 0 && S > g_tune.split_k) continue;
             if (S > 1 && K / S < 64) continue;
             const long long ctas = (long long)tiles * groups * S;
             const int budget = resident_ctas(S);
-            if (ctas > budget && !(S == 1 && tn == 256)) continue;
+            if (ctas > budget && !(S == 1 && tn == (g_tune.tile ? g_tune.tile : 256))) continue;
             const int fills = ((nchunks + S - 1) / S * 32 + cap - 1) / cap;
             const long long score = ctas > budget ? 0 : ctas * 64 + (63 - (fills < 63 ? fills : 63));
             if (score > best) { best = score; best_tn = tn; best_S = S; }
@@ -140,6 +141,7 @@ cudaError_t launch_fc(bool bf16, int mode, int xkind, int epi, const FcArgs &a, 
     }
     FcArgs f = a;
     f.l2_hints = g_tune.l2_hints;
+    f.status = tc_status_ptr();
     return bf16 ? launch_fc_w<true>(mode, xkind, epi, f, st) : launch_fc_w<false>(mode, xkind, epi, f, st);
 }
 
@@ -288,6 +290,11 @@ scap_status scap_tune(const char *key, int value) {
     }
     if (!strcmp(key, "l2_hints")) {
         g_tune.l2_hints = value != 0;
+        return SCAP_OK;
+    }
+    if (!strcmp(key, "tile")) {
+        if (value != 0 && value != 128 && value != 256) return SCAP_ERR_INVALID_ARG;
+        g_tune.tile = value;
         return SCAP_OK;
     }
     if (!strcmp(key, "tcgen05")) {

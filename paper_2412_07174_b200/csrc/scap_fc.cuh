@@ -68,6 +68,7 @@ struct FcArgs {
     int act;              // EPI_BIAS: 1 = the exact GELU is applied to the biased result (z_copy then gets a copy)
     const float *wscale;  // 8-bit weights only: one scale per input channel, W[k,n] = wscale[k] * Wq[k,n]
     int l2_hints;         // fp32-FMA body: 1 = loads carry L2 eviction hints (keep x and m, stream W)
+    int *status;          // device status word: set when a bounded wait runs out (NULL: not recorded)
 };
 
 template <bool BF16, int BT, int CAP>
@@ -128,6 +129,32 @@ __device__ __forceinline__ void reduce_push_round(const float *__restrict__ s_re
 #pragma unroll
             for (int q = 0; q < MAX_CLUSTER; ++q)
                 if (q == r) owner[q][slot] = v;
+        }
+    }
+}
+
+// The same reduction round with the asynchronous exchange: every element goes to its owner as a store that counts
+// down the owner's shared-memory barrier when it lands.
+template <int BT, int EPI, int TNT, int NRED, int RBX>
+__device__ __forceinline__ void reduce_send_round(const float *__restrict__ s_red, int b0, int B, int s, int per, uint32_t gather_local,
+                                                  uint32_t bar_local) {
+    constexpr int HALF = TNT / 2;
+    for (int i = threadIdx.x; i < RBX * TNT; i += FC_THREADS) {
+        const int rb = i / TNT, c = i - rb * TNT, b = b0 + rb;
+        float v = 0.0f;
+#pragma unroll
+        for (int g = 0; g < NRED; ++g) v += s_red[(g * RBX + rb) * TNT + c];
+        if (b < B) {
+            int r, slot;
+            if constexpr (EPI == EPI_GLU) {
+                const int j = c % HALF, hf = c / HALF;
+                r = j / per;
+                slot = ((s * BT + b) * 2 + hf) * per + (j - r * per);
+            } else {
+                r = c / per;
+                slot = (s * BT + b) * per + (c - r * per);
+            }
+            st_async_f32(cluster_addr(gather_local + 4u * (uint32_t)slot, (uint32_t)r), v, cluster_addr(bar_local, (uint32_t)r));
         }
     }
 }
@@ -212,6 +239,7 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
     uint32_t *s_bits = reinterpret_cast<uint32_t *>(s_gather + BT * GATHER_LD);
     int *s_rows = reinterpret_cast<int *>(s_bits + CAPC);  // source row of x per batch row (when a row map is given)
     int *s_wcnt = s_rows + 16;                             // kept channels per warp, this fill
+    const uint32_t bar = smem_addr(s_wcnt + FC_WARPS);     // 8 bytes: barrier the split-K partials of this rank's columns land on
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int rg = tid / LPR, cl = tid % LPR;  // row group and column lane of this thread
@@ -234,6 +262,17 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
 
     // columns (EPI_GLU: gate/up pairs) this rank finishes after the cluster exchange
     const int per = ((EPI == EPI_GLU ? HALF : TNT) + S - 1) / S;  // the last rank may own fewer
+    if (S > 1) {
+        // This rank will receive S * B * (columns it owns) partial sums (gate and up: twice that) on its barrier.
+        // The arrival half of a cluster barrier publishes the initialised barrier; the waiting half sits before the
+        // first send, by which time every rank has long arrived.
+        if (tid == 0) {
+            const int owned = max(0, min(per, (EPI == EPI_GLU ? HALF : TNT) - s * per));
+            mbarrier_init(bar, 1);
+            mbarrier_arrive_expect(bar, (uint32_t)(S * B * owned * (EPI == EPI_GLU ? 8 : 4)));
+        }
+        cluster_arrive();
+    }
     float bias0[2], bias1[2];
     prefetch_bias<BF16, EPI, TNT>(a, tile, s, per, bias0, bias1);
 
@@ -372,12 +411,14 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
             constexpr int G = U / 2;
             const int nrows = cnt > rg ? (cnt - rg + NR - 1) / NR : 0;
             uint4 ga[G], gb[G];
+            // the first 2 G requests go out without a branch (predicated loads; list entries beyond the count are
+            // never dereferenced)
 #pragma unroll
             for (int u = 0; u < G; ++u)
-                if (u < nrows) ga[u] = ld_stream16(Wb + (size_t)s_k[rg + NR * u] * row_bytes, pol_stream);
+                ga[u] = ld_stream16_if(Wb + (size_t)s_k[rg + NR * u] * row_bytes, u < nrows, pol_stream);
 #pragma unroll
             for (int u = 0; u < G; ++u)
-                if (G + u < nrows) gb[u] = ld_stream16(Wb + (size_t)s_k[rg + NR * (G + u)] * row_bytes, pol_stream);
+                gb[u] = ld_stream16_if(Wb + (size_t)s_k[rg + NR * (G + u)] * row_bytes, G + u < nrows, pol_stream);
             for (int t0 = 0; t0 < nrows; t0 += 2 * G) {
 #pragma unroll
                 for (int u = 0; u < G; ++u)
@@ -397,26 +438,31 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
     }
 
     // ---- reduction over the row groups in group order; each finished element of this CTA's partial tile is
-    // pushed into the shared memory of the cluster rank that owns its column (slot = this rank), so one cluster
-    // barrier later every rank holds all S partials of its columns and adds them in rank order.
-    cg::cluster_group cluster = cg::this_cluster();
-    float *owner[MAX_CLUSTER];
+    // sent to the shared memory of the cluster rank that owns its column (slot = this rank) as an asynchronous
+    // store that counts down the owner's barrier.  A rank finishes its columns as soon as its own S partials are
+    // in - it neither waits for the other ranks' exchanges nor for an acknowledgement of its own stores - and adds
+    // them in rank order.
+    static_assert(RB == BT, "one reduction round");
+    if (S > 1) cluster_wait();  // every rank's barrier is initialised (all ranks arrived at kernel start)
 #pragma unroll
-    for (int q = 0; q < MAX_CLUSTER; ++q) owner[q] = (S > 1 && q < S) ? cluster.map_shared_rank(s_gather, q) : s_gather;
+    for (int rb = 0; rb < RB; ++rb) {
+        float4 *dst = reinterpret_cast<float4 *>(s_red + ((rg * RB + rb) * TNT + cl * 8));
+        dst[0] = make_float4(acc[rb][0], acc[rb][1], acc[rb][2], acc[rb][3]);
+        dst[1] = make_float4(acc[rb][4], acc[rb][5], acc[rb][6], acc[rb][7]);
+    }
+    __syncthreads();
+    if (S > 1) {
+        reduce_send_round<BT, EPI, TNT, NR, RB>(s_red, 0, B, s, per, smem_addr(s_gather), bar);
+        bool landed = false;
+        for (uint32_t it = 0; it < (1u << 22) && !landed; ++it) landed = mbarrier_try_wait(bar, 0);
+        if (!landed && a.status) atomicCAS(a.status, 0, 2);  // never in a correct run; the result is then incomplete
+    } else {
+        float *owner[MAX_CLUSTER];
 #pragma unroll
-    for (int b0 = 0; b0 < BT; b0 += RB) {
-#pragma unroll
-        for (int rb = 0; rb < RB; ++rb) {
-            float4 *dst = reinterpret_cast<float4 *>(s_red + ((rg * RB + rb) * TNT + cl * 8));
-            dst[0] = make_float4(acc[b0 + rb][0], acc[b0 + rb][1], acc[b0 + rb][2], acc[b0 + rb][3]);
-            dst[1] = make_float4(acc[b0 + rb][4], acc[b0 + rb][5], acc[b0 + rb][6], acc[b0 + rb][7]);
-        }
-        __syncthreads();
-        reduce_push_round<BT, EPI, TNT, NR, RB>(s_red, b0, B, s, per, owner);
+        for (int q = 0; q < MAX_CLUSTER; ++q) owner[q] = s_gather;
+        reduce_push_round<BT, EPI, TNT, NR, RB>(s_red, 0, B, s, per, owner);
         __syncthreads();
     }
-    if (S > 1) cluster.sync();  // all pushes have landed; nothing remote is touched after this point
-    else __syncthreads();
 
     finish_columns<BF16, BT, EPI, TNT>(a, tile, s, per, s_gather, bias0, bias1);
 }
@@ -855,6 +901,7 @@ bool tc_applicable(const FcArgs &a, int epi, bool bf16);
 int tc_choose_split(int K, int Nh, int epi, int B, bool bf16);
 cudaError_t launch_fc_tc(bool bf16, int mode, int xkind, int epi, const FcArgs &a, cudaStream_t st);
 int tc_take_status();
+int *tc_status_ptr();  // device address of that status word on the current device (NULL if it cannot be had)
 
 // Launch with cluster dimension (1, S, 1) and, if enabled, programmatic dependent launch.
 template <typename... KArgs, typename... Args>

@@ -505,6 +505,18 @@ cudaError_t launch_fc_tc(bool bf16, int mode, int xkind, int epi, const FcArgs &
     return bf16 ? launch_tc_w<true>(mode, xkind, epi, a, st) : launch_tc_w<false>(mode, xkind, epi, a, st);
 }
 
+// Device address of the status word of the bounded waits, looked up once per device.
+int *tc_status_ptr() {
+    static int *cached[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+    if (dev >= 0 && dev < 64 && cached[dev]) return cached[dev];
+    int *p = nullptr;
+    if (cudaGetSymbolAddress(reinterpret_cast<void **>(&p), g_tc_status) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+    if (dev >= 0 && dev < 64) cached[dev] = p;
+    return p;
+}
+
 // Reads and clears the status word of the bounded waits (synchronises the device).
 int tc_take_status() {
     int v = 0, zero = 0;
