@@ -30,12 +30,12 @@
  *     SCAP_ERR_CUDA, a device that is not compute capability 10.x SCAP_ERR_UNSUPPORTED_ARCH.
  *     Nothing throws, aborts, traps or prints.  On error nothing has been enqueued.
  *   - Workspace contents are scratch: undefined on entry, undefined on exit.
- *   - Layer parameters (W, m, tau, biases) are read as soon as a kernel becomes resident, which with
- *     programmatic dependent launch can be before the previous scap_sparse_fc / scap_dense_fc /
- *     scap_glu_ffn / scap_moe_ffn call on the stream has finished; only activations (x, h, logits)
- *     wait for it.  So a parameter must not be an OUTPUT of such a call placed directly before on the
- *     same stream.  Parameters written by scap_calibrate, scap_fold_bias or any other kernel are safe:
- *     those complete before the next kernel starts.
+ *   - Every kernel of a call waits for the work placed before it on the stream before it reads anything - the
+ *     activations, and equally W, m, tau, the scales and the biases - and reads whatever a kernel may have
+ *     rewritten through L2.  So parameters may be produced on the same stream directly before the call that
+ *     uses them (scap_calibrate, scap_fold_bias, or any kernel or copy of the caller's), with no further
+ *     synchronisation.  Consecutive calls still overlap where they can: a kernel may become resident and set up
+ *     its shared memory while its predecessor drains (programmatic dependent launch, "pdl" below).
  */
 #ifndef SCAP_H_
 #define SCAP_H_

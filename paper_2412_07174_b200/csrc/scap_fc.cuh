@@ -98,8 +98,8 @@ __device__ __forceinline__ void store_result(const FcArgs &a, int row, int b, in
 
 template <bool BF16>
 __device__ __forceinline__ float load_bias(const FcArgs &a, int n) {
-    float bv = a.bias ? __ldg(a.bias + n) : 0.0f;
-    if (a.bias16) bv += widen_at<BF16>(a.bias16, n);
+    float bv = a.bias ? __ldcg(a.bias + n) : 0.0f;
+    if (a.bias16) bv += widen_bits<BF16>(__ldcg(reinterpret_cast<const unsigned short *>(a.bias16) + n));
     return bv;
 }
 
@@ -182,8 +182,8 @@ __device__ __forceinline__ void finish_columns(const FcArgs &a, int tile, int s,
         } else {
             const int F = a.Nh, f = tile * HALF + s * per + c;
             if (s * per + c < HALF && f < F) {
-                float g = it == 0 ? bias0[0] : it == 1 ? bias0[1] : (a.bias ? __ldg(a.bias + f) : 0.0f);
-                float u = it == 0 ? bias1[0] : it == 1 ? bias1[1] : (a.bias ? __ldg(a.bias + F + f) : 0.0f);
+                float g = it == 0 ? bias0[0] : it == 1 ? bias0[1] : (a.bias ? __ldcg(a.bias + f) : 0.0f);
+                float u = it == 0 ? bias1[0] : it == 1 ? bias1[1] : (a.bias ? __ldcg(a.bias + F + f) : 0.0f);
 #pragma unroll
                 for (int q = 0; q < MAX_CLUSTER; ++q)
                     if (q < S) {
@@ -198,7 +198,8 @@ __device__ __forceinline__ void finish_columns(const FcArgs &a, int tile, int s,
     }
 }
 
-// Bias of the columns this rank finishes, fetched at kernel start so that the load is off the critical path.
+// Bias of the columns this rank finishes, requested (through L2) before the row stream starts so that the load is off
+// the critical path.
 template <bool BF16, int EPI, int TNT>
 __device__ __forceinline__ void prefetch_bias(const FcArgs &a, int tile, int s, int per, float (&bias0)[2], float (&bias1)[2]) {
     constexpr int HALF = TNT / 2;
@@ -210,7 +211,7 @@ __device__ __forceinline__ void prefetch_bias(const FcArgs &a, int tile, int s, 
             const int c = i % per;
             if constexpr (EPI == EPI_GLU) {
                 const int f = tile * HALF + s * per + c;
-                if (s * per + c < HALF && f < a.Nh && a.bias) { bias0[it] = __ldg(a.bias + f); bias1[it] = __ldg(a.bias + a.Nh + f); }
+                if (s * per + c < HALF && f < a.Nh && a.bias) { bias0[it] = __ldcg(a.bias + f); bias1[it] = __ldcg(a.bias + a.Nh + f); }
             } else {
                 const int n = tile * TNT + s * per + c;
                 if (s * per + c < TNT && n < a.Nh) bias0[it] = load_bias<BF16>(a, n);
@@ -221,9 +222,10 @@ __device__ __forceinline__ void prefetch_bias(const FcArgs &a, int tile, int s, 
 
 // Body for column tile `tile` and cluster rank `s`; every thread of every CTA of the cluster calls it.
 // TNT = columns per CTA (256 or 128): a row segment is TNT/8 lanes wide, so a warp streams 1 or 2 rows per load.
-// With wait_inside the body itself waits for the previous kernel in the stream, and does so as late as it can:
-// W, m, tau and the biases are layer parameters, not outputs of the previous kernel, so they are read first and
-// only the activation x is read after the wait.
+// With wait_inside the body itself waits for the previous kernel in the stream before it reads anything: the
+// activations, and equally tau, m and the biases, may have been written by any earlier work on the stream.  No load
+// or prefetch goes out before that wait (measured: memory operations issued ahead of it delay its return for the
+// CTAs that become resident late, 0.15 - 0.2 us per call), and everything a kernel may rewrite is read through L2.
 template <bool BF16, int BT, int MODE, typename XT, int EPI, int TNT>
 __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const int s, const bool wait_inside) {
     constexpr int NT = FC_THREADS, PU = fc_pu(BT), CAP = fc_cap(BT), RB = fc_rb(BT), U = fc_unroll(BT);
@@ -274,7 +276,6 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
         cluster_arrive();
     }
     float bias0[2], bias1[2];
-    prefetch_bias<BF16, EPI, TNT>(a, tile, s, per, bias0, bias1);
 
     float acc[BT][8];
 #pragma unroll
@@ -285,20 +286,20 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
     const int nchunks = (K + 31) >> 5;
     const int my_chunks = nchunks > s ? (nchunks - s + S - 1) / S : 0;  // chunks s, s+S, ...
     float tau = 0.0f;
-    if constexpr (MODE == MODE_GATHER) tau = ld_nc(a.tau);
     // x and m are read again by every column tile of the call (and m by every later call): ask L2 to keep them and
     // to drop the weight rows, which are read once, first.
     const uint64_t pol_keep = a.l2_hints ? l2_policy_keep() : l2_policy_normal();
     const uint64_t pol_stream = a.l2_hints ? l2_policy_stream() : l2_policy_normal();
 
-    if (wait_inside && (my_chunks == 0 || a.in_rows)) {
-        griddep_wait();
-        griddep_launch_dependents();
+    if (wait_inside) {
+        griddep_wait();               // everything earlier work on the stream wrote (activations, parameters) is complete and visible
+        griddep_launch_dependents();  // the next kernel may begin launching; it waits for this grid itself
     }
     if (a.in_rows) {  // one L2 read per CTA and row (the map is an output of the previous kernel), then broadcast
         if (tid < BT) s_rows[tid] = __ldcg(a.in_rows + (tid < B ? tid : 0));
         __syncthreads();
     }
+    bool bias_done = false;
     for (int j0 = 0; j0 < my_chunks; j0 += CAPC) {
         const int nj = min(CAPC, my_chunks - j0);
         const int pw = (nj + FC_WARPS - 1) / FC_WARPS;  // chunks per warp this fill: warp w owns chunks w * pw .. w * pw + pw - 1
@@ -312,34 +313,23 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
         for (int p = 0; p < PU; ++p) {
             const int j = warp * pw + p;
             const int k = (s + S * (j0 + j)) * 32 + lane;
-            mk[p] = a.m ? ld_nc_if(a.m + k, p < pw && j < nj && k < K, pol_keep) : 0.0f;
-        }
-        if (wait_inside && j0 == 0 && !a.in_rows) {
-            // Pull this CTA's slice of x towards L2 while the previous kernel drains.  L2 is the coherence point,
-            // so a line the previous kernel still writes stays correct; the values are only read after the wait.
-#pragma unroll
-            for (int p = 0; p < PU; ++p) {
-                const int j = warp * pw + p;
-                const int k = (s + S * j) * 32 + lane;
-                if (p < pw && j < nj && k < K) {
-#pragma unroll
-                    for (int b = 0; b < BT; ++b)
-                        if (b < B) prefetch_l2(xg + (size_t)b * a.x_ld + k);
-                }
-            }
-            griddep_wait();               // x (produced by the previous kernel in the stream) is complete
-            griddep_launch_dependents();  // the next kernel may begin launching; it waits for this grid itself
-        }
-#pragma unroll
-        for (int p = 0; p < PU; ++p) {
-            const int j = warp * pw + p;
-            const int k = (s + S * (j0 + j)) * 32 + lane;
             const bool ok = p < pw && j < nj && k < K;
 #pragma unroll
             for (int b = 0; b < BT; ++b) {
                 const int bb = b < B ? b : 0;
                 xraw[p][b] = ld_act_if(xg + (size_t)(a.in_rows ? s_rows[bb] : bb) * a.x_ld + k, ok && b < B, pol_keep);
             }
+        }
+        if (MODE == MODE_GATHER && j0 == 0) {  // one request per warp, in flight together with the loads around it
+            float tv = 0.0f;
+            if (lane == 0) tv = ld_act(a.tau);
+            tau = __shfl_sync(0xffffffffu, tv, 0);
+        }
+#pragma unroll
+        for (int p = 0; p < PU; ++p) {
+            const int j = warp * pw + p;
+            const int k = (s + S * (j0 + j)) * 32 + lane;
+            mk[p] = a.m ? ld_act_if(a.m + k, p < pw && j < nj && k < K, pol_keep) : 0.0f;
         }
 #pragma unroll
         for (int p = 0; p < PU; ++p)
@@ -405,6 +395,7 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
         }
         __syncthreads();
 
+        if (!bias_done) { prefetch_bias<BF16, EPI, TNT>(a, tile, s, per, bias0, bias1); bias_done = true; }
         // ---- stream the kept rows: row group g takes rows g, g+NR, ...  Two register groups of G loads alternate
         // (one is consumed while the other is in flight).
         if (col_ok) {
@@ -437,6 +428,7 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
         __syncthreads();
     }
 
+    if (!bias_done) prefetch_bias<BF16, EPI, TNT>(a, tile, s, per, bias0, bias1);
     // ---- reduction over the row groups in group order; each finished element of this CTA's partial tile is
     // sent to the shared memory of the cluster rank that owns its column (slot = this rank) as an asynchronous
     // store that counts down the owner's barrier.  A rank finishes its columns as soon as its own S partials are
@@ -571,7 +563,6 @@ __device__ __forceinline__ void fc_body_mma(const FcArgs &a, const int tile, con
 
     const int per = ((EPI == EPI_GLU ? HALF : TNT) + S - 1) / S;  // the last rank may own fewer
     float bias0[2], bias1[2];
-    prefetch_bias<BF16, EPI, TNT>(a, tile, s, per, bias0, bias1);
 
     float acc[8][4];
 #pragma unroll
@@ -582,12 +573,17 @@ __device__ __forceinline__ void fc_body_mma(const FcArgs &a, const int tile, con
     const int nchunks = (K + 31) >> 5;
     const int my_chunks = nchunks > s ? (nchunks - s + S - 1) / S : 0;
     float tau = 0.0f;
-    if constexpr (MODE == MODE_GATHER) tau = ld_nc(a.tau);
 
-    if (wait_inside) {  // the row map and the activations are outputs of the previous kernel
+    if (wait_inside) {  // nothing is read before earlier work on the stream is complete
         griddep_wait();
         griddep_launch_dependents();
     }
+    if constexpr (MODE == MODE_GATHER) {
+        float tv = 0.0f;
+        if (lane == 0) tv = ld_act(a.tau);
+        tau = __shfl_sync(0xffffffffu, tv, 0);
+    }
+    prefetch_bias<BF16, EPI, TNT>(a, tile, s, per, bias0, bias1);
     if (a.in_rows) {  // one L2 read per CTA and row, then broadcast
         if (tid < BT) s_rows[tid] = __ldcg(a.in_rows + (tid < B ? tid : 0));
         __syncthreads();
@@ -607,7 +603,7 @@ __device__ __forceinline__ void fc_body_mma(const FcArgs &a, const int tile, con
         for (int p = 0; p < PU; ++p) {
             const int j = p * FC_WARPS + warp;
             const int k = (s + S * (j0 + j)) * 32 + lane;
-            mk[p] = a.m ? ld_nc_if(a.m + k, j < nj && k < K) : 0.0f;
+            mk[p] = a.m ? ld_act_if(a.m + k, j < nj && k < K) : 0.0f;
         }
         uint32_t km[PU];
         unsigned bal[PU];
@@ -854,8 +850,8 @@ __device__ __forceinline__ void fc_body_mma(const FcArgs &a, const int tile, con
                     pg[q] = q < S ? peer[q][b * TNT + s * per + c] : 0.0f;
                     pu[q] = q < S ? peer[q][b * TNT + HALF + s * per + c] : 0.0f;
                 }
-                float gt = it == 0 ? bias0[0] : it == 1 ? bias0[1] : (a.bias ? __ldg(a.bias + f) : 0.0f);
-                float up = it == 0 ? bias1[0] : it == 1 ? bias1[1] : (a.bias ? __ldg(a.bias + F + f) : 0.0f);
+                float gt = it == 0 ? bias0[0] : it == 1 ? bias0[1] : (a.bias ? __ldcg(a.bias + f) : 0.0f);
+                float up = it == 0 ? bias1[0] : it == 1 ? bias1[1] : (a.bias ? __ldcg(a.bias + F + f) : 0.0f);
 #pragma unroll
                 for (int q = 0; q < MAX_CLUSTER; ++q)
                     if (q < S) {

@@ -66,7 +66,6 @@ __global__ void __launch_bounds__(FC_THREADS, 2) fc_q8_kernel(const FcArgs a) {
 
     const int per = (TNT + S - 1) / S;
     float bias0[2], bias1[2];
-    prefetch_bias<true, EPI, TNT>(a, tile, s, per, bias0, bias1);
 
     float acc[BT][16];
 #pragma unroll
@@ -77,11 +76,16 @@ __global__ void __launch_bounds__(FC_THREADS, 2) fc_q8_kernel(const FcArgs a) {
     const int nchunks = (K + 31) >> 5;
     const int my_chunks = nchunks > s ? (nchunks - s + S - 1) / S : 0;
     float tau = 0.0f;
-    if constexpr (MODE == MODE_GATHER) tau = ld_nc(a.tau);
-    if (my_chunks == 0 || a.hold_dependents) {
-        griddep_wait();
-        if (!a.hold_dependents) griddep_launch_dependents();
+    // Nothing is read before earlier work on the stream is complete: tau, m, the scales and the biases may have been
+    // written by it just as the activations may; all of them are read through L2.
+    griddep_wait();
+    if (!a.hold_dependents) griddep_launch_dependents();
+    if constexpr (MODE == MODE_GATHER) {
+        float tv = 0.0f;
+        if (lane == 0) tv = ld_act(a.tau);
+        tau = __shfl_sync(0xffffffffu, tv, 0);
     }
+    prefetch_bias<true, EPI, TNT>(a, tile, s, per, bias0, bias1);
     for (int j0 = 0; j0 < my_chunks; j0 += CAPC) {
         const int nj = min(CAPC, my_chunks - j0);
         const int pw = (nj + FC_WARPS - 1) / FC_WARPS;  // chunks per warp this fill: warp w owns chunks w * pw .. w * pw + pw - 1
@@ -91,12 +95,8 @@ __global__ void __launch_bounds__(FC_THREADS, 2) fc_q8_kernel(const FcArgs a) {
         for (int p = 0; p < PU; ++p) {
             const int j = warp * pw + p;
             const int k = (s + S * (j0 + j)) * 32 + lane;
-            mk[p] = a.m ? ld_nc_if(a.m + k, p < pw && j < nj && k < K) : 0.0f;
-            sc[p] = ld_nc_if(a.wscale + k, p < pw && j < nj && k < K);
-        }
-        if (j0 == 0 && !a.hold_dependents) {
-            griddep_wait();
-            griddep_launch_dependents();
+            mk[p] = a.m ? ld_act_if(a.m + k, p < pw && j < nj && k < K) : 0.0f;
+            sc[p] = ld_act_if(a.wscale + k, p < pw && j < nj && k < K);
         }
 #pragma unroll
         for (int p = 0; p < PU; ++p) {

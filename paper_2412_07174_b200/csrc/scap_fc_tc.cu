@@ -152,15 +152,19 @@ __global__ void __launch_bounds__(FC_THREADS, 2) fc_tc_kernel(const FcArgs a) {
 
     const int per = ((EPI == EPI_GLU ? HALF : TNT) + S - 1) / S;
     float bias0[2], bias1[2];
-    prefetch_bias<BF16, EPI, TNT>(a, tile, s, per, bias0, bias1);
 
     const int nchunks = (K + 31) >> 5;
     const int my_chunks = nchunks > s ? (nchunks - s + S - 1) / S : 0;
     float tau = 0.0f;
-    if constexpr (MODE == MODE_GATHER) tau = ld_nc(a.tau);
 
-    griddep_wait();  // the row map and the activations are outputs of the previous kernel
+    griddep_wait();  // nothing (activations, row map, tau, m, biases) is read before earlier work on the stream is complete
     griddep_launch_dependents();
+    if constexpr (MODE == MODE_GATHER) {
+        float tv = 0.0f;
+        if (lane == 0) tv = ld_act(a.tau);
+        tau = __shfl_sync(0xffffffffu, tv, 0);
+    }
+    prefetch_bias<BF16, EPI, TNT>(a, tile, s, per, bias0, bias1);
     if (a.in_rows && tid < 16) misc->rows[tid] = __ldcg(a.in_rows + (tid < B ? tid : 0));
     tc_fence_before();
     __syncthreads();
@@ -184,7 +188,7 @@ __global__ void __launch_bounds__(FC_THREADS, 2) fc_tc_kernel(const FcArgs a) {
         for (int p = 0; p < PU; ++p) {
             const int j = warp * pu + p;
             const int k = (s + S * (j0 + j)) * 32 + lane;
-            mk[p] = a.m ? ld_nc_if(a.m + k, p < pu && j < nj && k < K) : 0.0f;
+            mk[p] = a.m ? ld_act_if(a.m + k, p < pu && j < nj && k < K) : 0.0f;
         }
 #pragma unroll
         for (int p = 0; p < PU; ++p) {
@@ -412,8 +416,8 @@ __global__ void __launch_bounds__(FC_THREADS, 2) fc_tc_kernel(const FcArgs a) {
         } else {
             const int F = a.Nh, f = tile * HALF + s * per + c;
             if (s * per + c < HALF && f < F) {
-                float gt = it == 0 ? bias0[0] : it == 1 ? bias0[1] : (a.bias ? __ldg(a.bias + f) : 0.0f);
-                float up = it == 0 ? bias1[0] : it == 1 ? bias1[1] : (a.bias ? __ldg(a.bias + F + f) : 0.0f);
+                float gt = it == 0 ? bias0[0] : it == 1 ? bias0[1] : (a.bias ? __ldcg(a.bias + f) : 0.0f);
+                float up = it == 0 ? bias1[0] : it == 1 ? bias1[1] : (a.bias ? __ldcg(a.bias + F + f) : 0.0f);
 #pragma unroll
                 for (int q = 0; q < MAX_CLUSTER; ++q)
                     if (q < S) {
