@@ -4,10 +4,10 @@
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--detail]
 
 Workload (N = 1): the Llama-2-7B-shaped FFN down projection, bf16, batch 1 - W[K=11008, N=4096] ~ N(0, 0.02^2),
-inputs silu(g)*u with g, u ~ N(0,1), mode and tau calibrated on 1024 tokens at sparsity targets 50 / 65 / 80 %.
-One step = one sparse FC call (one fused kernel: threshold + compaction + gather-GEMV + reduction) per sparsity target on
-each of R device copies of W, R chosen so that even the sparsest call pattern touches at least four times the L2 size
-per cycle: no call finds its weight rows in L2.
+inputs silu(g)*u with g, u ~ N(0,1), mode and tau calibrated on 1024 tokens at sparsity targets 50 / 60 / 65 / 80 / 90 %.
+One step = PASSES passes over R device copies of W, each pass one sparse FC call (one fused kernel: threshold +
+compaction + gather-GEMV + reduction) per sparsity target and copy; R is chosen so that even the sparsest call pattern
+touches at least four times the L2 size per cycle: no call finds its weight rows in L2.
 The metric is effective HBM GB/s on the bytes a call must touch (kept rows + activations + mode + bias + output),
 summed over the step; the JSON line also carries us/call per sparsity, the library's own dense GEMV on the same
 rotation, the speedup over it, the roofline fraction against the measured copy bandwidth, an end-to-end number
@@ -35,7 +35,9 @@ if ROOT not in sys.path:
 import scap_inputs as si  # noqa: E402
 
 K, N = 11008, 4096
-SPARSITIES = (0.5, 0.65, 0.8)
+SPARSITIES = (0.5, 0.6, 0.65, 0.8, 0.9)
+PASSES = 12          # passes over the weight rotation per step (one step is about 15 ms of device time)
+WORKLOAD = "llama2_7b_down_proj_bf16_b1 (K=11008,N=4096), sparsity targets 50/60/65/80/90%"
 N_INPUTS = 64
 NBINS = 2048
 T_CALIB = 1024
@@ -110,6 +112,16 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
+def cpu_model() -> str:
+    try:
+        for ln in open("/proc/cpuinfo"):
+            if ln.lower().startswith("model name"):
+                return ln.split(":", 1)[1].strip()
+    except OSError:
+        pass
+    return "unknown"
+
+
 def oracle_step(d, cal, x_rows, threads: int):
     """One bounded CPU sample: the oracle's sparse FC once per sparsity target (one weight copy)."""
     import oracle
@@ -161,7 +173,7 @@ def run_reference(args, rank):
         oracle_step(d, cal, d["x"], cores)
     tot_t, tot_b = 0.0, 0
     for k in range(args.steps):
-        t, b = oracle_step(d, cal, d["x"][3 * (k % 20):], cores)
+        t, b = oracle_step(d, cal, d["x"][len(SPARSITIES) * (k % 12):], cores)
         tot_t += t
         tot_b += b
     val = tot_b / tot_t / 1e9
@@ -169,10 +181,10 @@ def run_reference(args, rank):
         "impl": "reference", "metric": "sparse_fc_effective_hbm_gbs", "value": val, "unit": "GB/s", "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * tot_t / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": "llama2_7b_down_proj_bf16_b1 (K=11008,N=4096), sparsity 50/65/80%",
-                   "sample": "one oracle sparse-FC call per sparsity target per step (3 calls)"},
-        "cpu_baseline": {"value": val, "unit": "GB/s", "cores": cores, "kind": "oracle",
-                         "sample": "3 calls per step x %d steps" % args.steps},
+        "config": {"workload": WORKLOAD,
+                   "sample": "one oracle sparse-FC call per sparsity target per step (%d calls)" % len(SPARSITIES)},
+        "cpu_baseline": {"value": val, "unit": "GB/s", "cores": cores, "kind": "oracle", "cpu_model": cpu_model(),
+                         "sample": "%d calls per step x %d steps" % (len(SPARSITIES), args.steps)},
         "e2e": {"value": val, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
@@ -539,8 +551,8 @@ def run_suite(args):
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one fc_kernel launch from the ncu capture summarised under
 # profiles/ (None whenever the kernel has changed since that capture).
-NCU_TRAFFIC_BYTES = 31950592
-NCU_TRAFFIC_NOTE = "ncu capture of one launch at the 65% target (algorithmic bytes of that launch: 31.8 MB)"
+NCU_TRAFFIC_BYTES = None
+NCU_TRAFFIC_NOTE = "not re-captured since the kernel last changed"
 
 
 def main():
@@ -685,8 +697,14 @@ def main():
             stream.synchronize()
         return e0.elapsed_time(e1) / reps  # ms per replay
 
-    g_step, step_bytes = capture(lambda: sparse_calls(SPARSITIES, [0]))
-    calls_per_step = len(SPARSITIES) * R
+    def step_calls(counter):
+        nb = 0
+        for _ in range(PASSES):
+            nb += sparse_calls(SPARSITIES, counter)
+        return nb
+
+    g_step, step_bytes = capture(lambda: step_calls([0]))
+    calls_per_step = PASSES * len(SPARSITIES) * R
     launches_per_step = calls_per_step  # one fused kernel per call
 
     # ------------------------------------------------------------------ timed region: K steps, device time, max over ranks
@@ -697,18 +715,19 @@ def main():
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    marks = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
     with torch.cuda.stream(stream):
-        e0.record(stream)
-        for _ in range(args.steps):
+        marks[0].record(stream)
+        for k in range(args.steps):
             g_step.replay()
-        e1.record(stream)
+            marks[k + 1].record(stream)
     barrier()
     clocks = sampler.stop() if rank == 0 else None
-    ms = e0.elapsed_time(e1)
+    ms = marks[0].elapsed_time(marks[-1])
     ms = max_over_ranks(ms, world, "cuda")
     ms_per_step = ms / args.steps
     value = whole_job_gbs(step_bytes, world, ms_per_step * 1e-3)
+    step_us_per_call = np.array([marks[k].elapsed_time(marks[k + 1]) for k in range(args.steps)]) * 1e3 / calls_per_step
 
     # ------------------------------------------------------------------ per-sparsity and dense detail (rank 0 reports)
     detail = {}
@@ -723,10 +742,36 @@ def main():
     dense_us = 1e3 * t_dense / R
     dense_gbs = nb_dense / (t_dense * 1e-3) / 1e9
 
+    # the same calls as plain launches (no graph): every launch goes through the Python binding, so this figure is
+    # bound by the host's launch rate, not by the kernel
+    with torch.cuda.stream(stream):
+        sparse_calls(SPARSITIES, [0])
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        stream.synchronize()
+        e0.record(stream)
+        for _ in range(3):
+            sparse_calls(SPARSITIES, [0])
+        e1.record(stream)
+        stream.synchronize()
+    plain_us = e0.elapsed_time(e1) * 1e3 / (3 * len(SPARSITIES) * R)
+
+    # L2-warm: every call reads the same weight copy, so from about 65 % sparsity up the kept rows are found in L2
+    def warm_calls(s):
+        m, tau, bf = cal[s]
+        for r in range(R):
+            scap.scap_sparse_fc(xs[r % N_INPUTS:r % N_INPUTS + 1], Ws[0], m, tau, bf, y, ws)
+        return 0
+
+    l2_warm = {}
+    for s in SPARSITIES:
+        g, _ = capture(lambda s=s: warm_calls(s))
+        l2_warm["%d%%" % round(100 * s)] = round(1e3 * time_graph(g, reps, 5) / R, 3)
+
     # ------------------------------------------------------------------ end to end through the host-buffer entry point
     hws = torch.empty(scap.scap_fc_host_workspace(1, K, N), dtype=torch.uint8, device="cuda")
     x_host = si.as_torch(d["x"], dt).pin_memory()
     y_host = torch.zeros((1, N), dtype=torch.float32).pin_memory()
+    e2e_calls = len(SPARSITIES) * R  # one pass over the rotation per end-to-end step
 
     def host_step(counter):
         for s in SPARSITIES:
@@ -748,7 +793,7 @@ def main():
     barrier()
     e2e_s = time.perf_counter() - t0
     e2e_s = max_over_ranks(e2e_s, world, "cuda")
-    e2e_value = whole_job_gbs(step_bytes * e2e_steps, world, e2e_s)
+    e2e_value = whole_job_gbs(step_bytes / PASSES * e2e_steps, world, e2e_s)
 
     if rank != 0:
         if world > 1:
@@ -758,42 +803,65 @@ def main():
     peak, peak_kind = measured_peaks()
     per_call_s = ms_per_step * 1e-3 / calls_per_step
     achieved = step_bytes / calls_per_step / per_call_s / 1e9
+    pct = lambda s: "%d%%" % round(100 * s)
     line = {
         "metric": "sparse_fc_effective_hbm_gbs", "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32", "data": "synthetic",
         "config": {
-            "workload": "llama2_7b_down_proj_bf16_b1 (K=11008,N=4096), sparsity targets 50/65/80%",
-            "weights": "bf16", "accumulate": "f32", "batch": 1, "calls_per_step": calls_per_step,
+            "workload": WORKLOAD,
+            "weights": "bf16", "accumulate": "f32", "batch": 1, "calls_per_step": calls_per_step, "passes_per_step": PASSES,
             "l2_policy": "inputs larger than L2: %d weight copies (%.0f MB) rotated so that even the sparsest call pattern touches >= 4x L2 per cycle, %d input vectors" % (R, R * K * N * 2 / 1e6, N_INPUTS),
-            "launch": "CUDA graph replay of one step", "parallelism": "replicas only" if world > 1 else "single GPU",
+            "launch": "CUDA graph replay of one step; calls run back to back under programmatic dependent launch, so us per call is a throughput figure",
+            "parallelism": "replicas only" if world > 1 else "single GPU",
         },
-        "us_per_call": {("%d%%" % round(100 * s)): round(detail[s]["us_per_call"], 3) for s in SPARSITIES},
-        "gbs_per_sparsity": {("%d%%" % round(100 * s)): round(detail[s]["gbs"], 1) for s in SPARSITIES},
-        "kept_fraction": {("%d%%" % round(100 * s)): round(detail[s]["kept_fraction"], 4) for s in SPARSITIES},
-        "dense": {"us_per_call": round(dense_us, 3), "gbs": round(dense_gbs, 1)},
-        "speedup_vs_dense": {("%d%%" % round(100 * s)): round(dense_us / detail[s]["us_per_call"], 3) for s in SPARSITIES},
-        "calibrate_ms": {("%d%%" % round(100 * s)): round(cal_ms[s], 3) for s in SPARSITIES},
+        "us_per_call": {pct(s): round(detail[s]["us_per_call"], 3) for s in SPARSITIES},
+        "us_per_call_over_steps": {"p10": round(float(np.percentile(step_us_per_call, 10)), 3), "median": round(float(np.median(step_us_per_call)), 3),
+                                   "p90": round(float(np.percentile(step_us_per_call, 90)), 3), "note": "whole step (all sparsity targets), per timed step"},
+        "gbs_per_sparsity": {pct(s): round(detail[s]["gbs"], 1) for s in SPARSITIES},
+        "frac_of_peak_per_sparsity": {pct(s): round(detail[s]["gbs"] / peak, 3) for s in SPARSITIES},
+        "kept_fraction": {pct(s): round(detail[s]["kept_fraction"], 4) for s in SPARSITIES},
+        "dense": {"us_per_call": round(dense_us, 3), "gbs": round(dense_gbs, 1), "frac_of_peak": round(dense_gbs / peak, 3)},
+        "speedup_vs_dense": {pct(s): round(dense_us / detail[s]["us_per_call"], 3) for s in SPARSITIES},
+        "plain_launch_us_per_call": {"value": round(plain_us, 3), "note": "no CUDA graph; every launch goes through the Python binding (host-bound)"},
+        "l2_warm_us_per_call": dict(l2_warm, note="same weight copy every call: kept rows are L2 hits where they fit"),
+        "calibrate_ms": {pct(s): round(cal_ms[s], 3) for s in SPARSITIES},
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "traffic": NCU_TRAFFIC_BYTES, "traffic_note": NCU_TRAFFIC_NOTE, "peak_kind": peak_kind, "frac_of_nominal_8000": achieved / 8000.0,
                      "kernel": "fc_kernel (fused threshold + compaction + gather-GEMV + cluster reduction), one launch per call"},
-        "e2e": {"value": e2e_value, "unit": "GB/s", "h2d_bytes_per_step": calls_per_step * K * 2,
-                "d2h_bytes_per_step": calls_per_step * N * 4, "steps": e2e_steps},
+        "e2e": {"value": e2e_value, "unit": "GB/s", "h2d_bytes_per_step": e2e_calls * K * 2,
+                "d2h_bytes_per_step": e2e_calls * N * 4, "steps": e2e_steps, "calls_per_step": e2e_calls},
         "gpu_launches": launches_per_step * args.steps,
         "clocks": clocks,
     }
 
     if not args.no_cpu_baseline and world == 1:
+        import oracle
         cores = os.cpu_count() or 1
         cal_o = {s: (cal[s][0].cpu().numpy(), float(cal[s][1].item()), cal[s][2].cpu().numpy()) for s in SPARSITIES}
+        ns = len(SPARSITIES)
         tot_t, tot_b, n = 0.0, 0, 0
-        while tot_t < 10.0 and n < 2000:
-            t, b = oracle_step(d, cal_o, d["x"][3 * (n % 20):], cores)
+        while tot_t < 8.0 and n < 2000:
+            t, b = oracle_step(d, cal_o, d["x"][ns * (n % 12):], cores)
             tot_t += t
             tot_b += b
             n += 1
-        line["cpu_baseline"] = {"value": tot_b / tot_t / 1e9, "unit": "GB/s", "cores": cores, "kind": "oracle",
-                                "sample": "%d oracle sparse-FC calls (one per sparsity target, %d rounds), %.1f s" % (3 * n, n, tot_t)}
+        t1, b1 = oracle_step(d, cal_o, d["x"], 1)  # the same calls on one thread
+        # the oracle's other two entry points on bounded samples: calibration (256 of the 1024 tokens) and a SwiGLU block
+        xc = si.to_f32(d["x_calib"][:256], si.BF16)
+        tc0 = time.perf_counter()
+        oracle.calibrate(xc, 0.6, NBINS)
+        t_cal = time.perf_counter() - tc0
+        gb = si.glu_block(2, 512, 1376, si.BF16, 32, 1)
+        hf = si.to_f32(gb["h"], si.BF16)
+        tg0 = time.perf_counter()
+        oracle.glu_ffn(hf, gb["Wgu"], gb["Wd"], si.BF16, None, 0.3, None, None, 0.02, None)
+        t_glu = time.perf_counter() - tg0
+        line["cpu_baseline"] = {"value": tot_b / tot_t / 1e9, "unit": "GB/s", "cores": cores, "threads": cores, "kind": "oracle",
+                                "cpu_model": cpu_model(), "single_thread_value": b1 / t1 / 1e9,
+                                "sample": "%d oracle sparse-FC calls (one per sparsity target, %d rounds), %.1f s; single thread: %d calls, %.1f s" % (ns * n, n, tot_t, ns, t1),
+                                "calibrate_s": {"value": round(t_cal, 3), "sample": "oracle.calibrate on 256 tokens x %d channels, 2048 bins, one thread" % K},
+                                "glu_ffn_s": {"value": round(t_glu, 3), "sample": "oracle.glu_ffn, D=512, F=1376, batch 1, one thread"}}
     if args.detail:
         for s in SPARSITIES:
             print("sparsity %.0f%%: %.2f us/call  %.0f GB/s  kept %.3f" % (100 * s, detail[s]["us_per_call"], detail[s]["gbs"],

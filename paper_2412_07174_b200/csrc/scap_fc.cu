@@ -94,14 +94,29 @@ void choose_config(int K, int Nh, int epi, int groups, int B, int *tn_out, int *
     *S_out = best_S;
 }
 
-template <bool BF16, int BT, int MODE, typename XT, int EPI, int TNT>
-static cudaError_t launch_fc_tn(const FcArgs &a, cudaStream_t st) {
+template <bool BF16, int BT, int MODE, typename XT, int EPI, int TNT, int PUT>
+static cudaError_t launch_fc_pu(const FcArgs &a, cudaStream_t st) {
     static SmemOptIn opt_in;
-    auto kern = fc_kernel<BF16, BT, MODE, XT, EPI, TNT>;
+    auto kern = fc_kernel<BF16, BT, MODE, XT, EPI, TNT, PUT>;
     cudaError_t e0 = ensure_dynamic_smem(kern, fc_smem_for(BT), opt_in);
     if (e0 != cudaSuccess) return e0;
     return launch_cluster(kern, dim3(fc_tiles(a.Nh, EPI, TNT), a.S), dim3(FC_THREADS), fc_smem_for(BT), a.S, st,
                           g_tune.pdl != 0, a);
+}
+
+// The fp32-FMA bodies come unrolled for 2, 4, 6 (and, up to batch 2, 8) chunk slots per warp: the smallest one that takes
+// the rank's channels in one fill, else the largest (several fills).
+template <bool BF16, int BT, int MODE, typename XT, int EPI, int TNT>
+static cudaError_t launch_fc_tn(const FcArgs &a, cudaStream_t st) {
+    if constexpr (is_mma(BT)) {
+        return launch_fc_pu<BF16, BT, MODE, XT, EPI, TNT, fc_pu(BT)>(a, st);
+    } else {
+        const int per_rank = ((a.K + 31) / 32 + a.S - 1) / a.S, need = (per_rank + FC_WARPS - 1) / FC_WARPS;
+        if (need <= 2) return launch_fc_pu<BF16, BT, MODE, XT, EPI, TNT, 2>(a, st);
+        if (need <= 4) return launch_fc_pu<BF16, BT, MODE, XT, EPI, TNT, 4>(a, st);
+        if (need <= 6 || fc_pu(BT) == 6) return launch_fc_pu<BF16, BT, MODE, XT, EPI, TNT, 6>(a, st);
+        return launch_fc_pu<BF16, BT, MODE, XT, EPI, TNT, fc_pu(BT)>(a, st);
+    }
 }
 
 template <bool BF16, int BT, int MODE, typename XT, int EPI>

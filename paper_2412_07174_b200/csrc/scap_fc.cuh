@@ -226,10 +226,14 @@ __device__ __forceinline__ void prefetch_bias(const FcArgs &a, int tile, int s, 
 // activations, and equally tau, m and the biases, may have been written by any earlier work on the stream.  No load
 // or prefetch goes out before that wait (measured: memory operations issued ahead of it delay its return for the
 // CTAs that become resident late, 0.15 - 0.2 us per call), and everything a kernel may rewrite is read through L2.
-template <bool BF16, int BT, int MODE, typename XT, int EPI, int TNT>
+// PUT = chunk slots per warp and fill that the threshold code is unrolled for (at most fc_pu(BT), which sizes the
+// shared-memory list): that code is bound by instruction issue, so the launcher picks the smallest instantiation
+// that still takes the rank's channels in one fill.
+template <bool BF16, int BT, int MODE, typename XT, int EPI, int TNT, int PUT = fc_pu(BT)>
 __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const int s, const bool wait_inside) {
-    constexpr int NT = FC_THREADS, PU = fc_pu(BT), CAP = fc_cap(BT), RB = fc_rb(BT), U = fc_unroll(BT);
-    constexpr int CAPC = CAP / 32;    // chunks per fill
+    constexpr int NT = FC_THREADS, PU = PUT, CAP = fc_cap(BT), RB = fc_rb(BT), U = fc_unroll(BT);
+    constexpr int CAPC = FC_WARPS * PU;  // chunks per fill
+    static_assert(PUT >= 1 && PUT <= fc_pu(BT), "the list is sized for fc_pu(BT) slots per warp");
     constexpr int LPR = TNT / 8;      // lanes per row segment
     constexpr int NR = NT / LPR;      // row groups per CTA: group g streams rows g, g+NR, ...
     constexpr int HALF = TNT / 2;
@@ -299,37 +303,43 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
         if (tid < BT) s_rows[tid] = __ldcg(a.in_rows + (tid < B ? tid : 0));
         __syncthreads();
     }
+    // tau: one request per CTA (thousands of simultaneous requests for one address queue up in its L2 slice), issued
+    // first and handed to the other warps through shared memory once the loads of the first fill are in flight
+    float tau_reg = 0.0f;
+    if (MODE == MODE_GATHER && tid == 0) tau_reg = ld_act(a.tau);
     bool bias_done = false;
+    const int kstep = S * 32;  // channel distance between consecutive chunks of a rank
     for (int j0 = 0; j0 < my_chunks; j0 += CAPC) {
         const int nj = min(CAPC, my_chunks - j0);
         const int pw = (nj + FC_WARPS - 1) / FC_WARPS;  // chunks per warp this fill: warp w owns chunks w * pw .. w * pw + pw - 1
-        // ---- A: every warp loads PU chunks at once, centres and thresholds them (Alg. 3: one binary32
-        // subtraction, one compare per element) and keeps the values in registers.  Loads of unused slots are
-        // predicated off (no branch) and nothing consumes a value inside the load loops, so the PU * (BT + 1)
-        // loads of a lane are all in flight together.
+        // ---- A: every warp loads its chunks at once, centres and thresholds them (Alg. 3: one binary32 subtraction, one
+        // compare per element) and keeps the values in registers.  This code runs once per fill on all sixteen warps
+        // of the SM at the same moment, so it is bound by instruction issue: a slot costs one address add, one
+        // compare and the predicated load (unused slots are predicated off, no branch), and nothing consumes a value
+        // inside the load loops, so the loads of a lane are all in flight together.
+        const int nw = max(0, min(pw, nj - warp * pw));         // chunks of this warp
+        const int kbase = (s + S * (j0 + warp * pw)) * 32 + lane;  // this lane's channel in the warp's first chunk
+        const XT *xrow[BT];
+#pragma unroll
+        for (int b = 0; b < BT; ++b) xrow[b] = xg + (size_t)(a.in_rows ? s_rows[b < B ? b : 0] : (b < B ? b : 0)) * a.x_ld + kbase;
+        const float *mrow = a.m ? a.m + kbase : nullptr;
         XT xraw[PU][BT];
         float xv[PU][BT], mk[PU];
+        // (Skipping the unused slots of a fill with CTA-uniform branches was measured: 0.9 us per call slower - the
+        // branches break up the batch of loads.)
 #pragma unroll
         for (int p = 0; p < PU; ++p) {
-            const int j = warp * pw + p;
-            const int k = (s + S * (j0 + j)) * 32 + lane;
-            const bool ok = p < pw && j < nj && k < K;
+            const bool ok = p < nw && kbase + p * kstep < K;
 #pragma unroll
-            for (int b = 0; b < BT; ++b) {
-                const int bb = b < B ? b : 0;
-                xraw[p][b] = ld_act_if(xg + (size_t)(a.in_rows ? s_rows[bb] : bb) * a.x_ld + k, ok && b < B, pol_keep);
-            }
-        }
-        if (MODE == MODE_GATHER && j0 == 0) {  // one request per warp, in flight together with the loads around it
-            float tv = 0.0f;
-            if (lane == 0) tv = ld_act(a.tau);
-            tau = __shfl_sync(0xffffffffu, tv, 0);
+            for (int b = 0; b < BT; ++b) xraw[p][b] = ld_act_if(xrow[b] + p * kstep, ok && b < B, pol_keep);
         }
 #pragma unroll
-        for (int p = 0; p < PU; ++p) {
-            const int j = warp * pw + p;
-            const int k = (s + S * (j0 + j)) * 32 + lane;
-            mk[p] = a.m ? ld_act_if(a.m + k, p < pw && j < nj && k < K, pol_keep) : 0.0f;
+        for (int p = 0; p < PU; ++p) mk[p] = ld_act_if(mrow + p * kstep, mrow != nullptr && p < nw && kbase + p * kstep < K, pol_keep);
+        if (MODE == MODE_GATHER && j0 == 0) {
+            float *s_tau = reinterpret_cast<float *>(s_wcnt + FC_WARPS + 2);  // behind the 8-byte barrier
+            if (tid == 0) *s_tau = tau_reg;
+            __syncthreads();
+            tau = *s_tau;
         }
 #pragma unroll
         for (int p = 0; p < PU; ++p)
@@ -340,9 +350,7 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
         unsigned bal[PU];
 #pragma unroll
         for (int p = 0; p < PU; ++p) {
-            const int j = warp * pw + p;
-            const int k = (s + S * (j0 + j)) * 32 + lane;
-            const bool ok = p < pw && j < nj && k < K;
+            const bool ok = p < nw && kbase + p * kstep < K;
             uint32_t m_ = 0;
 #pragma unroll
             for (int b = 0; b < BT; ++b) {
@@ -385,9 +393,8 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
 #pragma unroll
         for (int p = 0; p < PU; ++p) {
             if (km[p]) {
-                const int j = warp * pw + p;
                 const int pos = wbase + my_off[p] + __popc(bal[p] & ((1u << lane) - 1u));
-                s_k[pos] = (uint32_t)((s + S * (j0 + j)) * 32 + lane);
+                s_k[pos] = (uint32_t)(kbase + p * kstep);
 #pragma unroll
                 for (int b = 0; b < BT; ++b)
                     s_xs[b * CAP + pos] = (MODE == MODE_DENSE || ((km[p] >> b) & 1u)) ? xv[p][b] : 0.0f;
@@ -867,15 +874,15 @@ __device__ __forceinline__ void fc_body_mma(const FcArgs &a, const int tile, con
     if (S > 1) cluster.sync();
 }
 
-template <bool BF16, int BT, int MODE, typename XT, int EPI, int TNT>
+template <bool BF16, int BT, int MODE, typename XT, int EPI, int TNT, int PUT = fc_pu(BT)>
 __global__ void __launch_bounds__(FC_THREADS, fc_min_blocks(BT)) fc_kernel(const FcArgs a) {
     if constexpr (is_mma(BT)) {
         fc_body_mma<BF16, BT, MODE, XT, EPI, TNT>(a, blockIdx.x, blockIdx.y, true);
     } else if (a.hold_dependents) {  // parameter-producing call: ordinary stream order on both sides
         griddep_wait();
-        fc_body<BF16, BT, MODE, XT, EPI, TNT>(a, blockIdx.x, blockIdx.y, false);
+        fc_body<BF16, BT, MODE, XT, EPI, TNT, PUT>(a, blockIdx.x, blockIdx.y, false);
     } else {
-        fc_body<BF16, BT, MODE, XT, EPI, TNT>(a, blockIdx.x, blockIdx.y, true);
+        fc_body<BF16, BT, MODE, XT, EPI, TNT, PUT>(a, blockIdx.x, blockIdx.y, true);
     }
 }
 
