@@ -83,6 +83,10 @@ int scap_version(void);
  *   "tcgen05"  tensor-core batches of the FC and SwiGLU entry points: 0 = always the mma.sync variants,
  *              1 = the tcgen05 (TMEM accumulator) kernel where its shared-memory operand region holds
  *              the call's kept channels in one pass, else mma.sync (default), 2 = always tcgen05
+ *   "tc_spin"  tcgen05 kernel: how often a wait on one of its shared-memory barriers polls before it gives up
+ *              (0 = the built-in limit of about a million polls, the default).  A limit of 1 makes the waits of
+ *              the next call run out at once, which is how the error path of scap_device_status() is exercised
+ *              without a fault; y of such a call is incomplete.
  *   "host_direct"  scap_sparse_fc_host: 1 = when x_host and y_host are page-locked and addressable by the
  *              device, a kernel pulls x and the FC kernel writes y to host memory (default), 0 = always copies
  *   "cal_strip"  scap_calibrate: channels per CTA of the per-channel histogram kernel, 16 (default: 256 threads,

@@ -23,6 +23,7 @@ struct Tuning {
     int cal_strip;    // channels per CTA of the calibration histogram kernel: 16 or 32
     int l2_hints;     // batch 1..4 FC kernel: L2 eviction hints (keep activations and modes, stream weights)
     int tile;         // columns per CTA of the FC kernel: 0 = automatic, else 128 or 256
+    int tc_spin;      // tcgen05 kernel: polls before a barrier wait gives up (0 = the built-in limit)
 };
 extern Tuning g_tune;
 

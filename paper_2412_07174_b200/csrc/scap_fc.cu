@@ -6,7 +6,7 @@
 
 namespace scap {
 
-Tuning g_tune = {0, 1, 1, 1, 4, 16, 1, 0};
+Tuning g_tune = {0, 1, 1, 1, 4, 16, 1, 0, 0};
 
 scap_status check_device() {
     static int cached[64];  // 0 unknown, 1 ok, 2 unsupported
@@ -152,6 +152,7 @@ cudaError_t launch_fc(bool bf16, int mode, int xkind, int epi, const FcArgs &a, 
         FcArgs t = a;
         t.tn = 256;
         t.S = tc_choose_split(a.K, a.Nh, epi, a.B, bf16);
+        t.spin = g_tune.tc_spin;
         return launch_fc_tc(bf16, mode, xkind, epi, t, st);
     }
     FcArgs f = a;
@@ -310,6 +311,11 @@ scap_status scap_tune(const char *key, int value) {
     if (!strcmp(key, "tile")) {
         if (value != 0 && value != 128 && value != 256) return SCAP_ERR_INVALID_ARG;
         g_tune.tile = value;
+        return SCAP_OK;
+    }
+    if (!strcmp(key, "tc_spin")) {
+        if (value < 0) return SCAP_ERR_INVALID_ARG;
+        g_tune.tc_spin = value;
         return SCAP_OK;
     }
     if (!strcmp(key, "tcgen05")) {

@@ -69,6 +69,7 @@ struct FcArgs {
     const float *wscale;  // 8-bit weights only: one scale per input channel, W[k,n] = wscale[k] * Wq[k,n]
     int l2_hints;         // fp32-FMA body: 1 = loads carry L2 eviction hints (keep x and m, stream W)
     int *status;          // device status word: set when a bounded wait runs out (NULL: not recorded)
+    int spin;             // tcgen05 kernel: polls before a shared-memory barrier wait gives up (0: the built-in limit)
 };
 
 template <bool BF16, int BT, int CAP>
@@ -295,9 +296,13 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
     const uint64_t pol_keep = a.l2_hints ? l2_policy_keep() : l2_policy_normal();
     const uint64_t pol_stream = a.l2_hints ? l2_policy_stream() : l2_policy_normal();
 
-    if (wait_inside) {
-        griddep_wait();               // everything earlier work on the stream wrote (activations, parameters) is complete and visible
-        griddep_launch_dependents();  // the next kernel may begin launching; it waits for this grid itself
+    // The wait for the previous kernel sits behind the address arithmetic of the first fill (pure register work, which
+    // so overlaps the previous kernel's tail); with a row map, or without channels, it comes first.
+    bool waited = !wait_inside;
+    if (!waited && (a.in_rows || my_chunks == 0)) {
+        griddep_wait();
+        griddep_launch_dependents();
+        waited = true;
     }
     if (a.in_rows) {  // one L2 read per CTA and row (the map is an output of the previous kernel), then broadcast
         if (tid < BT) s_rows[tid] = __ldcg(a.in_rows + (tid < B ? tid : 0));
@@ -306,7 +311,6 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
     // tau: one request per CTA (thousands of simultaneous requests for one address queue up in its L2 slice), issued
     // first and handed to the other warps through shared memory once the loads of the first fill are in flight
     float tau_reg = 0.0f;
-    if (MODE == MODE_GATHER && tid == 0) tau_reg = ld_act(a.tau);
     bool bias_done = false;
     const int kstep = S * 32;  // channel distance between consecutive chunks of a rank
     for (int j0 = 0; j0 < my_chunks; j0 += CAPC) {
@@ -323,18 +327,26 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
 #pragma unroll
         for (int b = 0; b < BT; ++b) xrow[b] = xg + (size_t)(a.in_rows ? s_rows[b < B ? b : 0] : (b < B ? b : 0)) * a.x_ld + kbase;
         const float *mrow = a.m ? a.m + kbase : nullptr;
+        bool okx[PU];
+#pragma unroll
+        for (int p = 0; p < PU; ++p) okx[p] = p < nw && kbase + p * kstep < K;
+        if (!waited) {
+            griddep_wait();               // everything earlier work on the stream wrote (activations, parameters) is complete and visible
+            griddep_launch_dependents();  // the next kernel may begin launching; it waits for this grid itself
+            waited = true;
+        }
+        if (MODE == MODE_GATHER && j0 == 0 && tid == 0) tau_reg = ld_act(a.tau);
         XT xraw[PU][BT];
         float xv[PU][BT], mk[PU];
         // (Skipping the unused slots of a fill with CTA-uniform branches was measured: 0.9 us per call slower - the
         // branches break up the batch of loads.)
 #pragma unroll
         for (int p = 0; p < PU; ++p) {
-            const bool ok = p < nw && kbase + p * kstep < K;
 #pragma unroll
-            for (int b = 0; b < BT; ++b) xraw[p][b] = ld_act_if(xrow[b] + p * kstep, ok && b < B, pol_keep);
+            for (int b = 0; b < BT; ++b) xraw[p][b] = ld_act_if(xrow[b] + p * kstep, okx[p] && b < B, pol_keep);
         }
 #pragma unroll
-        for (int p = 0; p < PU; ++p) mk[p] = ld_act_if(mrow + p * kstep, mrow != nullptr && p < nw && kbase + p * kstep < K, pol_keep);
+        for (int p = 0; p < PU; ++p) mk[p] = ld_act_if(mrow + p * kstep, mrow != nullptr && okx[p], pol_keep);
         if (MODE == MODE_GATHER && j0 == 0) {
             float *s_tau = reinterpret_cast<float *>(s_wcnt + FC_WARPS + 2);  // behind the 8-byte barrier
             if (tid == 0) *s_tau = tau_reg;
@@ -350,7 +362,7 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
         unsigned bal[PU];
 #pragma unroll
         for (int p = 0; p < PU; ++p) {
-            const bool ok = p < nw && kbase + p * kstep < K;
+            const bool ok = okx[p];
             uint32_t m_ = 0;
 #pragma unroll
             for (int b = 0; b < BT; ++b) {
@@ -402,7 +414,6 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
         }
         __syncthreads();
 
-        if (!bias_done) { prefetch_bias<BF16, EPI, TNT>(a, tile, s, per, bias0, bias1); bias_done = true; }
         // ---- stream the kept rows: row group g takes rows g, g+NR, ...  Two register groups of G loads alternate
         // (one is consumed while the other is in flight).
         if (col_ok) {
@@ -417,6 +428,10 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
 #pragma unroll
             for (int u = 0; u < G; ++u)
                 gb[u] = ld_stream16_if(Wb + (size_t)s_k[rg + NR * (G + u)] * row_bytes, G + u < nrows, pol_stream);
+            if (!bias_done) {  // behind the first row requests: needed only when the columns are finished
+                prefetch_bias<BF16, EPI, TNT>(a, tile, s, per, bias0, bias1);
+                bias_done = true;
+            }
             for (int t0 = 0; t0 < nrows; t0 += 2 * G) {
 #pragma unroll
                 for (int u = 0; u < G; ++u)
@@ -877,7 +892,12 @@ __device__ __forceinline__ void fc_body_mma(const FcArgs &a, const int tile, con
 template <bool BF16, int BT, int MODE, typename XT, int EPI, int TNT, int PUT = fc_pu(BT)>
 __global__ void __launch_bounds__(FC_THREADS, fc_min_blocks(BT)) fc_kernel(const FcArgs a) {
     if constexpr (is_mma(BT)) {
-        fc_body_mma<BF16, BT, MODE, XT, EPI, TNT>(a, blockIdx.x, blockIdx.y, true);
+        if (a.hold_dependents) {  // as below
+            griddep_wait();
+            fc_body_mma<BF16, BT, MODE, XT, EPI, TNT>(a, blockIdx.x, blockIdx.y, false);
+        } else {
+            fc_body_mma<BF16, BT, MODE, XT, EPI, TNT>(a, blockIdx.x, blockIdx.y, true);
+        }
     } else if (a.hold_dependents) {  // parameter-producing call: ordinary stream order on both sides
         griddep_wait();
         fc_body<BF16, BT, MODE, XT, EPI, TNT, PUT>(a, blockIdx.x, blockIdx.y, false);

@@ -37,7 +37,7 @@ constexpr int TC_CAP = 1408;                        // most kept channels per fi
 constexpr int TC_PLANE_DATA = TC_CAP * 32;          // A-operand bytes: 16 per channel and 8-row group, two groups at full capacity
 constexpr int TC_PLANE = TC_PLANE_DATA + 2048;      // + slack for the rows of M that nobody uses
 constexpr int TC_PART_LD = TC_TN + 1;               // row pitch of the accumulator copy (conflict-free)
-constexpr uint32_t TC_SPIN = 1u << 20;              // polls before a wait gives up (tens of milliseconds)
+constexpr uint32_t TC_SPIN = 1u << 20;              // polls before a wait gives up (tens of milliseconds); scap_tune("tc_spin") overrides
 __host__ __device__ constexpr int tc_pu(int ROWS) { return ROWS == 8 ? 6 : 3; }  // chunks per warp per fill, at most
 // 8-row groups of the A operand for B batch rows (parts stacked densely: row = part * B + b), and the chunks of 32
 // channels that fit in the A-operand region with that many groups
@@ -64,6 +64,7 @@ struct TcMisc {
     unsigned long long fill_done;
     uint32_t tmem_base;
     int abort;
+    int issued;  // the MMA lane has issued at least one MMA
     int wcnt[FC_WARPS];
     int rows[16];
 };
@@ -82,9 +83,10 @@ __device__ __forceinline__ bool mbar_test(unsigned long long *bar, uint32_t pari
                  : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
     return ok != 0;
 }
-// Bounded wait: false (and the status word set) when the phase did not complete within TC_SPIN polls.
-__device__ __forceinline__ bool mbar_wait(unsigned long long *bar, uint32_t parity, int code, volatile int *abort_flag) {
-    for (uint32_t i = 0; i < TC_SPIN; ++i) {
+// Bounded wait: false (and the status word set) when the phase did not complete within `limit` polls.
+__device__ __forceinline__ bool mbar_wait(unsigned long long *bar, uint32_t parity, int code, volatile int *abort_flag,
+                                          uint32_t limit) {
+    for (uint32_t i = 0; i < limit; ++i) {
         if (mbar_test(bar, parity)) return true;
         if (*abort_flag) return false;
         if (i > 64) __nanosleep(32);
@@ -125,6 +127,7 @@ __global__ void __launch_bounds__(FC_THREADS, 2) fc_tc_kernel(const FcArgs a) {
     TcMisc *misc = reinterpret_cast<TcMisc *>(smem + TC_OFF_MISC);
     float *s_part = reinterpret_cast<float *>(s_ring);                   // accumulator rows, after the stream
     volatile int *abort_flag = &misc->abort;
+    const uint32_t spin = a.spin ? (uint32_t)a.spin : TC_SPIN;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int tile = blockIdx.x, s = blockIdx.y;
@@ -142,6 +145,7 @@ __global__ void __launch_bounds__(FC_THREADS, 2) fc_tc_kernel(const FcArgs a) {
         }
         mbar_init(&misc->fill_done, 1);
         misc->abort = 0;
+        misc->issued = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 0) {  // the accumulator: 128 TMEM columns, allocated by warp 0 and freed by it at the end
@@ -301,7 +305,7 @@ __global__ void __launch_bounds__(FC_THREADS, 2) fc_tc_kernel(const FcArgs a) {
             for (uint32_t sq = 0; sq < nstg; ++sq) {
                 const uint32_t it = stages_done + sq, st = it % TC_NST;
                 bool ok = true;
-                if (lane == 0) ok = mbar_wait(&misc->empty[st], ((it / TC_NST) & 1u) ^ 1u, 1, abort_flag);
+                if (lane == 0) ok = mbar_wait(&misc->empty[st], ((it / TC_NST) & 1u) ^ 1u, 1, abort_flag, spin);
                 ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
                 if (!ok) break;
                 const int rows_here = min(TC_SROWS, cnt_pad - (int)sq * TC_SROWS);
@@ -324,11 +328,12 @@ __global__ void __launch_bounds__(FC_THREADS, 2) fc_tc_kernel(const FcArgs a) {
                 const uint32_t it = stages_done + sq, st = it % TC_NST;
                 bool ok = true;
                 if (lane == 0) {
-                    ok = mbar_wait(&misc->full[st], (it / TC_NST) & 1u, 2, abort_flag);
+                    ok = mbar_wait(&misc->full[st], (it / TC_NST) & 1u, 2, abort_flag, spin);
                     if (ok) {
                         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // copied rows -> tensor-core proxy
                         tc_fence_after();
                         const uint32_t kb_n = min(4u, nblk - sq * 4);
+                        misc->issued = 1;
                         for (uint32_t kb = 0; kb < kb_n; ++kb) {
                             const uint64_t da = tc_desc(smem_u32(s_plane) + (sq * 4 + kb) * BLK, LBO, 128, 0);
                             const uint64_t db = tc_desc(smem_u32(s_ring) + st * TC_STAGE + kb * TC_KB, 1024, 2048, 2);
@@ -345,8 +350,7 @@ __global__ void __launch_bounds__(FC_THREADS, 2) fc_tc_kernel(const FcArgs a) {
         }
         // ---- the A operand and the kept list are reused by the next fill: wait until this fill's MMAs are done
         if (nblk > 0) {
-            mbar_wait(&misc->fill_done, (uint32_t)fills_done & 1u, 3, abort_flag);
-            ++fills_done;
+            if (mbar_wait(&misc->fill_done, (uint32_t)fills_done & 1u, 3, abort_flag, spin)) ++fills_done;
         }
         stages_done += nstg;
         tc_fence_before();
@@ -356,6 +360,14 @@ __global__ void __launch_bounds__(FC_THREADS, 2) fc_tc_kernel(const FcArgs a) {
     }
 
     asm volatile("cp.async.wait_all;" ::: "memory");
+    // After a wait that ran out, MMAs issued before it may still be writing the accumulator: one more commit and a wait
+    // with the fixed limit (not the tunable one) let them finish before the TMEM columns are handed back.
+    if (*abort_flag && misc->issued) {
+        if (warp == 1 && lane == 0) tc_commit(&misc->fill_done);
+        __syncwarp();
+        int drain_abort = 0;
+        mbar_wait(&misc->fill_done, (uint32_t)fills_done & 1u, 4, &drain_abort, TC_SPIN);
+    }
     // ---- accumulator rows -> shared memory (the ring is idle now), parts added smallest first
     const bool have_acc = stages_done > 0 && !*abort_flag;
     const int acc_rows = racc;

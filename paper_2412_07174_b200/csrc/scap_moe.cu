@@ -17,6 +17,7 @@ struct Route {  // device-resident routing table
 struct MoeArgs {
     scap_expert ex[SCAP_MAX_EXPERTS];
     int E, top_k, B, D, F, S1, S2, tn1, tn2;
+    int l2_hints;  // as FcArgs::l2_hints, for the FMA bodies
     const void *h;
     const float *logits;
     unsigned char *groups;  // per-expert scratch: z[B, F]
@@ -91,6 +92,7 @@ __global__ void __launch_bounds__(FC_THREADS, fc_min_blocks(BT)) moe_fc_kernel(c
     float *z = reinterpret_cast<float *>(a.groups + (size_t)e * a.group_bytes);
     FcArgs g = {};
     g.B = nb;
+    g.l2_hints = a.l2_hints;
     if constexpr (STAGE == 1) {
         g.W = a.ex[e].Wgu; g.K = a.D; g.ldw = 2 * a.F; g.Nh = a.F; g.S = a.S1;
         g.x = a.h; g.x_ld = a.D; g.in_rows = a.route->rows[e];
@@ -210,6 +212,7 @@ scap_status scap_moe_ffn(const void *h, const float *logits, const scap_expert *
     memset(&a, 0, sizeof(a));
     memcpy(a.ex, experts_host, sizeof(scap_expert) * E);
     a.E = E; a.top_k = top_k; a.B = B; a.D = D; a.F = F;
+    a.l2_hints = g_tune.l2_hints;
     a.h = h; a.logits = logits;
     a.groups = w + M.groups;
     a.group_bytes = M.group_bytes;

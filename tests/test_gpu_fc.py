@@ -353,3 +353,77 @@ def test_tcgen05_and_mma_sync_paths_agree_closely(S):
         finally:
             S.scap_tune("tcgen05", 1)
     assert rel_l2_rows(ys[1], ys[0].astype(np.float64)) <= 1e-6
+
+
+# ---------------------------------------------------------------- parameters produced on the stream right before the call
+
+@pytest.mark.parametrize("B", [1, 4, 8])
+def test_parameters_rewritten_on_the_stream_directly_before_the_call(S, B):
+    """tau, m and the fused bias are rewritten by ordinary kernels (device copies and a fill) and the sparse FC is enqueued at
+    once on the same stream, several times over with alternating parameter sets and no synchronisation in between:
+    every call must see the values written just before it (kept list bit-exact, y within tolerance)."""
+    K, N = 2048, 1032
+    d = si.laplace_fc(4, K, N, si.BF16, 32, B)
+    dt = d["dt"]
+    xf = si.to_f32(d["x"], dt)
+    xcf = si.to_f32(d["x_calib"], dt)
+    sets = []
+    for i, (shift, s) in enumerate([(0.0, 0.5), (0.07, 0.8), (-0.05, 0.3)]):
+        m = (d["m_true"] + np.float32(shift)).astype(np.float32)
+        tau = oracle.tau(xcf, m, s)
+        bf64 = oracle.fold_bias(d["W"], dt, m, d.get("b"))
+        sets.append((m, float(tau), bf64))
+    x, W = dev(d["x"], dt), dev(d["W"], dt)
+    m_src = [f32(m) for m, _, _ in sets]
+    b_src = [f32(bf.astype(np.float32)) for _, _, bf in sets]
+    m_dev, b_dev = torch.empty_like(m_src[0]), torch.empty_like(b_src[0])
+    tau_dev = torch.zeros(1, dtype=torch.float32, device="cuda")
+    ws = workspace(S.scap_fc_workspace(B, K, N))
+    rounds = 9
+    ys = [torch.empty((B, N), dtype=torch.float32, device="cuda") for _ in range(rounds)]
+    idxs = [torch.full((K,), -1, dtype=torch.int32, device="cuda") for _ in range(rounds)]
+    nnzs = [torch.full((1,), -1, dtype=torch.int32, device="cuda") for _ in range(rounds)]
+    S.scap_tune("pdl", 1)
+    for r in range(rounds):
+        i = r % len(sets)
+        m_dev.copy_(m_src[i])           # device-to-device copy kernels and a fill kernel on the current stream ...
+        b_dev.copy_(b_src[i])
+        tau_dev.fill_(sets[i][1])
+        S.scap_sparse_fc(x, W, m_dev, tau_dev, b_dev, ys[r], ws.payload, idx_out=idxs[r], nnz_out=nnzs[r])  # ... and the call, at once
+    torch.cuda.synchronize()
+    assert ws.intact()
+    for r in range(rounds):
+        m, tau, bf64 = sets[r % len(sets)]
+        y64 = oracle.sparse_fc(xf, d["W"], dt, m, tau, None) + bf64[None, :]
+        idx_o = oracle.mask(xf, m, tau)[2]
+        n = int(nnzs[r].item())
+        assert n == idx_o.size and np.array_equal(idxs[r][:n].cpu().numpy().astype(np.uint32), idx_o), "round %d" % r
+        assert rel_l2_rows(ys[r].cpu().numpy(), y64) <= REL_L2_TOL
+
+
+# ---------------------------------------------------------------- the bounded waits of the tcgen05 kernel can run out
+
+def test_a_wait_that_runs_out_is_reported_once_and_the_next_call_is_correct(S):
+    """With the poll limit of the tcgen05 kernel's barrier waits set to 1 the waits of the next call give up at once:
+    the call must still return (every CTA passes its cluster barriers and frees its tensor memory),
+    scap_device_status must report the time-out exactly once, and an ordinary call afterwards must pass parity."""
+    from paper_2412_07174_b200 import ScapError
+    K, N, B = 2048, 512, 5
+    d = si.laplace_fc(4, K, N, si.BF16, 32, B)
+    m = d["m_true"]
+    tau = oracle.tau(si.to_f32(d["x_calib"], d["dt"]), m, 0.5)
+    try:
+        S.scap_tune("tcgen05", 2)      # batch 5 on the tcgen05 kernel
+        S.scap_device_status()         # clean slate (raises if an earlier test left a record)
+        S.scap_tune("tc_spin", 1)
+        run_sparse(S, d, m, tau, None, want_idx=False)   # returns; y is incomplete and not looked at
+        with pytest.raises(ScapError) as err:
+            S.scap_device_status()
+        assert err.value.code == 7     # SCAP_ERR_TIMEOUT
+        S.scap_device_status()         # reported once: the record is cleared
+        S.scap_tune("tc_spin", 0)
+        check_fc(S, d, m, tau)         # the same kernel with its normal limit
+        S.scap_device_status()
+    finally:
+        S.scap_tune("tc_spin", 0)
+        S.scap_tune("tcgen05", 1)

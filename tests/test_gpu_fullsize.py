@@ -94,14 +94,15 @@ def test_config3_mixtral_moe_layer(S):
         hc = si.to_f32(p["h_calib"], si.BF16)
         m1, tau1 = oracle.calibrate(hc, 0.4, 2048)
         b1 = oracle.fold_bias(p["Wgu"], si.BF16, m1, None).astype(np.float32)
-        # stage 2 is calibrated on the oracle's z of the first 256 calibration tokens (the full 2048 would take
-        # minutes of float64 matmul per expert on the host)
-        zc = oracle.glu_stage1_batch(hc[:256], p["Wgu"], si.BF16, m1, tau1, b1)
+        # stage 2 is calibrated on the oracle's z of all 2048 calibration tokens of this expert, as the workload
+        # description says (in slabs of 512 rows, to bound the host memory of the float64 product)
+        zc = np.concatenate([oracle.glu_stage1_batch(hc[t:t + 512], p["Wgu"], si.BF16, m1, tau1, b1) for t in range(0, hc.shape[0], 512)])
+        assert zc.shape == (2048, F)
         m2, tau2 = oracle.calibrate(zc, 0.6, 2048)
         b2 = oracle.fold_bias(p["Wd"], si.BF16, m2, None).astype(np.float32)
         p.update(m1=m1, tau1=tau1, bgu_fused=b1, m2=m2, tau2=tau2, bd_fused=b2)
     hf = si.to_f32(mo["h"], si.BF16)
-    for nb in (1, 4):
+    for nb in (1, 2, 3, 4):
         sub = dict(mo, h=mo["h"][:nb], logits=mo["logits"][:nb])
         y, ex, w = run_moe(S, sub, 2)
         y64, ex_o, w_o = oracle.moe_ffn(hf[:nb], sub["logits"], mo["experts"], si.BF16, 2)
@@ -119,7 +120,7 @@ def test_config4_sweep_points(S, K, N):
     bf64 = oracle.fold_bias(d["W"], dt, m_o, None)
     W = dev(d["W"], dt)
     m, bf = f32(m_o), f32(bf64)
-    for s, B in [(0.0, 1), (0.6, 1), (0.9, 1), (0.6, 4), (0.25, 16), (0.9, 16)]:
+    for s, B in [(0.0, 1), (0.6, 1), (0.9, 1), (0.6, 2), (0.6, 4), (0.8, 4), (0.5, 8), (0.25, 16), (0.9, 16)]:
         tau_o = oracle.tau(xcf, m_o, s)
         sparse_parity(S, d, W, m, f32([tau_o]), bf, d["x"][:B], m_o, tau_o, bf64)
     # dense baseline on the same layer
@@ -130,3 +131,16 @@ def test_config4_sweep_points(S, K, N):
     torch.cuda.synchronize()
     y64 = oracle.dense_fc(si.to_f32(d["x"][:4], dt), d["W"], dt, None)
     assert rel_l2_rows(y.cpu().numpy(), y64) <= REL_L2_TOL
+
+
+@pytest.mark.parametrize("B", [1, 4])
+def test_fused_qkv_projection_shares_one_mask(S, B):
+    """Q, K and V read the same input, so the fused projection is one sparse FC on the packed [D, 3D] weight with one
+    kept-channel list (Section 1 of the paper: projections that share their input share its mask)."""
+    D = 4096
+    d = si.config4_fc(D, 3 * D, 4, T_calib=256)
+    dt = d["dt"]
+    xcf = si.to_f32(d["x_calib"], dt)
+    m_o, tau_o = oracle.calibrate(xcf, 0.5, 2048)
+    bf64 = oracle.fold_bias(d["W"], dt, m_o, None)
+    sparse_parity(S, d, dev(d["W"], dt), f32(m_o), f32([tau_o]), f32(bf64), d["x"][:B], m_o, tau_o, bf64)
