@@ -246,7 +246,8 @@ scap_status scap_gelu_ffn(const void *h, const void *Wu, const void *Wd, const f
  *     until the process exits.  A shape needing more (scap_glu_workspace(B, D, F) > capacity, i.e.
  *     roughly B * F > 520000) is rejected with SCAP_ERR_WORKSPACE and nothing is enqueued.
  *   - The first call on each device looks up the array's device address (cudaGetSymbolAddress) and
- *     caches it; make that first call outside any stream capture.
+ *     caches it; make that first call outside any stream capture.  The cached address belongs to the
+ *     device's current context: it is not valid after a cudaDeviceReset.
  *   - All calls on a device share the one array.  It keeps whatever the last call left there; nothing
  *     needs clearing because each call writes every word before reading it.  Two calls that overlap
  *     on the GPU (different streams, or graphs replayed concurrently) race on it: keep them on one

@@ -74,6 +74,10 @@ def lib():
         L.scap_oracle_sparse_fc_q8.restype = None
         L.scap_oracle_fold_bias_q8.argtypes = [vp, vp, vp, vp, i, i, vp]
         L.scap_oracle_fold_bias_q8.restype = None
+        L.scap_oracle_sparse_fc_q4.argtypes = [vp, vp, vp, vp, i, vp, f, vp, i, i, i, vp]
+        L.scap_oracle_sparse_fc_q4.restype = None
+        L.scap_oracle_fold_bias_q4.argtypes = [vp, vp, vp, i, vp, vp, i, i, vp]
+        L.scap_oracle_fold_bias_q4.restype = None
         L.scap_oracle_router.argtypes = [vp, i, i, i, vp, vp]
         L.scap_oracle_router.restype = None
         L.scap_oracle_ffn_sparsity.argtypes = [d, d, d]
@@ -274,6 +278,33 @@ def fold_bias_q8(Wq, scale, m, b):
     K, N = Wq.shape
     out = np.empty(N, np.float64)
     lib().scap_oracle_fold_bias_q8(_p(Wq), _p(_f32(scale)), _p(_f32(m)), _p(_f32(b)), K, N, _p(out))
+    return out
+
+
+def sparse_fc_q4(xf, Wq, scale, zero, group, m, tau, b_fused):
+    """Eq. 2-3 on group-wise 4-bit weights: Wq[K, N/2] uint8 (two codes per byte, even column in the low nibble),
+    scale[K/group, N] float32, zero[K/group, N] uint8; W = scale * (q - zero).  Returns y[B,N] float64."""
+    xf = _f32(np.atleast_2d(xf))
+    B, K = xf.shape
+    Wq = np.ascontiguousarray(Wq, np.uint8)
+    N = Wq.shape[1] * 2
+    scale = _f32(scale)
+    zero = np.ascontiguousarray(zero, np.uint8)
+    G = (K + group - 1) // group
+    assert Wq.shape == (K, N // 2) and scale.shape == (G, N) and zero.shape == (G, N)
+    y = np.empty((B, N), np.float64)
+    lib().scap_oracle_sparse_fc_q4(_p(xf), _p(Wq), _p(scale), _p(zero), int(group), _p(_f32(m)), float(np.float32(tau)),
+                                   _p(_f32(b_fused)), B, K, N, _p(y))
+    return y
+
+
+def fold_bias_q4(Wq, scale, zero, group, m, b):
+    """Eq. 5-6 on group-wise 4-bit weights: b + m W in float64."""
+    Wq = np.ascontiguousarray(Wq, np.uint8)
+    K, N = Wq.shape[0], Wq.shape[1] * 2
+    out = np.empty(N, np.float64)
+    lib().scap_oracle_fold_bias_q4(_p(Wq), _p(_f32(scale)), _p(np.ascontiguousarray(zero, np.uint8)), int(group), _p(_f32(m)),
+                                   _p(_f32(b)), K, N, _p(out))
     return out
 
 

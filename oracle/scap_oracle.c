@@ -357,6 +357,42 @@ void scap_oracle_fold_bias_q8(const signed char *Wq, const float *scale, const f
     }
 }
 
+/* ---------------------------------------------------------------- group-wise 4-bit weights (Table 4: the AWQ rows)
+ * Storage reading (the paper names the models, not a layout): unsigned 4-bit codes q[k,n] in 0..15, two per byte in
+ * Wq[K, N/2] (row-major like W; column 2j in the low nibble of byte j, column 2j+1 in the high nibble); groups of
+ * `group` consecutive INPUT channels share, per output column, one binary32 scale and one zero point in 0..15:
+ *     W[k,n] = scale[k / group, n] * (q[k,n] - zero[k / group, n]).
+ * The sparse FC and the bias folding are Eq. 2-3 and Eq. 5-6 on that W, in binary64, ascending k.            */
+static double q4_weight(const uint8_t *Wq, const float *scale, const uint8_t *zero, int N, int group, int k, int n) {
+    const uint8_t byte = Wq[(long)k * (N / 2) + n / 2];
+    const int q = (n & 1) ? (byte >> 4) : (byte & 15);
+    const long g = k / group;
+    return (double)scale[g * N + n] * (double)(q - (int)zero[g * N + n]);
+}
+
+void scap_oracle_sparse_fc_q4(const float *xf, const uint8_t *Wq, const float *scale, const uint8_t *zero, int group,
+                              const float *m, float tau, const float *b_fused, int B, int K, int N, double *y) {
+    for (int b = 0; b < B; ++b)
+        for (int n = 0; n < N; ++n) {
+            double acc = b_fused ? (double)b_fused[n] : 0.0;
+            for (int k = 0; k < K; ++k) {
+                volatile float d = m ? xf[(long)b * K + k] - m[k] : xf[(long)b * K + k];   /* the decision: binary32 */
+                double xc = (double)xf[(long)b * K + k] - (m ? (double)m[k] : 0.0);      /* the product: exact difference */
+                if (fabsf(d) >= tau) acc += xc * q4_weight(Wq, scale, zero, N, group, k, n);
+            }
+            y[(long)b * N + n] = acc;
+        }
+}
+
+void scap_oracle_fold_bias_q4(const uint8_t *Wq, const float *scale, const uint8_t *zero, int group, const float *m,
+                              const float *b /*[N] nullable*/, int K, int N, double *b_fused) {
+    for (int n = 0; n < N; ++n) {
+        double acc = b ? (double)b[n] : 0.0;
+        for (int k = 0; k < K; ++k) acc += (double)m[k] * q4_weight(Wq, scale, zero, N, group, k, n);
+        b_fused[n] = acc;
+    }
+}
+
 /* ---------------------------------------------------------------- Alg. 2: SwiGLU block
  * Wgu[D,2F]: columns 0..F-1 are the gate projection, F..2F-1 the up projection; both read the
  * same pruned input (one tau_x, one mask).  z = up * silu(gate), silu(g) = g / (1 + exp(-g)),

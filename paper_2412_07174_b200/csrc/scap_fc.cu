@@ -2,6 +2,8 @@
 // variant, plus the launch plumbing shared with the SwiGLU and MoE entry points.
 #include <string.h>
 
+#include <atomic>
+
 #include "scap_fc.cuh"
 
 namespace scap {
@@ -9,32 +11,40 @@ namespace scap {
 Tuning g_tune = {0, 1, 1, 1, 4, 16, 1, 0, 0};
 
 scap_status check_device() {
-    static int cached[64];  // 0 unknown, 1 ok, 2 unsupported
+    static std::atomic<int> cached[64];  // 0 unknown, 1 ok, 2 unsupported
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) {
         cudaGetLastError();
         return SCAP_ERR_CUDA;
     }
-    if (dev >= 0 && dev < 64 && cached[dev]) return cached[dev] == 1 ? SCAP_OK : SCAP_ERR_UNSUPPORTED_ARCH;
+    if (dev >= 0 && dev < 64) {
+        const int hit = cached[dev].load(std::memory_order_relaxed);
+        if (hit) return hit == 1 ? SCAP_OK : SCAP_ERR_UNSUPPORTED_ARCH;
+    }
     int major = 0;
     if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) {
         cudaGetLastError();
         return SCAP_ERR_CUDA;
     }
-    if (dev >= 0 && dev < 64) cached[dev] = major == 10 ? 1 : 2;
+    if (dev >= 0 && dev < 64) cached[dev].store(major == 10 ? 1 : 2, std::memory_order_relaxed);
     return major == 10 ? SCAP_OK : SCAP_ERR_UNSUPPORTED_ARCH;
 }
 
 int sm_count() {
-    static int cached = 0;
-    if (cached) return cached;
+    static std::atomic<int> cached_by_dev[64];
     int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess && dev >= 0 && dev < 64) {
+        const int hit = cached_by_dev[dev].load(std::memory_order_relaxed);
+        if (hit) return hit;
+    } else {
+        cudaGetLastError();
+    }
     if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
         n <= 0) {
         cudaGetLastError();
         return 148;  // B200; used only so that queries work on a machine without a GPU
     }
-    cached = n;
+    if (dev >= 0 && dev < 64) cached_by_dev[dev].store(n, std::memory_order_relaxed);
     return n;
 }
 
@@ -43,8 +53,13 @@ int sm_count() {
 // little below 2 * SMs for S > 1).  Queried once per size for the batch-1 kernel, which has the launch shape of
 // all variants (256 threads, two CTAs per SM); 2 * SMs where the query is not possible.
 int resident_ctas(int S) {
-    static int cached[MAX_CLUSTER + 1];
-    if (cached[S]) return cached[S];
+    static std::atomic<int> cached_by_dev[64][MAX_CLUSTER + 1];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); dev = -1; }
+    if (dev >= 0 && dev < 64) {
+        const int hit = cached_by_dev[dev][S].load(std::memory_order_relaxed);
+        if (hit) return hit;
+    }
     int n = 2 * sm_count();
     if (S > 1) {
         auto kern = fc_kernel<true, 1, MODE_GATHER, __nv_bfloat16, EPI_BIAS, 128>;
@@ -63,7 +78,7 @@ int resident_ctas(int S) {
         if (cudaOccupancyMaxActiveClusters(&clusters, kern, &cfg) == cudaSuccess && clusters > 0) n = clusters * S;
         else cudaGetLastError();
     }
-    cached[S] = n;
+    if (dev >= 0 && dev < 64) cached_by_dev[dev][S].store(n, std::memory_order_relaxed);
     return n;
 }
 

@@ -24,6 +24,8 @@
 // still passes every cluster barrier and frees its TMEM.
 #include <string.h>
 
+#include <atomic>
+
 #include "scap_fc.cuh"
 
 namespace scap {
@@ -523,13 +525,16 @@ cudaError_t launch_fc_tc(bool bf16, int mode, int xkind, int epi, const FcArgs &
 
 // Device address of the status word of the bounded waits, looked up once per device.
 int *tc_status_ptr() {
-    static int *cached[64];
+    static std::atomic<int *> cached[64];
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return nullptr; }
-    if (dev >= 0 && dev < 64 && cached[dev]) return cached[dev];
+    if (dev >= 0 && dev < 64) {
+        int *hit = cached[dev].load(std::memory_order_acquire);
+        if (hit) return hit;
+    }
     int *p = nullptr;
     if (cudaGetSymbolAddress(reinterpret_cast<void **>(&p), g_tc_status) != cudaSuccess) { cudaGetLastError(); return nullptr; }
-    if (dev >= 0 && dev < 64) cached[dev] = p;
+    if (dev >= 0 && dev < 64) cached[dev].store(p, std::memory_order_release);
     return p;
 }
 

@@ -1,6 +1,7 @@
 // SwiGLU FFN block (Alg. 2): one fused FC kernel over the packed gate|up weight whose cluster
 // reduction also forms z = up * silu(gate), then one fused FC kernel over the down weight that
 // thresholds z itself.  z (fp32, B x F) is the only intermediate and stays L2-resident.
+#include <atomic>
 #include <string.h>
 
 #include "scap_fc.cuh"
@@ -124,22 +125,25 @@ constexpr size_t GLU_STATIC_BYTES = (size_t)2 << 20;
 static __device__ __align__(256) unsigned char g_glu_static_scratch[GLU_STATIC_BYTES];
 
 static scap_status glu_static_address(unsigned char **out) {
-    static unsigned char *cached[64];
+    static std::atomic<unsigned char *> cached[64];  // first calls may come from several host threads at once
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) {
         cudaGetLastError();
         return SCAP_ERR_CUDA;
     }
-    if (dev >= 0 && dev < 64 && cached[dev]) {
-        *out = cached[dev];
-        return SCAP_OK;
+    if (dev >= 0 && dev < 64) {
+        unsigned char *hit = cached[dev].load(std::memory_order_acquire);
+        if (hit) {
+            *out = hit;
+            return SCAP_OK;
+        }
     }
     void *p = nullptr;
     if (cudaGetSymbolAddress(&p, g_glu_static_scratch) != cudaSuccess || p == nullptr) {
         cudaGetLastError();
         return SCAP_ERR_CUDA;
     }
-    if (dev >= 0 && dev < 64) cached[dev] = static_cast<unsigned char *>(p);
+    if (dev >= 0 && dev < 64) cached[dev].store(static_cast<unsigned char *>(p), std::memory_order_release);
     *out = static_cast<unsigned char *>(p);
     return SCAP_OK;
 }

@@ -275,3 +275,26 @@ def quantise_q8(W_bits: np.ndarray, dt: int):
     scale = np.where(amax > 0, amax / 127.0, 1.0).astype(np.float32)
     q = np.clip(np.rint(Wf / scale.astype(np.float64)[:, None]), -127, 127).astype(np.int8)
     return q, scale
+
+
+def quantise_q4(W_bits: np.ndarray, dt: int, group: int = 128):
+    """Asymmetric group-wise 4-bit quantisation of a 16-bit weight: for every group of ``group`` consecutive input channels
+    (rows) and every output column, scale = (max - min) / 15 (1 where the group is constant), zero = round(-min / scale)
+    clipped to 0..15, q = round(W / scale) + zero clipped to 0..15.  Returns (packed uint8 [K, N/2] with the even column in
+    the low nibble, float32 scale [K/group, N], uint8 zero [K/group, N])."""
+    Wf = to_f32(W_bits, dt).astype(np.float64)
+    K, N = Wf.shape
+    assert N % 2 == 0
+    G = (K + group - 1) // group
+    scale = np.empty((G, N), np.float32)
+    zero = np.empty((G, N), np.uint8)
+    q = np.empty((K, N), np.uint8)
+    for g in range(G):
+        blk = Wf[g * group:(g + 1) * group]
+        lo, hi = blk.min(axis=0), blk.max(axis=0)
+        sc = np.where(hi > lo, (hi - lo) / 15.0, 1.0).astype(np.float32)
+        zp = np.clip(np.rint(-lo / sc.astype(np.float64)), 0, 15)
+        scale[g], zero[g] = sc, zp.astype(np.uint8)
+        q[g * group:(g + 1) * group] = np.clip(np.rint(blk / sc.astype(np.float64)[None, :]) + zp[None, :], 0, 15).astype(np.uint8)
+    packed = (q[:, 0::2] | (q[:, 1::2] << 4)).astype(np.uint8)
+    return packed, scale, zero

@@ -599,3 +599,61 @@ def test_q8_brute_force_on_a_tiny_case_and_quantiser_properties():
     Wf = si.to_f32(W, si.BF16)
     assert qq.dtype == np.int8 and np.abs(qq).max() == 127 and np.all(np.abs(qq).max(axis=1) == 127)
     assert np.all(np.abs(ss[:, None] * qq - Wf) <= 0.5 * ss[:, None] * (1 + 1e-3))
+
+
+# ---------------------------------------------------------------- group-wise 4-bit weights
+
+def _pack_q4(q):
+    return (q[:, 0::2] | (q[:, 1::2] << 4)).astype(np.uint8)
+
+
+def test_q4_oracle_reduces_to_the_16_bit_oracle_when_the_weights_are_representable():
+    # scale a power of two, q - zero in -15..15: scale * (q - zero) is exact in bf16, so both oracles see one real matrix
+    rng = np.random.default_rng(11)
+    K, N, B, group = 80, 24, 3, 32      # 2.5 groups: the last one is short
+    G = (K + group - 1) // group
+    q = rng.integers(0, 16, size=(K, N)).astype(np.uint8)
+    zero = rng.integers(0, 16, size=(G, N)).astype(np.uint8)
+    scale = (2.0 ** rng.integers(-9, -5, size=(G, N))).astype(np.float32)
+    gi = np.arange(K) // group
+    Wreal = scale[gi].astype(np.float64) * (q.astype(np.float64) - zero[gi].astype(np.float64))
+    W16 = si.to_bits(Wreal, si.BF16)
+    assert np.array_equal(si.to_f32(W16, si.BF16).astype(np.float64), Wreal)
+    d = si.laplace_fc(4, K, N, si.BF16, 8, B)
+    xf = si.to_f32(d["x"], si.BF16)
+    m, bf = d["m_true"], np.linspace(-1, 1, N).astype(np.float32)
+    for tau in (0.0, 0.2, 5.0):
+        assert np.array_equal(oracle.sparse_fc_q4(xf, _pack_q4(q), scale, zero, group, m, tau, bf),
+                              oracle.sparse_fc(xf, W16, si.BF16, m, tau, bf))
+    assert np.array_equal(oracle.fold_bias_q4(_pack_q4(q), scale, zero, group, m, None), oracle.fold_bias(W16, si.BF16, m, None))
+
+
+def test_q4_hand_case_pins_the_nibble_order_the_group_index_and_the_zero_point():
+    # K = 3 channels, group = 2 (channels 0, 1 | channel 2), N = 2 columns: one byte per row
+    q = np.uint8([[1, 14], [5, 2], [9, 7]])           # (column 0, column 1) per row
+    packed = np.uint8([[1 | (14 << 4)], [5 | (2 << 4)], [9 | (7 << 4)]])
+    assert np.array_equal(_pack_q4(q), packed)
+    scale = np.float32([[0.5, 0.25], [2.0, 4.0]])     # [group, column]
+    zero = np.uint8([[3, 8], [1, 15]])
+    x = np.float32([[1.0, -3.0, 2.0]])
+    # W = scale * (q - zero): row 0: 0.5 * -2, 0.25 * 6; row 1: 0.5 * 2, 0.25 * -6; row 2 (group 1): 2 * 8, 4 * -8
+    W = np.float64([[-1.0, 1.5], [1.0, -1.5], [16.0, -32.0]])
+    y = oracle.sparse_fc_q4(x, packed, scale, zero, 2, None, 0.0, np.float32([10, 20]))
+    assert np.array_equal(y, [[10 + 1.0 * W[0, 0] - 3.0 * W[1, 0] + 2.0 * W[2, 0], 20 + 1.0 * W[0, 1] - 3.0 * W[1, 1] + 2.0 * W[2, 1]]])
+    y = oracle.sparse_fc_q4(x, packed, scale, zero, 2, None, 1.5, None)     # channel 0 pruned (|1| < 1.5)
+    assert np.array_equal(y, [[-3.0 * W[1, 0] + 2.0 * W[2, 0], -3.0 * W[1, 1] + 2.0 * W[2, 1]]])
+    m = np.float32([0.5, 0.0, -1.0])
+    assert np.array_equal(oracle.fold_bias_q4(packed, scale, zero, 2, m, np.float32([1, 2])),
+                          [1 + 0.5 * W[0, 0] - 1.0 * W[2, 0], 2 + 0.5 * W[0, 1] - 1.0 * W[2, 1]])
+
+
+def test_q4_quantiser_properties():
+    W = si.weight(4, 200, 24, si.BF16)
+    packed, scale, zero = si.quantise_q4(W, si.BF16, 64)
+    Wf = si.to_f32(W, si.BF16).astype(np.float64)
+    q = np.empty((200, 24), np.int64)
+    q[:, 0::2], q[:, 1::2] = packed & 15, packed >> 4
+    gi = np.arange(200) // 64
+    back = scale[gi].astype(np.float64) * (q - zero[gi].astype(np.int64))
+    assert packed.shape == (200, 12) and scale.shape == (4, 24) and zero.shape == (4, 24) and q.min() >= 0 and q.max() == 15
+    assert np.all(np.abs(back - Wf) <= scale[gi] * (1.0 + 1e-6))      # within one step (zero-point rounding adds up to half a step)
