@@ -308,6 +308,49 @@ def suite_q8(torch, scap, peak, out):
                  "weight_copies": R})
 
 
+def suite_q4(torch, scap, peak, out):
+    """Group-wise 4-bit weights (groups of 128 input channels) at the bench shape, batch 1: a kept row is N/2 bytes, so a call
+    touches a quarter of the bf16 bytes plus the scales and zero points of the groups it meets; the fixed latencies stay."""
+    stream = torch.cuda.Stream()
+    l2 = torch.cuda.get_device_properties(0).L2_cache_size
+    Kk, Nn, group = 11008, 4096, 128
+    d = si.config4_fc(Kk, Nn, 16 * 8, T_calib=2048)
+    q, sc, zp = si.quantise_q4(d["W"], si.BF16, group)
+    Q0, S0, Z0 = torch.from_numpy(q).cuda(), torch.from_numpy(sc).cuda(), torch.from_numpy(zp).cuda()
+    xc = si.as_torch(d["x_calib"], si.BF16).cuda()
+    xs = si.as_torch(d["x"], si.BF16).cuda()
+    per_copy = Kk * Nn // 2 + sc.nbytes + zp.nbytes
+    Rmax = int(np.ceil(4 * l2 / (0.2 * per_copy)))
+    Qs = [(Q0, S0, Z0)] + [(Q0.clone(), S0.clone(), Z0.clone()) for _ in range(Rmax - 1)]
+    cws = torch.empty(scap.scap_calibrate_workspace(2048, Kk, NBINS), dtype=torch.uint8, device="cuda")
+    m = torch.empty(Kk, dtype=torch.float32, device="cuda")
+    bq = torch.empty(Nn, dtype=torch.float32, device="cuda")
+    nnz = torch.zeros(1, dtype=torch.int32, device="cuda")
+    idx = torch.empty(Kk, dtype=torch.int32, device="cuda")
+    B = 1
+    ws = torch.empty(scap.scap_fc_workspace(B, Kk, Nn), dtype=torch.uint8, device="cuda")
+    y = torch.empty((B, Nn), dtype=torch.float32, device="cuda")
+    xb = [xs[i * 16:i * 16 + B] for i in range(8)]
+    Rd = max(2, min(Rmax, int(np.ceil(4 * l2 / per_copy))))
+    t_dense = _time_graph(torch, stream, lambda: [scap.scap_dense_fc_q4(xb[r % 8], Qs[r][0], Qs[r][1], Qs[r][2], group, None, y, ws) for r in range(Rd)]) / Rd
+    G = (Kk + group - 1) // group
+    for s in (0.0, 0.5, 0.65, 0.8):
+        tau = torch.empty(1, dtype=torch.float32, device="cuda")
+        scap.scap_calibrate(xc, s, NBINS, m, tau, cws)
+        scap.scap_fold_bias_q4(Q0, S0, Z0, group, m, None, bq, ws)
+        kept = []
+        for i in range(8):
+            scap.scap_sparse_fc_q4(xb[i], Q0, S0, Z0, group, m, tau, bq, y, ws, idx_out=idx, nnz_out=nnz)
+            kept.append(int(nnz.item()))
+        rho = float(np.mean(kept)) / Kk
+        R = max(2, min(Rmax, int(np.ceil(4 * l2 / (max(rho, 0.2) * per_copy)))))
+        t = _time_graph(torch, stream, lambda: [scap.scap_sparse_fc_q4(xb[r % 8], Qs[r][0], Qs[r][1], Qs[r][2], group, m, tau, bq, y, ws) for r in range(R)]) / R
+        nb = float(np.mean(kept)) * Nn / 2 + G * Nn * 5 + B * Kk * 2 + 4 * Kk + 4 + 4 * Nn + 4 * B * Nn
+        out({"suite": "q4", "K": Kk, "N": Nn, "B": B, "group": group, "sparsity_target": s, "union_kept_fraction": round(rho, 4),
+             "us_per_call": round(t, 3), "gbs": round(nb / t / 1e3, 1), "frac_of_measured_peak": round(nb / t / 1e3 / peak, 3),
+             "dense_q4_us": round(t_dense, 3), "speedup_vs_dense_q4": round(t_dense / t, 3), "weight_copies": R})
+
+
 def suite_calibrate(torch, scap, out):
     """Config 4's timed calibration: 2048 tokens x 14336 channels, 2048 bins, plus the tau quantile."""
     T, Kk = 2048, 14336
@@ -533,6 +576,8 @@ def run_suite(args):
         suite_gelu(torch, scap, peak, out)
     if which in ("q8", "all"):
         suite_q8(torch, scap, peak, out)
+    if which in ("q4", "all"):
+        suite_q4(torch, scap, peak, out)
     if which in ("sweep", "all", "sweep-small"):
         shapes = [(4096, 4096), (4096, 11008), (11008, 4096), (14336, 4096)]
         if which == "sweep-small":
@@ -563,7 +608,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--detail", action="store_true", help="also print a per-sparsity table to stderr")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--suite", default="", choices=["", "calibrate", "glu", "gelu", "q8", "moe", "mamba", "sweep", "sweep-small", "all"],
+    ap.add_argument("--suite", default="", choices=["", "calibrate", "glu", "gelu", "q8", "q4", "moe", "mamba", "sweep", "sweep-small", "all"],
                     help="run the other workload descriptions instead of the headline line (one JSON object per line)")
     ap.add_argument("--copies", type=int, default=0,
                     help="number of weight copies to rotate (default: enough for the cold-HBM rule); a small value keeps "

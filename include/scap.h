@@ -190,6 +190,25 @@ scap_status scap_dense_fc_q8(const void *x, scap_dtype xdt, const signed char *W
 scap_status scap_fold_bias_q8(const signed char *Wq, const float *wscale, const float *m, const float *b, int K, int N,
                               float *b_fused, void *ws, size_t ws_bytes, scap_stream_t stream);
 
+/* Group-wise 4-bit weights (Table 4 applies SCAP to AWQ 4-bit models; the paper names the models, not a layout - this one is
+ * the library's).  Storage: Wq[K, N/2] bytes, two unsigned codes q in 0..15 per byte (column 2j in the low nibble of byte
+ * j, column 2j+1 in the high nibble), row-major like W, so a kept input channel is still one contiguous row; groups of
+ * `group` consecutive INPUT channels share, per output column, scale[K/group rounded up, N] (fp32) and a zero point
+ * zero[same shape] (one byte, 0..15):  W[k,n] = scale[k / group, n] * (q[k,n] - zero[k / group, n]).
+ * group: a multiple of 32, 32..2048 (else SCAP_ERR_SHAPE); N a multiple of 16.  Everything else - x of dtype xdt, m, tau,
+ * b_fused, y, the optional kept list, the batch rule (more than two rows run two at a time; idx_out / nnz_out only for
+ * B <= 2), the workspace query - as for the 8-bit calls above.  The sum over the kept channels of one group is formed
+ * on the integer codes, sum d * (q - zero) in fp32, and scaled once.                                                  */
+scap_status scap_sparse_fc_q4(const void *x, scap_dtype xdt, const unsigned char *Wq, const float *scale,
+                              const unsigned char *zero, int group, const float *m, const float *tau, const float *b_fused,
+                              float *y, int B, int K, int N, uint32_t *idx_out, int *nnz_out, void *ws, size_t ws_bytes,
+                              scap_stream_t stream);
+scap_status scap_dense_fc_q4(const void *x, scap_dtype xdt, const unsigned char *Wq, const float *scale,
+                             const unsigned char *zero, int group, const float *b, float *y, int B, int K, int N, void *ws,
+                             size_t ws_bytes, scap_stream_t stream);
+scap_status scap_fold_bias_q4(const unsigned char *Wq, const float *scale, const unsigned char *zero, int group, const float *m,
+                              const float *b, int K, int N, float *b_fused, void *ws, size_t ws_bytes, scap_stream_t stream);
+
 /* scap_sparse_fc for a caller whose activations live in HOST memory: copies x_host[B,K]
  * (dtype dt; pinned memory recommended) to the device, runs the sparse FC, and copies y back to
  * y_host[B,N] (fp32), all enqueued on `stream`; y_host is valid once the stream has drained.

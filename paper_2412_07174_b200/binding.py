@@ -11,6 +11,7 @@ __all__ = [
     "scap_calibrate_workspace", "scap_calibrate", "scap_calibrate_ex", "SCAP_MODE_HISTOGRAM", "SCAP_MODE_MEAN", "SCAP_MODE_MEDIAN", "SCAP_MODE_KDE",
     "SCAP_ETA_PER_CHANNEL", "SCAP_ETA_SCALAR", "scap_fold_bias_workspace", "scap_fold_bias",
     "scap_fc_workspace", "scap_sparse_fc", "scap_dense_fc", "scap_sparse_fc_q8", "scap_dense_fc_q8", "scap_fold_bias_q8",
+    "scap_sparse_fc_q4", "scap_dense_fc_q4", "scap_fold_bias_q4",
     "scap_fc_host_workspace", "scap_sparse_fc_host",
     "scap_glu_workspace", "scap_glu_ffn", "scap_gelu_ffn_workspace", "scap_gelu_ffn", "scap_glu_static_capacity", "scap_glu_ffn_static", "scap_moe_workspace",
     "scap_moe_ffn", "ScapExpert", "dtype_of", "EXPORTS",
@@ -23,7 +24,8 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 EXPORTS = [
     "scap_status_string", "scap_version", "scap_tune", "scap_device_status", "scap_calibrate_workspace", "scap_calibrate",
     "scap_calibrate_ex", "scap_fold_bias_workspace", "scap_fold_bias", "scap_fc_workspace", "scap_sparse_fc", "scap_dense_fc",
-    "scap_sparse_fc_q8", "scap_dense_fc_q8", "scap_fold_bias_q8", "scap_fc_host_workspace", "scap_sparse_fc_host", "scap_glu_workspace", "scap_glu_ffn", "scap_gelu_ffn_workspace",
+    "scap_sparse_fc_q8", "scap_dense_fc_q8", "scap_fold_bias_q8", "scap_sparse_fc_q4", "scap_dense_fc_q4", "scap_fold_bias_q4",
+    "scap_fc_host_workspace", "scap_sparse_fc_host", "scap_glu_workspace", "scap_glu_ffn", "scap_gelu_ffn_workspace",
     "scap_gelu_ffn", "scap_glu_static_capacity", "scap_glu_ffn_static", "scap_moe_workspace", "scap_moe_ffn",
 ]
 
@@ -86,6 +88,12 @@ def lib():
     L.scap_dense_fc_q8.restype = i
     L.scap_fold_bias_q8.argtypes = [vp, vp, vp, vp, i, i, vp, vp, sz, vp]
     L.scap_fold_bias_q8.restype = i
+    L.scap_sparse_fc_q4.argtypes = [vp, i, vp, vp, vp, i, vp, vp, vp, vp, i, i, i, vp, vp, vp, sz, vp]
+    L.scap_sparse_fc_q4.restype = i
+    L.scap_dense_fc_q4.argtypes = [vp, i, vp, vp, vp, i, vp, vp, i, i, i, vp, sz, vp]
+    L.scap_dense_fc_q4.restype = i
+    L.scap_fold_bias_q4.argtypes = [vp, vp, vp, i, vp, vp, i, i, vp, vp, sz, vp]
+    L.scap_fold_bias_q4.restype = i
     L.scap_fc_host_workspace.argtypes = [i, i, i]
     L.scap_fc_host_workspace.restype = sz
     L.scap_sparse_fc_host.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, vp, sz, vp]
@@ -236,6 +244,30 @@ def scap_fold_bias_q8(Wq, wscale, m, b, b_fused, ws, stream=None) -> None:
     p, n = _ws(ws)
     _check(lib().scap_fold_bias_q8(_ptr(Wq), _ptr(wscale), _ptr(m), _ptr(b), K, N, _ptr(b_fused), p, n, _stream(stream)),
            "scap_fold_bias_q8")
+
+
+def scap_sparse_fc_q4(x, Wq, scale, zero, group, m, tau, b_fused, y, ws, idx_out=None, nnz_out=None, stream=None) -> None:
+    """Sparse FC on group-wise 4-bit weights: Wq uint8 [K, N/2] (two codes per byte), scale fp32 and zero uint8 [K/group, N]."""
+    B, K = x.shape
+    N = Wq.shape[1] * 2
+    p, n = _ws(ws)
+    _check(lib().scap_sparse_fc_q4(_ptr(x), dtype_of(x), _ptr(Wq), _ptr(scale), _ptr(zero), int(group), _ptr(m), _ptr(tau), _ptr(b_fused),
+                                   _ptr(y), B, K, N, _ptr(idx_out), _ptr(nnz_out), p, n, _stream(stream)), "scap_sparse_fc_q4")
+
+
+def scap_dense_fc_q4(x, Wq, scale, zero, group, b, y, ws, stream=None) -> None:
+    B, K = x.shape
+    N = Wq.shape[1] * 2
+    p, n = _ws(ws)
+    _check(lib().scap_dense_fc_q4(_ptr(x), dtype_of(x), _ptr(Wq), _ptr(scale), _ptr(zero), int(group), _ptr(b), _ptr(y), B, K, N, p, n,
+                                  _stream(stream)), "scap_dense_fc_q4")
+
+
+def scap_fold_bias_q4(Wq, scale, zero, group, m, b, b_fused, ws, stream=None) -> None:
+    K, N = Wq.shape[0], Wq.shape[1] * 2
+    p, n = _ws(ws)
+    _check(lib().scap_fold_bias_q4(_ptr(Wq), _ptr(scale), _ptr(zero), int(group), _ptr(m), _ptr(b), K, N, _ptr(b_fused), p, n,
+                                   _stream(stream)), "scap_fold_bias_q4")
 
 
 def scap_fc_host_workspace(B: int, K: int, N: int) -> int:
