@@ -203,20 +203,32 @@ __global__ void __launch_bounds__(FC_THREADS, 2) fc_q4_kernel(const Q4Args qa) {
 #pragma unroll
                     for (int j = 0; j < 16; ++j) zc[j] = 8388608.0f + (float)((z4[j >> 2] >> (8 * (j & 3))) & 255u);
                 }
-                for (int tb = t; tb < t_end; tb += U) {   // batches of U rows: all requested, then all used
-                    uint2 v[U];
+                // two register groups of U / 2 row loads alternate: one is used while the other is in flight
+                constexpr int H = U / 2;
+                uint2 va[H], vb[H];
+                auto request = [&](uint2(&dst)[H], int first) {
 #pragma unroll
-                    for (int u = 0; u < U; ++u) {
-                        const bool on = tb + u < t_end;
-                        v[u] = ld_stream8_if(Wb + (size_t)(on ? s_k[tb + u] : 0u) * row_bytes, on);
+                    for (int u = 0; u < H; ++u) {
+                        const bool on = first + u < t_end;
+                        dst[u] = ld_stream8_if(Wb + (size_t)(on ? s_k[first + u] : 0u) * row_bytes, on);
                     }
+                };
+                auto use = [&](const uint2(&src)[H], int first) {
 #pragma unroll
-                    for (int u = 0; u < U; ++u) {
-                        if (tb + u < t_end) {
+                    for (int u = 0; u < H; ++u) {
+                        if (first + u < t_end) {
 #pragma unroll
-                            for (int b = 0; b < BT; ++b) fma_row_q4(acc[b], v[u], zc, s_xs[b * CAP + tb + u]);
+                            for (int b = 0; b < BT; ++b) fma_row_q4(acc[b], src[u], zc, s_xs[b * CAP + first + u]);
                         }
                     }
+                };
+                request(va, t);
+                request(vb, t + H);
+                for (int tb = t; tb < t_end; tb += U) {
+                    use(va, tb);
+                    request(va, tb + U);
+                    use(vb, tb + H);
+                    request(vb, tb + U + H);
                 }
                 const float sc[16] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w, s2.x, s2.y, s2.z, s2.w, s3.x, s3.y, s3.z, s3.w};
 #pragma unroll
