@@ -351,6 +351,62 @@ def suite_q4(torch, scap, peak, out):
              "dense_q4_us": round(t_dense, 3), "speedup_vs_dense_q4": round(t_dense / t, 3), "weight_copies": R})
 
 
+def suite_overlap(torch, scap, peak, out):
+    """Beyond one union mask per batch (Appendix C of the paper): rows whose large activations fall on a per-context set of
+    channels, overlap 0 (independent rows) to 1 (the rows of a context share one pattern).  Bench shape, 60 % target,
+    batch 8 and 16 in 1, 2 or 4 contexts: the union kept fraction over the whole batch and per context, the ordinary call
+    (one union over all rows) and the grouped call (one union per context, scap_sparse_fc_grouped), against the dense call."""
+    stream = torch.cuda.Stream()
+    l2 = torch.cuda.get_device_properties(0).L2_cache_size
+    Kk, Nn, s = 11008, 4096, 0.6
+    W0 = si.as_torch(si.weight(4, Kk, Nn, si.BF16), si.BF16).cuda()
+    Rmax = int(np.ceil(4 * l2 / (0.4 * Kk * Nn * 2)))
+    Ws = [W0] + [W0.clone() for _ in range(Rmax - 1)]
+    cws = torch.empty(scap.scap_calibrate_workspace(512, Kk, NBINS), dtype=torch.uint8, device="cuda")
+    gws = torch.empty(scap.scap_grouped_workspace(), dtype=torch.uint8, device="cuda")
+    m = torch.empty(Kk, dtype=torch.float32, device="cuda")
+    tau = torch.empty(1, dtype=torch.float32, device="cuda")
+    bf = torch.empty(Nn, dtype=torch.float32, device="cuda")
+    nnz = torch.zeros(1, dtype=torch.int32, device="cuda")
+    for B in (8, 16):
+        ws = torch.empty(scap.scap_fc_workspace(B, Kk, Nn), dtype=torch.uint8, device="cuda")
+        y = torch.empty((B, Nn), dtype=torch.float32, device="cuda")
+        t_dense = None
+        for n_ctx in (1, 2, 4):
+            for ov in (0.0, 0.5, 0.9, 1.0):
+                d = si.context_batch(4, Kk, Nn, si.BF16, 512, 4 * B, n_ctx, ov, weights=False)
+                xc = si.as_torch(d["x_calib"], si.BF16).cuda()
+                xs = si.as_torch(d["x"], si.BF16).cuda()      # four batches of B rows (row b: context b mod n_ctx)
+                scap.scap_calibrate(xc, s, NBINS, m, tau, cws)
+                scap.scap_fold_bias(W0, m, None, bf, ws)
+                xb = [xs[i * B:(i + 1) * B] for i in range(4)]
+                groups = [b % n_ctx for b in range(B)]
+                if t_dense is None:
+                    Rd = max(2, int(np.ceil(4 * l2 / (Kk * Nn * 2))))
+                    t_dense = _time_graph(torch, stream, lambda: [scap.scap_dense_fc(xb[r % 4], Ws[r], None, y, ws) for r in range(Rd)]) / Rd
+                u_all, u_grp = [], []
+                for i in range(4):
+                    scap.scap_sparse_fc(xb[i], W0, m, tau, bf, y, ws, nnz_out=nnz)
+                    u_all.append(int(nnz.item()))
+                    tot = 0
+                    for c in range(n_ctx):
+                        rows = xb[i][c::n_ctx].contiguous()
+                        scap.scap_sparse_fc(rows, W0, m, tau, bf, y[:rows.shape[0]], ws, nnz_out=nnz)
+                        tot += int(nnz.item())
+                    u_grp.append(tot)
+                rho_all, rho_grp = float(np.mean(u_all)) / Kk, float(np.mean(u_grp)) / Kk
+                R = max(2, min(Rmax, int(np.ceil(4 * l2 / (max(rho_all, 0.4) * Kk * Nn * 2)))))
+                t_one = _time_graph(torch, stream, lambda: [scap.scap_sparse_fc(xb[r % 4], Ws[r], m, tau, bf, y, ws) for r in range(R)]) / R
+                rec = {"suite": "overlap", "K": Kk, "N": Nn, "B": B, "contexts": n_ctx, "overlap": ov, "sparsity_target": s,
+                       "union_kept_fraction_whole_batch": round(rho_all, 4), "sum_of_union_kept_fractions_per_context": round(rho_grp, 4),
+                       "one_union_us": round(t_one, 2), "dense_us": round(t_dense, 2), "one_union_vs_dense": round(t_dense / t_one, 3)}
+                if n_ctx > 1:
+                    t_grp = _time_graph(torch, stream, lambda: [scap.scap_sparse_fc_grouped(xb[r % 4], Ws[r], m, tau, bf, y, groups, gws) for r in range(R)]) / R
+                    rec.update({"grouped_us": round(t_grp, 2), "grouped_vs_one_union": round(t_one / t_grp, 3), "grouped_vs_dense": round(t_dense / t_grp, 3),
+                                "kernels_per_grouped_call": 2})
+                out(rec)
+
+
 def suite_calibrate(torch, scap, out):
     """Config 4's timed calibration: 2048 tokens x 14336 channels, 2048 bins, plus the tau quantile."""
     T, Kk = 2048, 14336
@@ -578,6 +634,8 @@ def run_suite(args):
         suite_q8(torch, scap, peak, out)
     if which in ("q4", "all"):
         suite_q4(torch, scap, peak, out)
+    if which in ("overlap", "all"):
+        suite_overlap(torch, scap, peak, out)
     if which in ("sweep", "all", "sweep-small"):
         shapes = [(4096, 4096), (4096, 11008), (11008, 4096), (14336, 4096)]
         if which == "sweep-small":
@@ -608,7 +666,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--detail", action="store_true", help="also print a per-sparsity table to stderr")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--suite", default="", choices=["", "calibrate", "glu", "gelu", "q8", "q4", "moe", "mamba", "sweep", "sweep-small", "all"],
+    ap.add_argument("--suite", default="", choices=["", "calibrate", "glu", "gelu", "q8", "q4", "overlap", "moe", "mamba", "sweep", "sweep-small", "all"],
                     help="run the other workload descriptions instead of the headline line (one JSON object per line)")
     ap.add_argument("--copies", type=int, default=0,
                     help="number of weight copies to rotate (default: enough for the cold-HBM rule); a small value keeps "

@@ -209,6 +209,18 @@ scap_status scap_dense_fc_q4(const void *x, scap_dtype xdt, const unsigned char 
 scap_status scap_fold_bias_q4(const unsigned char *Wq, const float *scale, const unsigned char *zero, int group, const float *m,
                               const float *b, int K, int N, float *b_fused, void *ws, size_t ws_bytes, scap_stream_t stream);
 
+/* Appendix C ("overlapping sparsity"): the union mask of a batch keeps its sparsity only as far as the rows' patterns
+ * overlap.  scap_sparse_fc_grouped is scap_sparse_fc for up to 64 rows whose groups the caller names - rows that are
+ * expected to share their pattern, e.g. the beams of one prompt or the tokens of one request: group_of_row_host[b]
+ * (a HOST array, read during the call only) is the group 0..15 of row b; at most 16 rows per group (else
+ * SCAP_ERR_SHAPE).  Each group is pruned with the union mask of its own rows only and fetches only the weight rows
+ * that mask keeps, all groups in one launch; y[b] is the same function of x[b] as in scap_sparse_fc (pruning is per
+ * element), whatever the grouping.  No idx / nnz outputs.  Workspace: scap_grouped_workspace() bytes.              */
+size_t scap_grouped_workspace(void);
+scap_status scap_sparse_fc_grouped(const void *x, const void *W, const float *m, const float *tau, const float *b_fused,
+                                   float *y, int B, int K, int N, scap_dtype dt, const int *group_of_row_host, void *ws,
+                                   size_t ws_bytes, scap_stream_t stream);
+
 /* scap_sparse_fc for a caller whose activations live in HOST memory: copies x_host[B,K]
  * (dtype dt; pinned memory recommended) to the device, runs the sparse FC, and copies y back to
  * y_host[B,N] (fp32), all enqueued on `stream`; y_host is valid once the stream has drained.

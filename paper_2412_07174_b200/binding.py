@@ -11,7 +11,7 @@ __all__ = [
     "scap_calibrate_workspace", "scap_calibrate", "scap_calibrate_ex", "SCAP_MODE_HISTOGRAM", "SCAP_MODE_MEAN", "SCAP_MODE_MEDIAN", "SCAP_MODE_KDE",
     "SCAP_ETA_PER_CHANNEL", "SCAP_ETA_SCALAR", "scap_fold_bias_workspace", "scap_fold_bias",
     "scap_fc_workspace", "scap_sparse_fc", "scap_dense_fc", "scap_sparse_fc_q8", "scap_dense_fc_q8", "scap_fold_bias_q8",
-    "scap_sparse_fc_q4", "scap_dense_fc_q4", "scap_fold_bias_q4",
+    "scap_sparse_fc_q4", "scap_dense_fc_q4", "scap_fold_bias_q4", "scap_grouped_workspace", "scap_sparse_fc_grouped",
     "scap_fc_host_workspace", "scap_sparse_fc_host",
     "scap_glu_workspace", "scap_glu_ffn", "scap_gelu_ffn_workspace", "scap_gelu_ffn", "scap_glu_static_capacity", "scap_glu_ffn_static", "scap_moe_workspace",
     "scap_moe_ffn", "ScapExpert", "dtype_of", "EXPORTS",
@@ -25,7 +25,7 @@ EXPORTS = [
     "scap_status_string", "scap_version", "scap_tune", "scap_device_status", "scap_calibrate_workspace", "scap_calibrate",
     "scap_calibrate_ex", "scap_fold_bias_workspace", "scap_fold_bias", "scap_fc_workspace", "scap_sparse_fc", "scap_dense_fc",
     "scap_sparse_fc_q8", "scap_dense_fc_q8", "scap_fold_bias_q8", "scap_sparse_fc_q4", "scap_dense_fc_q4", "scap_fold_bias_q4",
-    "scap_fc_host_workspace", "scap_sparse_fc_host", "scap_glu_workspace", "scap_glu_ffn", "scap_gelu_ffn_workspace",
+    "scap_grouped_workspace", "scap_sparse_fc_grouped", "scap_fc_host_workspace", "scap_sparse_fc_host", "scap_glu_workspace", "scap_glu_ffn", "scap_gelu_ffn_workspace",
     "scap_gelu_ffn", "scap_glu_static_capacity", "scap_glu_ffn_static", "scap_moe_workspace", "scap_moe_ffn",
 ]
 
@@ -94,6 +94,10 @@ def lib():
     L.scap_dense_fc_q4.restype = i
     L.scap_fold_bias_q4.argtypes = [vp, vp, vp, i, vp, vp, i, i, vp, vp, sz, vp]
     L.scap_fold_bias_q4.restype = i
+    L.scap_grouped_workspace.argtypes = []
+    L.scap_grouped_workspace.restype = sz
+    L.scap_sparse_fc_grouped.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, C.POINTER(C.c_int), vp, sz, vp]
+    L.scap_sparse_fc_grouped.restype = i
     L.scap_fc_host_workspace.argtypes = [i, i, i]
     L.scap_fc_host_workspace.restype = sz
     L.scap_sparse_fc_host.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, vp, sz, vp]
@@ -268,6 +272,20 @@ def scap_fold_bias_q4(Wq, scale, zero, group, m, b, b_fused, ws, stream=None) ->
     p, n = _ws(ws)
     _check(lib().scap_fold_bias_q4(_ptr(Wq), _ptr(scale), _ptr(zero), int(group), _ptr(m), _ptr(b), K, N, _ptr(b_fused), p, n,
                                    _stream(stream)), "scap_fold_bias_q4")
+
+
+def scap_grouped_workspace() -> int:
+    return lib().scap_grouped_workspace()
+
+
+def scap_sparse_fc_grouped(x, W, m, tau, b_fused, y, groups, ws, stream=None) -> None:
+    """Sparse FC with one union mask per group of rows; ``groups`` is a host sequence of B group numbers 0..15."""
+    B, K = x.shape
+    N = W.shape[1]
+    p, n = _ws(ws)
+    arr = (C.c_int * B)(*[int(g) for g in groups])
+    _check(lib().scap_sparse_fc_grouped(_ptr(x), _ptr(W), _ptr(m), _ptr(tau), _ptr(b_fused), _ptr(y), B, K, N, dtype_of(W), arr, p, n,
+                                        _stream(stream)), "scap_sparse_fc_grouped")
 
 
 def scap_fc_host_workspace(B: int, K: int, N: int) -> int:

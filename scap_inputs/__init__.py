@@ -186,6 +186,38 @@ def laplace_fc(config: int, K: int, N: int, dt: int, T_calib: int, B: int, with_
     return d
 
 
+def context_batch(config: int, K: int, N: int, dt: int, T_calib: int, B: int, n_ctx: int, overlap: float,
+                  active_frac: float = 0.5, hi: float = 0.3, lo: float = 0.01, weights: bool = True) -> dict:
+    """Rows whose large activations fall on a per-context set of channels (Appendix C of the paper: the rows of one batch
+    - beams of one prompt, tokens of one request - share part of their sparsity pattern).
+
+    Every context c has an active set A_c (each channel with probability active_frac).  Row b belongs to context
+    b mod n_ctx; channel k of row b is "on" if it is in A_c - with probability ``overlap`` per (row, channel) - or else
+    by an independent draw with probability active_frac.  x[b,k] = m_k + Laplace(0, hi) where on, Laplace(0, lo)
+    elsewhere.  overlap = 1: all rows of a context share one pattern; overlap = 0: the rows are independent.
+    With the defaults and a 60 % sparsity target the threshold falls between the two populations: a row keeps about
+    four fifths of its "on" channels and next to none of the others, so the union over a context's rows is bounded by
+    the context's active set (half the channels) at overlap 1 and approaches all channels at overlap 0.
+    The calibration rows are drawn the same way (context t mod n_ctx).  Returns also ``ctx`` [B]."""
+    m_true = uniform(stream_seed(config, S_MODE), K, -0.5, 0.5)
+    A = uniform(stream_seed(config, S_GAMMA), n_ctx * K).reshape(n_ctx, K) < active_frac
+
+    def rows(stream, T):
+        pick = uniform(stream_seed(config, stream, 1), T * K).reshape(T, K) < overlap
+        own = uniform(stream_seed(config, stream, 2), T * K).reshape(T, K) < active_frac
+        on = np.where(pick, A[np.arange(T) % n_ctx], own)
+        noise = laplace(stream_seed(config, stream), T * K, 1.0).reshape(T, K)
+        return m_true[None, :] + noise * np.where(on, hi, lo), on
+
+    xc, _ = rows(S_XCALIB, T_calib)
+    xt, on = rows(S_XTEST, B)
+    d = {"dt": dt, "K": K, "N": N, "m_true": m_true.astype(np.float32), "x_calib": to_bits(xc, dt), "x": to_bits(xt, dt),
+         "ctx": (np.arange(B) % n_ctx).astype(np.int32), "on": on, "b": None}
+    if weights:
+        d["W"] = weight(config, K, N, dt)
+    return d
+
+
 def _silu(g: np.ndarray) -> np.ndarray:
     return g / (1.0 + np.exp(-g))
 

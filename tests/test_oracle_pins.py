@@ -657,3 +657,20 @@ def test_q4_quantiser_properties():
     back = scale[gi].astype(np.float64) * (q - zero[gi].astype(np.int64))
     assert packed.shape == (200, 12) and scale.shape == (4, 24) and zero.shape == (4, 24) and q.min() >= 0 and q.max() == 15
     assert np.all(np.abs(back - Wf) <= scale[gi] * (1.0 + 1e-6))      # within one step (zero-point rounding adds up to half a step)
+
+
+# ---------------------------------------------------------------- input recipe with overlapping sparsity (Appendix C)
+
+def test_overlapping_rows_keep_the_union_sparse():
+    """The recipe behind the test above: with full overlap the union over a context's rows stays near the per-row kept
+    fraction, with none it grows like independent draws (CPU check of the generator through the oracle's mask)."""
+    K = 4096
+    fr = {}
+    for ov in (0.0, 1.0):
+        d = si.context_batch(4, K, 8, si.BF16, 64, 8, 1, ov, weights=False)
+        xf = si.to_f32(d["x"], si.BF16)
+        tau = oracle.tau(si.to_f32(d["x_calib"], si.BF16), d["m_true"], 0.6)
+        keep, U, idx = oracle.mask(xf, d["m_true"], tau)
+        fr[ov] = (keep.mean(), idx.size / K)
+    assert abs(fr[0.0][0] - 0.4) < 0.05 and abs(fr[1.0][0] - 0.4) < 0.05
+    assert fr[1.0][1] < 0.55 and fr[0.0][1] > 0.8
