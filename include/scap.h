@@ -83,7 +83,12 @@ int scap_version(void);
  *   "tcgen05"  tensor-core batches of the FC and SwiGLU entry points: 0 = always the mma.sync variants,
  *              1 = the tcgen05 (TMEM accumulator) kernel where its shared-memory operand region holds
  *              the call's kept channels in one pass, else mma.sync (default), 2 = always tcgen05
- *   "tc_spin"  tcgen05 kernel: how often a wait on one of its shared-memory barriers polls before it gives up
+ *   "dense_stream"  batches above "fma_rows": 1 (default) = the dense-stream tensor-core kernel, which reads every row of
+ *              its weight tile with TMA box loads and prunes on the activation operand (with that many rows the union
+ *              mask of unrelated rows keeps nearly every channel anyway); 0 = the gather kernels, which fetch kept rows
+ *              only (better when the rows of a batch share their pattern and the union keeps less than about half);
+ *              2 = the dense-stream kernel from batch 3 on
+ *   "tc_spin"  tcgen05 kernels: how often a wait on one of its shared-memory barriers polls before it gives up
  *              (0 = the built-in limit of about a million polls, the default).  A limit of 1 makes the waits of
  *              the next call run out at once, which is how the error path of scap_device_status() is exercised
  *              without a fault; y of such a call is incomplete.
@@ -115,7 +120,8 @@ scap_status scap_device_status(void);
  *   tau_out[1] the `sparsity` quantile (linear interpolation between order statistics) of the
  *              importance |x - m| pooled over all T*K values; sparsity <= 0 gives tau = 0.
  * Binary32 arithmetic with every operation rounded separately, so results are bit-reproducible.
- * Inputs must be finite.  sparsity must lie in [0, 1); T*K < 2^31; T <= 65535.
+ * Inputs must be finite.  sparsity must lie in [0, 1); T*K < 2^31; T <= 65535; K a multiple of 8
+ * (else SCAP_ERR_ALIGN).
  * ------------------------------------------------------------------------------------------ */
 size_t scap_calibrate_workspace(int T, int K, int nbins);
 scap_status scap_calibrate(const void *x_calib, int T, int K, scap_dtype dt, double sparsity, int nbins,
@@ -161,10 +167,12 @@ scap_status scap_fold_bias(const void *W, const float *m, const void *b, int K, 
  * Optional outputs for inspection: idx_out[K] receives the ascending list of fetched channels
  * (first *nnz_out entries valid), nnz_out[1] their number.  m, b_fused, idx_out, nnz_out may
  * be NULL.  Results are bitwise reproducible for fixed shapes and tuning.
- * Arithmetic: batch 1-2 multiply-accumulates in fp32 FMAs.  Batch 3-16 runs on the tensor cores
- * with d split exactly into parts of the weight dtype (bf16: three parts, fp16: two) and fp32
- * accumulation, so the result carries the same information as the FMA path; with fp16 weights
- * the parts overflow for |d| > 65504 (such an activation yields inf/NaN in its row only).
+ * Arithmetic: batches up to the tuning value "fma_rows" (default 4) multiply-accumulate in fp32 FMAs.
+ * Larger batches (up to 16) run on the tensor cores with d split exactly into parts of the weight dtype
+ * (bf16: three parts, fp16: two) and fp32 accumulation, so the result carries the same information as
+ * the FMA path; with fp16 weights the parts overflow for |d| > 65504 (such an activation yields inf/NaN
+ * in its row only).  In the tensor-core forms a non-finite weight makes its column non-finite whether
+ * or not its channel is kept (0 * inf): weights must be finite.
  * ------------------------------------------------------------------------------------------ */
 size_t scap_fc_workspace(int B, int K, int N);
 scap_status scap_sparse_fc(const void *x, const void *W, const float *m, const float *tau, const float *b_fused,

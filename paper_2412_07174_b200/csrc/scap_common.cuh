@@ -24,6 +24,7 @@ struct Tuning {
     int l2_hints;     // batch 1..4 FC kernel: L2 eviction hints (keep activations and modes, stream weights)
     int tile;         // columns per CTA of the FC kernel: 0 = automatic, else 128 or 256
     int tc_spin;      // tcgen05 kernel: polls before a barrier wait gives up (0 = the built-in limit)
+    int dense_stream; // batch 5..16: 1 = the dense-stream tcgen05 kernel (TMA box loads of all rows), 0 = the gather kernels, 2 = from batch 3
 };
 extern Tuning g_tune;
 
@@ -182,6 +183,18 @@ __device__ __forceinline__ unsigned short ld_act_if_u16(const void *p, bool on) 
 }
 __device__ __forceinline__ __nv_bfloat16 ld_act_if(const __nv_bfloat16 *p, bool on) { return __ushort_as_bfloat16(ld_act_if_u16(p, on)); }
 __device__ __forceinline__ __half ld_act_if(const __half *p, bool on) { return __ushort_as_half(ld_act_if_u16(p, on)); }
+
+// 16-byte activation / parameter load through L2, predicated (zeros where off).
+__device__ __forceinline__ uint4 ld_act16_if(const void *p, bool on) {
+    uint4 v;
+    asm volatile(
+        "{ .reg .pred q; setp.ne.u32 q, %5, 0; mov.u32 %0, 0; mov.u32 %1, 0; mov.u32 %2, 0; mov.u32 %3, 0;"
+        " @q ld.global.cg.v4.u32 {%0,%1,%2,%3}, [%4]; }"
+        : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+        : "l"(p), "r"((unsigned)on)
+        : "memory");
+    return v;
+}
 
 // L2 eviction policies for loads that carry a cache hint.  keep: small data every column tile of a call reads again
 // (activations, modes); stream: weight rows, read once.

@@ -8,7 +8,7 @@
 
 namespace scap {
 
-Tuning g_tune = {0, 1, 1, 1, 4, 16, 1, 0, 0};
+Tuning g_tune = {0, 1, 1, 1, 4, 16, 1, 0, 0, 1};
 
 scap_status check_device() {
     static std::atomic<int> cached[64];  // 0 unknown, 1 ok, 2 unsupported
@@ -163,6 +163,14 @@ static cudaError_t launch_fc_w(int mode, int xkind, int epi, const FcArgs &a, cu
 }
 
 cudaError_t launch_fc(bool bf16, int mode, int xkind, int epi, const FcArgs &a, cudaStream_t st) {
+    if (ds_applicable(a, epi, bf16)) {
+        FcArgs t = a;
+        t.tn = 128;
+        t.S = ds_choose_split(a.K, a.Nh, epi);
+        t.spin = g_tune.tc_spin;
+        t.status = tc_status_ptr();
+        return launch_fc_ds(bf16, mode, xkind, epi, t, st);
+    }
     if (tc_applicable(a, epi, bf16)) {
         FcArgs t = a;
         t.tn = 256;
@@ -326,6 +334,11 @@ scap_status scap_tune(const char *key, int value) {
     if (!strcmp(key, "tile")) {
         if (value != 0 && value != 128 && value != 256) return SCAP_ERR_INVALID_ARG;
         g_tune.tile = value;
+        return SCAP_OK;
+    }
+    if (!strcmp(key, "dense_stream")) {
+        if (value < 0 || value > 2) return SCAP_ERR_INVALID_ARG;
+        g_tune.dense_stream = value;
         return SCAP_OK;
     }
     if (!strcmp(key, "tc_spin")) {

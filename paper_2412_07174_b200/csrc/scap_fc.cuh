@@ -924,6 +924,10 @@ bool tc_applicable(const FcArgs &a, int epi, bool bf16);
 int tc_choose_split(int K, int Nh, int epi, int B, bool bf16);
 cudaError_t launch_fc_tc(bool bf16, int mode, int xkind, int epi, const FcArgs &a, cudaStream_t st);
 int tc_take_status();
+// Dense-stream tcgen05 kernel (scap_fc_tc.cu): TMA box loads of all rows, pruning on the activation operand.
+bool ds_applicable(const FcArgs &a, int epi, bool bf16);
+int ds_choose_split(int K, int Nh, int epi);
+cudaError_t launch_fc_ds(bool bf16, int mode, int xkind, int epi, const FcArgs &a, cudaStream_t st);
 int *tc_status_ptr();  // device address of that status word on the current device (NULL if it cannot be had)
 
 // Launch with cluster dimension (1, S, 1) and, if enabled, programmatic dependent launch.

@@ -22,6 +22,7 @@
 // first and was no faster on this access pattern.)
 // Every wait on an mbarrier is bounded; a wait that runs out sets a device status word, the CTA stops issuing work,
 // still passes every cluster barrier and frees its TMEM.
+#include <cuda.h>
 #include <string.h>
 
 #include <atomic>
@@ -447,6 +448,317 @@ __global__ void __launch_bounds__(FC_THREADS, 2) fc_tc_kernel(const FcArgs a) {
     if (S > 1) cluster.sync();
 }
 
+// ------------------------------------------------------------------------------------------------
+// Dense-stream variant (batch 5..16).  With that many rows the union mask of independent rows keeps nearly every channel
+// (Appendix C), so gathering kept rows buys nothing and costs the memory-level parallelism of the copy engine.  Here
+// the CTA streams ALL rows of its share of the tile - blocks of 64 consecutive rows, block q of rank s = rows
+// (q S + s) 64 .. + 63 - with two TMA box loads per block (64 columns x 64 rows each, 128-byte swizzle: exactly the
+// MN-major B operand of the MMA, no address arithmetic, one instruction per 8 KB), and pruning happens on the small
+// operand instead: a dropped channel gets a zero activation.  Roles: warp 0 issues the TMA loads, warp 1 the MMAs,
+// warps 2-7 threshold one 32-channel chunk at a time (d = x - m, |d| >= tau, ballot for the mask words, exact split into
+// parts of the weight dtype) and write it as the A operand of its stage; W ring and A ring have DS_NST stages each and
+// share the stage's "empty" barrier.  The epilogue is that of the gather kernel.  Every wait is bounded.
+// ------------------------------------------------------------------------------------------------
+constexpr int DS_NST = 4;
+constexpr int DS_STAGE_W = 64 * TC_TN * 2;                      // 16 KB: two boxes of 64 rows x 64 columns
+__host__ __device__ constexpr int ds_a_stage(int groups) { return 4 * 2 * groups * 128; }  // A operand of 64 channels
+constexpr int DS_OFF_W = 0;
+constexpr int DS_OFF_A = DS_OFF_W + DS_NST * DS_STAGE_W;
+constexpr int DS_OFF_GATHER = DS_OFF_A + DS_NST * ds_a_stage(6) + 2560;  // + slack: the MMA reads 128 rows of M, used or not
+constexpr int DS_OFF_MISC = DS_OFF_GATHER + 16 * TC_TN * 4;
+constexpr int DS_SMEM = DS_OFF_MISC + 512 + 1024;               // misc block + alignment slack
+static_assert(48 * TC_PART_LD * 4 <= DS_NST * DS_STAGE_W, "accumulator copy must fit in the W ring");
+static_assert(2 * (DS_SMEM + 1024) <= 233472, "two CTAs must fit in the shared memory of an SM");
+
+struct DsMisc {
+    unsigned long long wfull[DS_NST];   // TMA bytes of the stage have landed
+    unsigned long long afull[DS_NST];   // both chunks of the stage's A operand are written
+    unsigned long long empty[DS_NST];   // the stage's MMAs have read W and A
+    unsigned long long done;
+    uint32_t tmem_base;
+    int abort;
+    int issued;
+    int rows[16];
+};
+
+__device__ __forceinline__ void mbar_arrive_expect_tx(unsigned long long *bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+// One box of the tensor map (64 columns x 64 rows) to shared memory; completion counts bytes on `bar`.  No multicast.
+__device__ __forceinline__ void tma_box_2d(uint32_t dst, const CUtensorMap *map, int x, int y, unsigned long long *bar) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
+                 "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar))
+                 : "memory");
+}
+
+template <bool BF16, int ROWS, int MODE, typename XT, int EPI>
+__global__ void __launch_bounds__(FC_THREADS, 2) fc_ds_kernel(const FcArgs a, const __grid_constant__ CUtensorMap tmap) {
+    constexpr int TNT = TC_TN, HALF = TNT / 2, NSPLIT = mma_nsplit(BF16);
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    unsigned char *s_w = smem + DS_OFF_W;
+    unsigned char *s_a = smem + DS_OFF_A;
+    float *s_gather = reinterpret_cast<float *>(smem + DS_OFF_GATHER);
+    DsMisc *misc = reinterpret_cast<DsMisc *>(smem + DS_OFF_MISC);
+    float *s_part = reinterpret_cast<float *>(s_w);  // accumulator rows, after the stream
+    volatile int *abort_flag = &misc->abort;
+    const uint32_t spin = a.spin ? (uint32_t)a.spin : TC_SPIN;
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int tile = blockIdx.x, s = blockIdx.y;
+    const int B = a.B, S = a.S, K = a.K;
+    const int racc = NSPLIT * B;
+    const int G = tc_groups(B, NSPLIT);
+    const uint32_t LBO = G * 128, BLK = 2 * LBO, ASTG = 4 * BLK;
+    const XT *xg = reinterpret_cast<const XT *>(a.x);
+    const int nblk64 = (K + 63) >> 6;
+    const int nq = nblk64 > s ? (nblk64 - s + S - 1) / S : 0;  // 64-row blocks (= stages) of this rank
+
+    if (tid == 0) {
+        for (int i = 0; i < DS_NST; ++i) {
+            mbar_init(&misc->wfull[i], 1);
+            mbar_init(&misc->afull[i], 2);
+            mbar_init(&misc->empty[i], 1);
+        }
+        mbar_init(&misc->done, 1);
+        misc->abort = 0;
+        misc->issued = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&misc->tmem_base)), "r"(TNT) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    const int per = ((EPI == EPI_GLU ? HALF : TNT) + S - 1) / S;
+    float bias0[2], bias1[2];
+
+    griddep_wait();  // nothing is read before earlier work on the stream is complete
+    griddep_launch_dependents();
+    float tau = 0.0f;
+    if constexpr (MODE == MODE_GATHER) {
+        float tv = 0.0f;
+        if (lane == 0) tv = ld_act(a.tau);
+        tau = __shfl_sync(0xffffffffu, tv, 0);
+    }
+    prefetch_bias<BF16, EPI, TNT>(a, tile, s, per, bias0, bias1);
+    if (a.in_rows && tid < 16) misc->rows[tid] = __ldcg(a.in_rows + (tid < B ? tid : 0));
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = misc->tmem_base;
+    const uint32_t idesc = (1u << 4) | ((BF16 ? 1u : 0u) << 7) | ((BF16 ? 1u : 0u) << 10) | (0u << 15) | (1u << 16) |
+                           ((uint32_t)(TNT >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+
+    if (warp == 0) {
+        // ---- TMA producer: two boxes per stage
+        if (lane == 0) {
+            const int x0 = EPI == EPI_GLU ? tile * HALF : tile * TNT;
+            const int x1 = EPI == EPI_GLU ? a.Nh + tile * HALF : tile * TNT + HALF;
+            int q = 0;
+            for (; q < nq; ++q) {
+                const uint32_t st = (uint32_t)q % DS_NST;
+                if (!mbar_wait(&misc->empty[st], (((uint32_t)q / DS_NST) & 1u) ^ 1u, 1, abort_flag, spin)) break;
+                mbar_arrive_expect_tx(&misc->wfull[st], DS_STAGE_W);
+                const int row0 = (q * S + s) * 64;
+                const uint32_t dst = smem_u32(s_w) + st * DS_STAGE_W;
+                tma_box_2d(dst, &tmap, x0, row0, &misc->wfull[st]);
+                tma_box_2d(dst + DS_STAGE_W / 2, &tmap, x1, row0, &misc->wfull[st]);
+            }
+            // After a wait that ran out the MMA lane no longer consumes stages, but loads already issued still write
+            // this CTA's shared memory: wait for them (fixed limit; they land within microseconds) before anyone leaves.
+            if (*abort_flag) {
+                int drain_abort = 0;
+                for (int qq = q > DS_NST ? q - DS_NST : 0; qq < q; ++qq)
+                    mbar_wait(&misc->wfull[(uint32_t)qq % DS_NST], ((uint32_t)qq / DS_NST) & 1u, 5, &drain_abort, TC_SPIN);
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        // ---- MMA issuer: per stage four MMAs of 16 rows
+        if (lane == 0) {
+            for (int q = 0; q < nq; ++q) {
+                const uint32_t st = (uint32_t)q % DS_NST, par = ((uint32_t)q / DS_NST) & 1u;
+                if (!mbar_wait(&misc->afull[st], par, 2, abort_flag, spin)) break;
+                if (!mbar_wait(&misc->wfull[st], par, 2, abort_flag, spin)) break;
+                tc_fence_after();
+                misc->issued = 1;
+#pragma unroll
+                for (uint32_t kb = 0; kb < 4; ++kb) {
+                    const uint64_t da = tc_desc(smem_u32(s_a) + st * ASTG + kb * BLK, LBO, 128, 0);
+                    const uint64_t db = tc_desc(smem_u32(s_w) + st * DS_STAGE_W + kb * 2048, DS_STAGE_W / 2, 1024, 2);
+                    tc_mma(tmem, da, db, idesc, (q > 0 || kb > 0) ? 1u : 0u);
+                }
+                tc_commit(&misc->empty[st]);
+            }
+            if (nq > 0 && !*abort_flag) tc_commit(&misc->done);
+        }
+        __syncwarp();
+    } else {
+        // ---- A operand: chunk jc = stage 2 q + half h; element (row r = part * B + b, position pos of the stage): block
+        // pos / 16, K half (pos / 8) & 1, 8-row group r / 8, 16 bytes per row of the group, 2 bytes per position.
+        // A lane takes ONE batch row and ROWS consecutive channels of the chunk (lane = channel group * ROWS + row): its
+        // activations are one or two 16-byte loads, and the eight positions of a row inside a K half are one 16-byte
+        // store per part.  (Rows of x that are not 16-byte aligned - K not a multiple of 8 - take scalar loads.)
+        const int pw = warp - 2;
+        constexpr int CPL = ROWS;                   // channels per lane
+        constexpr int XV = CPL * (int)sizeof(XT) / 16;  // 16-byte loads of x per lane
+        const int b = lane % ROWS, cgp = lane / ROWS, ch0 = cgp * CPL;
+        const bool vec_ok = ((size_t)a.x_ld * sizeof(XT)) % 16 == 0;
+        const int xrow = a.in_rows ? misc->rows[b < B ? b : 0] : (b < B ? b : 0);
+        for (int jc = pw; jc < 2 * nq; jc += FC_WARPS - 2) {
+            const int q = jc >> 1, h = jc & 1;
+            const uint32_t st = (uint32_t)q % DS_NST;
+            const int c = 2 * (q * S + s) + h;  // global 32-channel chunk
+            const int k0 = c * 32 + ch0;        // this lane's first channel
+            float xv[CPL], mv[CPL];
+            if (vec_ok) {
+                uint4 raw[XV];
+#pragma unroll
+                for (int v = 0; v < XV; ++v) {
+                    const int kk = k0 + v * (16 / (int)sizeof(XT));
+                    raw[v] = ld_act16_if(reinterpret_cast<const unsigned char *>(xg + (size_t)xrow * a.x_ld + kk), b < B && kk < K);
+                }
+                const XT *xe = reinterpret_cast<const XT *>(raw);
+#pragma unroll
+                for (int i = 0; i < CPL; ++i) xv[i] = widen1(xe[i]);
+            } else {
+#pragma unroll
+                for (int i = 0; i < CPL; ++i) xv[i] = widen1(ld_act_if(xg + (size_t)xrow * a.x_ld + k0 + i, b < B && k0 + i < K));
+            }
+            if (K % 4 == 0) {
+#pragma unroll
+                for (int v = 0; v < CPL / 4; ++v) {
+                    uint4 r4 = make_uint4(0, 0, 0, 0);
+                    if (MODE == MODE_GATHER && a.m) r4 = ld_act16_if(reinterpret_cast<const unsigned char *>(a.m + k0 + 4 * v), b < B && k0 + 4 * v < K);
+                    mv[4 * v] = __uint_as_float(r4.x); mv[4 * v + 1] = __uint_as_float(r4.y);
+                    mv[4 * v + 2] = __uint_as_float(r4.z); mv[4 * v + 3] = __uint_as_float(r4.w);
+                }
+            } else {
+#pragma unroll
+                for (int i = 0; i < CPL; ++i) mv[i] = (MODE == MODE_GATHER && a.m) ? ld_act_if(a.m + k0 + i, b < B && k0 + i < K) : 0.0f;
+            }
+            bool go = true;
+            if (lane == 0) go = mbar_wait(&misc->empty[st], (((uint32_t)q / DS_NST) & 1u) ^ 1u, 1, abort_flag, spin);
+            go = __shfl_sync(0xffffffffu, go ? 1 : 0, 0) != 0;
+            if (!go) break;
+            uint32_t mine = 0;
+            unsigned short part[CPL][3];
+#pragma unroll
+            for (int i = 0; i < CPL; ++i) {
+                const float dv = (MODE == MODE_GATHER && a.m) ? __fsub_rn(xv[i], mv[i]) : xv[i];
+                const bool kept = b < B && k0 + i < K && (MODE == MODE_DENSE || fabsf(dv) >= tau);
+                mine |= kept ? (1u << i) : 0u;
+                split_parts<BF16>(kept ? dv : 0.0f, part[i]);
+            }
+            if (b < B) {
+#pragma unroll
+                for (int v = 0; v < CPL / 8; ++v) {
+                    const int pos = h * 32 + ch0 + 8 * v;   // first of eight consecutive positions: one K half of one block
+                    unsigned char *dst = s_a + st * ASTG + (size_t)(pos >> 4) * BLK + ((pos >> 3) & 1) * LBO;
+#pragma unroll
+                    for (int p = 0; p < NSPLIT; ++p) {
+                        const int r = p * B + b;
+                        uint4 w;
+                        w.x = (uint32_t)part[8 * v + 0][p] | ((uint32_t)part[8 * v + 1][p] << 16);
+                        w.y = (uint32_t)part[8 * v + 2][p] | ((uint32_t)part[8 * v + 3][p] << 16);
+                        w.z = (uint32_t)part[8 * v + 4][p] | ((uint32_t)part[8 * v + 5][p] << 16);
+                        w.w = (uint32_t)part[8 * v + 6][p] | ((uint32_t)part[8 * v + 7][p] << 16);
+                        *reinterpret_cast<uint4 *>(dst + (r >> 3) * 128 + (r & 7) * 16) = w;
+                    }
+                }
+            }
+            const unsigned bal = __reduce_or_sync(0xffffffffu, mine << ch0);   // union over the rows, all 32 channels
+            if (MODE == MODE_GATHER && a.bits && tile == 0 && lane == 0 && c * 32 < K) a.bits[c] = bal;
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes -> visible to the tensor core
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&misc->afull[st]);
+        }
+    }
+    // ---- all threads: wait until the last MMA has finished
+    if (nq > 0) mbar_wait(&misc->done, 0, 3, abort_flag, spin);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    if (*abort_flag && misc->issued) {  // MMAs issued before a wait ran out may still be writing the accumulator
+        if (warp == 1 && lane == 0) tc_commit(&misc->done);
+        __syncwarp();
+        int drain_abort = 0;
+        mbar_wait(&misc->done, 0, 4, &drain_abort, TC_SPIN);
+    }
+    const bool have_acc = nq > 0 && !*abort_flag;
+    if (have_acc && warp * 32 < racc && warp < 2) {
+#pragma unroll 1
+        for (int c0 = 0; c0 < TNT; c0 += 32) {
+            uint32_t v[32];
+            asm volatile(
+                "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+                "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+                : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+                  "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
+                  "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
+                  "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+                : "r"(tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0));
+            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+            const int r = warp * 32 + lane;
+            if (r < racc) {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) s_part[r * TC_PART_LD + c0 + j] = __uint_as_float(v[j]);
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TNT) : "memory");
+    for (int i = tid; i < 16 * TNT; i += FC_THREADS) {
+        const int b = i / TNT, c = i - b * TNT;
+        float v = 0.0f;
+        if (have_acc && b < B) {
+#pragma unroll
+            for (int p = NSPLIT - 1; p >= 0; --p) v += s_part[(p * B + b) * TC_PART_LD + c];
+        }
+        s_gather[i] = v;
+    }
+    // ---- cluster exchange, pull form, and the bias / SwiGLU epilogue (as in the gather kernel)
+    cg::cluster_group cluster = cg::this_cluster();
+    if (S > 1) cluster.sync();
+    else __syncthreads();
+    const float *peer[MAX_CLUSTER];
+#pragma unroll
+    for (int q = 0; q < MAX_CLUSTER; ++q) peer[q] = (S > 1 && q < S) ? cluster.map_shared_rank(s_gather, q) : s_gather;
+    for (int it = 0; tid + it * FC_THREADS < per * B; ++it) {
+        const int i = tid + it * FC_THREADS;
+        const int b = i / per, c = i - b * per;
+        const int row = a.out_rows ? __ldcg(a.out_rows + b) : b;
+        if constexpr (EPI == EPI_BIAS) {
+            const int n = tile * TNT + s * per + c;
+            if (s * per + c < TNT && n < a.Nh) {
+                float v = it == 0 ? bias0[0] : it == 1 ? bias0[1] : load_bias<BF16>(a, n);
+#pragma unroll
+                for (int q = 0; q < MAX_CLUSTER; ++q)
+                    if (q < S) v += peer[q][b * TNT + s * per + c];
+                store_result(a, row, b, n, v);
+            }
+        } else {
+            const int F = a.Nh, f = tile * HALF + s * per + c;
+            if (s * per + c < HALF && f < F) {
+                float gt = it == 0 ? bias0[0] : it == 1 ? bias0[1] : (a.bias ? __ldcg(a.bias + f) : 0.0f);
+                float up = it == 0 ? bias1[0] : it == 1 ? bias1[1] : (a.bias ? __ldcg(a.bias + F + f) : 0.0f);
+#pragma unroll
+                for (int q = 0; q < MAX_CLUSTER; ++q)
+                    if (q < S) {
+                        gt += peer[q][b * TNT + s * per + c];
+                        up += peer[q][b * TNT + HALF + s * per + c];
+                    }
+                const float z = up * (gt / (1.0f + expf(-gt)));  // up * silu(gate)
+                a.y[(size_t)row * a.y_ld + f] = z;
+                if (a.z_copy) a.z_copy[(size_t)b * F + f] = z;
+            }
+        }
+    }
+    if (S > 1) cluster.sync();
+}
+
 // ---- host side ------------------------------------------------------------------------------------------------
 
 template <bool BF16, int ROWS, int MODE, typename XT, int EPI>
@@ -517,6 +829,95 @@ int tc_choose_split(int K, int Nh, int epi, int B, bool bf16) {
         if (score > best) { best = score; best_S = S; }
     }
     return best_S;
+}
+
+
+// ---- dense-stream kernel: tensor map and launch ----------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
+                                  const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_tiled_fn() {
+    static std::atomic<EncodeTiledFn> cached{nullptr};
+    EncodeTiledFn fn = cached.load(std::memory_order_acquire);
+    if (fn) return fn;
+    void *p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess || q != cudaDriverEntryPointSuccess || !p) {
+        cudaGetLastError();
+        return nullptr;
+    }
+    fn = reinterpret_cast<EncodeTiledFn>(p);
+    cached.store(fn, std::memory_order_release);
+    return fn;
+}
+
+// W[K, ldw] of 16-bit elements as a 2-D tensor (columns innermost), boxes of 64 columns x 64 rows, 128-byte swizzle,
+// rows and columns beyond the matrix read as zeros.  The map covers this GPU's own W only; no multicast anywhere.
+static bool ds_tensor_map(CUtensorMap *map, const void *W, int K, int ldw, bool bf16) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)ldw, (cuuint64_t)K};
+    const cuuint64_t strides[1] = {(cuuint64_t)ldw * 2};
+    const cuuint32_t box[2] = {64, 64};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(map, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void *>(W), dims, strides, box,
+              estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <bool BF16, int ROWS, int MODE, typename XT, int EPI>
+static cudaError_t launch_ds_r(const FcArgs &a, const CUtensorMap &map, cudaStream_t st) {
+    static SmemOptIn opt_in;
+    auto kern = fc_ds_kernel<BF16, ROWS, MODE, XT, EPI>;
+    cudaError_t e0 = ensure_dynamic_smem(kern, DS_SMEM, opt_in);
+    if (e0 != cudaSuccess) return e0;
+    return launch_cluster(kern, dim3(fc_tiles(a.Nh, EPI, TC_TN), a.S), dim3(FC_THREADS), DS_SMEM, a.S, st, g_tune.pdl != 0, a, map);
+}
+template <bool BF16, int MODE, typename XT, int EPI>
+static cudaError_t launch_ds_t(const FcArgs &a, const CUtensorMap &map, cudaStream_t st) {
+    return a.B <= 8 ? launch_ds_r<BF16, 8, MODE, XT, EPI>(a, map, st) : launch_ds_r<BF16, 16, MODE, XT, EPI>(a, map, st);
+}
+template <bool BF16, int MODE, typename XT>
+static cudaError_t launch_ds_e(int epi, const FcArgs &a, const CUtensorMap &map, cudaStream_t st) {
+    return epi == EPI_GLU ? launch_ds_t<BF16, MODE, XT, EPI_GLU>(a, map, st) : launch_ds_t<BF16, MODE, XT, EPI_BIAS>(a, map, st);
+}
+template <bool BF16>
+static cudaError_t launch_ds_w(int mode, int xkind, int epi, const FcArgs &a, const CUtensorMap &map, cudaStream_t st) {
+    using ST = typename std::conditional<BF16, __nv_bfloat16, __half>::type;
+    if (mode == MODE_DENSE)
+        return xkind == 2 ? launch_ds_e<BF16, MODE_DENSE, float>(epi, a, map, st) : launch_ds_e<BF16, MODE_DENSE, ST>(epi, a, map, st);
+    return xkind == 2 ? launch_ds_e<BF16, MODE_GATHER, float>(epi, a, map, st) : launch_ds_e<BF16, MODE_GATHER, ST>(epi, a, map, st);
+}
+
+// tune "dense_stream": 0 never, 1 (default) batches above the fp32-FMA limit, 2 every batch 3..16 call.
+bool ds_applicable(const FcArgs &a, int epi, bool bf16) {
+    (void)epi; (void)bf16;
+    if (g_tune.dense_stream == 0 || a.no_tc || a.B < 3 || a.B > 16 || a.ldw % 8 != 0 || !aligned16(a.W) || a.hold_dependents) return false;
+    if (a.K < 64) return false;
+    if (g_tune.dense_stream >= 2) return true;
+    return a.B > g_tune.fma_rows;
+}
+
+// Split-K factor: the most CTAs (128-column tiles x S) that are all resident, at least one 64-row block per rank.
+int ds_choose_split(int K, int Nh, int epi) {
+    const int tiles = fc_tiles(Nh, epi, TC_TN), blocks = (K + 63) / 64;
+    int best_S = 1;
+    long long best = -1;
+    for (int S = 1; S <= MAX_CLUSTER; ++S) {
+        if (g_tune.split_k > 0 && S > g_tune.split_k) continue;
+        if (S > blocks) continue;
+        const long long ctas = (long long)tiles * S;
+        if (S > 1 && ctas > tc_resident(S)) continue;
+        if (ctas > best) { best = ctas; best_S = S; }
+    }
+    return best_S;
+}
+
+cudaError_t launch_fc_ds(bool bf16, int mode, int xkind, int epi, const FcArgs &a, cudaStream_t st) {
+    CUtensorMap map;
+    if (!ds_tensor_map(&map, a.W, a.K, a.ldw, bf16)) return cudaErrorNotSupported;
+    return bf16 ? launch_ds_w<true>(mode, xkind, epi, a, map, st) : launch_ds_w<false>(mode, xkind, epi, a, map, st);
 }
 
 cudaError_t launch_fc_tc(bool bf16, int mode, int xkind, int epi, const FcArgs &a, cudaStream_t st) {

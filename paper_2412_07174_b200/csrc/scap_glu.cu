@@ -72,7 +72,9 @@ static scap_status ffn_impl(bool gated, const void *h, const void *Wgu, const vo
     if (idx2_out || nnz2_out) d.bits = reinterpret_cast<uint32_t *>(w + G.bits2);
     // The two stages run back to back: either both take the tcgen05 kernel or neither does (measured: a stage on
     // it between two mma.sync stages loses more at the kernel boundaries than it gains).
-    if (!(tc_applicable(a, epi1, bf16) && tc_applicable(d, EPI_BIAS, bf16))) a.no_tc = d.no_tc = 1;
+    // The dense-stream kernel (batches above the FMA limit) takes both stages whenever it takes one.
+    const bool ds_both = ds_applicable(a, epi1, bf16) && ds_applicable(d, EPI_BIAS, bf16);
+    if (!ds_both && !(tc_applicable(a, epi1, bf16) && tc_applicable(d, EPI_BIAS, bf16))) a.no_tc = d.no_tc = 1;
 
     cudaError_t e = launch_fc(bf16, MODE_GATHER, bf16 ? 1 : 0, epi1, a, st);
     if (e != cudaSuccess) return cuda_status(e);

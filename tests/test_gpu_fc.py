@@ -87,19 +87,21 @@ def test_sparsity_levels(S, s):
 
 # ---------------------------------------------------------------- degenerate cases
 
-# the three forms of the kernel a batch of three can run on: (fma_rows, tcgen05) tune values
-ROUTES = {"fma": (4, 0), "mma_sync": (2, 0), "tcgen05": (2, 2)}
+# the four forms of the kernel a batch of three can run on: (fma_rows, tcgen05, dense_stream) tune values
+ROUTES = {"fma": (4, 0, 0), "mma_sync": (2, 0, 0), "tcgen05": (2, 2, 0), "dense_stream": (2, 0, 2)}
 
 
 def set_route(S, route):
-    rows, tc = ROUTES[route]
+    rows, tc, ds = ROUTES[route]
     S.scap_tune("fma_rows", rows)
     S.scap_tune("tcgen05", tc)
+    S.scap_tune("dense_stream", ds)
 
 
 def reset_route(S):
     S.scap_tune("fma_rows", 4)
     S.scap_tune("tcgen05", 1)
+    S.scap_tune("dense_stream", 1)
 
 
 @pytest.mark.parametrize("route", sorted(ROUTES))
@@ -323,12 +325,14 @@ def test_tcgen05_kernel_matches_the_oracle(S, K, N, B, dt, split):
     d = si.laplace_fc(4, K, N, dt, 16, B)
     try:
         S.scap_tune("tcgen05", 2)
+        S.scap_tune("dense_stream", 0)
         S.scap_tune("split_k", split)
         check_fc(S, d, d["m_true"], 0.25)
         check_fc(S, d, None, 0.4, with_bias=False)
         S.scap_device_status()
     finally:
         S.scap_tune("tcgen05", 1)
+        S.scap_tune("dense_stream", 1)
         S.scap_tune("split_k", 0)
 
 
@@ -403,8 +407,9 @@ def test_parameters_rewritten_on_the_stream_directly_before_the_call(S, B):
 
 # ---------------------------------------------------------------- the bounded waits of the tcgen05 kernel can run out
 
-def test_a_wait_that_runs_out_is_reported_once_and_the_next_call_is_correct(S):
-    """With the poll limit of the tcgen05 kernel's barrier waits set to 1 the waits of the next call give up at once:
+@pytest.mark.parametrize("kernel", ["gather", "dense_stream"])
+def test_a_wait_that_runs_out_is_reported_once_and_the_next_call_is_correct(S, kernel):
+    """With the poll limit of the tcgen05 kernels' barrier waits set to 1 the waits of the next call give up at once:
     the call must still return (every CTA passes its cluster barriers and frees its tensor memory),
     scap_device_status must report the time-out exactly once, and an ordinary call afterwards must pass parity."""
     from paper_2412_07174_b200 import ScapError
@@ -413,7 +418,8 @@ def test_a_wait_that_runs_out_is_reported_once_and_the_next_call_is_correct(S):
     m = d["m_true"]
     tau = oracle.tau(si.to_f32(d["x_calib"], d["dt"]), m, 0.5)
     try:
-        S.scap_tune("tcgen05", 2)      # batch 5 on the tcgen05 kernel
+        S.scap_tune("tcgen05", 2)      # batch 5 on the gather tcgen05 kernel, or on the dense-stream one
+        S.scap_tune("dense_stream", 2 if kernel == "dense_stream" else 0)
         S.scap_device_status()         # clean slate (raises if an earlier test left a record)
         S.scap_tune("tc_spin", 1)
         run_sparse(S, d, m, tau, None, want_idx=False)   # returns; y is incomplete and not looked at
@@ -427,3 +433,28 @@ def test_a_wait_that_runs_out_is_reported_once_and_the_next_call_is_correct(S):
     finally:
         S.scap_tune("tc_spin", 0)
         S.scap_tune("tcgen05", 1)
+        S.scap_tune("dense_stream", 1)
+
+
+# ---------------------------------------------------------------- batch 3..16 on the dense-stream tcgen05 kernel (forced)
+
+@pytest.mark.parametrize("K,N,B,dt,split", [
+    (2048, 512, 8, si.BF16, 0), (2048, 512, 16, si.BF16, 0), (1000, 264, 5, si.BF16, 0), (777, 520, 3, si.F16, 0),
+    (4096, 1032, 12, si.F16, 0), (640, 128, 16, si.BF16, 1), (2500, 256, 7, si.BF16, 3), (11008, 4096, 8, si.BF16, 0),
+    (64, 16, 4, si.BF16, 0), (100, 2048, 9, si.F16, 0),
+])
+def test_dense_stream_kernel_matches_the_oracle(S, K, N, B, dt, split):
+    """Every row of W is streamed with TMA box loads and pruning happens on the activation operand: same results as the
+    gather kernels (kept list bit-exact, y within tolerance), for ragged K (not a multiple of 64), ragged N and all cluster sizes."""
+    d = si.laplace_fc(4, K, N, dt, 32, B)
+    m = d["m_true"]
+    tau = oracle.tau(si.to_f32(d["x_calib"], dt), m, 0.6)
+    try:
+        S.scap_tune("dense_stream", 2)
+        S.scap_tune("split_k", split)
+        check_fc(S, d, m, tau)
+        check_fc(S, d, None, 0.0, with_bias=False)
+        S.scap_device_status()
+    finally:
+        S.scap_tune("dense_stream", 1)
+        S.scap_tune("split_k", 0)

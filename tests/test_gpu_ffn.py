@@ -104,10 +104,25 @@ def test_glu_on_the_tcgen05_kernel(S, D, F, B):
     c = calibrate_glu(g, 0.4, 0.7)
     try:
         S.scap_tune("tcgen05", 2)
+        S.scap_tune("dense_stream", 0)
         check_glu(S, g, c)
         S.scap_device_status()
     finally:
         S.scap_tune("tcgen05", 1)
+        S.scap_tune("dense_stream", 1)
+
+
+@pytest.mark.parametrize("D,F,B", [(520, 1000, 3), (1024, 776, 8), (2048, 520, 16), (200, 264, 5), (4096, 1376, 12)])
+def test_glu_on_the_dense_stream_kernel(S, D, F, B):
+    """Both stages on the TMA dense-stream kernel: packed gate|up boxes in the first, fp32 z as the input of the second."""
+    g = si.glu_block(2, D, F, si.BF16, 64, B)
+    c = calibrate_glu(g, 0.4, 0.7)
+    try:
+        S.scap_tune("dense_stream", 2)
+        check_glu(S, g, c)
+        S.scap_device_status()
+    finally:
+        S.scap_tune("dense_stream", 1)
 
 
 def test_glu_fp16_and_no_centring(S):
@@ -243,9 +258,11 @@ def test_gelu_ffn_small_shapes(S, D, F, B, tc_mode):
     c = calibrate_gelu(g, 0.3, 0.5)
     try:
         S.scap_tune("tcgen05", tc_mode)
+        S.scap_tune("dense_stream", 0 if tc_mode == 2 else 1)   # 2: the gather tcgen05 kernel, 1: the default routes
         kept2 = check_gelu(S, g, c)
     finally:
         S.scap_tune("tcgen05", 1)
+        S.scap_tune("dense_stream", 1)
     assert kept2 < 0.95
 
 
