@@ -30,13 +30,14 @@ __device__ __forceinline__ void widen8(const uint4 &v, float (&f)[8]) {
 // beyond T are skipped (their slots keep zeros and `valid` says how many are real).
 constexpr int CAL_U = 16;  // with 128 rows per sweep: 2048 rows of a strip live in registers at once
 __device__ __forceinline__ int load_rows(const uint16_t *xp, int K, int T, int t0, uint4 (&v)[CAL_U]) {
+    const uint64_t pol = l2_policy_keep();  // the radix passes read the tensor again: it fits in L2, ask for it to stay
     int valid = 0;
 #pragma unroll
     for (int u = 0; u < CAL_U; ++u) {
         const int t = t0 + u * CAL_ROWS;
         v[u] = make_uint4(0, 0, 0, 0);
         if (t < T) {
-            v[u] = __ldg(reinterpret_cast<const uint4 *>(xp + (size_t)t * K));
+            v[u] = ld_keep16(xp + (size_t)t * K, pol);
             valid = u + 1;
         }
     }
@@ -377,13 +378,14 @@ __global__ void __launch_bounds__(256) radix_pass_kernel(const uint16_t *__restr
     if (kc < K) {
         const int step = 8 * gridDim.y;
         const uint16_t *xp = x + kc;
+        const uint64_t pol = l2_policy_keep();
         for (int t0 = blockIdx.y * 8 + ty; t0 < T; t0 += step * RP_U) {
             uint4 v[RP_U];
 #pragma unroll
             for (int u = 0; u < RP_U; ++u) {
                 const int t = t0 + step * u;
                 v[u] = make_uint4(0, 0, 0, 0);
-                if (t < T) v[u] = __ldg(reinterpret_cast<const uint4 *>(xp + (size_t)t * K));
+                if (t < T) v[u] = ld_keep16(xp + (size_t)t * K, pol);
             }
 #pragma unroll
             for (int u = 0; u < RP_U; ++u) {

@@ -283,6 +283,15 @@ __device__ __forceinline__ void st_async_f32(uint32_t remote_addr, float v, uint
 __device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
 __device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
 
+// 16-byte read-only load that asks L2 to keep the line (the calibration tensor is read again by the following passes).
+__device__ __forceinline__ uint4 ld_keep16(const void *p, uint64_t pol) {
+    uint4 v;
+    asm volatile("ld.global.nc.L2::cache_hint.v4.u32 {%0,%1,%2,%3}, [%4], %5;"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p), "l"(pol));
+    return v;
+}
+
 // Hint: bring the line that holds *p into L2 (no register result, no ordering effect).
 __device__ __forceinline__ void prefetch_l2(const void *p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
 
