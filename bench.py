@@ -216,7 +216,7 @@ def _time_graph(torch, stream, fn, reps=30, warm=5):
     return e0.elapsed_time(e1) / reps * 1e3  # us per replay
 
 
-def suite_sweep(torch, scap, peak, shapes, sparsities, batches, out):
+def suite_sweep(torch, scap, peak, shapes, sparsities, batches, out, max_copies=0):
     """Config 4: sparse FC over sparsity x batch x shape, bf16, Laplace-around-mode inputs, vs the dense GEMV."""
     stream = torch.cuda.Stream()
     l2 = torch.cuda.get_device_properties(0).L2_cache_size
@@ -226,6 +226,8 @@ def suite_sweep(torch, scap, peak, shapes, sparsities, batches, out):
         xc = si.as_torch(d["x_calib"], si.BF16).cuda()
         xs = si.as_torch(d["x"], si.BF16).cuda()          # 128 rows = 8 batches of 16
         Rmax = int(np.ceil(4 * l2 / (0.1 * Kk * Nn * 2)))
+        if max_copies > 0:
+            Rmax = min(Rmax, max_copies)   # a profiler capture keeps device memory low
         Ws = [W0] + [W0.clone() for _ in range(Rmax - 1)]
         cws = torch.empty(scap.scap_calibrate_workspace(2048, Kk, NBINS), dtype=torch.uint8, device="cuda")
         m = torch.empty(Kk, dtype=torch.float32, device="cuda")
@@ -235,7 +237,7 @@ def suite_sweep(torch, scap, peak, shapes, sparsities, batches, out):
             ws = torch.empty(scap.scap_fc_workspace(B, Kk, Nn), dtype=torch.uint8, device="cuda")
             y = torch.empty((B, Nn), dtype=torch.float32, device="cuda")
             xb = [xs[i * 16:i * 16 + B] for i in range(8)]
-            Rd = max(2, int(np.ceil(4 * l2 / (Kk * Nn * 2))))
+            Rd = max(2, min(Rmax, int(np.ceil(4 * l2 / (Kk * Nn * 2)))))
             t_dense = _time_graph(torch, stream, lambda: [scap.scap_dense_fc(xb[r % 8], Ws[r], None, y, ws) for r in range(Rd)]) / Rd
             dense_b = Kk * Nn * 2 + B * Kk * 2 + 4 * Nn + 4 * B * Nn
             for s in sparsities:
@@ -639,7 +641,7 @@ def run_suite(args):
     if which in ("sweep", "all", "sweep-small"):
         shapes = [(4096, 4096), (4096, 11008), (11008, 4096), (14336, 4096)]
         if which == "sweep-small":
-            suite_sweep(torch, scap, peak, [(11008, 4096)], (0.0, 0.5, 0.8), (1, 4, 8, 16), out)
+            suite_sweep(torch, scap, peak, [(11008, 4096)], (0.0, 0.5, 0.8), (1, 4, 8, 16), out, args.copies)
         else:
             suite_sweep(torch, scap, peak, shapes, (0.0, 0.25, 0.5, 0.6, 0.7, 0.8, 0.9), (1, 2, 4, 8, 16), out)
     if which in ("moe", "all"):
