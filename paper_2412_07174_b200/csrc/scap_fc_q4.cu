@@ -18,11 +18,11 @@
 
 namespace scap {
 
-constexpr int Q4_TN = 256;   // columns per CTA: a row segment is 128 bytes = 16 lanes x 8 bytes
+constexpr int Q4_TN = 128;   // columns per CTA: a row segment is 64 bytes = 8 lanes x 8 bytes (two CTAs per SM: the unpack arithmetic needs the warps)
 constexpr int Q4_CPT = 16;   // columns per thread (one 8-byte load)
 __host__ __device__ constexpr int q4_unroll(int BT) { return BT <= 1 ? 16 : 8; }  // row loads in flight per thread
 constexpr int Q4_MAXG = 64;  // most groups per fill (2048 channels of 32)
-// list region, overlaid by the reduction buffer of the 16 row groups
+// list region, overlaid by the reduction buffer of the row groups
 __host__ __device__ constexpr int q4_main_bytes(int BT) {
     const int red = (FC_THREADS / (Q4_TN / Q4_CPT)) * fc_rb(BT) * Q4_TN * 4;
     return fc_main_bytes(BT) > red ? fc_main_bytes(BT) : red;
@@ -60,8 +60,8 @@ __global__ void __launch_bounds__(FC_THREADS, 2) fc_q4_kernel(const Q4Args qa) {
     const FcArgs &a = qa.f;
     constexpr int TNT = Q4_TN, EPI = EPI_BIAS, U = q4_unroll(BT);
     constexpr int PU = fc_pu(BT), CAP = fc_cap(BT), RB = fc_rb(BT);
-    constexpr int LPR = TNT / Q4_CPT;      // 16 lanes per row segment
-    constexpr int NR = FC_THREADS / LPR;   // 16 row groups per CTA
+    constexpr int LPR = TNT / Q4_CPT;      // 8 lanes per row segment
+    constexpr int NR = FC_THREADS / LPR;   // 32 row groups per CTA
     static_assert(RB == BT, "one reduction round");
     extern __shared__ __align__(16) unsigned char smem[];
     uint32_t *s_k = reinterpret_cast<uint32_t *>(smem);
@@ -241,7 +241,7 @@ __global__ void __launch_bounds__(FC_THREADS, 2) fc_q4_kernel(const Q4Args qa) {
         __syncthreads();
     }
 
-    // ---- reduction over the 16 row groups (group order), cluster exchange, bias: as in the 16-bit kernel
+    // ---- reduction over the row groups (group order), cluster exchange, bias: as in the 16-bit kernel
     cg::cluster_group cluster = cg::this_cluster();
     float *owner[MAX_CLUSTER];
 #pragma unroll
@@ -263,7 +263,7 @@ __global__ void __launch_bounds__(FC_THREADS, 2) fc_q4_kernel(const Q4Args qa) {
 
 constexpr int q4_smem(int BT) { return q4_main_bytes(BT) + BT * GATHER_LD * 4 + FC_WARPS * 4 + (Q4_MAXG + 1) * 4 + 16; }
 
-// Split-K factor: the most CTAs (tiles of 256 columns x S) that are all resident, with at least one group per rank.
+// Split-K factor: the most CTAs (column tiles x S) that are all resident, with at least one group per rank.
 static int q4_split(int K, int N, int group) {
     const int tiles = (N + Q4_TN - 1) / Q4_TN, G = (K + group - 1) / group;
     int best_S = 1;
