@@ -385,7 +385,7 @@ def suite_overlap(torch, scap, peak, out):
                 groups = [b % n_ctx for b in range(B)]
                 if t_dense is None:
                     Rd = max(2, int(np.ceil(4 * l2 / (Kk * Nn * 2))))
-                    t_dense = _time_graph(torch, stream, lambda: [scap.scap_dense_fc(xb[r % 4], Ws[r], None, y, ws) for r in range(Rd)]) / Rd
+                    t_dense = _time_graph(torch, stream, lambda: [scap.scap_dense_fc(xb[r % 4], Ws[r], None, y, ws) for r in range(Rd)]) / Rd   # dense-stream kernel
                 u_all, u_grp = [], []
                 for i in range(4):
                     scap.scap_sparse_fc(xb[i], W0, m, tau, bf, y, ws, nnz_out=nnz)
@@ -398,10 +398,16 @@ def suite_overlap(torch, scap, peak, out):
                     u_grp.append(tot)
                 rho_all, rho_grp = float(np.mean(u_all)) / Kk, float(np.mean(u_grp)) / Kk
                 R = max(2, min(Rmax, int(np.ceil(4 * l2 / (max(rho_all, 0.4) * Kk * Nn * 2)))))
-                t_one = _time_graph(torch, stream, lambda: [scap.scap_sparse_fc(xb[r % 4], Ws[r], m, tau, bf, y, ws) for r in range(R)]) / R
+                t_stream = _time_graph(torch, stream, lambda: [scap.scap_sparse_fc(xb[r % 4], Ws[r], m, tau, bf, y, ws) for r in range(R)]) / R
+                scap.scap_tune("dense_stream", 0)   # the gather kernels: rows the union drops are not fetched
+                try:
+                    t_one = _time_graph(torch, stream, lambda: [scap.scap_sparse_fc(xb[r % 4], Ws[r], m, tau, bf, y, ws) for r in range(R)]) / R
+                finally:
+                    scap.scap_tune("dense_stream", 1)
                 rec = {"suite": "overlap", "K": Kk, "N": Nn, "B": B, "contexts": n_ctx, "overlap": ov, "sparsity_target": s,
                        "union_kept_fraction_whole_batch": round(rho_all, 4), "sum_of_union_kept_fractions_per_context": round(rho_grp, 4),
-                       "one_union_us": round(t_one, 2), "dense_us": round(t_dense, 2), "one_union_vs_dense": round(t_dense / t_one, 3)}
+                       "one_union_gather_us": round(t_one, 2), "one_union_dense_stream_us": round(t_stream, 2), "dense_us": round(t_dense, 2),
+                       "one_union_gather_vs_dense": round(t_dense / t_one, 3)}
                 if n_ctx > 1:
                     t_grp = _time_graph(torch, stream, lambda: [scap.scap_sparse_fc_grouped(xb[r % 4], Ws[r], m, tau, bf, y, groups, gws) for r in range(R)]) / R
                     rec.update({"grouped_us": round(t_grp, 2), "grouped_vs_one_union": round(t_one / t_grp, 3), "grouped_vs_dense": round(t_dense / t_grp, 3),
