@@ -13,28 +13,48 @@ namespace scap {
 constexpr int Q8_TN = 128;   // columns per CTA
 constexpr int Q8_CPT = 16;   // columns per thread (one 16-byte load)
 
-// 16 signed bytes -> floats.  (byte ^ 0x80) placed in the mantissa of 2^23 reads as 2^23 + (q + 128); subtracting
-// 2^23 + 128 gives q exactly.
-__device__ __forceinline__ void unpack_q8(const uint4 &v, float (&w)[16]) {
-    const uint32_t u[4] = {v.x ^ 0x80808080u, v.y ^ 0x80808080u, v.z ^ 0x80808080u, v.w ^ 0x80808080u};
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        w[4 * i + 0] = __uint_as_float(__byte_perm(u[i], 0x4B000000u, 0x7650)) - 8388736.0f;
-        w[4 * i + 1] = __uint_as_float(__byte_perm(u[i], 0x4B000000u, 0x7651)) - 8388736.0f;
-        w[4 * i + 2] = __uint_as_float(__byte_perm(u[i], 0x4B000000u, 0x7652)) - 8388736.0f;
-        w[4 * i + 3] = __uint_as_float(__byte_perm(u[i], 0x4B000000u, 0x7653)) - 8388736.0f;
-    }
+// Two fp32 values in one 64-bit register, for the packed fp32 instructions of sm_100 (add.f32x2 / fma.rn.f32x2: one
+// instruction per two weights; the unpack is bound by instruction issue, so this is worth a third of its time).
+__device__ __forceinline__ unsigned long long pack2(float lo, float hi) {
+    unsigned long long r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(__float_as_uint(lo)), "r"(__float_as_uint(hi)));
+    return r;
+}
+__device__ __forceinline__ unsigned long long add2(unsigned long long a, unsigned long long b) {
+    unsigned long long r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ unsigned long long fma2(unsigned long long a, unsigned long long b, unsigned long long c) {
+    unsigned long long r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+__device__ __forceinline__ void unpack2(unsigned long long v, float &lo, float &hi) {
+    uint32_t a, b;
+    asm("mov.b64 {%0, %1}, %2;" : "=r"(a), "=r"(b) : "l"(v));
+    lo = __uint_as_float(a);
+    hi = __uint_as_float(b);
 }
 
+// acc[b][j] (pairs of columns) += xv * q for the 16 signed bytes of v.  (byte ^ 0x80) placed in the mantissa of 2^23 reads
+// as 2^23 + (q + 128); adding -(2^23 + 128) gives q exactly; both steps and the multiply-add run two columns at a time.
 template <int BT, int CAP>
-__device__ __forceinline__ void fma_row_q8(float (&acc)[BT][16], const uint4 &v, const float *__restrict__ s_xs, int i) {
-    float w[16];
-    unpack_q8(v, w);
+__device__ __forceinline__ void fma_row_q8(unsigned long long (&acc)[BT][8], const uint4 &v, const float *__restrict__ s_xs, int i) {
+    const uint32_t u[4] = {v.x ^ 0x80808080u, v.y ^ 0x80808080u, v.z ^ 0x80808080u, v.w ^ 0x80808080u};
+    const unsigned long long neg = pack2(-8388736.0f, -8388736.0f);
+    unsigned long long w[8];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        w[2 * q] = add2(pack2(__uint_as_float(__byte_perm(u[q], 0x4B000000u, 0x7650)), __uint_as_float(__byte_perm(u[q], 0x4B000000u, 0x7651))), neg);
+        w[2 * q + 1] = add2(pack2(__uint_as_float(__byte_perm(u[q], 0x4B000000u, 0x7652)), __uint_as_float(__byte_perm(u[q], 0x4B000000u, 0x7653))), neg);
+    }
 #pragma unroll
     for (int b = 0; b < BT; ++b) {
         const float xv = s_xs[b * CAP + i];
+        const unsigned long long x2 = pack2(xv, xv);
 #pragma unroll
-        for (int j = 0; j < 16; ++j) acc[b][j] = fmaf(xv, w[j], acc[b][j]);
+        for (int j = 0; j < 8; ++j) acc[b][j] = fma2(x2, w[j], acc[b][j]);
     }
 }
 
@@ -67,11 +87,11 @@ __global__ void __launch_bounds__(FC_THREADS, 2) fc_q8_kernel(const FcArgs a) {
     const int per = (TNT + S - 1) / S;
     float bias0[2], bias1[2];
 
-    float acc[BT][16];
+    unsigned long long acc2[BT][8];  // 16 columns per batch row as 8 packed pairs
 #pragma unroll
     for (int b = 0; b < BT; ++b)
 #pragma unroll
-        for (int j = 0; j < 16; ++j) acc[b][j] = 0.0f;
+        for (int j = 0; j < 8; ++j) acc2[b][j] = 0ull;
 
     const int nchunks = (K + 31) >> 5;
     const int my_chunks = nchunks > s ? (nchunks - s + S - 1) / S : 0;
@@ -179,13 +199,13 @@ __global__ void __launch_bounds__(FC_THREADS, 2) fc_q8_kernel(const FcArgs a) {
             for (int t0 = 0; t0 < nrows; t0 += 2 * G) {
 #pragma unroll
                 for (int u = 0; u < G; ++u)
-                    if (t0 + u < nrows) fma_row_q8<BT, CAP>(acc, ga[u], s_xs, rg + NR * (t0 + u));
+                    if (t0 + u < nrows) fma_row_q8<BT, CAP>(acc2, ga[u], s_xs, rg + NR * (t0 + u));
 #pragma unroll
                 for (int u = 0; u < G; ++u)
                     if (t0 + 2 * G + u < nrows) ga[u] = ld_stream16(Wb + (size_t)s_k[rg + NR * (t0 + 2 * G + u)] * row_bytes);
 #pragma unroll
                 for (int u = 0; u < G; ++u)
-                    if (t0 + G + u < nrows) fma_row_q8<BT, CAP>(acc, gb[u], s_xs, rg + NR * (t0 + G + u));
+                    if (t0 + G + u < nrows) fma_row_q8<BT, CAP>(acc2, gb[u], s_xs, rg + NR * (t0 + G + u));
 #pragma unroll
                 for (int u = 0; u < G; ++u)
                     if (t0 + 3 * G + u < nrows) gb[u] = ld_stream16(Wb + (size_t)s_k[rg + NR * (t0 + 3 * G + u)] * row_bytes);
@@ -194,6 +214,11 @@ __global__ void __launch_bounds__(FC_THREADS, 2) fc_q8_kernel(const FcArgs a) {
         __syncthreads();
     }
 
+    float acc[BT][16];
+#pragma unroll
+    for (int b = 0; b < BT; ++b)
+#pragma unroll
+        for (int j = 0; j < 8; ++j) unpack2(acc2[b][j], acc[b][2 * j], acc[b][2 * j + 1]);
     // the four row groups of a warp (lanes l, l ^ 8, l ^ 16, l ^ 24 hold the same columns) are added by shuffles
     // in a fixed order; lanes 0-7 then hold the warp's partial of its 128 columns
 #pragma unroll
