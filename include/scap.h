@@ -30,12 +30,16 @@
  *     SCAP_ERR_CUDA, a device that is not compute capability 10.x SCAP_ERR_UNSUPPORTED_ARCH.
  *     Nothing throws, aborts, traps or prints.  On error nothing has been enqueued.
  *   - Workspace contents are scratch: undefined on entry, undefined on exit.
- *   - Every kernel of a call waits for the work placed before it on the stream before it reads anything - the
- *     activations, and equally W, m, tau, the scales and the biases - and reads whatever a kernel may have
- *     rewritten through L2.  So parameters may be produced on the same stream directly before the call that
- *     uses them (scap_calibrate, scap_fold_bias, or any kernel or copy of the caller's), with no further
- *     synchronisation.  Consecutive calls still overlap where they can: a kernel may become resident and set up
- *     its shared memory while its predecessor drains (programmatic dependent launch, "pdl" below).
+ *   - Every kernel of a call waits for the work placed before it on the stream before it reads the activations,
+ *     m, tau, the scales, the biases or a row map, and reads whatever a kernel may have rewritten through L2.  So
+ *     these may be produced on the same stream directly before the call that uses them (scap_calibrate,
+ *     scap_fold_bias, or any kernel or copy of the caller's), with no further synchronisation.  The weight matrix W
+ *     is the exception: it is a constant of the layer and must be complete in device memory when the call is
+ *     ISSUED (not written by work still pending on the stream), because the batch 5..16 kernel requests its first
+ *     weight blocks before that wait - their addresses do not depend on the activations - so that the memory
+ *     system does not idle between consecutive calls.  Consecutive calls overlap where they can: a kernel may
+ *     become resident and set up its shared memory while its predecessor drains (programmatic dependent launch,
+ *     "pdl" below).
  */
 #ifndef SCAP_H_
 #define SCAP_H_

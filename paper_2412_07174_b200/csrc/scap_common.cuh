@@ -196,6 +196,17 @@ __device__ __forceinline__ uint4 ld_act16_if(const void *p, bool on) {
     return v;
 }
 
+__device__ __forceinline__ uint4 ld_act16_if(const void *p, bool on, uint64_t pol) {
+    uint4 v;
+    asm volatile(
+        "{ .reg .pred q; setp.ne.u32 q, %5, 0; mov.u32 %0, 0; mov.u32 %1, 0; mov.u32 %2, 0; mov.u32 %3, 0;"
+        " @q ld.global.cg.L2::cache_hint.v4.u32 {%0,%1,%2,%3}, [%4], %6; }"
+        : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+        : "l"(p), "r"((unsigned)on), "l"(pol)
+        : "memory");
+    return v;
+}
+
 // L2 eviction policies for loads that carry a cache hint.  keep: small data every column tile of a call reads again
 // (activations, modes); stream: weight rows, read once.
 __device__ __forceinline__ uint64_t l2_policy_keep() {
@@ -281,6 +292,9 @@ __device__ __forceinline__ void st_async_f32(uint32_t remote_addr, float v, uint
 }
 // Split cluster barrier: arrive early, wait where the guarantee is needed.
 __device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
+// Arrival without memory ordering of its own: enough after mbarrier_init, whose fence publishes the barriers, and it
+// does not wait for loads that are under way.
+__device__ __forceinline__ void cluster_arrive_relaxed() { asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory"); }
 __device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
 
 // 16-byte read-only load that asks L2 to keep the line (the calibration tensor is read again by the following passes).
@@ -294,5 +308,7 @@ __device__ __forceinline__ uint4 ld_keep16(const void *p, uint64_t pol) {
 
 // Hint: bring the line that holds *p into L2 (no register result, no ordering effect).
 __device__ __forceinline__ void prefetch_l2(const void *p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
+// The same, and L2 is asked to keep the line (small data that many CTAs and later calls read again).
+__device__ __forceinline__ void prefetch_l2_keep(const void *p) { asm volatile("prefetch.global.L2::evict_last [%0];" ::"l"(p)); }
 
 }  // namespace scap

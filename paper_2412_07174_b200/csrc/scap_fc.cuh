@@ -271,14 +271,16 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
     const int per = ((EPI == EPI_GLU ? HALF : TNT) + S - 1) / S;  // the last rank may own fewer
     if (S > 1) {
         // This rank will receive S * B * (columns it owns) partial sums (gate and up: twice that) on its barrier.
-        // The arrival half of a cluster barrier publishes the initialised barrier; the waiting half sits before the
-        // first send, by which time every rank has long arrived.
+        // The fence after the initialisation publishes the barrier; the arrival half of a cluster barrier follows (with
+        // no ordering of its own, so it waits for nothing: the releasing form took 0.3 - 0.8 us, measured, on the
+        // critical path of a CTA that became resident late) and the waiting half sits before the first send, by which
+        // time every rank has long arrived.
         if (tid == 0) {
             const int owned = max(0, min(per, (EPI == EPI_GLU ? HALF : TNT) - s * per));
             mbarrier_init(bar, 1);
             mbarrier_arrive_expect(bar, (uint32_t)(S * B * owned * (EPI == EPI_GLU ? 8 : 4)));
         }
-        cluster_arrive();
+        cluster_arrive_relaxed();
     }
     float bias0[2], bias1[2];
 

@@ -475,6 +475,7 @@ struct DsMisc {
     unsigned long long afull[DS_NST];   // both chunks of the stage's A operand are written
     unsigned long long empty[DS_NST];   // the stage's MMAs have read W and A
     unsigned long long done;
+    unsigned long long recv;            // split-K partials of this rank's columns have landed
     uint32_t tmem_base;
     int abort;
     int issued;
@@ -514,6 +515,8 @@ __global__ void __launch_bounds__(FC_THREADS, 2) fc_ds_kernel(const FcArgs a, co
     const int nblk64 = (K + 63) >> 6;
     const int nq = nblk64 > s ? (nblk64 - s + S - 1) / S : 0;  // 64-row blocks (= stages) of this rank
 
+    const int per = ((EPI == EPI_GLU ? HALF : TNT) + S - 1) / S;   // columns (gate/up pairs) a rank finishes
+    const uint32_t recv_bar = smem_addr(&misc->recv);
     if (tid == 0) {
         for (int i = 0; i < DS_NST; ++i) {
             mbar_init(&misc->wfull[i], 1);
@@ -524,21 +527,68 @@ __global__ void __launch_bounds__(FC_THREADS, 2) fc_ds_kernel(const FcArgs a, co
         misc->abort = 0;
         misc->issued = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        if (S > 1) {
+            // S B (columns this rank finishes) partial sums (gate and up: twice that) will land on the receive barrier
+            const int owned = max(0, min(per, (EPI == EPI_GLU ? HALF : TNT) - s * per));
+            mbarrier_init(recv_bar, 1);
+            mbarrier_arrive_expect(recv_bar, (uint32_t)(S * B * owned * (EPI == EPI_GLU ? 8 : 4)));
+        }
+    }
+    // The arrival half of a cluster barrier (the fence after the initialisation publishes the receive barrier; the
+    // arrival itself carries no ordering and so does not wait for anything); the waiting half sits before the first
+    // send, long after every rank has arrived.
+    if (S > 1) cluster_arrive_relaxed();
+    // The first ring of weight blocks is requested at once, by the thread that initialised the barriers and BEFORE the
+    // wait for earlier work on the stream: the weights are constants of the layer (the interface requires them to be
+    // complete when the call is issued), their addresses do not depend on the activations, and so the stream of this
+    // call starts while the previous call is still finishing its columns - the memory system does not idle between
+    // calls.  Everything else (x, m, tau, biases, row maps) is read after the wait.
+    const int x0 = EPI == EPI_GLU ? tile * HALF : tile * TNT;
+    const int x1 = EPI == EPI_GLU ? a.Nh + tile * HALF : tile * TNT + HALF;
+    const int nq_first = nq < DS_NST ? nq : DS_NST;
+    if (tid == 0) {
+        for (int q = 0; q < nq_first; ++q) {
+            mbar_arrive_expect_tx(&misc->wfull[q], DS_STAGE_W);
+            const uint32_t dst = smem_u32(s_w) + q * DS_STAGE_W;
+            tma_box_2d(dst, &tmap, x0, (q * S + s) * 64, &misc->wfull[q]);
+            tma_box_2d(dst + DS_STAGE_W / 2, &tmap, x1, (q * S + s) * 64, &misc->wfull[q]);
+        }
     }
     if (warp == 0) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&misc->tmem_base)), "r"(TNT) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-    const int per = ((EPI == EPI_GLU ? HALF : TNT) + S - 1) / S;
     float bias0[2], bias1[2];
 
-    griddep_wait();  // nothing is read before earlier work on the stream is complete
+    griddep_wait();  // x, m, tau, the biases and the row maps may be outputs of the work just before this call
     griddep_launch_dependents();
+    // x and m are read again by every column tile of the call (and m by every later call): ask L2 to keep them.
+    const uint64_t pol_keep = a.l2_hints ? l2_policy_keep() : l2_policy_normal();
+    // This rank's share of m and x is asked into L2 now, ahead of the weight stream: a request that misses L2 later
+    // queues behind megabytes of weight reads (measured: 1.8 us, which made the operand warps the limit of the stream).
+    // One line per thread and turn; every tile of the call asks for the same lines, L2 merges them.
+    if (warp >= 2) {
+        const int t = tid - 64;
+        if (MODE == MODE_GATHER && a.m) {
+            for (int i = t; i < 2 * nq; i += FC_THREADS - 64) {
+                const int k = ((i >> 1) * S + s) * 64 + (i & 1) * 32;
+                if (k < K) prefetch_l2_keep(a.m + k);
+            }
+        }
+        if (!a.in_rows) {  // (with a row map the rows are not known yet)
+            constexpr int XL = (64 * (int)sizeof(XT) + 127) / 128;  // lines per row and block
+            for (int i = t; i < nq * B * XL; i += FC_THREADS - 64) {
+                const int l = i % XL, rb = i / XL, b = rb % B, q = rb / B;
+                const int k = (q * S + s) * 64 + l * (128 / (int)sizeof(XT));
+                if (k < K) prefetch_l2_keep(xg + (size_t)b * a.x_ld + k);
+            }
+        }
+    }
+    // Only the thresholding warps need tau; each of their lanes asks for it here and first uses it after its first
+    // activations have arrived, so the two round trips to L2 overlap.
     float tau = 0.0f;
     if constexpr (MODE == MODE_GATHER) {
-        float tv = 0.0f;
-        if (lane == 0) tv = ld_act(a.tau);
-        tau = __shfl_sync(0xffffffffu, tv, 0);
+        if (warp >= 2) tau = ld_act(a.tau);
     }
     prefetch_bias<BF16, EPI, TNT>(a, tile, s, per, bias0, bias1);
     if (a.in_rows && tid < 16) misc->rows[tid] = __ldcg(a.in_rows + (tid < B ? tid : 0));
@@ -552,9 +602,7 @@ __global__ void __launch_bounds__(FC_THREADS, 2) fc_ds_kernel(const FcArgs a, co
     if (warp == 0) {
         // ---- TMA producer: two boxes per stage
         if (lane == 0) {
-            const int x0 = EPI == EPI_GLU ? tile * HALF : tile * TNT;
-            const int x1 = EPI == EPI_GLU ? a.Nh + tile * HALF : tile * TNT + HALF;
-            int q = 0;
+            int q = nq_first;  // the first ring went out above
             for (; q < nq; ++q) {
                 const uint32_t st = (uint32_t)q % DS_NST;
                 if (!mbar_wait(&misc->empty[st], (((uint32_t)q / DS_NST) & 1u) ^ 1u, 1, abort_flag, spin)) break;
@@ -616,7 +664,7 @@ __global__ void __launch_bounds__(FC_THREADS, 2) fc_ds_kernel(const FcArgs a, co
 #pragma unroll
                 for (int v = 0; v < XV; ++v) {
                     const int kk = k0 + v * (16 / (int)sizeof(XT));
-                    raw[v] = ld_act16_if(reinterpret_cast<const unsigned char *>(xg + (size_t)xrow * a.x_ld + kk), b < B && kk < K);
+                    raw[v] = ld_act16_if(reinterpret_cast<const unsigned char *>(xg + (size_t)xrow * a.x_ld + kk), b < B && kk < K, pol_keep);
                 }
                 const XT *xe = reinterpret_cast<const XT *>(raw);
 #pragma unroll
@@ -629,7 +677,7 @@ __global__ void __launch_bounds__(FC_THREADS, 2) fc_ds_kernel(const FcArgs a, co
 #pragma unroll
                 for (int v = 0; v < CPL / 4; ++v) {
                     uint4 r4 = make_uint4(0, 0, 0, 0);
-                    if (MODE == MODE_GATHER && a.m) r4 = ld_act16_if(reinterpret_cast<const unsigned char *>(a.m + k0 + 4 * v), b < B && k0 + 4 * v < K);
+                    if (MODE == MODE_GATHER && a.m) r4 = ld_act16_if(reinterpret_cast<const unsigned char *>(a.m + k0 + 4 * v), b < B && k0 + 4 * v < K, pol_keep);
                     mv[4 * v] = __uint_as_float(r4.x); mv[4 * v + 1] = __uint_as_float(r4.y);
                     mv[4 * v + 2] = __uint_as_float(r4.z); mv[4 * v + 3] = __uint_as_float(r4.w);
                 }
@@ -686,9 +734,12 @@ __global__ void __launch_bounds__(FC_THREADS, 2) fc_ds_kernel(const FcArgs a, co
         mbar_wait(&misc->done, 0, 4, &drain_abort, TC_SPIN);
     }
     const bool have_acc = nq > 0 && !*abort_flag;
-    if (have_acc && warp * 32 < racc && warp < 2) {
+    // Accumulator rows (part p of batch row b = row p B + b = TMEM lane) to shared memory.  A warp reaches the 32 lanes
+    // of its quarter (warp mod 4), so warps 0 and 4 share lanes 0-31 and warps 1 and 5 lanes 32-63, half the columns each.
+    if (have_acc && (warp & 3) * 32 < racc && (warp & 3) < 2) {
+        const int lq = warp & 3;
 #pragma unroll 1
-        for (int c0 = 0; c0 < TNT; c0 += 32) {
+        for (int c0 = (warp >> 2) * 64; c0 < (warp >> 2) * 64 + 64; c0 += 32) {
             uint32_t v[32];
             asm volatile(
                 "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
@@ -697,9 +748,9 @@ __global__ void __launch_bounds__(FC_THREADS, 2) fc_ds_kernel(const FcArgs a, co
                   "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
                   "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
                   "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
-                : "r"(tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0));
+                : "r"(tmem + ((uint32_t)(lq * 32) << 16) + (uint32_t)c0));
             asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-            const int r = warp * 32 + lane;
+            const int r = lq * 32 + lane;
             if (r < racc) {
 #pragma unroll
                 for (int j = 0; j < 32; ++j) s_part[r * TC_PART_LD + c0 + j] = __uint_as_float(v[j]);
@@ -710,53 +761,40 @@ __global__ void __launch_bounds__(FC_THREADS, 2) fc_ds_kernel(const FcArgs a, co
     __syncthreads();
     tc_fence_after();
     if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TNT) : "memory");
+    // ---- cluster exchange, push form: the parts of an element are added (smallest first) and the sum goes straight to
+    // the cluster rank that finishes its column - slot (this rank, row) of that rank's gather buffer - as an asynchronous
+    // store that counts down the owner's barrier.  No cluster-wide barrier after the prologue: a rank finishes its columns
+    // as soon as its own S partials are in, and may leave while its stores to the others are still under way.
+    if (S > 1) cluster_wait();  // every rank's barrier is initialised (all ranks arrived before their streams)
     for (int i = tid; i < 16 * TNT; i += FC_THREADS) {
         const int b = i / TNT, c = i - b * TNT;
-        float v = 0.0f;
-        if (have_acc && b < B) {
+        if (b < B) {
+            float v = 0.0f;
+            if (have_acc) {
 #pragma unroll
-            for (int p = NSPLIT - 1; p >= 0; --p) v += s_part[(p * B + b) * TC_PART_LD + c];
-        }
-        s_gather[i] = v;
-    }
-    // ---- cluster exchange, pull form, and the bias / SwiGLU epilogue (as in the gather kernel)
-    cg::cluster_group cluster = cg::this_cluster();
-    if (S > 1) cluster.sync();
-    else __syncthreads();
-    const float *peer[MAX_CLUSTER];
-#pragma unroll
-    for (int q = 0; q < MAX_CLUSTER; ++q) peer[q] = (S > 1 && q < S) ? cluster.map_shared_rank(s_gather, q) : s_gather;
-    for (int it = 0; tid + it * FC_THREADS < per * B; ++it) {
-        const int i = tid + it * FC_THREADS;
-        const int b = i / per, c = i - b * per;
-        const int row = a.out_rows ? __ldcg(a.out_rows + b) : b;
-        if constexpr (EPI == EPI_BIAS) {
-            const int n = tile * TNT + s * per + c;
-            if (s * per + c < TNT && n < a.Nh) {
-                float v = it == 0 ? bias0[0] : it == 1 ? bias0[1] : load_bias<BF16>(a, n);
-#pragma unroll
-                for (int q = 0; q < MAX_CLUSTER; ++q)
-                    if (q < S) v += peer[q][b * TNT + s * per + c];
-                store_result(a, row, b, n, v);
+                for (int p = NSPLIT - 1; p >= 0; --p) v += s_part[(p * B + b) * TC_PART_LD + c];
             }
-        } else {
-            const int F = a.Nh, f = tile * HALF + s * per + c;
-            if (s * per + c < HALF && f < F) {
-                float gt = it == 0 ? bias0[0] : it == 1 ? bias0[1] : (a.bias ? __ldcg(a.bias + f) : 0.0f);
-                float up = it == 0 ? bias1[0] : it == 1 ? bias1[1] : (a.bias ? __ldcg(a.bias + F + f) : 0.0f);
-#pragma unroll
-                for (int q = 0; q < MAX_CLUSTER; ++q)
-                    if (q < S) {
-                        gt += peer[q][b * TNT + s * per + c];
-                        up += peer[q][b * TNT + HALF + s * per + c];
-                    }
-                const float z = up * (gt / (1.0f + expf(-gt)));  // up * silu(gate)
-                a.y[(size_t)row * a.y_ld + f] = z;
-                if (a.z_copy) a.z_copy[(size_t)b * F + f] = z;
+            int r, slot;
+            if constexpr (EPI == EPI_GLU) {
+                const int j = c % HALF, hf = c / HALF;
+                r = j / per;
+                slot = ((s * 16 + b) * 2 + hf) * per + (j - r * per);
+            } else {
+                r = c / per;
+                slot = (s * 16 + b) * per + (c - r * per);
             }
+            if (S > 1) st_async_f32(cluster_addr(smem_addr(s_gather) + 4u * (uint32_t)slot, (uint32_t)r), v, cluster_addr(recv_bar, (uint32_t)r));
+            else s_gather[slot] = v;
         }
     }
-    if (S > 1) cluster.sync();
+    if (S > 1) {
+        bool landed = false;
+        for (uint32_t it = 0; it < (1u << 22) && !landed; ++it) landed = mbarrier_try_wait(recv_bar, 0);
+        if (!landed) atomicCAS(&g_tc_status, 0, 6);  // never in a correct run; the result is then incomplete
+    } else {
+        __syncthreads();
+    }
+    finish_columns<BF16, 16, EPI, TNT>(a, tile, s, per, s_gather, bias0, bias1);
 }
 
 // ---- host side ------------------------------------------------------------------------------------------------
