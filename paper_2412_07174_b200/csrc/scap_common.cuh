@@ -24,6 +24,7 @@ struct Tuning {
     int l2_hints;     // batch 1..4 FC kernel: L2 eviction hints (keep activations and modes, stream weights)
     int tile;         // columns per CTA of the FC kernel: 0 = automatic, else 128 or 256
     int tc_spin;      // tcgen05 kernel: polls before a barrier wait gives up (0 = the built-in limit)
+    int head_rows;    // batch 1..4 FC kernel: 32-channel chunks per CTA whose weight rows are asked into L2 before the kept set is known
     int dense_stream; // batch 5..16: 1 = the dense-stream tcgen05 kernel (TMA box loads of all rows), 0 = the gather kernels, 2 = from batch 3
 };
 extern Tuning g_tune;

@@ -8,7 +8,7 @@
 
 namespace scap {
 
-Tuning g_tune = {0, 1, 1, 1, 4, 16, 1, 0, 0, 1};
+Tuning g_tune = {0, 1, 1, 1, 4, 16, 1, 0, 0, 0, 1};
 
 scap_status check_device() {
     static std::atomic<int> cached[64];  // 0 unknown, 1 ok, 2 unsupported
@@ -180,6 +180,9 @@ cudaError_t launch_fc(bool bf16, int mode, int xkind, int epi, const FcArgs &a, 
     }
     FcArgs f = a;
     f.l2_hints = g_tune.l2_hints;
+    // A dense call needs every row, so the head of its stream is always asked for early (nothing is wasted); a sparse
+    // call only on request (tune key "head_rows"): what it asks for and then prunes is extra traffic.
+    f.head_rows = g_tune.head_rows > 0 ? g_tune.head_rows : (mode == MODE_DENSE ? 4 : 0);
     f.status = tc_status_ptr();
     return bf16 ? launch_fc_w<true>(mode, xkind, epi, f, st) : launch_fc_w<false>(mode, xkind, epi, f, st);
 }
@@ -329,6 +332,11 @@ scap_status scap_tune(const char *key, int value) {
     }
     if (!strcmp(key, "l2_hints")) {
         g_tune.l2_hints = value != 0;
+        return SCAP_OK;
+    }
+    if (!strcmp(key, "head_rows")) {
+        if (value < 0 || value > 64) return SCAP_ERR_INVALID_ARG;
+        g_tune.head_rows = value;
         return SCAP_OK;
     }
     if (!strcmp(key, "tile")) {

@@ -67,6 +67,7 @@ struct FcArgs {
     int no_tc;            // 1: keep this call off the tcgen05 kernel
     int act;              // EPI_BIAS: 1 = the exact GELU is applied to the biased result (z_copy then gets a copy)
     const float *wscale;  // 8-bit weights only: one scale per input channel, W[k,n] = wscale[k] * Wq[k,n]
+    int head_rows;        // fp32-FMA body: chunks per CTA whose rows are asked into L2 at kernel start (0: none)
     int l2_hints;         // fp32-FMA body: 1 = loads carry L2 eviction hints (keep x and m, stream W)
     int *status;          // device status word: set when a bounded wait runs out (NULL: not recorded)
     int spin;             // tcgen05 kernel: polls before a shared-memory barrier wait gives up (0: the built-in limit)
@@ -266,6 +267,20 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
     }
     const unsigned char *Wb = reinterpret_cast<const unsigned char *>(a.W) + (size_t)col * 2;
     const size_t row_bytes = (size_t)a.ldw * 2;
+
+    // Head of the stream, asked into L2 before anything is known about the activations: between the end of the
+    // previous call and the first row request of this one (hand-over, activations and parameters through L2, compaction:
+    // about 2 us) the memory system would otherwise idle.  The rows of the rank's first head_rows chunks are requested
+    // as L2 hints - all of them, kept or not, so the part that is pruned is extra traffic, bought with idle time -
+    // and the row requests proper then meet them in L2.  The weights are constants of the layer, so this precedes
+    // the wait for earlier work on the stream.  One 128-byte line per hint: the lanes that start a line issue them.
+    if (a.head_rows > 0 && col_ok && (cl & 7) == 0) {
+        const int nhead = min(a.head_rows, (((K + 31) >> 5) - s + S - 1) / S) * 32;
+        for (int t = rg; t < nhead; t += NR) {
+            const int k = (s + S * (t >> 5)) * 32 + (t & 31);
+            if (k < K) prefetch_l2(Wb + (size_t)k * row_bytes);
+        }
+    }
 
     // columns (EPI_GLU: gate/up pairs) this rank finishes after the cluster exchange
     const int per = ((EPI == EPI_GLU ? HALF : TNT) + S - 1) / S;  // the last rank may own fewer

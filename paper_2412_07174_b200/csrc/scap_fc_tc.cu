@@ -538,6 +538,29 @@ __global__ void __launch_bounds__(FC_THREADS, 2) fc_ds_kernel(const FcArgs a, co
     // arrival itself carries no ordering and so does not wait for anything); the waiting half sits before the first
     // send, long after every rank has arrived.
     if (S > 1) cluster_arrive_relaxed();
+    // This rank's share of m and x is asked into L2 first of all, ahead of the weight stream: a request that misses L2
+    // later queues behind megabytes of weight reads (measured: 1.8 - 2.8 us, which made the operand warps the limit of
+    // the stream and of its start).  These are hints without a result: L2 is the point of coherence, so a line that
+    // earlier work on the stream rewrites after the hint is rewritten there, and the loads proper - after the wait,
+    // through L2 - see the final contents.  One line per thread and turn; every tile of the call asks for the same
+    // lines, L2 merges them.
+    if (warp >= 2) {
+        const int t = tid - 64;
+        if (MODE == MODE_GATHER && a.m) {
+            for (int i = t; i < 2 * nq; i += FC_THREADS - 64) {
+                const int k = ((i >> 1) * S + s) * 64 + (i & 1) * 32;
+                if (k < K) prefetch_l2_keep(a.m + k);
+            }
+        }
+        if (!a.in_rows) {  // (with a row map the rows are not known yet)
+            constexpr int XL = (64 * (int)sizeof(XT) + 127) / 128;  // lines per row and block
+            for (int i = t; i < nq * B * XL; i += FC_THREADS - 64) {
+                const int l = i % XL, rb = i / XL, b = rb % B, q = rb / B;
+                const int k = (q * S + s) * 64 + l * (128 / (int)sizeof(XT));
+                if (k < K) prefetch_l2_keep(xg + (size_t)b * a.x_ld + k);
+            }
+        }
+    }
     // The first ring of weight blocks is requested at once, by the thread that initialised the barriers and BEFORE the
     // wait for earlier work on the stream: the weights are constants of the layer (the interface requires them to be
     // complete when the call is issued), their addresses do not depend on the activations, and so the stream of this
@@ -564,26 +587,6 @@ __global__ void __launch_bounds__(FC_THREADS, 2) fc_ds_kernel(const FcArgs a, co
     griddep_launch_dependents();
     // x and m are read again by every column tile of the call (and m by every later call): ask L2 to keep them.
     const uint64_t pol_keep = a.l2_hints ? l2_policy_keep() : l2_policy_normal();
-    // This rank's share of m and x is asked into L2 now, ahead of the weight stream: a request that misses L2 later
-    // queues behind megabytes of weight reads (measured: 1.8 us, which made the operand warps the limit of the stream).
-    // One line per thread and turn; every tile of the call asks for the same lines, L2 merges them.
-    if (warp >= 2) {
-        const int t = tid - 64;
-        if (MODE == MODE_GATHER && a.m) {
-            for (int i = t; i < 2 * nq; i += FC_THREADS - 64) {
-                const int k = ((i >> 1) * S + s) * 64 + (i & 1) * 32;
-                if (k < K) prefetch_l2_keep(a.m + k);
-            }
-        }
-        if (!a.in_rows) {  // (with a row map the rows are not known yet)
-            constexpr int XL = (64 * (int)sizeof(XT) + 127) / 128;  // lines per row and block
-            for (int i = t; i < nq * B * XL; i += FC_THREADS - 64) {
-                const int l = i % XL, rb = i / XL, b = rb % B, q = rb / B;
-                const int k = (q * S + s) * 64 + l * (128 / (int)sizeof(XT));
-                if (k < K) prefetch_l2_keep(xg + (size_t)b * a.x_ld + k);
-            }
-        }
-    }
     // Only the thresholding warps need tau; each of their lanes asks for it here and first uses it after its first
     // activations have arrived, so the two round trips to L2 overlap.
     float tau = 0.0f;
@@ -766,25 +769,31 @@ __global__ void __launch_bounds__(FC_THREADS, 2) fc_ds_kernel(const FcArgs a, co
     // store that counts down the owner's barrier.  No cluster-wide barrier after the prologue: a rank finishes its columns
     // as soon as its own S partials are in, and may leave while its stores to the others are still under way.
     if (S > 1) cluster_wait();  // every rank's barrier is initialised (all ranks arrived before their streams)
-    for (int i = tid; i < 16 * TNT; i += FC_THREADS) {
-        const int b = i / TNT, c = i - b * TNT;
-        if (b < B) {
+    {
+        // A thread keeps one column and walks the rows (two row phases per CTA), so owner, slot and the owner's
+        // addresses are computed once.
+        const int c = tid % TNT;
+        int r, slot0, bstride;
+        if constexpr (EPI == EPI_GLU) {
+            const int j = c % HALF, hf = c / HALF;
+            r = j / per;
+            slot0 = (s * 16 * 2 + hf) * per + (j - r * per);
+            bstride = 2 * per;
+        } else {
+            r = c / per;
+            slot0 = s * 16 * per + (c - r * per);
+            bstride = per;
+        }
+        const uint32_t dst0 = S > 1 ? cluster_addr(smem_addr(s_gather) + 4u * (uint32_t)slot0, (uint32_t)r) : 0u;
+        const uint32_t dbar = S > 1 ? cluster_addr(recv_bar, (uint32_t)r) : 0u;
+        for (int b = tid / TNT; b < B; b += FC_THREADS / TNT) {
             float v = 0.0f;
             if (have_acc) {
 #pragma unroll
                 for (int p = NSPLIT - 1; p >= 0; --p) v += s_part[(p * B + b) * TC_PART_LD + c];
             }
-            int r, slot;
-            if constexpr (EPI == EPI_GLU) {
-                const int j = c % HALF, hf = c / HALF;
-                r = j / per;
-                slot = ((s * 16 + b) * 2 + hf) * per + (j - r * per);
-            } else {
-                r = c / per;
-                slot = (s * 16 + b) * per + (c - r * per);
-            }
-            if (S > 1) st_async_f32(cluster_addr(smem_addr(s_gather) + 4u * (uint32_t)slot, (uint32_t)r), v, cluster_addr(recv_bar, (uint32_t)r));
-            else s_gather[slot] = v;
+            if (S > 1) st_async_f32(dst0 + 4u * (uint32_t)(b * bstride), v, dbar);
+            else s_gather[slot0 + b * bstride] = v;
         }
     }
     if (S > 1) {
