@@ -88,6 +88,51 @@ __device__ __forceinline__ void fma_row(float (&acc)[BT][8], const uint4 &v, con
     }
 }
 
+// ---- 8-bit weights (WB = 1 in the body below): a 16-byte load holds 16 columns of a row.
+// Two fp32 values in one 64-bit register, for the packed fp32 instructions of sm_100 (add.f32x2 / fma.rn.f32x2: one
+// instruction per two weights).
+__device__ __forceinline__ unsigned long long pack2(float lo, float hi) {
+    unsigned long long r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(__float_as_uint(lo)), "r"(__float_as_uint(hi)));
+    return r;
+}
+__device__ __forceinline__ unsigned long long add2(unsigned long long a, unsigned long long b) {
+    unsigned long long r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ unsigned long long fma2(unsigned long long a, unsigned long long b, unsigned long long c) {
+    unsigned long long r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+__device__ __forceinline__ void unpack2(unsigned long long v, float &lo, float &hi) {
+    uint32_t a, b;
+    asm("mov.b64 {%0, %1}, %2;" : "=r"(a), "=r"(b) : "l"(v));
+    lo = __uint_as_float(a);
+    hi = __uint_as_float(b);
+}
+// acc[b][j] (pairs of columns) += xv * q for the 16 signed bytes of v.  (byte ^ 0x80) placed in the mantissa of 2^23 reads
+// as 2^23 + (q + 128); adding -(2^23 + 128) gives q exactly; both steps and the multiply-add run two columns at a time.
+template <int BT, int CAP>
+__device__ __forceinline__ void fma_row_q8(unsigned long long (&acc)[BT][8], const uint4 &v, const float *__restrict__ s_xs, int i) {
+    const uint32_t u[4] = {v.x ^ 0x80808080u, v.y ^ 0x80808080u, v.z ^ 0x80808080u, v.w ^ 0x80808080u};
+    const unsigned long long neg = pack2(-8388736.0f, -8388736.0f);
+    unsigned long long w[8];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        w[2 * q] = add2(pack2(__uint_as_float(__byte_perm(u[q], 0x4B000000u, 0x7650)), __uint_as_float(__byte_perm(u[q], 0x4B000000u, 0x7651))), neg);
+        w[2 * q + 1] = add2(pack2(__uint_as_float(__byte_perm(u[q], 0x4B000000u, 0x7652)), __uint_as_float(__byte_perm(u[q], 0x4B000000u, 0x7653))), neg);
+    }
+#pragma unroll
+    for (int b = 0; b < BT; ++b) {
+        const float xv = s_xs[b * CAP + i];
+        const unsigned long long x2 = pack2(xv, xv);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) acc[b][j] = fma2(x2, w[j], acc[b][j]);
+    }
+}
+
 // Exact GELU, gelu(v) = v/2 (1 + erf(v / sqrt 2)), binary32.
 __device__ __forceinline__ float gelu_exact(float v) { return 0.5f * v * (1.0f + erff(v * 0.70710678118654752f)); }
 
@@ -231,12 +276,17 @@ __device__ __forceinline__ void prefetch_bias(const FcArgs &a, int tile, int s, 
 // PUT = chunk slots per warp and fill that the threshold code is unrolled for (at most fc_pu(BT), which sizes the
 // shared-memory list): that code is bound by instruction issue, so the launcher picks the smallest instantiation
 // that still takes the rank's channels in one fill.
-template <bool BF16, int BT, int MODE, typename XT, int EPI, int TNT, int PUT = fc_pu(BT)>
+// WB = bytes per weight: 2 (fp16 / bf16) or 1 (signed 8-bit with one binary32 scale per input channel, which is folded
+// into the pruned activation once per kept channel, so the stream multiplies by the raw integers).  A thread's 16-byte
+// load then covers 16 columns and 8 lanes cover a row of a 128-column tile.
+template <bool BF16, int BT, int MODE, typename XT, int EPI, int TNT, int PUT = fc_pu(BT), int WB = 2>
 __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const int s, const bool wait_inside) {
     constexpr int NT = FC_THREADS, PU = PUT, CAP = fc_cap(BT), RB = fc_rb(BT), U = fc_unroll(BT);
     constexpr int CAPC = FC_WARPS * PU;  // chunks per fill
     static_assert(PUT >= 1 && PUT <= fc_pu(BT), "the list is sized for fc_pu(BT) slots per warp");
-    constexpr int LPR = TNT / 8;      // lanes per row segment
+    static_assert(WB == 2 || (WB == 1 && EPI == EPI_BIAS && TNT == 128), "8-bit weights: plain FC, 128-column tiles");
+    constexpr int CPT = 16 / WB;      // columns per thread (one 16-byte load)
+    constexpr int LPR = TNT / CPT;    // lanes per row segment
     constexpr int NR = NT / LPR;      // row groups per CTA: group g streams rows g, g+NR, ...
     constexpr int HALF = TNT / 2;
     extern __shared__ __align__(16) unsigned char smem[];
@@ -262,11 +312,11 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
         col_ok = f < a.Nh;
         col = (cl / (LPR / 2)) * a.Nh + f;
     } else {
-        col = tile * TNT + cl * 8;
+        col = tile * TNT + cl * CPT;
         col_ok = col < a.Nh;
     }
-    const unsigned char *Wb = reinterpret_cast<const unsigned char *>(a.W) + (size_t)col * 2;
-    const size_t row_bytes = (size_t)a.ldw * 2;
+    const unsigned char *Wb = reinterpret_cast<const unsigned char *>(a.W) + (size_t)col * WB;
+    const size_t row_bytes = (size_t)a.ldw * WB;
 
     // Head of the stream, asked into L2 before anything is known about the activations: between the end of the
     // previous call and the first row request of this one (hand-over, activations and parameters through L2, compaction:
@@ -299,11 +349,15 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
     }
     float bias0[2], bias1[2];
 
-    float acc[BT][8];
+    float acc[BT][CPT];
+    unsigned long long acc2[BT][8];  // WB = 1: 16 columns per batch row as 8 packed pairs
 #pragma unroll
-    for (int b = 0; b < BT; ++b)
+    for (int b = 0; b < BT; ++b) {
 #pragma unroll
-        for (int j = 0; j < 8; ++j) acc[b][j] = 0.0f;
+        for (int j = 0; j < CPT; ++j) acc[b][j] = 0.0f;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) acc2[b][j] = 0ull;
+    }
 
     const int nchunks = (K + 31) >> 5;
     const int my_chunks = nchunks > s ? (nchunks - s + S - 1) / S : 0;  // chunks s, s+S, ...
@@ -364,6 +418,11 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
         }
 #pragma unroll
         for (int p = 0; p < PU; ++p) mk[p] = ld_act_if(mrow + p * kstep, mrow != nullptr && okx[p], pol_keep);
+        float sc[WB == 1 ? PU : 1];
+        if constexpr (WB == 1) {
+#pragma unroll
+            for (int p = 0; p < PU; ++p) sc[p] = ld_act_if(a.wscale + kbase + p * kstep, okx[p], pol_keep);
+        }
         if (MODE == MODE_GATHER && j0 == 0) {
             float *s_tau = reinterpret_cast<float *>(s_wcnt + FC_WARPS + 2);  // behind the 8-byte barrier
             if (tid == 0) *s_tau = tau_reg;
@@ -425,8 +484,11 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
                 const int pos = wbase + my_off[p] + __popc(bal[p] & ((1u << lane) - 1u));
                 s_k[pos] = (uint32_t)(kbase + p * kstep);
 #pragma unroll
-                for (int b = 0; b < BT; ++b)
-                    s_xs[b * CAP + pos] = (MODE == MODE_DENSE || ((km[p] >> b) & 1u)) ? xv[p][b] : 0.0f;
+                for (int b = 0; b < BT; ++b) {
+                    float v = (MODE == MODE_DENSE || ((km[p] >> b) & 1u)) ? xv[p][b] : 0.0f;
+                    if constexpr (WB == 1) v = __fmul_rn(v, sc[p]);  // the channel's weight scale, once per kept channel
+                    s_xs[b * CAP + pos] = v;
+                }
             }
         }
         __syncthreads();
@@ -452,13 +514,19 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
             for (int t0 = 0; t0 < nrows; t0 += 2 * G) {
 #pragma unroll
                 for (int u = 0; u < G; ++u)
-                    if (t0 + u < nrows) fma_row<BF16, BT, CAP>(acc, ga[u], s_xs, rg + NR * (t0 + u));
+                    if (t0 + u < nrows) {
+                        if constexpr (WB == 2) fma_row<BF16, BT, CAP>(acc, ga[u], s_xs, rg + NR * (t0 + u));
+                        else fma_row_q8<BT, CAP>(acc2, ga[u], s_xs, rg + NR * (t0 + u));
+                    }
 #pragma unroll
                 for (int u = 0; u < G; ++u)
                     if (t0 + 2 * G + u < nrows) ga[u] = ld_stream16(Wb + (size_t)s_k[rg + NR * (t0 + 2 * G + u)] * row_bytes, pol_stream);
 #pragma unroll
                 for (int u = 0; u < G; ++u)
-                    if (t0 + G + u < nrows) fma_row<BF16, BT, CAP>(acc, gb[u], s_xs, rg + NR * (t0 + G + u));
+                    if (t0 + G + u < nrows) {
+                        if constexpr (WB == 2) fma_row<BF16, BT, CAP>(acc, gb[u], s_xs, rg + NR * (t0 + G + u));
+                        else fma_row_q8<BT, CAP>(acc2, gb[u], s_xs, rg + NR * (t0 + G + u));
+                    }
 #pragma unroll
                 for (int u = 0; u < G; ++u)
                     if (t0 + 3 * G + u < nrows) gb[u] = ld_stream16(Wb + (size_t)s_k[rg + NR * (t0 + 3 * G + u)] * row_bytes, pol_stream);
@@ -475,15 +543,34 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
     // them in rank order.
     static_assert(RB == BT, "one reduction round");
     if (S > 1) cluster_wait();  // every rank's barrier is initialised (all ranks arrived at kernel start)
+    // WB = 1: the four row groups of a warp (lanes l, l ^ 8, l ^ 16, l ^ 24 hold the same columns) are added by shuffles
+    // in a fixed order first, so that the cross-warp reduction sees one partial per warp.
+    constexpr int NRED = WB == 1 ? FC_WARPS : NR;
+    if constexpr (WB == 1) {
 #pragma unroll
-    for (int rb = 0; rb < RB; ++rb) {
-        float4 *dst = reinterpret_cast<float4 *>(s_red + ((rg * RB + rb) * TNT + cl * 8));
-        dst[0] = make_float4(acc[rb][0], acc[rb][1], acc[rb][2], acc[rb][3]);
-        dst[1] = make_float4(acc[rb][4], acc[rb][5], acc[rb][6], acc[rb][7]);
+        for (int b = 0; b < BT; ++b) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) unpack2(acc2[b][j], acc[b][2 * j], acc[b][2 * j + 1]);
+#pragma unroll
+            for (int j = 0; j < CPT; ++j) {
+                acc[b][j] += __shfl_xor_sync(0xffffffffu, acc[b][j], 8);
+                acc[b][j] += __shfl_xor_sync(0xffffffffu, acc[b][j], 16);
+            }
+        }
+    }
+    if (WB == 2 || lane < LPR) {
+        const int g = WB == 1 ? warp : rg;
+#pragma unroll
+        for (int rb = 0; rb < RB; ++rb) {
+            float4 *dst = reinterpret_cast<float4 *>(s_red + ((g * RB + rb) * TNT + cl * CPT));
+#pragma unroll
+            for (int q = 0; q < CPT / 4; ++q)
+                dst[q] = make_float4(acc[rb][4 * q], acc[rb][4 * q + 1], acc[rb][4 * q + 2], acc[rb][4 * q + 3]);
+        }
     }
     __syncthreads();
     if (S > 1) {
-        reduce_send_round<BT, EPI, TNT, NR, RB>(s_red, 0, B, s, per, smem_addr(s_gather), bar);
+        reduce_send_round<BT, EPI, TNT, NRED, RB>(s_red, 0, B, s, per, smem_addr(s_gather), bar);
         bool landed = false;
         for (uint32_t it = 0; it < (1u << 22) && !landed; ++it) landed = mbarrier_try_wait(bar, 0);
         if (!landed && a.status) atomicCAS(a.status, 0, 2);  // never in a correct run; the result is then incomplete
@@ -491,7 +578,7 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
         float *owner[MAX_CLUSTER];
 #pragma unroll
         for (int q = 0; q < MAX_CLUSTER; ++q) owner[q] = s_gather;
-        reduce_push_round<BT, EPI, TNT, NR, RB>(s_red, 0, B, s, per, owner);
+        reduce_push_round<BT, EPI, TNT, NRED, RB>(s_red, 0, B, s, per, owner);
         __syncthreads();
     }
 
@@ -906,7 +993,7 @@ __device__ __forceinline__ void fc_body_mma(const FcArgs &a, const int tile, con
     if (S > 1) cluster.sync();
 }
 
-template <bool BF16, int BT, int MODE, typename XT, int EPI, int TNT, int PUT = fc_pu(BT)>
+template <bool BF16, int BT, int MODE, typename XT, int EPI, int TNT, int PUT = fc_pu(BT), int WB = 2>
 __global__ void __launch_bounds__(FC_THREADS, fc_min_blocks(BT)) fc_kernel(const FcArgs a) {
     if constexpr (is_mma(BT)) {
         if (a.hold_dependents) {  // as below
@@ -917,9 +1004,9 @@ __global__ void __launch_bounds__(FC_THREADS, fc_min_blocks(BT)) fc_kernel(const
         }
     } else if (a.hold_dependents) {  // parameter-producing call: ordinary stream order on both sides
         griddep_wait();
-        fc_body<BF16, BT, MODE, XT, EPI, TNT, PUT>(a, blockIdx.x, blockIdx.y, false);
+        fc_body<BF16, BT, MODE, XT, EPI, TNT, PUT, WB>(a, blockIdx.x, blockIdx.y, false);
     } else {
-        fc_body<BF16, BT, MODE, XT, EPI, TNT, PUT>(a, blockIdx.x, blockIdx.y, true);
+        fc_body<BF16, BT, MODE, XT, EPI, TNT, PUT, WB>(a, blockIdx.x, blockIdx.y, true);
     }
 }
 
