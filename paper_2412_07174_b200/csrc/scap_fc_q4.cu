@@ -42,16 +42,25 @@ __device__ __forceinline__ uint2 ld_stream8_if(const void *p, bool on) {
     return v;
 }
 
-// acc[j] += xv * (q_j - zero_j) for the 16 codes of v; zc[j] = 2^23 + zero_j.
-__device__ __forceinline__ void fma_row_q4(float (&acc)[16], const uint2 &v, const float (&zc)[16], float xv) {
+// acc[j] (pairs of columns) += xv * q_j for the 16 codes of v.  The zero point is not subtracted per weight: over the rows
+// of one group sum xv (q - z) = sum xv q - z sum xv, and the second sum is one addition per row (the caller keeps it).
+// A code becomes a float by placing it in the mantissa of 2^23 and subtracting 2^23 (exact); the even and the odd codes
+// of a word are masked out together, then one byte permute per code; subtraction and multiply-add run two columns at a time.
+__device__ __forceinline__ void fma_row_q4(unsigned long long (&acc)[8], const uint2 &v, float xv) {
+    const unsigned long long neg = pack2(-8388608.0f, -8388608.0f);
+    const unsigned long long x2 = pack2(xv, xv);
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
         const uint32_t w = h ? v.y : v.x;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const float q = __uint_as_float(((w >> (4 * i)) & 15u) | 0x4B000000u) - zc[8 * h + i];
-            acc[8 * h + i] = fmaf(xv, q, acc[8 * h + i]);
-        }
+        const uint32_t ev = w & 0x0F0F0F0Fu, od = (w >> 4) & 0x0F0F0F0Fu;  // codes 0,2,4,6 and 1,3,5,7, one per byte
+        const unsigned long long q01 = add2(pack2(__uint_as_float(__byte_perm(ev, 0x4B000000u, 0x7650)), __uint_as_float(__byte_perm(od, 0x4B000000u, 0x7650))), neg);
+        const unsigned long long q23 = add2(pack2(__uint_as_float(__byte_perm(ev, 0x4B000000u, 0x7651)), __uint_as_float(__byte_perm(od, 0x4B000000u, 0x7651))), neg);
+        const unsigned long long q45 = add2(pack2(__uint_as_float(__byte_perm(ev, 0x4B000000u, 0x7652)), __uint_as_float(__byte_perm(od, 0x4B000000u, 0x7652))), neg);
+        const unsigned long long q67 = add2(pack2(__uint_as_float(__byte_perm(ev, 0x4B000000u, 0x7653)), __uint_as_float(__byte_perm(od, 0x4B000000u, 0x7653))), neg);
+        acc[4 * h + 0] = fma2(x2, q01, acc[4 * h + 0]);
+        acc[4 * h + 1] = fma2(x2, q23, acc[4 * h + 1]);
+        acc[4 * h + 2] = fma2(x2, q45, acc[4 * h + 2]);
+        acc[4 * h + 3] = fma2(x2, q67, acc[4 * h + 3]);
     }
 }
 
@@ -192,16 +201,13 @@ __global__ void __launch_bounds__(FC_THREADS, 2) fc_q4_kernel(const Q4Args qa) {
                 const float4 *sp = reinterpret_cast<const float4 *>(qa.scale + gofs);
                 const float4 s0 = __ldcg(sp), s1 = __ldcg(sp + 1), s2 = __ldcg(sp + 2), s3 = __ldcg(sp + 3);
                 const uint4 zw = __ldcg(reinterpret_cast<const uint4 *>(qa.zero + gofs));
-                float acc[BT][16];
+                unsigned long long acc2[BT][8];  // sum xv q of the stretch, 16 columns as 8 packed pairs
+                float sx[BT];                    // sum xv of the stretch
 #pragma unroll
-                for (int b = 0; b < BT; ++b)
+                for (int b = 0; b < BT; ++b) {
+                    sx[b] = 0.0f;
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) acc[b][j] = 0.0f;
-                float zc[16];
-                {
-                    const uint32_t z4[4] = {zw.x, zw.y, zw.z, zw.w};
-#pragma unroll
-                    for (int j = 0; j < 16; ++j) zc[j] = 8388608.0f + (float)((z4[j >> 2] >> (8 * (j & 3))) & 255u);
+                    for (int j = 0; j < 8; ++j) acc2[b][j] = 0ull;
                 }
                 // two register groups of U / 2 row loads alternate: one is used while the other is in flight
                 constexpr int H = U / 2;
@@ -218,7 +224,11 @@ __global__ void __launch_bounds__(FC_THREADS, 2) fc_q4_kernel(const Q4Args qa) {
                     for (int u = 0; u < H; ++u) {
                         if (first + u < t_end) {
 #pragma unroll
-                            for (int b = 0; b < BT; ++b) fma_row_q4(acc[b], src[u], zc, s_xs[b * CAP + first + u]);
+                            for (int b = 0; b < BT; ++b) {
+                                const float xv = s_xs[b * CAP + first + u];
+                                sx[b] += xv;
+                                fma_row_q4(acc2[b], src[u], xv);
+                            }
                         }
                     }
                 };
@@ -230,11 +240,20 @@ __global__ void __launch_bounds__(FC_THREADS, 2) fc_q4_kernel(const Q4Args qa) {
                     use(vb, tb + H);
                     request(vb, tb + U + H);
                 }
+                // the stretch's contribution: scale (sum xv q - zero sum xv)
                 const float sc[16] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w, s2.x, s2.y, s2.z, s2.w, s3.x, s3.y, s3.z, s3.w};
+                const uint32_t z4[4] = {zw.x, zw.y, zw.z, zw.w};
 #pragma unroll
-                for (int b = 0; b < BT; ++b)
+                for (int b = 0; b < BT; ++b) {
+                    float acc[16];
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) y_acc[b][j] = fmaf(sc[j], acc[b][j], y_acc[b][j]);
+                    for (int j = 0; j < 8; ++j) unpack2(acc2[b][j], acc[2 * j], acc[2 * j + 1]);
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        const float zf = (float)((z4[j >> 2] >> (8 * (j & 3))) & 255u);
+                        y_acc[b][j] = fmaf(sc[j], fmaf(-zf, sx[b], acc[j]), y_acc[b][j]);
+                    }
+                }
                 t = t_end;
             }
         }
