@@ -507,22 +507,38 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
                 prefetch_bias<BF16, EPI, TNT>(a, tile, s, per, bias0, bias1);
                 bias_done = true;
             }
-            for (int t0 = 0; t0 < nrows; t0 += 2 * G) {
+            auto use = [&](const uint4 &v, int t) {
+                if constexpr (WB == 2) fma_row<BF16, BT, CAP>(acc, v, s_xs, rg + NR * t);
+                else fma_row_q8<BT, CAP>(acc2, v, s_xs, rg + NR * t);
+            };
+            // Full rounds first: while every row of this round and of the next exists the body carries no compares and
+            // no branches (they cost about as many instructions as the arithmetic of a row at batch 1); the guarded form
+            // finishes the list.
+            // (At batch 1 the second copy of the body costs more than it saves - measured, +0.2 us per sparse call on
+            // either weight format - so only the instantiations for two and more rows take the full rounds:
+            // -1.0 .. -1.7 us per call at batch 2 and 4, -2 .. -3 us at batch 2 on 8-bit weights.)
+            constexpr bool FULL_ROUNDS = BT >= 2;
+            int t0 = 0;
+            for (; FULL_ROUNDS && t0 + 4 * G <= nrows; t0 += 2 * G) {
+#pragma unroll
+                for (int u = 0; u < G; ++u) use(ga[u], t0 + u);
+#pragma unroll
+                for (int u = 0; u < G; ++u) ga[u] = ld_stream16(Wb + (size_t)s_k[rg + NR * (t0 + 2 * G + u)] * row_bytes, pol_stream);
+#pragma unroll
+                for (int u = 0; u < G; ++u) use(gb[u], t0 + G + u);
+#pragma unroll
+                for (int u = 0; u < G; ++u) gb[u] = ld_stream16(Wb + (size_t)s_k[rg + NR * (t0 + 3 * G + u)] * row_bytes, pol_stream);
+            }
+            for (; t0 < nrows; t0 += 2 * G) {
 #pragma unroll
                 for (int u = 0; u < G; ++u)
-                    if (t0 + u < nrows) {
-                        if constexpr (WB == 2) fma_row<BF16, BT, CAP>(acc, ga[u], s_xs, rg + NR * (t0 + u));
-                        else fma_row_q8<BT, CAP>(acc2, ga[u], s_xs, rg + NR * (t0 + u));
-                    }
+                    if (t0 + u < nrows) use(ga[u], t0 + u);
 #pragma unroll
                 for (int u = 0; u < G; ++u)
                     if (t0 + 2 * G + u < nrows) ga[u] = ld_stream16(Wb + (size_t)s_k[rg + NR * (t0 + 2 * G + u)] * row_bytes, pol_stream);
 #pragma unroll
                 for (int u = 0; u < G; ++u)
-                    if (t0 + G + u < nrows) {
-                        if constexpr (WB == 2) fma_row<BF16, BT, CAP>(acc, gb[u], s_xs, rg + NR * (t0 + G + u));
-                        else fma_row_q8<BT, CAP>(acc2, gb[u], s_xs, rg + NR * (t0 + G + u));
-                    }
+                    if (t0 + G + u < nrows) use(gb[u], t0 + G + u);
 #pragma unroll
                 for (int u = 0; u < G; ++u)
                     if (t0 + 3 * G + u < nrows) gb[u] = ld_stream16(Wb + (size_t)s_k[rg + NR * (t0 + 3 * G + u)] * row_bytes, pol_stream);

@@ -215,6 +215,24 @@ def test_pdl_off_gives_identical_bits(S):
     assert np.array_equal(y1, y2)
 
 
+@pytest.mark.parametrize("B", [1, 2, 4])
+@pytest.mark.parametrize("chunks", [1, 6, 64])
+def test_early_row_hints_change_no_bit(S, B, chunks):
+    """The optional L2 hints for the head of a sparse call's row stream (tune key head_rows) are requests without a
+    result: the kept list and every output bit stay as they are, also when the hint reaches past the rank's channels."""
+    d = si.laplace_fc(B, 1500, 520, si.BF16, 16, 2)
+    y1, idx1, nnz1 = run_sparse(S, d, d["m_true"], 0.2, None)
+    try:
+        S.scap_tune("head_rows", chunks)
+        y2, idx2, nnz2 = run_sparse(S, d, d["m_true"], 0.2, None)
+    finally:
+        S.scap_tune("head_rows", 0)
+    assert nnz1 == nnz2 and np.array_equal(idx1, idx2)
+    assert np.array_equal(y1, y2)
+    with pytest.raises(Exception):
+        S.scap_tune("head_rows", 65)
+
+
 def test_back_to_back_calls_share_a_workspace(S):
     # many calls in a row on one stream with different inputs: each must see only its own lists
     d = si.laplace_fc(4, 1024, 512, si.BF16, 16, 8)
