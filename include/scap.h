@@ -215,7 +215,7 @@ scap_status scap_fold_bias_q8(const signed char *Wq, const float *wscale, const 
  * group: a multiple of 32, 32..2048 (else SCAP_ERR_SHAPE); N a multiple of 16.  Everything else - x of dtype xdt, m, tau,
  * b_fused, y, the optional kept list, the batch rule (more than two rows run two at a time; idx_out / nnz_out only for
  * B <= 2), the workspace query - as for the 8-bit calls above.  The sum over the kept channels of one group is formed
- * on the integer codes, sum d * (q - zero) in fp32, and scaled once.                                                  */
+ * on the integer codes in fp32 as sum d * q - zero * sum d, and scaled once.                                          */
 scap_status scap_sparse_fc_q4(const void *x, scap_dtype xdt, const unsigned char *Wq, const float *scale,
                               const unsigned char *zero, int group, const float *m, const float *tau, const float *b_fused,
                               float *y, int B, int K, int N, uint32_t *idx_out, int *nnz_out, void *ws, size_t ws_bytes,
