@@ -45,7 +45,7 @@ def run_q8(S, d, m, tau, bf, want_idx=True):
 
 @pytest.mark.parametrize("K,N,B,dt", [
     (1024, 1024, 1, si.F16), (1500, 528, 1, si.BF16), (1500, 528, 2, si.BF16), (4100, 272, 2, si.F16), (96, 16, 1, si.BF16),
-    (11008, 4096, 1, si.BF16),
+    (11008, 4096, 1, si.BF16), (11008, 4096, 2, si.BF16), (14336, 512, 1, si.BF16), (14336, 512, 2, si.F16),
 ])
 def test_q8_sparse_fc_matches_the_oracle(S, K, N, B, dt):
     d = case(K, N, B, dt)
