@@ -485,7 +485,7 @@ struct DsMisc {
 __device__ __forceinline__ void mbar_arrive_expect_tx(unsigned long long *bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
 }
-// One box of the tensor map (64 columns x 64 rows) to shared memory; completion counts bytes on `bar`.  No multicast.
+// One box of the tensor map (64 columns x 64 rows) to shared memory; completion counts bytes on `bar`.  The copy goes to this CTA only.
 __device__ __forceinline__ void tma_box_2d(uint32_t dst, const CUtensorMap *map, int x, int y, unsigned long long *bar) {
     asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
                  "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar))
@@ -900,7 +900,7 @@ static EncodeTiledFn encode_tiled_fn() {
 }
 
 // W[K, ldw] of 16-bit elements as a 2-D tensor (columns innermost), boxes of 64 columns x 64 rows, 128-byte swizzle,
-// rows and columns beyond the matrix read as zeros.  The map covers this GPU's own W only; no multicast anywhere.
+// rows and columns beyond the matrix read as zeros.  The map covers this GPU's own W only, and every box is copied to the one CTA that asked for it.
 static bool ds_tensor_map(CUtensorMap *map, const void *W, int K, int ldw, bool bf16) {
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) return false;
