@@ -107,14 +107,12 @@ __global__ void __launch_bounds__(FC_THREADS, 2) fc_q4_kernel(const Q4Args qa) {
 
     griddep_wait();  // nothing is read before earlier work on the stream is complete
     if (!a.hold_dependents) griddep_launch_dependents();
-    float tau = 0.0f;
-    if constexpr (MODE == MODE_GATHER) {
-        float tv = 0.0f;
-        if (lane == 0) tv = ld_act(a.tau);
-        tau = __shfl_sync(0xffffffffu, tv, 0);
-    }
+    // tau: one request per CTA, issued first and handed to the other warps through shared memory once the activation
+    // requests of the first fill are out (as in the 16-bit kernel: the two round trips to L2 overlap)
+    float tau = 0.0f, tau_reg = 0.0f;
+    if (MODE == MODE_GATHER && tid == 0) tau_reg = ld_act(a.tau);
     float bias0[2], bias1[2];
-    prefetch_bias<true, EPI, TNT>(a, tile, s, per, bias0, bias1);
+    bool first_fill = true;
 
     for (int g0 = g_lo; g0 < g_hi; g0 += fill_groups) {
         const int ng = min(fill_groups, g_hi - g0);         // groups of this fill
@@ -132,6 +130,16 @@ __global__ void __launch_bounds__(FC_THREADS, 2) fc_q4_kernel(const Q4Args qa) {
 #pragma unroll
             for (int b = 0; b < BT; ++b) xraw[p][b] = ld_act_if(xg + (size_t)(b < B ? b : 0) * a.x_ld + k, ok && b < B);
             mk[p] = (MODE == MODE_GATHER && a.m) ? ld_act_if(a.m + k, ok) : 0.0f;
+        }
+        if (first_fill) {
+            if constexpr (MODE == MODE_GATHER) {
+                float *s_tau = reinterpret_cast<float *>(s_goff + Q4_MAXG + 1);
+                if (tid == 0) *s_tau = tau_reg;
+                __syncthreads();
+                tau = *s_tau;
+            }
+            prefetch_bias<true, EPI, TNT>(a, tile, s, per, bias0, bias1);  // behind the activation requests
+            first_fill = false;
         }
         uint32_t km[PU];
         unsigned bal[PU];
@@ -276,6 +284,7 @@ __global__ void __launch_bounds__(FC_THREADS, 2) fc_q4_kernel(const Q4Args qa) {
         __syncthreads();
     }
 
+    if (first_fill) prefetch_bias<true, EPI, TNT>(a, tile, s, per, bias0, bias1);  // a rank without groups
     // ---- reduction over the row groups (group order), cluster exchange, bias: as in the 16-bit kernel
     cg::cluster_group cluster = cg::this_cluster();
     float *owner[MAX_CLUSTER];
