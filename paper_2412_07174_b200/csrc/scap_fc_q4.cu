@@ -209,7 +209,22 @@ __global__ void __launch_bounds__(FC_THREADS, 2) fc_q4_kernel(const Q4Args qa) {
             constexpr int RGW = decltype(rgw_tag)::value;  // positions between two rows of a row group: 4 or 1
             constexpr bool interleave = RGW > 1;
             const int rows_per = interleave ? (cnt + FC_WARPS - 1) / FC_WARPS : (cnt + NR - 1) / NR;
-            const int r_lo = min(cnt, (interleave ? warp : rg) * rows_per), r_hi = min(cnt, r_lo + rows_per);
+            int r_lo = min(cnt, (interleave ? warp : rg) * rows_per), r_hi = min(cnt, r_lo + rows_per);
+            if constexpr (!interleave) {
+                // Short lists are bound by latency, not by balance: an end of a range that lies within half a range of a
+                // group boundary moves onto it, so that a row group mostly streams ONE group - all its row requests go
+                // out together instead of one dependent batch per group.
+                auto snap = [&](int b) {
+                    int best = 0, dist = cnt + 1;
+                    for (int g = 0; g <= ng; ++g) {
+                        const int d = abs(s_goff[g] - b);
+                        if (d < dist) { dist = d; best = s_goff[g]; }
+                    }
+                    return 2 * dist <= rows_per ? best : b;
+                };
+                r_lo = snap(min(cnt, rg * rows_per));
+                r_hi = snap(min(cnt, (rg + 1) * rows_per));
+            }
             const int jrg = interleave ? rg % (32 / LPR) : 0;
             int gl = 0;
             for (int t = r_lo; t < r_hi;) {
