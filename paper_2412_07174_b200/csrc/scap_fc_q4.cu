@@ -201,7 +201,7 @@ __global__ void __launch_bounds__(FC_THREADS, 2) fc_q4_kernel(const Q4Args qa) {
         // position of it (row group j the positions = r_lo + j mod 4), so that all lanes of the warp meet the group
         // boundaries in the same iteration and run the same number of rounds (with a contiguous range per row group
         // the four ranges of a warp crossed their boundaries at different places and the warp ran up to twice the rounds).
-        // Inside the range: one stretch per group.  Short lists (fewer than 16 rows per row group) keep a contiguous range
+        // Inside the range: one stretch per group.  Shorter lists (fewer than 24 rows per row group) keep a contiguous range
         // per row group instead: there every row group of the interleaved form would open and close every group of the
         // warp's range, and that bookkeeping costs more than the idle rounds (measured: 13.3 against 11.7 us at 80 %).
         // (Two copies of the loop, so that the distance between two rows of a row group is a constant in each.)
@@ -293,7 +293,7 @@ __global__ void __launch_bounds__(FC_THREADS, 2) fc_q4_kernel(const Q4Args qa) {
             }
         };
         if (col_ok) {
-            if (cnt >= NR * 16) stream(std::integral_constant<int, 32 / LPR>{});
+            if (cnt >= NR * 24) stream(std::integral_constant<int, 32 / LPR>{});
             else stream(std::integral_constant<int, 1>{});
         }
         __syncthreads();
