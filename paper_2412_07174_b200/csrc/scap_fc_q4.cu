@@ -105,6 +105,16 @@ __global__ void __launch_bounds__(FC_THREADS, 2) fc_q4_kernel(const Q4Args qa) {
     const int cpg = group >> 5;            // chunks per group
     const int fill_groups = CAP / group;   // whole groups per fill
 
+    // The barrier the split-K partials of this rank's columns will land on (asynchronous exchange, as in the 16-bit kernel)
+    const uint32_t bar = smem_addr(s_goff + Q4_MAXG + 2);
+    if (S > 1) {
+        if (tid == 0) {
+            const int owned = max(0, min(per, TNT - s * per));
+            mbarrier_init(bar, 1);
+            mbarrier_arrive_expect(bar, (uint32_t)(S * B * owned * 4));
+        }
+        cluster_arrive_relaxed();
+    }
     griddep_wait();  // nothing is read before earlier work on the stream is complete
     if (!a.hold_dependents) griddep_launch_dependents();
     // tau: one request per CTA, issued first and handed to the other warps through shared memory once the activation
@@ -300,11 +310,10 @@ __global__ void __launch_bounds__(FC_THREADS, 2) fc_q4_kernel(const Q4Args qa) {
     }
 
     if (first_fill) prefetch_bias<true, EPI, TNT>(a, tile, s, per, bias0, bias1);  // a rank without groups
-    // ---- reduction over the row groups (group order), cluster exchange, bias: as in the 16-bit kernel
-    cg::cluster_group cluster = cg::this_cluster();
-    float *owner[MAX_CLUSTER];
-#pragma unroll
-    for (int q = 0; q < MAX_CLUSTER; ++q) owner[q] = (S > 1 && q < S) ? cluster.map_shared_rank(s_gather, q) : s_gather;
+    // ---- reduction over the row groups (group order) and asynchronous cluster exchange, as in the 16-bit kernel: every
+    // sum goes to the rank that owns its column as a store that counts down that rank's barrier; a rank finishes when
+    // its own S partials are in.
+    if (S > 1) cluster_wait();  // every rank's barrier is initialised (all ranks arrived at kernel start)
 #pragma unroll
     for (int rb = 0; rb < RB; ++rb) {
         float4 *dst = reinterpret_cast<float4 *>(s_red + ((rg * RB + rb) * TNT + cl * Q4_CPT));
@@ -313,10 +322,18 @@ __global__ void __launch_bounds__(FC_THREADS, 2) fc_q4_kernel(const Q4Args qa) {
             dst[q] = make_float4(y_acc[rb][4 * q], y_acc[rb][4 * q + 1], y_acc[rb][4 * q + 2], y_acc[rb][4 * q + 3]);
     }
     __syncthreads();
-    reduce_push_round<BT, EPI, TNT, NR, RB>(s_red, 0, B, s, per, owner);
-    __syncthreads();
-    if (S > 1) cluster.sync();
-    else __syncthreads();
+    if (S > 1) {
+        reduce_send_round<BT, EPI, TNT, NR, RB>(s_red, 0, B, s, per, smem_addr(s_gather), bar);
+        bool landed = false;
+        for (uint32_t it = 0; it < (1u << 22) && !landed; ++it) landed = mbarrier_try_wait(bar, 0);
+        if (!landed && a.status) atomicCAS(a.status, 0, 2);  // never in a correct run; the result is then incomplete
+    } else {
+        float *owner[MAX_CLUSTER];
+#pragma unroll
+        for (int q = 0; q < MAX_CLUSTER; ++q) owner[q] = s_gather;
+        reduce_push_round<BT, EPI, TNT, NR, RB>(s_red, 0, B, s, per, owner);
+        __syncthreads();
+    }
     finish_columns<true, BT, EPI, TNT>(a, tile, s, per, s_gather, bias0, bias1);
 }
 
@@ -395,6 +412,7 @@ static void q4_fill(Q4Args &qa, const void *x, const void *Wq, const float *scal
     qa.f.W = Wq; qa.f.K = K; qa.f.ldw = N; qa.f.Nh = N; qa.f.B = B; qa.f.tn = Q4_TN; qa.f.S = q4_split(K, N, group);
     qa.f.x = x; qa.f.x_ld = K; qa.f.y = y; qa.f.y_ld = N;
     qa.scale = scale; qa.zero = zero; qa.group = group;
+    qa.f.status = tc_status_ptr();
 }
 
 scap_status scap_sparse_fc_q4(const void *x, scap_dtype xdt, const unsigned char *Wq, const float *scale, const unsigned char *zero,
