@@ -65,11 +65,16 @@ __device__ __forceinline__ void fma_row_q4(unsigned long long (&acc)[8], const u
     }
 }
 
-template <int BT, int MODE, typename XT>
+// PUT = chunk slots per warp and fill that the threshold code is unrolled for (at most fc_pu(BT), which sizes the list):
+// that code is bound by instruction issue, so the launcher picks the smallest instantiation whose fill still holds a
+// whole group and the rank's channels.
+template <int BT, int MODE, typename XT, int PUT = fc_pu(BT)>
 __global__ void __launch_bounds__(FC_THREADS, 2) fc_q4_kernel(const Q4Args qa) {
     const FcArgs &a = qa.f;
     constexpr int TNT = Q4_TN, EPI = EPI_BIAS, U = q4_unroll(BT);
-    constexpr int PU = fc_pu(BT), CAP = fc_cap(BT), RB = fc_rb(BT);
+    constexpr int PU = PUT, CAP = fc_cap(BT), RB = fc_rb(BT);
+    constexpr int FILL = FC_WARPS * PU * 32;  // channels per fill
+    static_assert(PUT >= 1 && PUT <= fc_pu(BT), "the list is sized for fc_pu(BT) slots per warp");
     constexpr int LPR = TNT / Q4_CPT;      // 8 lanes per row segment
     constexpr int NR = FC_THREADS / LPR;   // 32 row groups per CTA
     static_assert(RB == BT, "one reduction round");
@@ -103,7 +108,7 @@ __global__ void __launch_bounds__(FC_THREADS, 2) fc_q4_kernel(const Q4Args qa) {
     const int G = (K + group - 1) / group, gper = (G + S - 1) / S;
     const int g_lo = min(G, s * gper), g_hi = min(G, g_lo + gper);
     const int cpg = group >> 5;            // chunks per group
-    const int fill_groups = CAP / group;   // whole groups per fill
+    const int fill_groups = FILL / group;  // whole groups per fill (the launcher guarantees at least one)
 
     // The barrier the split-K partials of this rank's columns will land on (asynchronous exchange, as in the 16-bit kernel)
     const uint32_t bar = smem_addr(s_goff + Q4_MAXG + 2);
@@ -354,13 +359,24 @@ static int q4_split(int K, int N, int group) {
     return best_S;
 }
 
-template <int BT, int MODE, typename XT>
-static cudaError_t launch_q4_t(const Q4Args &qa, cudaStream_t st) {
+template <int BT, int MODE, typename XT, int PUT>
+static cudaError_t launch_q4_pu(const Q4Args &qa, cudaStream_t st) {
     static SmemOptIn opt_in;
-    auto kern = fc_q4_kernel<BT, MODE, XT>;
+    auto kern = fc_q4_kernel<BT, MODE, XT, PUT>;
     cudaError_t e0 = ensure_dynamic_smem(kern, q4_smem(BT), opt_in);
     if (e0 != cudaSuccess) return e0;
     return launch_cluster(kern, dim3((qa.f.ldw + Q4_TN - 1) / Q4_TN, qa.f.S), dim3(FC_THREADS), q4_smem(BT), qa.f.S, st, g_tune.pdl != 0, qa);
+}
+
+// 4, 6 or 8 chunk slots per warp: the fewest whose fill (slots x 256 channels) holds a whole group and, if possible,
+// all groups of a rank.
+template <int BT, int MODE, typename XT>
+static cudaError_t launch_q4_t(const Q4Args &qa, cudaStream_t st) {
+    const int group = qa.group, G = (qa.f.K + group - 1) / group, gper = (G + qa.f.S - 1) / qa.f.S;
+    const int need = (gper * group / 32 + FC_WARPS - 1) / FC_WARPS;  // slots that take the rank's channels in one fill
+    if (need <= 4 && group <= 4 * FC_WARPS * 32) return launch_q4_pu<BT, MODE, XT, 4>(qa, st);
+    if (need <= 6 && group <= 6 * FC_WARPS * 32) return launch_q4_pu<BT, MODE, XT, 6>(qa, st);
+    return launch_q4_pu<BT, MODE, XT, fc_pu(BT)>(qa, st);
 }
 
 // xkind: 0 fp16, 1 bf16, 2 float activations.  Batches beyond two rows run two rows at a time (row results are
