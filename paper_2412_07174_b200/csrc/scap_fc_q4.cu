@@ -135,17 +135,26 @@ __global__ void __launch_bounds__(FC_THREADS, 2) fc_q4_kernel(const Q4Args qa) {
         const int nj = min((ng * group) >> 5, ((K - k0) + 31) >> 5);  // chunks of the fill
         const int pw = (nj + FC_WARPS - 1) / FC_WARPS;      // consecutive chunks per warp
         // ---- threshold: as in the 16-bit kernel, with the rank's chunks contiguous
+        // (addresses and predicates first, then all requests of the lane back to back: the code runs on every warp of the
+        // SM at the same moment and is bound by instruction issue)
+        const int nw = max(0, min(pw, nj - warp * pw));      // chunks of this warp
+        const int kbase = k0 + warp * pw * 32 + lane;        // this lane's channel in the warp's first chunk
+        const XT *xrow[BT];
+#pragma unroll
+        for (int b = 0; b < BT; ++b) xrow[b] = xg + (size_t)(b < B ? b : 0) * a.x_ld + kbase;
+        const float *mrow = (MODE == MODE_GATHER && a.m) ? a.m + kbase : nullptr;
+        bool okx[PU];
+#pragma unroll
+        for (int p = 0; p < PU; ++p) okx[p] = p < nw && kbase + p * 32 < K;
         XT xraw[PU][BT];
         float xv[PU][BT], mk[PU];
 #pragma unroll
         for (int p = 0; p < PU; ++p) {
-            const int j = warp * pw + p;
-            const int k = k0 + j * 32 + lane;
-            const bool ok = p < pw && j < nj && k < K;
 #pragma unroll
-            for (int b = 0; b < BT; ++b) xraw[p][b] = ld_act_if(xg + (size_t)(b < B ? b : 0) * a.x_ld + k, ok && b < B);
-            mk[p] = (MODE == MODE_GATHER && a.m) ? ld_act_if(a.m + k, ok) : 0.0f;
+            for (int b = 0; b < BT; ++b) xraw[p][b] = ld_act_if(xrow[b] + p * 32, okx[p] && b < B);
         }
+#pragma unroll
+        for (int p = 0; p < PU; ++p) mk[p] = ld_act_if(mrow + p * 32, mrow != nullptr && okx[p]);
         if (first_fill) {
             if constexpr (MODE == MODE_GATHER) {
                 float *s_tau = reinterpret_cast<float *>(s_goff + Q4_MAXG + 1);
@@ -161,9 +170,7 @@ __global__ void __launch_bounds__(FC_THREADS, 2) fc_q4_kernel(const Q4Args qa) {
         int my_off[PU], wtotal = 0;
 #pragma unroll
         for (int p = 0; p < PU; ++p) {
-            const int j = warp * pw + p;
-            const int k = k0 + j * 32 + lane;
-            const bool ok = p < pw && j < nj && k < K;
+            const bool ok = okx[p];
             uint32_t m_ = 0;
 #pragma unroll
             for (int b = 0; b < BT; ++b) {
@@ -203,7 +210,7 @@ __global__ void __launch_bounds__(FC_THREADS, 2) fc_q4_kernel(const Q4Args qa) {
             if (lane == 0 && p < pw && j < nj && j % cpg == 0) s_goff[j / cpg] = wbase + my_off[p];  // the chunk opens a group
             if (km[p]) {
                 const int pos = wbase + my_off[p] + __popc(bal[p] & ((1u << lane) - 1u));
-                s_k[pos] = (uint32_t)(k0 + j * 32 + lane);
+                s_k[pos] = (uint32_t)(kbase + p * 32);
 #pragma unroll
                 for (int b = 0; b < BT; ++b)
                     s_xs[b * CAP + pos] = (MODE == MODE_DENSE || ((km[p] >> b) & 1u)) ? xv[p][b] : 0.0f;
