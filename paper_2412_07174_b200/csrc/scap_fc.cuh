@@ -517,7 +517,7 @@ __device__ __forceinline__ void fc_body(const FcArgs &a, const int tile, const i
             // (At batch 1 the second copy of the body costs more than it saves - measured, +0.2 us per sparse call on
             // either weight format - so only the instantiations for two and more rows take the full rounds:
             // -1.0 .. -1.7 us per call at batch 2 and 4, -2 .. -3 us at batch 2 on 8-bit weights.)
-            constexpr bool FULL_ROUNDS = BT >= 2;
+            constexpr bool FULL_ROUNDS = BT >= 2 || (WB == 1 && MODE == MODE_DENSE);  // (the dense 8-bit call gains 0.1 us)
             int t0 = 0;
             for (; FULL_ROUNDS && t0 + 4 * G <= nrows; t0 += 2 * G) {
 #pragma unroll
